@@ -1,0 +1,142 @@
+"""ctypes front end of the fp64 CPU oracle (oracle/pdattn_oracle.cpp).
+
+TEST INFRASTRUCTURE: only tests, the smoke check and the benchmark's CPU-baseline leg may
+import this.  It never touches the CUDA library and the CUDA library never touches it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pdattn_oracle.cpp")
+_LIB = os.path.join(_HERE, "libpdattn_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with plain g++ (no CUDA headers)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-pthread",
+                               "-ffp-contract=off", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    with _lock:
+        if _lib is None:
+            build()
+            L = ctypes.CDLL(_LIB)
+            vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
+            common = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i64, i64, i64, f32]
+            L.pdattn_oracle_decode.argtypes = common + [vp, i64, vp, i32, vp]
+            L.pdattn_oracle_decode.restype = i32
+            L.pdattn_oracle_partial.argtypes = common + [i32, i32, i32, i32, vp, vp, vp]
+            L.pdattn_oracle_partial.restype = i32
+            L.pdattn_oracle_merge.argtypes = [vp, vp, vp, i32, i32, vp]
+            L.pdattn_oracle_merge.restype = i32
+            L.pdattn_oracle_bf16_rne.argtypes = [ctypes.c_double]
+            L.pdattn_oracle_bf16_rne.restype = ctypes.c_uint16
+            L.pdattn_oracle_bf16_to_double.argtypes = [ctypes.c_uint16]
+            L.pdattn_oracle_bf16_to_double.restype = ctypes.c_double
+            _lib = L
+    return _lib
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def _cpu(t: torch.Tensor) -> torch.Tensor:
+    return t.detach().to("cpu").contiguous()
+
+
+def _common_args(q, k_cache, v_cache, block_table, context_lens, scale, keep):
+    q, block_table, context_lens = _cpu(q), _cpu(block_table).to(torch.int32), _cpu(context_lens).to(torch.int32)
+    k_cache, v_cache = k_cache.detach().to("cpu"), v_cache.detach().to("cpu")
+    assert q.dtype == torch.bfloat16 and k_cache.dtype == torch.bfloat16 and v_cache.dtype == torch.bfloat16
+    assert k_cache.stride() == v_cache.stride() and k_cache.shape == v_cache.shape
+    assert k_cache.stride(3) == 1
+    S, Hq, d = q.shape
+    NB, Hkv, bs, d2 = k_cache.shape          # logical [page, kv head, slot, dim]; any strides
+    assert d2 == d
+    MB = block_table.shape[1] if block_table.dim() == 2 else 0
+    keep.extend([q, k_cache, v_cache, block_table, context_lens])
+    args = [q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), block_table.data_ptr(), context_lens.data_ptr(),
+            S, Hq, Hkv, d, bs, MB, NB, k_cache.stride(0), k_cache.stride(1), k_cache.stride(2),
+            float(scale)]
+    return args, (S, Hq, d)
+
+
+def decode(q, k_cache, v_cache, block_table, context_lens, scale, pairs=None, num_threads=None,
+           return_bad=False):
+    """fp64 attention output.  k_cache / v_cache are indexed [page, kv_head, slot, dim] with any
+    strides (pass a permuted view for a token-major pool).  pairs: optional int array [n,2] of
+    (seq, q_head) to compute; the result is then [n, d], else [S, Hq, d]."""
+    keep = []
+    args, (S, Hq, d) = _common_args(q, k_cache, v_cache, block_table, context_lens, scale, keep)
+    if pairs is not None:
+        pairs = np.ascontiguousarray(np.asarray(pairs, dtype=np.int32).reshape(-1, 2))
+        n = pairs.shape[0]
+        out = np.empty((n, d), dtype=np.float64)
+        pptr = pairs.ctypes.data
+    else:
+        n = 0
+        out = np.empty((S, Hq, d), dtype=np.float64)
+        pptr = None
+    bad = ctypes.c_int64(0)
+    nt = int(num_threads) if num_threads else host_cores()
+    rc = lib().pdattn_oracle_decode(*args, pptr, n, out.ctypes.data, nt, ctypes.addressof(bad))
+    if rc != 0:
+        raise ValueError("pdattn_oracle_decode: invalid arguments")
+    return (out, bad.value) if return_bad else out
+
+
+def decode_workload(w, **kw):
+    return decode(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, **kw)
+
+
+def partial(q, k_cache, v_cache, block_table, context_lens, scale, s, h, t0, t1):
+    """(m, l, acc[d]) of tokens [t0, t1) for one (seq, head): natural-log-domain maximum,
+    sum of exp(x - m) and the un-normalised weighted V sum."""
+    keep = []
+    args, (S, Hq, d) = _common_args(q, k_cache, v_cache, block_table, context_lens, scale, keep)
+    m, l = ctypes.c_double(0), ctypes.c_double(0)
+    acc = np.empty(d, dtype=np.float64)
+    rc = lib().pdattn_oracle_partial(*args, int(s), int(h), int(t0), int(t1),
+                                     ctypes.addressof(m), ctypes.addressof(l), acc.ctypes.data)
+    if rc != 0:
+        raise ValueError("pdattn_oracle_partial: invalid arguments")
+    return m.value, l.value, acc
+
+
+def merge(ms, ls, accs):
+    ms = np.ascontiguousarray(ms, dtype=np.float64)
+    ls = np.ascontiguousarray(ls, dtype=np.float64)
+    accs = np.ascontiguousarray(accs, dtype=np.float64)
+    n, d = accs.shape
+    out = np.empty(d, dtype=np.float64)
+    lib().pdattn_oracle_merge(ms.ctypes.data, ls.ctypes.data, accs.ctypes.data, n, d, out.ctypes.data)
+    return out
+
+
+def bf16_rne(x: np.ndarray) -> np.ndarray:
+    """Round fp64 values to bf16 (nearest even), returned as float64 values."""
+    L = lib()
+    flat = np.asarray(x, dtype=np.float64).ravel()
+    out = np.empty_like(flat)
+    for i, v in enumerate(flat):
+        out[i] = L.pdattn_oracle_bf16_to_double(L.pdattn_oracle_bf16_rne(float(v)))
+    return out.reshape(np.shape(x))

@@ -1,0 +1,255 @@
+"""Pins of the fp64 oracle against closed forms, invariants and brute force (CPU only).
+
+Each test would fail under a plausible mistake in the oracle: a dropped or doubled token, a
+wrong page/slot/head index, a missing scale, a sign error in the exponent, a transposed operand.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import pdattn_oracle as orc
+from paper_2607_09207_b200 import workloads as W
+
+BF16 = torch.bfloat16
+
+
+def f64(t):
+    return t.to(torch.float32).to(torch.float64).numpy()
+
+
+def dense_kv(w, s):
+    """Independent gather of sequence s into dense [L, Hkv, d] fp64 arrays (numpy indexing)."""
+    L = int(w.context_lens_host[s])
+    bs = w.block_size
+    k = f64(w.k_cache)
+    v = f64(w.v_cache)
+    bt = w.block_table.numpy()
+    K = np.stack([k[bt[s, t // bs], :, t % bs, :] for t in range(L)]) if L else np.zeros((0, w.num_kv_heads, w.head_dim))
+    V = np.stack([v[bt[s, t // bs], :, t % bs, :] for t in range(L)]) if L else np.zeros((0, w.num_kv_heads, w.head_dim))
+    return K, V
+
+
+def brute(w):
+    """Textbook softmax(q K^T scale) V per head on the dense gather."""
+    S, Hq, d = w.q.shape
+    G = Hq // w.num_kv_heads
+    q = f64(w.q)
+    out = np.zeros((S, Hq, d))
+    for s in range(S):
+        K, V = dense_kv(w, s)
+        if K.shape[0] == 0:
+            continue
+        for h in range(Hq):
+            x = (K[:, h // G, :] @ q[s, h]) * float(np.float32(w.scale))
+            p = np.exp(x - x.max())
+            p /= p.sum()
+            out[s, h] = p @ V[:, h // G, :]
+    return out
+
+
+def test_context_len_one_returns_v_exactly():
+    w = W.make_custom([1, 1, 1], Hq=6, Hkv=2, d=64, seed=11)
+    out = orc.decode_workload(w)
+    v = f64(w.v_cache)
+    bt = w.block_table.numpy()
+    for s in range(3):
+        for h in range(6):
+            assert np.array_equal(out[s, h], v[bt[s, 0], h // 3, 0])
+
+
+@pytest.mark.parametrize("how", ["equal_keys", "zero_scale", "zero_q"])
+def test_uniform_weights_return_mean_of_v(how):
+    w = W.make_custom([37, 64, 5], Hq=4, Hkv=2, d=64, seed=12, poison=False)
+    if how == "equal_keys":
+        w.k_cache[:] = w.k_cache[0, 0, 0][None, None, None, :]
+    elif how == "zero_scale":
+        w.scale = 0.0
+    else:
+        w.q.zero_()
+    out = orc.decode_workload(w)
+    for s in range(3):
+        _, V = dense_kv(w, s)
+        for h in range(4):
+            np.testing.assert_allclose(out[s, h], V[:, h // 2].mean(0), rtol=1e-13, atol=1e-15)
+
+
+def test_page_permutation_leaves_bits_unchanged():
+    w = W.make_custom([100, 33, 256], Hq=4, Hkv=1, d=64, seed=13, num_blocks=64)
+    ref = orc.decode_workload(w)
+    rng = np.random.default_rng(5)
+    perm = rng.permutation(64)                      # new id of old page p is perm[p]
+    w2 = w.clone()
+    inv = np.argsort(perm)
+    w2.k_cache = w.k_cache[torch.from_numpy(inv)]
+    w2.v_cache = w.v_cache[torch.from_numpy(inv)]
+    bt = w.block_table.numpy().copy()
+    valid = bt >= 0
+    bt[valid] = perm[bt[valid]]
+    w2.block_table = torch.from_numpy(bt.astype(np.int32))
+    out = orc.decode_workload(w2)
+    assert np.array_equal(ref, out)
+
+
+def test_brute_force_dense_on_tiny_inputs():
+    for seed, (Hq, Hkv, d) in enumerate([(4, 1, 64), (6, 2, 32), (7, 7, 16), (8, 2, 128)]):
+        w = W.make_custom([1, 2, 15, 16, 17, 50, 0], Hq=Hq, Hkv=Hkv, d=d, seed=20 + seed, num_blocks=32)
+        np.testing.assert_allclose(orc.decode_workload(w), brute(w), rtol=1e-12, atol=1e-14)
+
+
+def test_tiny_config_matches_brute_force():
+    w = W.make_config(1)
+    np.testing.assert_allclose(orc.decode_workload(w), brute(w), rtol=1e-12, atol=1e-14)
+
+
+def test_context_len_two_is_a_sigmoid_blend():
+    w = W.make_custom([2], Hq=2, Hkv=1, d=32, seed=14)
+    out = orc.decode_workload(w)
+    K, V = dense_kv(w, 0)
+    q = f64(w.q)
+    for h in range(2):
+        x = (K[:, 0] @ q[0, h]) * float(np.float32(w.scale))
+        sg = 1.0 / (1.0 + math.exp(-(x[0] - x[1])))
+        np.testing.assert_allclose(out[0, h], sg * V[0, 0] + (1 - sg) * V[1, 0], rtol=1e-13, atol=1e-15)
+
+
+def test_dominant_key_selects_its_value():
+    w = W.make_custom([70], Hq=1, Hkv=1, d=64, seed=15, poison=False)
+    w.k_cache.zero_()
+    w.q[:] = 1.0
+    w.scale = 1.0
+    bt = w.block_table.numpy()
+    t = 37
+    w.k_cache[bt[0, t // 16], 0, t % 16, :] = 1.0      # score 64, all others 0
+    out = orc.decode_workload(w)
+    _, V = dense_kv(w, 0)
+    # the 69 other weights are e^-64 = 1.6e-28 each
+    assert np.abs(out[0, 0] - V[t, 0]).max() < 1e-20
+
+
+def test_score_shift_invariance():
+    """Adding the same constant to every score of a head (an extra dimension with q = 1 and a
+    constant key) must not change the output."""
+    w = W.make_custom([45, 16], Hq=2, Hkv=1, d=32, seed=16, poison=False)
+    base = orc.decode_workload(w)
+    S, Hq, d = w.q.shape
+    q2 = torch.zeros(S, Hq, d + 32, dtype=BF16)
+    q2[..., :d] = w.q
+    q2[..., d] = 1.0
+    k2 = torch.zeros(w.num_blocks, 1, 16, d + 32, dtype=BF16)
+    k2[..., :d] = w.k_cache
+    k2[..., d] = 3.0
+    v2 = torch.zeros_like(k2)
+    v2[..., :d] = w.v_cache
+    out = orc.decode(q2, k2, v2, w.block_table, w.context_lens, w.scale)
+    np.testing.assert_allclose(out[..., :d], base, rtol=1e-12, atol=1e-14)
+    assert np.all(out[..., d:] == 0)
+
+
+def test_convex_hull_and_linearity_in_v():
+    w = W.make_custom([90, 3], Hq=4, Hkv=2, d=64, seed=17, poison=False)
+    out = orc.decode_workload(w)
+    for s in range(2):
+        _, V = dense_kv(w, s)
+        for h in range(4):
+            lo, hi = V[:, h // 2].min(0), V[:, h // 2].max(0)
+            assert np.all(out[s, h] >= lo - 1e-12) and np.all(out[s, h] <= hi + 1e-12)
+    w2 = w.clone()
+    w2.v_cache = (w.v_cache.to(torch.float32) * 2.0).to(BF16)     # exact in bf16
+    np.testing.assert_allclose(orc.decode_workload(w2), 2.0 * out, rtol=1e-14, atol=0)
+
+
+def test_split_merge_identity():
+    """Attention over [0,L) equals the (m, l, acc) merge of partials over [0,c) and [c,L): pins
+    the combine formula independently of any GPU code."""
+    w = W.make_custom([200], Hq=4, Hkv=2, d=64, seed=18)
+    full = orc.decode_workload(w)
+    args = (w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale)
+    for h in range(4):
+        for cuts in ([64], [1], [199], [64, 128], [16, 17, 150]):
+            edges = [0] + cuts + [200]
+            parts = [orc.partial(*args, 0, h, a, b) for a, b in zip(edges[:-1], edges[1:])]
+            ms, ls, accs = zip(*parts)
+            got = orc.merge(ms, ls, np.stack(accs))
+            np.testing.assert_allclose(got, full[0, h], rtol=1e-12, atol=1e-15)
+
+
+def test_library_softmax_matmul_on_identity_table():
+    """With an identity block table the pool is a dense [L, d] array: compare with torch's fp64
+    softmax and matmul."""
+    L, d, Hq, Hkv = 80, 64, 4, 2
+    w = W.make_custom([L], Hq=Hq, Hkv=Hkv, d=d, seed=19, num_blocks=8, poison=False)
+    w.block_table = torch.arange(5, dtype=torch.int32)[None, :]
+    out = orc.decode_workload(w)
+    K = w.k_cache.to(torch.float64).permute(1, 0, 2, 3).reshape(Hkv, -1, d)[:, :L]
+    V = w.v_cache.to(torch.float64).permute(1, 0, 2, 3).reshape(Hkv, -1, d)[:, :L]
+    q = w.q.to(torch.float64)[0]
+    for h in range(Hq):
+        p = torch.softmax((K[h // 2] @ q[h]) * float(np.float32(w.scale)), dim=0)
+        np.testing.assert_allclose(out[0, h], (p @ V[h // 2]).numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_gqa_head_map_is_contiguous_groups():
+    """q head h reads KV head h // G: make KV head 1 the only one that differs."""
+    w = W.make_custom([20], Hq=6, Hkv=3, d=32, seed=21, poison=False)
+    w.v_cache.zero_()
+    w.v_cache[:, 1] = 1.0
+    out = orc.decode_workload(w)
+    for h in range(6):
+        expect = 1.0 if h // 2 == 1 else 0.0
+        np.testing.assert_allclose(out[0, h], expect, rtol=1e-14)
+
+
+def test_poisoned_tail_and_unowned_pages_do_not_matter():
+    w = W.make_custom([1, 17, 100], Hq=4, Hkv=1, d=64, seed=22, num_blocks=32, poison=False)
+    clean = orc.decode_workload(w)
+    W.poison_unused(w)
+    assert torch.isnan(w.k_cache.float()).any()
+    out = orc.decode_workload(w)
+    assert np.array_equal(clean, out)
+
+
+def test_zero_length_and_empty_batch():
+    w = W.make_custom([0, 5], Hq=2, Hkv=1, d=32, seed=23)
+    out = orc.decode_workload(w)
+    assert np.all(out[0] == 0) and np.isfinite(out).all()
+    e = W.make_custom([], Hq=2, Hkv=1, d=32, seed=23)
+    assert orc.decode_workload(e).shape == (0, 2, 32)
+
+
+def test_out_of_range_pages_are_skipped_and_counted():
+    w = W.make_custom([48], Hq=2, Hkv=1, d=32, seed=24, num_blocks=16, poison=False)
+    ref_w = w.clone()
+    bt = w.block_table.clone()
+    bt[0, 1] = 99                                     # tokens 16..31 unreachable
+    w.block_table = bt
+    out, bad = orc.decode_workload(w, return_bad=True)
+    assert bad == 16 * 2
+    # equals attention over tokens 0..15 and 32..47 of the intact cache
+    args = (ref_w.q, ref_w.k_cache, ref_w.v_cache, ref_w.block_table, ref_w.context_lens, ref_w.scale)
+    for h in range(2):
+        a = orc.partial(*args, 0, h, 0, 16)
+        b = orc.partial(*args, 0, h, 32, 48)
+        got = orc.merge([a[0], b[0]], [a[1], b[1]], np.stack([a[2], b[2]]))
+        np.testing.assert_allclose(out[0, h], got, rtol=1e-12, atol=1e-15)
+
+
+def test_strided_token_major_pool_gives_same_result():
+    """The same logical cache stored [page, slot, head, dim] (token-major) through strides."""
+    w = W.make_custom([40, 9], Hq=4, Hkv=2, d=32, seed=25)
+    ref = orc.decode_workload(w)
+    k_nhd = w.k_cache.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    v_nhd = w.v_cache.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert k_nhd.stride() != w.k_cache.stride()
+    out = orc.decode(w.q, k_nhd, v_nhd, w.block_table, w.context_lens, w.scale)
+    assert np.array_equal(ref, out)
+
+
+def test_bf16_rounding_helper():
+    xs = np.array([0.0, 1.0, 1.00390625, 1.005859375, -2.5, 3.3895313892515355e38, 1e-40, 0.1])
+    got = orc.bf16_rne(xs)
+    want = torch.tensor(xs, dtype=torch.float64).to(torch.float32).to(BF16).to(torch.float64).numpy()
+    # 1.00390625 = 1 + 2^-8 is a tie: rounds to even (1.0); 1.005859375 = 1 + 1.5*2^-8 rounds up
+    assert got[2] == 1.0 and got[3] == 1.0078125
+    np.testing.assert_array_equal(got, want)
