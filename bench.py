@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of libpdattn: one step = one paged-decode-attention call (split-KV kernel + combine
+kernel) over one rollout batch, through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--cfg 2]
+
+Workload: benchmark configs[1], the 7B-shaped rollout step (256 sequences, 28 q heads / 4 KV
+heads, head_dim 128, page size 16, context = 512-token prompt + lognormal response), synthetic and
+seeded.  With N > 1 (torchrun, one rank per GPU) every rank runs its own batch of that shape
+(sequences are independent: no collective on the data path) and the value is the sum over ranks
+divided by the slowest rank's time: weak scaling.
+
+Prints ONE JSON line.  `value` is seq-steps/s with everything resident in HBM; `e2e` is the same
+metric through pdattn_decode_host with the step's q / block_table / context_lens in pinned host
+memory and `out` read back every step; `roofline` is the split-KV kernel's algorithmic KV bytes
+over its own CUDA-event duration against the measured HBM copy bandwidth; `cpu_baseline` is the
+fp64 oracle timed on this machine's host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import re
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+METRIC = "paged decode attn: seq-steps/s (achieved HBM TB/s in roofline) at N GPUs"
+UNIT = "seq-steps/s"
+CFG_DESC = {
+    1: "configs[0] tiny: 4 seqs, 4/1 heads, d64",
+    2: "configs[1] 7B-shaped rollout step: 256 seqs, 28 q / 4 kv heads, d128, page 16, "
+       "ctx = 512 + lognormal(median 2048, sigma 0.8) capped 8192, seed 1",
+    3: "configs[2] GRPO group sharing: 64x8 seqs, 40/8 heads, d128, shared 1024-token prompt pages",
+    4: "configs[3] 32B-shaped long context: 128 seqs, 64/8 heads, d128",
+    5: "configs[4] long-tail straggler phase: 8 seqs, 28/4 heads, d128, ctx U[32768,65536]",
+}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cfg", type=int, default=2, help="BASELINE.json config index + 1 (default: the metric's config)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, STREAM-style copy)"
+    except Exception:
+        return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+def profiled_traffic(cfg):
+    """dram bytes per decode_kernel launch from the committed ncu summary, or None."""
+    p = os.path.join(ROOT, "profiles", f"decode_kernel_cfg{cfg}_ncu.md")
+    try:
+        m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)", open(p).read())
+        return float(m.group(1)) if m else None
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Polls NVML for SM clock and throttle reasons while the timed regions run."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._stop.clear()
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        if self._thr is not None:
+            self._stop.set()
+            self._thr.join()
+            self._thr = None
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_pass(wc, n_seqs):
+    """Time the oracle, as it stands, on the first n_seqs sequences of the host copy of the workload."""
+    from oracle import pdattn_oracle as orc
+    cores = orc.host_cores()
+    sl = slice(0, n_seqs)
+    t0 = time.perf_counter()
+    orc.decode(wc.q[sl], wc.k_cache, wc.v_cache, wc.block_table[sl], wc.context_lens[sl], wc.scale,
+               num_threads=cores)
+    return time.perf_counter() - t0, cores
+
+
+def run_reference(args):
+    """The reference arm is the fp64 CPU oracle (there is no reference implementation of this path):
+    each step is one oracle pass over a bounded sample of the workload, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2607_09207_b200 import workloads as W
+    w = W.make_config(args.cfg, device="cpu", poison=True)
+    S = w.num_seqs
+    t_probe, cores = oracle_pass(w, min(S, 8))
+    per_seq = t_probe / min(S, 8)
+    budget = 150.0 / max(1, args.steps + args.warmup)          # whole run within a few minutes
+    n = int(max(1, min(S, min(budget, 3.0) / max(per_seq, 1e-9))))
+    for _ in range(args.warmup):
+        oracle_pass(w, n)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(w, n)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = f"first {n} of {S} sequences of the workload per step, {args.steps} steps"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": CFG_DESC[args.cfg], "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    from paper_2607_09207_b200 import pdattn
+    from paper_2607_09207_b200 import workloads as W
+    pdattn.lib()   # fail loudly if the CUDA library is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    K, Wm = args.steps, max(3, args.warmup)
+    # ---- inputs: this rank's batch, in two physically distinct copies (pools, tables, q) so that
+    # consecutive steps never find the previous step's pages in L2
+    base = W.make_config(args.cfg, device=dev)
+    if world > 1:
+        # every rank gets its own lengths and values: same shape, different seed stream
+        lens = W.config_lengths(args.cfg)
+        rng = np.random.default_rng(1000 + rank)
+        base = W.make_config(args.cfg, device=dev) if rank == 0 else _reseeded(W, args.cfg, rank, dev, lens, rng)
+    copies = [base]
+    if base.unique_kv_bytes() < (40 << 30):
+        copies.append(_physical_copy(base, seed=77 + rank))
+    S = base.num_seqs
+    uniq = base.unique_kv_bytes()
+    logical = base.logical_kv_bytes()
+    ws = pdattn.alloc_workspace(S, base.num_q_heads, base.num_kv_heads, base.head_dim, base.block_size, device=dev)
+    outs = [torch.empty_like(c.q) for c in copies]
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local)
+
+    def step(i):
+        c = copies[i % len(copies)]
+        pdattn.decode_ex(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale, outs[i % len(copies)],
+                         ws, context_lens_host=c.context_lens_host, stream=stream)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- region A: headline
+    for i in range(Wm):
+        step(i)
+    launches_per_step = pdattn.last_launch_count()
+    assert pdattn.check(ws) == pdattn.OK
+    sync_all()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(K):
+        step(i)
+    e1.record(stream)
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / K
+    value = world * S / (ms_step * 1e-3)
+
+    # ---- region B: the split-KV kernel's own duration, CUDA events recorded around it by the library
+    nb = min(K, 200)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nb)]
+    for a, b in evs:                      # force creation of the underlying CUDA events
+        a.record(stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    L = pdattn.lib()
+    for i, (a, b) in enumerate(evs):
+        L.pdattn_profile_events(a.cuda_event, b.cuda_event)
+        step(i)
+    L.pdattn_profile_events(None, None)
+    torch.cuda.synchronize()
+    k1_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    peak, peak_src = measured_peak()
+    achieved = uniq / (k1_ms * 1e-3) / 1e9
+
+    # ---- region C: end to end from pinned host buffers through pdattn_decode_host
+    c0 = copies[0]
+    qh, bth, lh = c0.q.cpu().pin_memory(), c0.block_table.cpu().pin_memory(), c0.context_lens.cpu().pin_memory()
+    oh = torch.empty_like(qh).pin_memory()
+    staging = torch.empty(pdattn.host_staging_size(S, c0.num_q_heads, c0.head_dim, c0.max_blocks_per_seq),
+                          dtype=torch.uint8, device=dev)
+    ke = min(K, 500)
+
+    def e2e_step():
+        pdattn.decode_host(qh, bth, lh, oh, c0.k_cache, c0.v_cache, c0.scale, staging, ws, stream=stream)
+        stream.synchronize()              # the caller reads `out` on the host every step
+        return float(oh[0, 0, 0])
+
+    for _ in range(5):
+        e2e_step()
+    sync_all()
+    t0 = time.perf_counter()
+    for _ in range(ke):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    sampler.stop()
+    e2e_value = world * S * ke / e2e_s
+    h2d = qh.numel() * 2 + bth.numel() * 4 + lh.numel() * 4
+    d2h = oh.numel() * 2
+    assert pdattn.check(ws) == pdattn.OK
+
+    # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only)
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        wc = base.to("cpu")
+        t_probe, cores = oracle_pass(wc, min(S, 8))
+        n = int(max(1, min(S, 20.0 / max(t_probe / min(S, 8), 1e-9))))
+        dt, cores = oracle_pass(wc, n)
+        cpu_baseline = {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"one oracle pass over the first {n} of {S} sequences ({dt:.2f} s)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": CFG_DESC[args.cfg], "num_seqs_per_gpu": S,
+                       "unique_kv_bytes_per_step": uniq, "logical_kv_bytes_per_step": logical,
+                       "l2": f"inputs ({uniq / 1e9:.2f} GB) larger than L2 and steps rotate over {len(copies)} "
+                             "physically distinct copies of pools/tables",
+                       "parallelism": f"dp{world} (independent batches, no collective)"},
+            "hbm_tbs_step": uniq / (ms_step * 1e-3) / 1e12 * 1.0,
+            "pct_of_8tbs_nominal_step": uniq / (ms_step * 1e-3) / 8e12 * 100.0,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": profiled_traffic(args.cfg),
+                         "kernel": "decode_kernel", "kernel_ms": k1_ms, "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": uniq,
+                         "pct_of_8tbs_nominal": achieved / 8000.0 * 100.0},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": ke, "note": "q/block_table/context_lens from pinned host memory, out read back "
+                                         "and the stream synchronised every step; KV pools are resident state"},
+            "gpu_launches": launches_per_step * K,
+            "clocks": sampler.summary(),
+            "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def _physical_copy(w, seed):
+    """Same logical batch in a second, differently permuted set of physical pages."""
+    import dataclasses
+    NB = w.num_blocks
+    dev = w.k_cache.device
+    perm = torch.from_numpy(np.random.default_rng(seed).permutation(NB)).to(dev)
+    inv = torch.argsort(perm)
+    bt = w.block_table.clone().long()
+    valid = bt >= 0
+    bt[valid] = perm[bt[valid]]
+    return dataclasses.replace(w, q=w.q.clone(), k_cache=w.k_cache[inv].contiguous(),
+                               v_cache=w.v_cache[inv].contiguous(), block_table=bt.to(torch.int32),
+                               context_lens=w.context_lens.clone())
+
+
+def _reseeded(W, cfg, rank, dev, lens, rng):
+    """Another batch of the same configuration for rank > 0: lengths shuffled, values reseeded."""
+    lens = rng.permutation(lens)
+    shapes = {2: (28, 4), 3: (40, 8), 4: (64, 8), 5: (28, 4), 1: (4, 1)}
+    Hq, Hkv = shapes[cfg]
+    d = 64 if cfg == 1 else 128
+    return W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, seed=1000 * cfg + rank, device=dev)
+
+
+if __name__ == "__main__":
+    main()

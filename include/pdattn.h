@@ -1,0 +1,164 @@
+/*
+ * libpdattn -- paged decode attention for RL rollout on NVIDIA B200 (sm_100a).
+ *
+ * One call = one layer's attention for one autoregressive decode step of a whole rollout
+ * batch: a single query token per sequence attends over that sequence's history in a paged
+ * bf16 KV cache (the "autoregressive decoding" of the rollout stage, Section 2.1 and Section 2.3
+ * of the paper; the cache's per-token size is the b_kv formula of Appendix A.1.2, and the cost
+ * the paper models as linear in history tokens is the beta_hist * H_dec term of the same appendix).
+ *
+ *     out[s,h,:] = softmax_t( scale * <q[s,h,:], K_s[t, h/G, :]> ) . V_s[t, h/G, :],  t in [0, L_s)
+ *
+ * G = num_q_heads / num_kv_heads; token t of sequence s is slot t % block_size of physical page
+ * block_table[s, t / block_size]; L_s = context_lens[s] counts the current token (its K/V are
+ * already in the cache).  Scores and accumulation are fp32, the output is rounded to bf16
+ * (nearest even).
+ *
+ * Conventions for every entry point
+ *   - C ABI, no exceptions, no aborts: a negative pdattn_status reports failure.
+ *   - Pointers marked DEVICE must be device memory of the current device, HOST ordinary host
+ *     memory.  All memory is caller-owned; the library never allocates, frees or keeps device
+ *     memory, creates no streams, and synchronises only where stated.
+ *   - Work is enqueued on `stream`; outputs are valid once the stream reaches that point.
+ *   - The only state is the thread-local binding made by pdattn_bind().
+ */
+#ifndef PDATTN_H_
+#define PDATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int pdattn_status;
+#define PDATTN_OK                   0
+#define PDATTN_INVALID_ARG         (-1) /* null pointer, negative size, Hq % Hkv != 0, ...           */
+#define PDATTN_UNSUPPORTED         (-2) /* head_dim not in {64,128}, block_size != 16, G > 16, or a
+                                           cache stride that is not a multiple of 8 elements          */
+#define PDATTN_WORKSPACE_TOO_SMALL (-3)
+#define PDATTN_MISALIGNED          (-4) /* q / k_cache / v_cache / out / workspace not 16-byte aligned */
+#define PDATTN_NOT_BOUND           (-5) /* pdattn_decode() without pdattn_bind() on this thread       */
+#define PDATTN_CUDA_ERROR          (-6) /* a CUDA call failed; text in pdattn_last_cuda_error()       */
+#define PDATTN_BAD_PAGE_INDEX      (-7) /* reported by pdattn_check(): a used block_table entry was
+                                           outside [0, num_blocks)                                   */
+#define PDATTN_DEVICE_TIMEOUT      (-8) /* reported by pdattn_check(): a bounded wait inside a kernel
+                                           gave up; that call's output is undefined                  */
+
+typedef struct CUstream_st* pdattn_stream_t; /* a cudaStream_t */
+
+/*
+ * Size of the scratch area a decode call needs (the partial (m, l, acc) triples of split
+ * sequences, the per-CTA work spans and one sticky error word).  max_context_len is accepted
+ * for forward compatibility and does not change the result today.  pinned_host_bytes (optional)
+ * receives 0: no pinned staging is needed.
+ */
+pdattn_status pdattn_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                                    int block_size, int max_context_len,
+                                    size_t* device_bytes, size_t* pinned_host_bytes);
+
+/*
+ * Clear the workspace's error word.  Call once after allocating a workspace (and at will later);
+ * enqueued on `stream`.  workspace: DEVICE.
+ */
+pdattn_status pdattn_workspace_init(void* workspace, size_t workspace_bytes, pdattn_stream_t stream);
+
+/* All arguments of one decode step.  Strides are in ELEMENTS; head_dim is contiguous. */
+typedef struct {
+  const void* q;                    /* DEVICE bf16 [num_seqs, num_q_heads, head_dim], dense          */
+  const void* k_cache;              /* DEVICE bf16, element (page, kv_head, slot, j) at               */
+  const void* v_cache;              /*   page*kv_block_stride + kv_head*kv_head_stride +              */
+                                    /*   slot*kv_token_stride + j.  Both caches use the same strides. */
+  void* out;                        /* DEVICE bf16 [num_seqs, num_q_heads, head_dim], dense          */
+  const int32_t* block_table;       /* DEVICE int32 [num_seqs, max_blocks_per_seq], row-major.        */
+                                    /*   Entries at or past ceil(L_s/block_size) are never read.      */
+  const int32_t* context_lens;      /* DEVICE int32 [num_seqs]                                        */
+  const int32_t* context_lens_host; /* HOST copy of context_lens for the host partitioner, or NULL:   */
+                                    /*   then a small planning kernel runs on the device instead.      */
+                                    /*   Read during the call only.  Must equal the device array.      */
+  int num_seqs, num_q_heads, num_kv_heads, head_dim, block_size;
+  int max_blocks_per_seq;           /* row stride of block_table                                      */
+  int num_blocks;                   /* pages in each pool; used entries must be in [0, num_blocks)    */
+  int64_t kv_block_stride, kv_head_stride, kv_token_stride;
+  float scale;                      /* multiplies q.k before the softmax                              */
+  void* workspace;                  /* DEVICE, >= pdattn_workspace_size() bytes, 256-byte aligned     */
+  size_t workspace_bytes;
+} pdattn_args;
+
+/*
+ * The decode step (Section 2.3's decoding loop body, attention part).  Launches the split-KV
+ * kernel and the split-combine kernel on `stream`; never synchronises.
+ *   - num_seqs == 0: PDATTN_OK, nothing launched.  L_s == 0: out[s] = +0.
+ *   - The same page may appear in many rows (shared prompt pages of a GRPO group) or twice in one.
+ *   - Cache slots at or past L_s and pages no row references may hold anything (NaN included)
+ *     and do not influence `out`.
+ *   - A used block_table entry outside [0, num_blocks) is not dereferenced: its tokens are left
+ *     out of the softmax and the workspace's sticky error word is set (see pdattn_check).
+ *   - The result is a pure function of the logical inputs: bit-identical from run to run, under
+ *     any renumbering of physical pages, and for shared versus privately copied prefix pages.
+ *   - Two calls that share a workspace must not overlap on the GPU.
+ */
+pdattn_status pdattn_decode_ex(const pdattn_args* args, pdattn_stream_t stream);
+
+/*
+ * Thread-local binding of the arguments the short form below does not carry.
+ * context_lens_host may be NULL.  The pointers must stay valid while bound.
+ */
+pdattn_status pdattn_bind(int max_blocks_per_seq, int num_blocks, void* workspace,
+                          size_t workspace_bytes, const int32_t* context_lens_host);
+
+/*
+ * Short form: dense caches [num_blocks, num_kv_heads, block_size, head_dim]; everything else as
+ * pdattn_decode_ex with the values bound on this thread.
+ */
+pdattn_status pdattn_decode(const void* q, const void* k_cache, const void* v_cache,
+                            const int32_t* block_table, const int32_t* context_lens,
+                            int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                            int block_size, float scale, void* out, pdattn_stream_t stream);
+
+/*
+ * End-to-end form for a caller whose per-step inputs live in HOST memory (pinned for real
+ * asynchrony): copies q, block_table and context_lens to the device staging area, runs
+ * pdattn_decode_ex (host partitioner on context_lens_host = the given lengths), copies `out`
+ * back.  All on `stream`; the caller synchronises.  The KV pools are resident device state.
+ * staging: DEVICE, >= pdattn_host_staging_size() bytes, 256-byte aligned.
+ */
+pdattn_status pdattn_host_staging_size(int num_seqs, int num_q_heads, int head_dim,
+                                       int max_blocks_per_seq, size_t* device_bytes);
+pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_host,
+                                 const int32_t* context_lens_host, void* out_host,
+                                 const void* k_cache, const void* v_cache,
+                                 int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                                 int block_size, int max_blocks_per_seq, int num_blocks, float scale,
+                                 void* staging, size_t staging_bytes,
+                                 void* workspace, size_t workspace_bytes, pdattn_stream_t stream);
+
+/*
+ * The host partitioner on its own (no GPU needed): splits the batch's KV stream into n_ctas
+ * contiguous spans of 64-token tiles so that long-tail sequences are spread over all SMs.
+ * Units are (sequence, kv head) pairs in the order unit = s * num_kv_heads + kv_head; unit u has
+ * ceil(L_s / 64) tiles.  Span c starts at tile spans[2c+1] of unit spans[2c] and holds
+ * *tiles_q + (c < *tiles_r) tiles.  spans: HOST int32 [2 * n_ctas].  Returns the total tile
+ * count in *total_tiles.  Depends on the context lengths only, never on page ids.
+ */
+pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, int num_kv_heads,
+                               int n_ctas, int32_t* spans, int* tiles_q, int* tiles_r,
+                               int64_t* total_tiles);
+
+/*
+ * Synchronises `stream`, reads and clears the workspace's sticky error word.
+ * Returns PDATTN_OK, PDATTN_BAD_PAGE_INDEX or PDATTN_DEVICE_TIMEOUT.
+ */
+pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream);
+
+/* Number of kernels the last pdattn_decode_ex on this thread launched (2 or 3). */
+int pdattn_last_launch_count(void);
+
+const char* pdattn_status_string(pdattn_status status);
+const char* pdattn_last_cuda_error(void); /* thread-local text of the last CUDA failure */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PDATTN_H_ */

@@ -1,0 +1,780 @@
+// Device code of libpdattn (sm_100a only).
+//
+//   decode_kernel  : split-KV flash decoding.  One persistent CTA per SM walks a contiguous span
+//                    of the batch's 64-token KV tiles.  A producer warp streams K/V pages from HBM
+//                    into a shared-memory ring with TMA tensor copies (128-byte swizzle) signalled
+//                    through mbarriers; the consumer warps each take whole tiles, compute
+//                    S^T = K.Q^T and O^T += V^T.P^T with bf16 tensor-core MMAs (tokens on M, the
+//                    packed GQA query heads of the KV head on N) and keep the online-softmax
+//                    running max / sum in fp32.
+//   combine_kernel : merges the (m, l, acc) triples of units that a span boundary cut.
+//   plan_kernel    : device-side twin of the host partitioner for callers without host lengths.
+//
+// No kernel waits on another CTA.  Every mbarrier wait is bounded (kWaitLimitNs); on expiry the
+// CTA raises ERR_TIMEOUT in the error word, stops consuming and returns normally.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace pdattn {
+
+constexpr int TILE = 64;                         // tokens per pipeline stage
+constexpr int MAX_PARAM_SPANS = 320;             // spans that travel in kernel parameters
+constexpr int MAX_CTAS = 592;                    // upper bound used for workspace sizing
+constexpr int MAX_STAGES = 12;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2 };
+
+// Workspace header (first 256 bytes of the workspace)
+struct WsHeader {
+  int32_t err;       // sticky error bits
+  int32_t tiles_q;   // written by plan_kernel
+  int32_t tiles_r;
+  int32_t pad[61];
+};
+
+struct DecodeParams {
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  const int32_t* block_table;
+  const int32_t* context_lens;
+  WsHeader* hdr;
+  const int2* spans_ws;     // spans written by plan_kernel (used when use_ws_plan)
+  int4* rec;                // per-CTA record: (first_unit, first_tile, own_unit, own_slot)
+  float* partials;          // [cta][2][HP*(D+2)] fp32
+  int S, Hq, Hkv, G, MB, NB;
+  float scale_log2;         // scale * log2(e)
+  int tiles_q, tiles_r;
+  int use_ws_plan;
+  int2 spans[MAX_PARAM_SPANS];
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when the limit expired.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
+  }
+  return true;
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+// 4-D tiled TMA load (no multicast), completion counted in bytes on an mbarrier of this CTA.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, int w,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+template <int NCT>
+__device__ __forceinline__ void bar_consumers() {   // named barrier 1: the NCT consumer threads
+  asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
+// Shared-memory plan
+// ------------------------------------------------------------------------------------------
+template <int D, int NT, int BS>
+struct Cfg {
+  static constexpr int PAGES = TILE / BS;              // pages per tile
+  static constexpr int HALVES = D / 64;                // 128-byte column blocks per row
+  static constexpr int HALF_BYTES = BS * 128;          // one TMA box: BS rows x 128 bytes
+  static constexpr int PAGE_BYTES = BS * D * 2;
+  static constexpr int KV_BYTES = TILE * D * 2;
+  static constexpr int STAGE_BYTES = 2 * KV_BYTES;     // K tile then V tile
+  static constexpr int HP = 8 * NT;                    // padded query heads per KV head
+  static constexpr int KSTEPS = D / 16;
+  // Consumer warp w owns the tiles with index = w (mod NCW) and tile i lives in ring slot i mod
+  // NSTAGES.  NSTAGES must be a multiple of NCW: then the tile that used a slot one ring turn
+  // earlier belonged to the same warp, so a warp can never wait on a slot's next mbarrier phase
+  // while the previous one is still pending (a parity wait cannot tell those apart).
+  static constexpr int NCW = (D == 128 && NT == 2) ? 5 : 6;            // consumer warps
+  static constexpr int NSTAGES = (D == 128) ? NCW : 2 * NCW;
+  static constexpr int NCT = NCW * 32;                                 // consumer threads
+  static constexpr int NTHREADS = NCT + 32;                            // + 1 producer warp
+  static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the scratch stores conflict-free
+  static constexpr int SCRATCH_BYTES = NCW * HP * ACC_STRIDE * 4;
+  static constexpr int ML_BYTES = NCW * HP * 2 * 4;
+  static constexpr int CTRL_BYTES = 256;
+  static constexpr int SMEM_MAX = 232448;              // 227 KB
+  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + SCRATCH_BYTES + ML_BYTES + CTRL_BYTES;
+  static constexpr int SLOT_FLOATS = HP * (D + 2);     // one partial: m[HP], l[HP], acc[HP][D]
+  static_assert(NSTAGES % NCW == 0 && NSTAGES <= MAX_STAGES, "ring/warp mapping");
+  static_assert(DYN_BYTES <= SMEM_MAX, "shared memory");
+  static_assert(TILE % BS == 0 && BS % 16 == 0, "block size");
+};
+
+struct Ctrl {                 // lives in the CTRL_BYTES area
+  uint64_t full[MAX_STAGES];
+  uint64_t empty[MAX_STAGES];
+  uint32_t meta[MAX_STAGES];  // per stage: bit j set = page j of the tile had a bad id
+  uint32_t abort;
+};
+static_assert(sizeof(Ctrl) <= 256, "control block");
+
+// ------------------------------------------------------------------------------------------
+// The walk over a span: pieces = (unit, tile range) in order.  Every warp runs the same walk.
+// ------------------------------------------------------------------------------------------
+struct Piece {
+  int unit, s, g, L, nt, tb, te;
+};
+struct Walker {
+  const int32_t* ctx;
+  int Hkv, nunits, unit, tb, rem;
+  __device__ __forceinline__ bool next(Piece& p) {
+    while (rem > 0 && unit < nunits) {
+      const int s = unit / Hkv;
+      const int L = __ldg(ctx + s);
+      const int nt = L > 0 ? (L + TILE - 1) / TILE : 0;
+      if (tb >= nt) {
+        ++unit;
+        tb = 0;
+        continue;
+      }
+      p.unit = unit;
+      p.s = s;
+      p.g = unit - s * Hkv;
+      p.L = L;
+      p.nt = nt;
+      p.tb = tb;
+      p.te = min(nt, tb + rem);
+      rem -= p.te - p.tb;
+      ++unit;
+      tb = 0;
+      return true;
+    }
+    return false;
+  }
+};
+
+// ------------------------------------------------------------------------------------------
+// One 64-token tile on one warp
+// ------------------------------------------------------------------------------------------
+template <int D, int NT, int BS, bool TAIL>
+__device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uint32_t (&qf)[NT][D / 16][2],
+                                             float (&acc)[NT][D / 16][4], float (&m)[NT][2], float (&l)[NT][2],
+                                             float sl2, int n_valid, uint32_t badmask, int lane) {
+  using C = Cfg<D, NT, BS>;
+  constexpr int GROUPS = TILE / 16;     // 16-token MMA groups per tile
+  const float NEG_INF = __int_as_float(0xff800000);
+
+  // per-lane pieces of the ldmatrix addresses
+  const int l8 = lane & 7;
+  const int mi = lane >> 3;
+  // K (A operand, row-major [token][d]): matrices (tok 0-7,c), (tok 8-15,c), (tok 0-7,c+1), (tok 8-15,c+1)
+  const int k_row = l8 + 8 * (mi & 1);
+  const int k_csel = mi >> 1;
+  // V (A operand = V^T via .trans): matrices (tok 0-7,c), (tok 0-7,c+1), (tok 8-15,c), (tok 8-15,c+1)
+  const int v_row = l8 + 8 * (mi >> 1);
+  const int v_csel = mi & 1;
+
+  if (TAIL) {
+    // Zero the V rows past the last valid token inside its 16-token group: P is 0 there, but
+    // 0 * NaN would still poison the accumulator.
+    const int g_last = (n_valid - 1) >> 4;
+    const int r_beg = n_valid - (g_last << 4);   // 1..16
+    const int nrows = 16 - r_beg;
+    const int tok0 = (g_last << 4) + r_beg;
+    for (int idx = lane; idx < nrows * (D / 8); idx += 32) {
+      const int tok = tok0 + idx / (D / 8);
+      const int ch = idx % (D / 8);
+      const int page = tok / BS, row = tok % BS;
+      const uint32_t a = sV + page * C::PAGE_BYTES + (ch >> 3) * C::HALF_BYTES + row * 128 + ((ch & 7) << 4);
+      asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+    }
+    __syncwarp();
+  }
+
+  // ---- S^T = K . Q^T : [64 tokens] x [8*NT heads]
+  float sc[GROUPS][NT][4];
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) sc[j][nt][0] = sc[j][nt][1] = sc[j][nt][2] = sc[j][nt][3] = 0.f;
+    if (!TAIL || j * 16 < n_valid) {
+      const int page = (j * 16) / BS, row0 = (j * 16) % BS;
+      const int row = row0 + k_row;
+      const uint32_t base = sK + page * C::PAGE_BYTES + row * 128;
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const int half = kk >> 2;
+        const int ch = ((kk & 3) * 2 + k_csel) ^ (row & 7);
+        uint32_t a[4];
+        ldsm_x4(a, base + half * C::HALF_BYTES + (ch << 4));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_bf16(sc[j][nt], a, qf[nt][kk][0], qf[nt][kk][1]);
+      }
+    }
+  }
+
+  // ---- scale, mask
+  const int trow = lane >> 2;
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j) {
+    bool dead_page = false;
+    if (badmask) dead_page = (badmask >> ((j * 16) / BS)) & 1u;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        float v = sc[j][nt][r] * sl2;
+        if (TAIL) {
+          const int tok = j * 16 + trow + ((r & 2) ? 8 : 0);
+          if (tok >= n_valid) v = NEG_INF;
+        }
+        if (dead_page) v = NEG_INF;
+        sc[j][nt][r] = v;
+      }
+  }
+
+  // ---- online softmax: running max per head (2 heads per thread per N tile)
+  float alpha[NT][2], muse[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      float mx = NEG_INF;
+#pragma unroll
+      for (int j = 0; j < GROUPS; ++j) mx = fmaxf(mx, fmaxf(sc[j][nt][e], sc[j][nt][e + 2]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+      const float m_new = fmaxf(m[nt][e], mx);
+      const float mu = (m_new == NEG_INF) ? 0.f : m_new;
+      alpha[nt][e] = fast_exp2(m[nt][e] - mu);
+      muse[nt][e] = mu;
+      m[nt][e] = m_new;
+      l[nt][e] *= alpha[nt][e];
+    }
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int jm = 0; jm < D / 16; ++jm) {
+      acc[nt][jm][0] *= alpha[nt][0];
+      acc[nt][jm][1] *= alpha[nt][1];
+      acc[nt][jm][2] *= alpha[nt][0];
+      acc[nt][jm][3] *= alpha[nt][1];
+    }
+
+  // ---- P = exp2(S - m), transposed into the B-operand layout.  bf16 keeps 8 bits of P, which is
+  // not enough when a few tokens carry the weight (short contexts, peaked softmax), so P goes
+  // to the tensor cores as hi + lo, two bf16 terms (16 bits of significand).
+  uint32_t pb[GROUPS][NT][2], pl[GROUPS][NT][2];
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float p0 = fast_exp2(sc[j][nt][0] - muse[nt][0]);
+      const float p1 = fast_exp2(sc[j][nt][1] - muse[nt][1]);
+      const float p2 = fast_exp2(sc[j][nt][2] - muse[nt][0]);
+      const float p3 = fast_exp2(sc[j][nt][3] - muse[nt][1]);
+      l[nt][0] += p0 + p2;
+      l[nt][1] += p1 + p3;
+      const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);
+      const uint32_t l01 = pack_bf16x2(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u));
+      const uint32_t l23 = pack_bf16x2(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xffff0000u));
+      pb[j][nt][0] = movmatrix_trans(h01);
+      pb[j][nt][1] = movmatrix_trans(h23);
+      pl[j][nt][0] = movmatrix_trans(l01);
+      pl[j][nt][1] = movmatrix_trans(l23);
+    }
+
+  // ---- O^T += V^T . P^T : [D] x [8*NT heads], K = 64 tokens
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j) {
+    if (!TAIL || j * 16 < n_valid) {
+      const int page = (j * 16) / BS, row0 = (j * 16) % BS;
+      const int row = row0 + v_row;
+      const uint32_t base = sV + page * C::PAGE_BYTES + row * 128;
+#pragma unroll
+      for (int jm = 0; jm < D / 16; ++jm) {
+        const int half = jm >> 2;
+        const int ch = ((jm & 3) * 2 + v_csel) ^ (row & 7);
+        uint32_t a[4];
+        ldsm_x4_trans(a, base + half * C::HALF_BYTES + (ch << 4));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          mma_bf16(acc[nt][jm], a, pb[j][nt][0], pb[j][nt][1]);
+          mma_bf16(acc[nt][jm], a, pl[j][nt][0], pl[j][nt][1]);
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// The decode kernel
+// ------------------------------------------------------------------------------------------
+template <int D, int NT, int BS>
+__global__ void __launch_bounds__(Cfg<D, NT, BS>::NTHREADS, 1)
+decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+              const __grid_constant__ DecodeParams P) {
+  using C = Cfg<D, NT, BS>;
+  constexpr int NST = C::NSTAGES;
+  constexpr int NCW = C::NCW;
+  constexpr int NCT = C::NCT;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;
+  const uint32_t ring = raw + pad;                                        // NST stages, 1024-aligned
+  float* scratch = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);  // [NCW][HP][ACC_STRIDE]
+  float* sm_m = scratch + NCW * C::HP * C::ACC_STRIDE;                     // [NCW][HP]
+  float* sm_l = sm_m + NCW * C::HP;                                        // [NCW][HP]
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm_l + NCW * C::HP);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int cta = blockIdx.x;
+  const float NEG_INF = __int_as_float(0xff800000);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NST; ++i) {
+      mbar_init(smem_u32(&ctrl->full[i]), 1);
+      mbar_init(smem_u32(&ctrl->empty[i]), 1);
+    }
+    ctrl->abort = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  // this CTA's span
+  int unit0, tile0, ntiles;
+  {
+    int2 sp;
+    int tq, tr;
+    if (P.use_ws_plan) {
+      sp = P.spans_ws[cta];
+      tq = P.hdr->tiles_q;
+      tr = P.hdr->tiles_r;
+    } else {
+      sp = P.spans[cta];
+      tq = P.tiles_q;
+      tr = P.tiles_r;
+    }
+    unit0 = sp.x;
+    tile0 = sp.y;
+    ntiles = tq + (cta < tr ? 1 : 0);
+  }
+  Walker walk{P.context_lens, P.Hkv, P.S * P.Hkv, unit0, tile0, ntiles};
+  Piece pc;
+  int it = 0;   // tile counter within this CTA: tile `it` uses ring slot it % NST
+
+  if (warp == NCW) {
+    // ================= producer warp =================
+    constexpr int IDS_PER_BATCH = 32;
+    constexpr int TILES_PER_BATCH = IDS_PER_BATCH / C::PAGES;
+    bool any_bad = false;
+    bool aborted = false;
+    while (!aborted && walk.next(pc)) {
+      const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
+      const int npages = (pc.L + BS - 1) / BS;
+      const int pbase = pc.tb * C::PAGES;
+      int ids_cur = (pbase + lane < npages) ? __ldg(row + pbase + lane) : 0;
+      int ids_nxt = (pbase + IDS_PER_BATCH + lane < npages) ? __ldg(row + pbase + IDS_PER_BATCH + lane) : 0;
+      for (int t = pc.tb; t < pc.te; ++t, ++it) {
+        const int rel = t - pc.tb;
+        const int k = rel % TILES_PER_BATCH;
+        if (k == 0 && rel != 0) {
+          ids_cur = ids_nxt;
+          const int nb = pbase + rel * C::PAGES + IDS_PER_BATCH;
+          ids_nxt = (nb + lane < npages) ? __ldg(row + nb + lane) : 0;
+        }
+        const int slot = it % NST;
+        const uint32_t phase = (it / NST) & 1;
+        if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) {
+          aborted = true;
+          break;
+        }
+        const int np = min(C::PAGES, npages - t * C::PAGES);
+        const int j = lane % C::PAGES;
+        int id = __shfl_sync(0xffffffffu, ids_cur, k * C::PAGES + j);
+        const bool bad = (lane < C::PAGES) && (j < np) && (id < 0 || id >= P.NB);
+        const uint32_t badmask = __ballot_sync(0xffffffffu, bad);
+        if (id < 0 || id >= P.NB) id = P.NB;   // out-of-bounds coordinate: TMA fills zeros, nothing is read
+        const uint32_t bar = smem_u32(&ctrl->full[slot]);
+        if (lane == 0) {
+          ctrl->meta[slot] = badmask;
+          mbar_arrive_expect_tx(bar, static_cast<uint32_t>(np) * 2u * C::PAGE_BYTES);
+        }
+        __syncwarp();
+        if (lane < 2 * C::PAGES && j < np) {
+          const bool isV = lane >= C::PAGES;
+          const uint32_t dst = ring + slot * C::STAGE_BYTES + (isV ? C::KV_BYTES : 0) + j * C::PAGE_BYTES;
+          const CUtensorMap* tm = isV ? &tmV : &tmK;
+#pragma unroll
+          for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, tm, h * 64, 0, pc.g, id, bar);
+        }
+        any_bad |= (badmask != 0);
+      }
+    }
+    if (lane == 0) {
+      if (any_bad) atomicOr(&P.hdr->err, ERR_BAD_PAGE);
+      if (aborted) {
+        atomicOr(&P.hdr->err, ERR_TIMEOUT);
+        atomicExch(&ctrl->abort, 1u);
+      }
+    }
+    return;
+  }
+
+  // ================= consumer warps =================
+  const int ct = threadIdx.x;   // 0..NCT-1
+  // sequences with no context produce zeros
+  for (int s = cta; s < P.S; s += gridDim.x) {
+    if (__ldg(P.context_lens + s) <= 0) {
+      uint32_t* o = reinterpret_cast<uint32_t*>(P.out + static_cast<int64_t>(s) * P.Hq * D);
+      for (int i = ct; i < P.Hq * D / 2; i += NCT) o[i] = 0u;
+    }
+  }
+
+  int first_unit = -1, first_tb = 0, own_unit = -1, own_slot = 0, piece_idx = 0;
+  bool aborted = false;
+  const int hq0 = lane >> 2;         // B-operand column (head) this lane feeds
+  const int qcol = (lane & 3) * 2;
+
+  while (walk.next(pc)) {
+    // ---- packed query rows of this KV head as MMA B fragments
+    uint32_t qf[NT][D / 16][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int head = nt * 8 + hq0;
+      const bool live = head < P.G;
+      const uint32_t* qp = reinterpret_cast<const uint32_t*>(
+          P.q + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + (live ? head : 0)) * D);
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        qf[nt][kk][0] = live ? __ldg(qp + (kk * 16 + qcol) / 2) : 0u;
+        qf[nt][kk][1] = live ? __ldg(qp + (kk * 16 + 8 + qcol) / 2) : 0u;
+      }
+    }
+    float acc[NT][D / 16][4];
+    float m[NT][2], l[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      m[nt][0] = m[nt][1] = NEG_INF;
+      l[nt][0] = l[nt][1] = 0.f;
+#pragma unroll
+      for (int jm = 0; jm < D / 16; ++jm) acc[nt][jm][0] = acc[nt][jm][1] = acc[nt][jm][2] = acc[nt][jm][3] = 0.f;
+    }
+
+    for (int t = pc.tb; t < pc.te; ++t, ++it) {
+      if (it % NCW != warp) continue;
+      if (!aborted && *reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) aborted = true;
+      if (aborted) continue;
+      const int slot = it % NST;
+      const uint32_t phase = (it / NST) & 1;
+      if (!mbar_wait(smem_u32(&ctrl->full[slot]), phase)) {
+        aborted = true;
+        if (lane == 0) {
+          atomicOr(&P.hdr->err, ERR_TIMEOUT);
+          atomicExch(&ctrl->abort, 1u);
+        }
+        continue;
+      }
+      const uint32_t sK = ring + slot * C::STAGE_BYTES;
+      const uint32_t sV = sK + C::KV_BYTES;
+      const uint32_t badmask = ctrl->meta[slot];
+      const int n_valid = min(TILE, pc.L - t * TILE);
+      if (n_valid == TILE) {
+        compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane);
+      } else {
+        compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_valid, badmask, lane);
+        fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
+    }
+
+    // ---- merge the NCW warp states of this piece
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float v = l[nt][e];
+        v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        l[nt][e] = v;
+      }
+    {
+      float* my = scratch + warp * C::HP * C::ACC_STRIDE;
+      const int drow = lane >> 2;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const int h0 = nt * 8 + qcol;
+#pragma unroll
+        for (int jm = 0; jm < D / 16; ++jm) {
+          my[h0 * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][0];
+          my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][1];
+          my[h0 * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][2];
+          my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][3];
+        }
+        if (lane < 4) {
+          sm_m[warp * C::HP + h0] = m[nt][0];
+          sm_m[warp * C::HP + h0 + 1] = m[nt][1];
+          sm_l[warp * C::HP + h0] = l[nt][0];
+          sm_l[warp * C::HP + h0 + 1] = l[nt][1];
+        }
+      }
+    }
+    bar_consumers<NCT>();
+    const bool complete = (pc.tb == 0 && pc.te == pc.nt);
+    const int slot_idx = piece_idx == 0 ? 0 : 1;
+    float* part = P.partials + (static_cast<int64_t>(cta) * 2 + slot_idx) * C::SLOT_FLOATS;
+    for (int idx = ct; idx < C::HP * (D / 4); idx += NCT) {
+      const int h = idx / (D / 4);
+      const int dq = idx % (D / 4);
+      float M = NEG_INF;
+#pragma unroll
+      for (int w = 0; w < NCW; ++w) M = fmaxf(M, sm_m[w * C::HP + h]);
+      const float Mu = (M == NEG_INF) ? 0.f : M;
+      float Ls = 0.f;
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int w = 0; w < NCW; ++w) {
+        const float f = fast_exp2(sm_m[w * C::HP + h] - Mu);
+        Ls += sm_l[w * C::HP + h] * f;
+        const float4 v = *reinterpret_cast<const float4*>(scratch + (w * C::HP + h) * C::ACC_STRIDE + dq * 4);
+        a.x += v.x * f;
+        a.y += v.y * f;
+        a.z += v.z * f;
+        a.w += v.w * f;
+      }
+      if (complete) {
+        if (h < P.G) {
+          const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
+          uint2 o;
+          o.x = pack_bf16x2(a.x * inv, a.y * inv);
+          o.y = pack_bf16x2(a.z * inv, a.w * inv);
+          *reinterpret_cast<uint2*>(P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + h) * D + dq * 4) = o;
+        }
+      } else {
+        if (dq == 0) {
+          part[h] = M;
+          part[C::HP + h] = Ls;
+        }
+        *reinterpret_cast<float4*>(part + 2 * C::HP + h * D + dq * 4) = a;
+      }
+    }
+    bar_consumers<NCT>();   // scratch is reused by the next piece
+    if (piece_idx == 0) {
+      first_unit = pc.unit;
+      first_tb = pc.tb;
+    }
+    if (!complete && pc.tb == 0) {
+      own_unit = pc.unit;
+      own_slot = slot_idx;
+    }
+    ++piece_idx;
+  }
+  if (ct == 0) P.rec[cta] = make_int4(first_unit, first_tb, own_unit, own_slot);
+}
+
+// ------------------------------------------------------------------------------------------
+// Split-combine: block c merges the unit that started in CTA c's span and ran past its end.
+// The pieces live in consecutive CTAs (slot 0 of each follower), merged in ascending token
+// order:  M = max m_c;  Lsum = sum l_c 2^(m_c - M);  out = bf16( sum acc_c 2^(m_c - M) / Lsum ).
+// ------------------------------------------------------------------------------------------
+template <int D, int NT>
+__global__ void __launch_bounds__(256)
+combine_kernel(const int4* __restrict__ rec, const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
+               int n_ctas, int Hq, int Hkv, int G) {
+  constexpr int HP = 8 * NT;
+  constexpr int SLOT_FLOATS = HP * (D + 2);
+  const int c = blockIdx.x;
+  const int4 r = rec[c];
+  const int unit = r.z;
+  if (unit < 0) return;
+  // followers: CTAs c+1.. whose first piece continues `unit`
+  __shared__ int n_follow;
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int cc = c + 1; cc < n_ctas; ++cc) {
+      const int4 rr = rec[cc];
+      if (rr.x != unit || rr.y <= 0) break;
+      ++n;
+    }
+    n_follow = n;
+  }
+  __syncthreads();
+  const int np = n_follow + 1;
+  const int s = unit / Hkv, g = unit - s * Hkv;
+  const float NEG_INF = __int_as_float(0xff800000);
+  for (int idx = threadIdx.x; idx < HP * (D / 4); idx += blockDim.x) {
+    const int h = idx / (D / 4);
+    const int dq = idx % (D / 4);
+    if (h >= G) continue;
+    float M = NEG_INF;
+    for (int p = 0; p < np; ++p) {
+      const float* part = partials + (static_cast<int64_t>(c + p) * 2 + (p == 0 ? r.w : 0)) * SLOT_FLOATS;
+      M = fmaxf(M, part[h]);
+    }
+    const float Mu = (M == NEG_INF) ? 0.f : M;
+    float Ls = 0.f;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = 0; p < np; ++p) {
+      const float* part = partials + (static_cast<int64_t>(c + p) * 2 + (p == 0 ? r.w : 0)) * SLOT_FLOATS;
+      const float f = fast_exp2(part[h] - Mu);
+      Ls += part[HP + h] * f;
+      const float4 v = *reinterpret_cast<const float4*>(part + 2 * HP + h * D + dq * 4);
+      a.x += v.x * f;
+      a.y += v.y * f;
+      a.z += v.z * f;
+      a.w += v.w * f;
+    }
+    const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
+    uint2 o;
+    o.x = pack_bf16x2(a.x * inv, a.y * inv);
+    o.y = pack_bf16x2(a.z * inv, a.w * inv);
+    *reinterpret_cast<uint2*>(out + (static_cast<int64_t>(s) * Hq + g * G + h) * D + dq * 4) = o;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Device twin of the host partitioner (one block).  prefix: [S+1] ints of scratch.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_ctas, int32_t* __restrict__ prefix,
+            int2* __restrict__ spans, WsHeader* hdr) {
+  __shared__ int warp_sums[32];
+  __shared__ int carry_s;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) {
+    carry_s = 0;
+    prefix[0] = 0;
+  }
+  __syncthreads();
+  for (int base = 0; base < S; base += 1024) {
+    const int s = base + tid;
+    int v = 0;
+    if (s < S) {
+      const int L = context_lens[s];
+      v = L > 0 ? ((L + TILE - 1) / TILE) * Hkv : 0;
+    }
+    int x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) warp_sums[wid] = x;
+    __syncthreads();
+    if (wid == 0) {
+      int w = warp_sums[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, w, o);
+        if (lane >= o) w += y;
+      }
+      warp_sums[lane] = w;
+    }
+    __syncthreads();
+    const int incl = x + (wid > 0 ? warp_sums[wid - 1] : 0) + carry_s;
+    if (s < S) prefix[s + 1] = incl;
+    __syncthreads();
+    if (tid == 1023) carry_s = incl;
+    __syncthreads();
+  }
+  const int total = carry_s;
+  const int tq = total / n_ctas, tr = total % n_ctas;
+  if (tid == 0) {
+    hdr->tiles_q = tq;
+    hdr->tiles_r = tr;
+  }
+  __threadfence_block();
+  __syncthreads();
+  for (int c = tid; c < n_ctas; c += 1024) {
+    const int start = c * tq + min(c, tr);
+    int2 sp = make_int2(S * Hkv, 0);
+    if (start < total) {
+      int lo = 0, hi = S;   // find s with prefix[s] <= start < prefix[s+1]
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (prefix[mid] <= start) lo = mid; else hi = mid;
+      }
+      const int L = context_lens[lo];
+      const int nt = (L + TILE - 1) / TILE;
+      const int off = start - prefix[lo];
+      sp = make_int2(lo * Hkv + off / nt, off % nt);
+    }
+    spans[c] = sp;
+  }
+}
+
+}  // namespace pdattn

@@ -1,0 +1,453 @@
+// Host side of libpdattn: argument checks, the host partitioner call, TMA tensor maps, launches.
+// No allocation, no synchronisation (except pdattn_check), no state beyond thread-locals.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/pdattn.h"
+#include "kernels.cuh"
+#include "partition.h"
+
+namespace {
+
+using namespace pdattn;
+
+thread_local char g_cuda_err[256] = "";
+thread_local int g_last_launches = 0;
+
+struct Binding {
+  bool set = false;
+  int max_blocks_per_seq = 0, num_blocks = 0;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  const int32_t* context_lens_host = nullptr;
+};
+thread_local Binding g_bind;
+
+pdattn_status cuda_fail(const char* what, cudaError_t e) {
+  snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", what, cudaGetErrorString(e));
+  return PDATTN_CUDA_ERROR;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- workspace layout ----------------------------------------------------------------------
+struct WsLayout {
+  size_t hdr, spans, rec, prefix, partials, total;
+};
+WsLayout ws_layout(int num_seqs, int G, int head_dim) {
+  const int NT = G > 8 ? 2 : 1;
+  const size_t slot_bytes = static_cast<size_t>(8 * NT) * (head_dim + 2) * 4;
+  WsLayout w;
+  w.hdr = 0;
+  w.spans = 256;
+  w.rec = w.spans + align_up(static_cast<size_t>(MAX_CTAS) * sizeof(int2), 256);
+  w.prefix = w.rec + align_up(static_cast<size_t>(MAX_CTAS) * sizeof(int4), 256);
+  w.partials = w.prefix + align_up(static_cast<size_t>(num_seqs + 1) * 4, 256);
+  w.total = w.partials + align_up(static_cast<size_t>(MAX_CTAS) * 2 * slot_bytes, 256);
+  return w;
+}
+
+pdattn_status check_shape(int num_seqs, int Hq, int Hkv, int d, int bs) {
+  if (num_seqs < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || bs <= 0) return PDATTN_INVALID_ARG;
+  if (Hq % Hkv != 0) return PDATTN_INVALID_ARG;
+  if (d != 64 && d != 128) return PDATTN_UNSUPPORTED;
+  if (bs != 16) return PDATTN_UNSUPPORTED;
+  if (Hq / Hkv > 16) return PDATTN_UNSUPPORTED;
+  return PDATTN_OK;
+}
+
+// ---- per-device facts ------------------------------------------------------------------------
+struct DevInfo {
+  bool ready = false;
+  int sm_count = 0;
+  bool attr_set[2][2] = {{false, false}, {false, false}};   // [D==128][NT==2]
+};
+constexpr int kMaxDevices = 64;
+DevInfo g_dev[kMaxDevices];
+std::mutex g_dev_mu;
+
+pdattn_status device_info(int* dev_out, DevInfo** info) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+  if (dev < 0 || dev >= kMaxDevices) return PDATTN_UNSUPPORTED;
+  DevInfo& di = g_dev[dev];
+  if (!di.ready) {
+    std::lock_guard<std::mutex> lk(g_dev_mu);
+    if (!di.ready) {
+      int sms = 0, major = 0;
+      e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute", e);
+      e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+      if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute", e);
+      if (major != 10) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "libpdattn is built for sm_100a only (device has major %d)", major);
+        return PDATTN_CUDA_ERROR;
+      }
+      di.sm_count = sms;
+      di.ready = true;
+    }
+  }
+  *dev_out = dev;
+  *info = &di;
+  return PDATTN_OK;
+}
+
+// ---- TMA tensor maps ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+pdattn_status get_encode() {
+  if (g_encode) return PDATTN_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return cuda_fail("cudaGetDriverEntryPoint", e);
+  if (!fn || qres != cudaDriverEntryPointSuccess) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled not available in this driver");
+    return PDATTN_CUDA_ERROR;
+  }
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return PDATTN_OK;
+}
+
+struct MapKey {
+  const void* ptr;
+  int d, bs, hkv, nb;
+  int64_t sb, sh, st;
+  bool operator==(const MapKey& o) const {
+    return ptr == o.ptr && d == o.d && bs == o.bs && hkv == o.hkv && nb == o.nb && sb == o.sb && sh == o.sh && st == o.st;
+  }
+};
+struct MapCacheEntry {
+  bool valid = false;
+  MapKey key;
+  CUtensorMap map;
+};
+thread_local MapCacheEntry g_maps[8];
+thread_local int g_map_next = 0;
+
+// View of a cache as a 4-D tensor (dim, slot, kv head, page); one box = one page-head's
+// 64-element column block: [64, block_size, 1, 1], 128-byte swizzle, zero fill out of bounds.
+pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t sb, int64_t sh, int64_t st,
+                       CUtensorMap* out) {
+  MapKey key{ptr, d, bs, hkv, nb, sb, sh, st};
+  for (auto& e : g_maps)
+    if (e.valid && e.key == key) {
+      *out = e.map;
+      return PDATTN_OK;
+    }
+  pdattn_status s = get_encode();
+  if (s != PDATTN_OK) return s;
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(hkv),
+                        static_cast<cuuint64_t>(nb > 0 ? nb : 1)};
+  cuuint64_t strides[3] = {static_cast<cuuint64_t>(st) * 2, static_cast<cuuint64_t>(sh) * 2,
+                           static_cast<cuuint64_t>(sb) * 2};
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(bs), 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUtensorMap m;
+  CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+    return PDATTN_CUDA_ERROR;
+  }
+  MapCacheEntry& e = g_maps[g_map_next];
+  g_map_next = (g_map_next + 1) % 8;
+  e.valid = true;
+  e.key = key;
+  e.map = m;
+  *out = m;
+  return PDATTN_OK;
+}
+
+// ---- launches ------------------------------------------------------------------------------------
+template <int D, int NT>
+pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, DevInfo* di,
+                     cudaStream_t stream) {
+  using C = Cfg<D, NT, 16>;
+  auto kern = decode_kernel<D, NT, 16>;
+  bool& done = di->attr_set[D == 128][NT == 2];
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
+    if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
+    done = true;
+  }
+  kern<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
+  combine_kernel<D, NT><<<grid, 256, 0, stream>>>(P.rec, P.partials, P.out, grid, P.Hq, P.Hkv, P.G);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("combine_kernel launch", e);
+  return PDATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+pdattn_status pdattn_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim, int block_size,
+                                    int max_context_len, size_t* device_bytes, size_t* pinned_host_bytes) {
+  (void)max_context_len;
+  if (!device_bytes) return PDATTN_INVALID_ARG;
+  pdattn_status s = check_shape(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size);
+  if (s != PDATTN_OK) return s;
+  *device_bytes = ws_layout(num_seqs, num_q_heads / num_kv_heads, head_dim).total;
+  if (pinned_host_bytes) *pinned_host_bytes = 0;
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_workspace_init(void* workspace, size_t workspace_bytes, pdattn_stream_t stream) {
+  if (!workspace || workspace_bytes < 256) return PDATTN_INVALID_ARG;
+  cudaError_t e = cudaMemsetAsync(workspace, 0, 256, reinterpret_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, int num_kv_heads, int n_ctas,
+                               int32_t* spans, int* tiles_q, int* tiles_r, int64_t* total_tiles) {
+  Plan plan;
+  if (!plan_spans(context_lens_host, num_seqs, num_kv_heads, n_ctas, spans, &plan)) return PDATTN_INVALID_ARG;
+  if (tiles_q) *tiles_q = plan.tiles_q;
+  if (tiles_r) *tiles_r = plan.tiles_r;
+  if (total_tiles) *total_tiles = plan.total_tiles;
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
+  g_last_launches = 0;
+  if (!a) return PDATTN_INVALID_ARG;
+  pdattn_status s = check_shape(a->num_seqs, a->num_q_heads, a->num_kv_heads, a->head_dim, a->block_size);
+  if (s != PDATTN_OK) return s;
+  if (a->num_seqs == 0) return PDATTN_OK;
+  if (!a->q || !a->k_cache || !a->v_cache || !a->out || !a->block_table || !a->context_lens || !a->workspace)
+    return PDATTN_INVALID_ARG;
+  if (a->max_blocks_per_seq <= 0 || a->num_blocks <= 0) return PDATTN_INVALID_ARG;
+  if (a->kv_block_stride <= 0 || a->kv_head_stride <= 0 || a->kv_token_stride < a->head_dim) return PDATTN_INVALID_ARG;
+  if ((a->kv_block_stride | a->kv_head_stride | a->kv_token_stride) % 8 != 0) return PDATTN_UNSUPPORTED;
+  auto mis = [](const void* p, size_t al) { return (reinterpret_cast<uintptr_t>(p) & (al - 1)) != 0; };
+  if (mis(a->q, 16) || mis(a->k_cache, 16) || mis(a->v_cache, 16) || mis(a->out, 16) || mis(a->workspace, 256))
+    return PDATTN_MISALIGNED;
+  const int G = a->num_q_heads / a->num_kv_heads;
+  const WsLayout wl = ws_layout(a->num_seqs, G, a->head_dim);
+  if (a->workspace_bytes < wl.total) return PDATTN_WORKSPACE_TOO_SMALL;
+
+  int dev = 0;
+  DevInfo* di = nullptr;
+  s = device_info(&dev, &di);
+  if (s != PDATTN_OK) return s;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+
+  static_assert(sizeof(DecodeParams) + 2 * sizeof(CUtensorMap) <= 4000, "kernel parameters");
+  DecodeParams P;
+  P.q = static_cast<const __nv_bfloat16*>(a->q);
+  P.out = static_cast<__nv_bfloat16*>(a->out);
+  P.block_table = a->block_table;
+  P.context_lens = a->context_lens;
+  P.hdr = reinterpret_cast<WsHeader*>(ws + wl.hdr);
+  P.spans_ws = reinterpret_cast<const int2*>(ws + wl.spans);
+  P.rec = reinterpret_cast<int4*>(ws + wl.rec);
+  P.partials = reinterpret_cast<float*>(ws + wl.partials);
+  P.S = a->num_seqs;
+  P.Hq = a->num_q_heads;
+  P.Hkv = a->num_kv_heads;
+  P.G = G;
+  P.MB = a->max_blocks_per_seq;
+  P.NB = a->num_blocks;
+  P.scale_log2 = a->scale * 1.4426950408889634f;
+  P.tiles_q = P.tiles_r = 0;
+  P.use_ws_plan = 0;
+
+  int n_ctas = di->sm_count;
+  if (n_ctas > MAX_PARAM_SPANS) n_ctas = MAX_PARAM_SPANS;
+  int grid = n_ctas;
+  if (a->context_lens_host) {
+    Plan plan;
+    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, reinterpret_cast<int32_t*>(P.spans),
+                    &plan))
+      return PDATTN_INVALID_ARG;
+    P.tiles_q = plan.tiles_q;
+    P.tiles_r = plan.tiles_r;
+    if (plan.total_tiles < n_ctas) grid = plan.total_tiles > 0 ? static_cast<int>(plan.total_tiles) : 1;
+  } else {
+    P.use_ws_plan = 1;
+    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas,
+                                         reinterpret_cast<int32_t*>(ws + wl.prefix),
+                                         reinterpret_cast<int2*>(ws + wl.spans), P.hdr);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
+    g_last_launches += 1;
+  }
+
+  CUtensorMap mk, mv;
+  s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+               a->kv_head_stride, a->kv_token_stride, &mk);
+  if (s != PDATTN_OK) return s;
+  s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+               a->kv_head_stride, a->kv_token_stride, &mv);
+  if (s != PDATTN_OK) return s;
+
+  const bool nt2 = G > 8;
+  if (a->head_dim == 128)
+    s = nt2 ? launch<128, 2>(mk, mv, P, grid, di, stream) : launch<128, 1>(mk, mv, P, grid, di, stream);
+  else
+    s = nt2 ? launch<64, 2>(mk, mv, P, grid, di, stream) : launch<64, 1>(mk, mv, P, grid, di, stream);
+  if (s == PDATTN_OK) g_last_launches += 2;
+  return s;
+}
+
+pdattn_status pdattn_bind(int max_blocks_per_seq, int num_blocks, void* workspace, size_t workspace_bytes,
+                          const int32_t* context_lens_host) {
+  if (max_blocks_per_seq <= 0 || num_blocks <= 0 || !workspace) return PDATTN_INVALID_ARG;
+  g_bind.set = true;
+  g_bind.max_blocks_per_seq = max_blocks_per_seq;
+  g_bind.num_blocks = num_blocks;
+  g_bind.workspace = workspace;
+  g_bind.workspace_bytes = workspace_bytes;
+  g_bind.context_lens_host = context_lens_host;
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_decode(const void* q, const void* k_cache, const void* v_cache, const int32_t* block_table,
+                            const int32_t* context_lens, int num_seqs, int num_q_heads, int num_kv_heads,
+                            int head_dim, int block_size, float scale, void* out, pdattn_stream_t stream) {
+  if (!g_bind.set) return PDATTN_NOT_BOUND;
+  pdattn_args a;
+  memset(&a, 0, sizeof a);
+  a.q = q;
+  a.k_cache = k_cache;
+  a.v_cache = v_cache;
+  a.out = out;
+  a.block_table = block_table;
+  a.context_lens = context_lens;
+  a.context_lens_host = g_bind.context_lens_host;
+  a.num_seqs = num_seqs;
+  a.num_q_heads = num_q_heads;
+  a.num_kv_heads = num_kv_heads;
+  a.head_dim = head_dim;
+  a.block_size = block_size;
+  a.max_blocks_per_seq = g_bind.max_blocks_per_seq;
+  a.num_blocks = g_bind.num_blocks;
+  a.kv_token_stride = head_dim;
+  a.kv_head_stride = static_cast<int64_t>(block_size) * head_dim;
+  a.kv_block_stride = static_cast<int64_t>(num_kv_heads) * block_size * head_dim;
+  a.scale = scale;
+  a.workspace = g_bind.workspace;
+  a.workspace_bytes = g_bind.workspace_bytes;
+  return pdattn_decode_ex(&a, stream);
+}
+
+pdattn_status pdattn_host_staging_size(int num_seqs, int num_q_heads, int head_dim, int max_blocks_per_seq,
+                                       size_t* device_bytes) {
+  if (num_seqs < 0 || num_q_heads <= 0 || head_dim <= 0 || max_blocks_per_seq <= 0 || !device_bytes)
+    return PDATTN_INVALID_ARG;
+  const size_t qb = align_up(static_cast<size_t>(num_seqs) * num_q_heads * head_dim * 2, 256);
+  const size_t tb = align_up(static_cast<size_t>(num_seqs) * max_blocks_per_seq * 4, 256);
+  const size_t lb = align_up(static_cast<size_t>(num_seqs) * 4, 256);
+  *device_bytes = 2 * qb + tb + lb;
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_host,
+                                 const int32_t* context_lens_host, void* out_host, const void* k_cache,
+                                 const void* v_cache, int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                                 int block_size, int max_blocks_per_seq, int num_blocks, float scale, void* staging,
+                                 size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                 pdattn_stream_t stream_) {
+  if (num_seqs == 0) return PDATTN_OK;
+  if (!q_host || !block_table_host || !context_lens_host || !out_host || !staging) return PDATTN_INVALID_ARG;
+  size_t need = 0;
+  pdattn_status s = pdattn_host_staging_size(num_seqs, num_q_heads, head_dim, max_blocks_per_seq, &need);
+  if (s != PDATTN_OK) return s;
+  if (staging_bytes < need) return PDATTN_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(staging) & 255) return PDATTN_MISALIGNED;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  const size_t q_bytes = static_cast<size_t>(num_seqs) * num_q_heads * head_dim * 2;
+  const size_t t_bytes = static_cast<size_t>(num_seqs) * max_blocks_per_seq * 4;
+  const size_t l_bytes = static_cast<size_t>(num_seqs) * 4;
+  uint8_t* st = static_cast<uint8_t*>(staging);
+  void* q_dev = st;
+  void* out_dev = st + align_up(q_bytes, 256);
+  void* bt_dev = st + 2 * align_up(q_bytes, 256);
+  void* len_dev = st + 2 * align_up(q_bytes, 256) + align_up(t_bytes, 256);
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+    return cuda_fail("cudaMemcpyAsync(q)", e);
+  if ((e = cudaMemcpyAsync(bt_dev, block_table_host, t_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+    return cuda_fail("cudaMemcpyAsync(block_table)", e);
+  if ((e = cudaMemcpyAsync(len_dev, context_lens_host, l_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+    return cuda_fail("cudaMemcpyAsync(context_lens)", e);
+  pdattn_args a;
+  memset(&a, 0, sizeof a);
+  a.q = q_dev;
+  a.k_cache = k_cache;
+  a.v_cache = v_cache;
+  a.out = out_dev;
+  a.block_table = static_cast<const int32_t*>(bt_dev);
+  a.context_lens = static_cast<const int32_t*>(len_dev);
+  a.context_lens_host = context_lens_host;
+  a.num_seqs = num_seqs;
+  a.num_q_heads = num_q_heads;
+  a.num_kv_heads = num_kv_heads;
+  a.head_dim = head_dim;
+  a.block_size = block_size;
+  a.max_blocks_per_seq = max_blocks_per_seq;
+  a.num_blocks = num_blocks;
+  a.kv_token_stride = head_dim;
+  a.kv_head_stride = static_cast<int64_t>(block_size) * head_dim;
+  a.kv_block_stride = static_cast<int64_t>(num_kv_heads) * block_size * head_dim;
+  a.scale = scale;
+  a.workspace = workspace;
+  a.workspace_bytes = workspace_bytes;
+  s = pdattn_decode_ex(&a, stream_);
+  if (s != PDATTN_OK) return s;
+  if ((e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+    return cuda_fail("cudaMemcpyAsync(out)", e);
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream_) {
+  if (!workspace) return PDATTN_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  int32_t word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, stream);
+  if (e != cudaSuccess) return cuda_fail("cudaMemcpyAsync", e);
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+  if (word == 0) return PDATTN_OK;
+  e = cudaMemsetAsync(workspace, 0, 4, stream);
+  if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+  if (word & ERR_TIMEOUT) return PDATTN_DEVICE_TIMEOUT;
+  return PDATTN_BAD_PAGE_INDEX;
+}
+
+int pdattn_last_launch_count(void) { return g_last_launches; }
+
+const char* pdattn_status_string(pdattn_status st) {
+  switch (st) {
+    case PDATTN_OK: return "ok";
+    case PDATTN_INVALID_ARG: return "invalid argument";
+    case PDATTN_UNSUPPORTED: return "unsupported shape or stride";
+    case PDATTN_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case PDATTN_MISALIGNED: return "misaligned pointer";
+    case PDATTN_NOT_BOUND: return "pdattn_bind was not called on this thread";
+    case PDATTN_CUDA_ERROR: return "CUDA error";
+    case PDATTN_BAD_PAGE_INDEX: return "block_table entry out of range";
+    case PDATTN_DEVICE_TIMEOUT: return "bounded wait expired inside a kernel";
+    default: return "unknown status";
+  }
+}
+
+const char* pdattn_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

@@ -1,0 +1,217 @@
+"""ctypes binding of libpdattn (include/pdattn.h): argument marshalling only.
+
+Every step of the decode path runs in the library's CUDA kernels.  torch is used for device
+memory and streams.  There is no CPU fallback: if the library has not been built, importing
+`lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libpdattn.so")
+
+OK = 0
+INVALID_ARG = -1
+UNSUPPORTED = -2
+WORKSPACE_TOO_SMALL = -3
+MISALIGNED = -4
+NOT_BOUND = -5
+CUDA_ERROR = -6
+BAD_PAGE_INDEX = -7
+DEVICE_TIMEOUT = -8
+
+EXPORTS = [
+    "pdattn_workspace_size", "pdattn_workspace_init", "pdattn_decode_ex", "pdattn_bind", "pdattn_decode",
+    "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
+    "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error",
+]
+
+
+class PdattnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        L = lib()
+        msg = L.pdattn_status_string(status).decode()
+        if status == CUDA_ERROR:
+            msg += ": " + L.pdattn_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({status})")
+
+
+class Args(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+        ("out", ctypes.c_void_p), ("block_table", ctypes.c_void_p), ("context_lens", ctypes.c_void_p),
+        ("context_lens_host", ctypes.c_void_p),
+        ("num_seqs", ctypes.c_int), ("num_q_heads", ctypes.c_int), ("num_kv_heads", ctypes.c_int),
+        ("head_dim", ctypes.c_int), ("block_size", ctypes.c_int),
+        ("max_blocks_per_seq", ctypes.c_int), ("num_blocks", ctypes.c_int),
+        ("kv_block_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64), ("kv_token_stride", ctypes.c_int64),
+        ("scale", ctypes.c_float),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it has not been built (see build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2607_09207_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+        L.pdattn_workspace_size.argtypes = [i32] * 6 + [ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.pdattn_workspace_init.argtypes = [vp, sz, vp]
+        L.pdattn_decode_ex.argtypes = [ctypes.POINTER(Args), vp]
+        L.pdattn_bind.argtypes = [i32, i32, vp, sz, vp]
+        L.pdattn_decode.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, vp, vp]
+        L.pdattn_host_staging_size.argtypes = [i32, i32, i32, i32, ctypes.POINTER(sz)]
+        L.pdattn_decode_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32,
+                                         vp, sz, vp, sz, vp]
+        L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                       ctypes.POINTER(i64)]
+        L.pdattn_check.argtypes = [vp, vp]
+        L.pdattn_last_launch_count.argtypes = []
+        L.pdattn_status_string.argtypes = [i32]
+        L.pdattn_status_string.restype = ctypes.c_char_p
+        L.pdattn_last_cuda_error.argtypes = []
+        L.pdattn_last_cuda_error.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size=16, max_context_len=0) -> int:
+    dev, pin = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    st = lib().pdattn_workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size, max_context_len,
+                                     ctypes.byref(dev), ctypes.byref(pin))
+    if st != OK:
+        raise PdattnError(st, "pdattn_workspace_size")
+    return dev.value
+
+
+def alloc_workspace(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size=16, device="cuda", stream=None):
+    """torch-owned workspace, error word cleared."""
+    n = workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    st = lib().pdattn_workspace_init(ws.data_ptr(), n, _stream_ptr(stream))
+    if st != OK:
+        raise PdattnError(st, "pdattn_workspace_init")
+    return ws
+
+
+def decode_ex(q, k_cache, v_cache, block_table, context_lens, scale, out, workspace,
+              context_lens_host: Optional[np.ndarray] = None, num_blocks: Optional[int] = None,
+              stream=None, check: bool = True) -> int:
+    """pdattn_decode_ex.  k_cache / v_cache: bf16 tensors indexed [page, kv_head, slot, dim] with any
+    strides whose last dimension is contiguous.  Returns the status (raises unless check=False)."""
+    S, Hq, d = q.shape
+    NB, Hkv, bs, _ = k_cache.shape
+    a = Args()
+    a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr()
+    a.block_table, a.context_lens = block_table.data_ptr(), context_lens.data_ptr()
+    keep = None
+    if context_lens_host is not None:
+        keep = np.ascontiguousarray(context_lens_host, dtype=np.int32)
+        a.context_lens_host = keep.ctypes.data
+    else:
+        a.context_lens_host = None
+    a.num_seqs, a.num_q_heads, a.num_kv_heads, a.head_dim, a.block_size = S, Hq, Hkv, d, bs
+    a.max_blocks_per_seq = block_table.shape[1] if block_table.dim() == 2 else 0
+    a.num_blocks = NB if num_blocks is None else num_blocks
+    a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
+    a.scale = float(scale)
+    a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    st = lib().pdattn_decode_ex(ctypes.byref(a), _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_ex")
+    return st
+
+
+def bind(max_blocks_per_seq, num_blocks, workspace, context_lens_host: Optional[np.ndarray] = None):
+    """pdattn_bind.  The caller keeps `workspace` and `context_lens_host` alive while bound."""
+    hp = context_lens_host.ctypes.data if context_lens_host is not None else None
+    st = lib().pdattn_bind(max_blocks_per_seq, num_blocks, workspace.data_ptr(), workspace.numel(), hp)
+    if st != OK:
+        raise PdattnError(st, "pdattn_bind")
+
+
+def decode(q, k_cache, v_cache, block_table, context_lens, num_seqs, num_q_heads, num_kv_heads, head_dim,
+           block_size, scale, out, stream=None, check: bool = True) -> int:
+    """pdattn_decode (13-argument form, dense [NB, Hkv, bs, d] caches, uses the thread's binding)."""
+    st = lib().pdattn_decode(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), block_table.data_ptr(),
+                             context_lens.data_ptr(), num_seqs, num_q_heads, num_kv_heads, head_dim, block_size,
+                             float(scale), out.data_ptr(), _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode")
+    return st
+
+
+def host_staging_size(num_seqs, num_q_heads, head_dim, max_blocks_per_seq) -> int:
+    n = ctypes.c_size_t(0)
+    st = lib().pdattn_host_staging_size(num_seqs, num_q_heads, head_dim, max_blocks_per_seq, ctypes.byref(n))
+    if st != OK:
+        raise PdattnError(st, "pdattn_host_staging_size")
+    return n.value
+
+
+def decode_host(q_host, block_table_host, context_lens_host, out_host, k_cache, v_cache, scale, staging, workspace,
+                stream=None, check: bool = True) -> int:
+    """pdattn_decode_host: q / block_table / context_lens / out are HOST tensors (pinned), caches on device."""
+    S, Hq, d = q_host.shape
+    NB, Hkv, bs, _ = k_cache.shape
+    st = lib().pdattn_decode_host(q_host.data_ptr(), block_table_host.data_ptr(), context_lens_host.data_ptr(),
+                                  out_host.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), S, Hq, Hkv, d, bs,
+                                  block_table_host.shape[1], NB, float(scale), staging.data_ptr(), staging.numel(),
+                                  workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_host")
+    return st
+
+
+def plan_host(context_lens_host, num_kv_heads, n_ctas):
+    """pdattn_plan_host -> (spans[n_ctas,2], tiles_q, tiles_r, total_tiles).  Needs no GPU."""
+    lens = np.ascontiguousarray(context_lens_host, dtype=np.int32)
+    spans = np.zeros((n_ctas, 2), dtype=np.int32)
+    tq, tr, tot = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int64(0)
+    st = lib().pdattn_plan_host(lens.ctypes.data if lens.size else None, lens.size, num_kv_heads, n_ctas,
+                                spans.ctypes.data, ctypes.byref(tq), ctypes.byref(tr), ctypes.byref(tot))
+    if st != OK:
+        raise PdattnError(st, "pdattn_plan_host")
+    return spans, tq.value, tr.value, tot.value
+
+
+def check(workspace, stream=None) -> int:
+    """pdattn_check: synchronises, returns OK / BAD_PAGE_INDEX / DEVICE_TIMEOUT and clears the word."""
+    return lib().pdattn_check(workspace.data_ptr(), _stream_ptr(stream))
+
+
+def last_launch_count() -> int:
+    return lib().pdattn_last_launch_count()
+
+
+def decode_workload(w, out=None, workspace=None, use_host_lens: bool = True, stream=None):
+    """Convenience for tests and the benchmark: run one step on a workloads.Workload living on the GPU."""
+    if out is None:
+        out = torch.empty_like(w.q)
+    if workspace is None:
+        workspace = alloc_workspace(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size,
+                                    device=w.q.device)
+    decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, workspace,
+              context_lens_host=w.context_lens_host if use_host_lens else None, stream=stream)
+    return out

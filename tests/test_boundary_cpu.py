@@ -1,0 +1,151 @@
+"""C-ABI boundary and host partitioner, without a GPU: the library loads, exports every symbol the
+header declares, validates arguments before touching CUDA, and the partitioner covers every tile once."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2607_09207_b200 import build as pd_build
+from paper_2607_09207_b200 import pdattn
+from paper_2607_09207_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    pd_build.build()
+
+
+def declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if f.endswith(".h"):
+            text = open(os.path.join(inc, f)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names.update(re.findall(r"\b(pdattn_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_library_exports_every_declared_symbol():
+    L = pdattn.lib()
+    syms = declared_symbols()
+    assert len(syms) >= 12
+    for name in syms:
+        assert hasattr(L, name), name
+    assert set(pdattn.EXPORTS) <= set(syms)
+
+
+def test_status_strings():
+    L = pdattn.lib()
+    assert L.pdattn_status_string(0) == b"ok"
+    seen = {L.pdattn_status_string(-i) for i in range(0, 9)}
+    assert len(seen) == 9
+
+
+def test_workspace_size_and_shape_checks():
+    n = pdattn.workspace_size(256, 28, 4, 128)
+    assert 0 < n < 64 << 20 and n % 256 == 0
+    assert pdattn.workspace_size(256, 64, 4, 128) > n          # G = 16 needs wider partial slots
+    for bad, code in [((4, 28, 4, 96, 16), pdattn.UNSUPPORTED), ((4, 28, 4, 128, 8), pdattn.UNSUPPORTED),
+                      ((4, 30, 4, 128, 16), pdattn.INVALID_ARG), ((4, 68, 4, 128, 16), pdattn.UNSUPPORTED),
+                      ((-1, 28, 4, 128, 16), pdattn.INVALID_ARG)]:
+        with pytest.raises(pdattn.PdattnError) as e:
+            pdattn.workspace_size(*bad)
+        assert e.value.status == code
+
+
+def test_decode_rejects_bad_arguments_before_any_cuda_call():
+    L = pdattn.lib()
+    assert L.pdattn_decode_ex(None, None) == pdattn.INVALID_ARG
+    a = pdattn.Args()
+    a.num_seqs, a.num_q_heads, a.num_kv_heads, a.head_dim, a.block_size = 0, 4, 1, 64, 16
+    assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.OK          # empty batch: no-op
+    a.num_seqs = 2
+    assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.INVALID_ARG  # null pointers
+    for f in ("q", "k_cache", "v_cache", "out", "block_table", "context_lens"):
+        setattr(a, f, 0x1000)
+    a.workspace = 0x1000
+    a.max_blocks_per_seq, a.num_blocks = 4, 8
+    a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = 1024, 1024, 64
+    a.workspace_bytes = 16
+    assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.WORKSPACE_TOO_SMALL
+    a.workspace_bytes = 1 << 30
+    a.q = 0x1004
+    assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.MISALIGNED
+    a.q = 0x1000
+    a.kv_token_stride = 68
+    assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.UNSUPPORTED
+    a.head_dim = 80
+    assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.UNSUPPORTED
+
+
+def test_short_form_needs_a_binding():
+    import threading
+    res = []
+    t = threading.Thread(target=lambda: res.append(
+        pdattn.lib().pdattn_decode(None, None, None, None, None, 1, 4, 1, 64, 16, 1.0, None, None)))
+    t.start()
+    t.join()
+    assert res == [pdattn.NOT_BOUND]
+
+
+def walk_spans(lens, Hkv, n_ctas):
+    """Re-walk the plan the way a CTA does and return the set of (unit, tile) each CTA covers."""
+    spans, tq, tr, total = pdattn.plan_host(lens, Hkv, n_ctas)
+    nt = [(int(L) + 63) // 64 if L > 0 else 0 for L in lens]
+    cover = []
+    for c in range(n_ctas):
+        unit, tb = int(spans[c, 0]), int(spans[c, 1])
+        rem = tq + (1 if c < tr else 0)
+        mine = []
+        while rem > 0 and unit < len(lens) * Hkv:
+            n = nt[unit // Hkv]
+            if tb >= n:
+                unit, tb = unit + 1, 0
+                continue
+            te = min(n, tb + rem)
+            mine += [(unit, t) for t in range(tb, te)]
+            rem -= te - tb
+            unit, tb = unit + 1, 0
+        assert rem == 0
+        cover.append(mine)
+    return cover, total
+
+
+@pytest.mark.parametrize("case", ["cfg1", "cfg2", "cfg5", "zeros", "short", "one"])
+@pytest.mark.parametrize("n_ctas", [1, 7, 148, 320])
+def test_partitioner_covers_every_tile_exactly_once(case, n_ctas):
+    lens, Hkv = {
+        "cfg1": (W.config_lengths(1), 1), "cfg2": (W.config_lengths(2), 4), "cfg5": (W.config_lengths(5), 4),
+        "zeros": (np.array([0, 5, 0, 0, 300, 0]), 2), "short": (np.arange(1, 40), 3), "one": (np.array([1]), 8),
+    }[case]
+    cover, total = walk_spans(lens, Hkv, n_ctas)
+    want = [(s * Hkv + g, t) for s, L in enumerate(lens) for g in range(Hkv) for t in range((int(L) + 63) // 64)]
+    flat = [x for mine in cover for x in mine]
+    assert total == len(want)
+    assert flat == want                      # contiguous, ordered, nothing twice, nothing missing
+    sizes = [len(m) for m in cover]
+    assert max(sizes) - min(sizes) <= 1      # balanced to within one tile
+
+
+def test_partitioner_spreads_the_straggler_phase_over_all_sms():
+    """8 sequences x 4 KV heads = 32 units must still occupy all 148 CTAs."""
+    lens = W.config_lengths(5)
+    cover, total = walk_spans(lens, 4, 148)
+    assert all(len(m) > 0 for m in cover)
+    splits = {}
+    for c, mine in enumerate(cover):
+        for u, _ in mine:
+            splits.setdefault(u, set()).add(c)
+    assert min(len(v) for v in splits.values()) >= 3
+
+
+def test_partitioner_depends_on_lengths_only():
+    lens = W.config_lengths(2, num_seqs=32)
+    a = pdattn.plan_host(lens, 4, 148)
+    b = pdattn.plan_host(lens.copy(), 4, 148)
+    assert np.array_equal(a[0], b[0]) and a[1:] == b[1:]
