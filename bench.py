@@ -53,6 +53,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cfg", type=int, default=2, help="BASELINE.json config index + 1 (default: the metric's config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--num-seqs", type=int, default=None,
+                    help="shrink the batch (profiling captures only; not the metric's workload)")
     return ap.parse_args()
 
 
@@ -201,7 +203,7 @@ def main():
     K, Wm = args.steps, max(3, args.warmup)
     # ---- inputs: this rank's batch, in two physically distinct copies (pools, tables, q) so that
     # consecutive steps never find the previous step's pages in L2
-    base = W.make_config(args.cfg, device=dev)
+    base = W.make_config(args.cfg, device=dev, num_seqs=args.num_seqs)
     if world > 1:
         # every rank gets its own lengths and values: same shape, different seed stream
         lens = W.config_lengths(args.cfg)
@@ -313,7 +315,8 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": CFG_DESC[args.cfg], "num_seqs_per_gpu": S,
+            "config": {"workload": CFG_DESC[args.cfg] + (f" [REDUCED to {S} seqs]" if args.num_seqs else ""),
+                       "num_seqs_per_gpu": S,
                        "unique_kv_bytes_per_step": uniq, "logical_kv_bytes_per_step": logical,
                        "l2": f"inputs ({uniq / 1e9:.2f} GB) larger than L2 and steps rotate over {len(copies)} "
                              "physically distinct copies of pools/tables",

@@ -152,6 +152,25 @@ pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, i
  */
 pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream);
 
+/*
+ * Measurement aid (roofline accounting of the split-KV kernel, Appendix A.1.2's history-token
+ * term being the bytes it moves): while two CUDA events are registered on this thread, every
+ * decode call records `start` just before and `stop` just after the split-KV kernel on its
+ * stream.  start / stop are cudaEvent_t handles owned by the caller; pass NULLs to stop.
+ */
+pdattn_status pdattn_profile_events(void* start_event, void* stop_event);
+
+/*
+ * Bandwidth ceilings for the same roofline accounting (no paper counterpart beyond the bytes of
+ * Appendix A.1.2's per-token footprint): measurement aids, they compute nothing.
+ *   pdattn_gather_probe      : the decode step's exact memory access stream (same partition, page
+ *                              lookups and TMA ring) with the math and all output removed.
+ *   pdattn_stream_read_probe : a plain sequential read of `bytes` bytes (16-byte aligned DEVICE
+ *                              src); sink is 4 bytes of DEVICE scratch.
+ */
+pdattn_status pdattn_gather_probe(const pdattn_args* args, pdattn_stream_t stream);
+pdattn_status pdattn_stream_read_probe(const void* src, size_t bytes, void* sink, pdattn_stream_t stream);
+
 /* Number of kernels the last pdattn_decode_ex on this thread launched (2 or 3). */
 int pdattn_last_launch_count(void);
 

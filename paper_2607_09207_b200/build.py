@@ -28,19 +28,22 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, defines=(), out: str = None) -> str:
+    """defines / out build a tuning variant (e.g. defines=["PDATTN_NCW=4"]) to another path."""
+    target = out or LIB
+    if out is None and not force and not needs_build():
         return LIB
-    os.makedirs(LIB_DIR, exist_ok=True)
-    tmp = LIB + ".tmp%d" % os.getpid()
+    os.makedirs(os.path.dirname(target), exist_ok=True)
+    tmp = target + ".tmp%d" % os.getpid()
     cmd = [_nvcc(), "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += ["-D" + d for d in defines]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, target)
+    return target
 
 
 if __name__ == "__main__":

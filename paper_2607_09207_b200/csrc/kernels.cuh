@@ -1,9 +1,9 @@
 // Device code of libpdattn (sm_100a only).
 //
 //   decode_kernel  : split-KV flash decoding.  One persistent CTA per SM walks a contiguous span
-//                    of the batch's 64-token KV tiles.  A producer warp streams K/V pages from HBM
-//                    into a shared-memory ring with TMA tensor copies (128-byte swizzle) signalled
-//                    through mbarriers; the consumer warps each take whole tiles, compute
+//                    of the batch's 64-token KV tiles.  Producer warps stream K/V pages from HBM
+//                    into a shared-memory ring with TMA tensor copies (128-byte swizzle, one copy
+//                    per page-head) signalled through mbarriers; the consumer warps each take whole tiles, compute
 //                    S^T = K.Q^T and O^T += V^T.P^T with bf16 tensor-core MMAs (tokens on M, the
 //                    packed GQA query heads of the KV head on N) and keep the online-softmax
 //                    running max / sum in fp32.
@@ -19,12 +19,21 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "partition.h"
+
+#ifndef PDATTN_NCW
+#define PDATTN_NCW 6
+#endif
+#ifndef PDATTN_NPW
+#define PDATTN_NPW 3              // producer warps (tile i is issued by producer i mod NPW)
+#endif
+
 namespace pdattn {
 
-constexpr int TILE = 64;                         // tokens per pipeline stage
+constexpr int TILE = kTileTokens;                // tokens per pipeline stage
 constexpr int MAX_PARAM_SPANS = 320;             // spans that travel in kernel parameters
 constexpr int MAX_CTAS = 592;                    // upper bound used for workspace sizing
-constexpr int MAX_STAGES = 12;
+constexpr int MAX_STAGES = 24;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2 };
@@ -50,6 +59,7 @@ struct DecodeParams {
   float scale_log2;         // scale * log2(e)
   int tiles_q, tiles_r;
   int use_ws_plan;
+  int box5d;                // 1: the tensor maps are 5-D and one TMA op brings a whole page-head
   int2 spans[MAX_PARAM_SPANS];
 };
 
@@ -109,6 +119,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
       : "memory");
 }
+// 5-D variant: (dim-in-half, slot, half, kv head, page)
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, int c4,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+      : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -163,18 +181,31 @@ struct Cfg {
   // NSTAGES.  NSTAGES must be a multiple of NCW: then the tile that used a slot one ring turn
   // earlier belonged to the same warp, so a warp can never wait on a slot's next mbarrier phase
   // while the previous one is still pending (a parity wait cannot tell those apart).
-  static constexpr int NCW = (D == 128 && NT == 2) ? 5 : 6;            // consumer warps
-  static constexpr int NSTAGES = (D == 128) ? NCW : 2 * NCW;
-  static constexpr int NCT = NCW * 32;                                 // consumer threads
-  static constexpr int NTHREADS = NCT + 32;                            // + 1 producer warp
   static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the scratch stores conflict-free
+  static constexpr int SMEM_MAX = 232448;              // 227 KB
+  static constexpr int CTRL_BYTES = 512;
+  static constexpr int fixed_bytes(int ncw) { return 1024 + ncw * HP * ACC_STRIDE * 4 + ncw * HP * 2 * 4 + CTRL_BYTES; }
+  static constexpr int stages_for(int ncw) {
+    int fit = (SMEM_MAX - fixed_bytes(ncw)) / STAGE_BYTES;
+    if (fit > MAX_STAGES) fit = MAX_STAGES;
+    return fit / ncw * ncw;
+  }
+  static constexpr int pick_ncw() {   // the requested warp count, lowered until a ring of >= NCW stages fits
+    int ncw = PDATTN_NCW;
+    while (ncw > 1 && stages_for(ncw) < ncw) --ncw;
+    return ncw;
+  }
+  static constexpr int NCW = pick_ncw();                               // consumer warps
+  static constexpr int NSTAGES = stages_for(NCW);
+  static constexpr int NCT = NCW * 32;                                 // consumer threads
+  static constexpr int NPW = (NSTAGES % PDATTN_NPW == 0) ? PDATTN_NPW : 1;   // producer warps
+  static constexpr int NTHREADS = NCT + 32 * NPW;
   static constexpr int SCRATCH_BYTES = NCW * HP * ACC_STRIDE * 4;
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
-  static constexpr int CTRL_BYTES = 256;
-  static constexpr int SMEM_MAX = 232448;              // 227 KB
   static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + SCRATCH_BYTES + ML_BYTES + CTRL_BYTES;
   static constexpr int SLOT_FLOATS = HP * (D + 2);     // one partial: m[HP], l[HP], acc[HP][D]
-  static_assert(NSTAGES % NCW == 0 && NSTAGES <= MAX_STAGES, "ring/warp mapping");
+  static_assert(NSTAGES >= NCW && NSTAGES % NCW == 0 && NSTAGES <= MAX_STAGES, "ring/warp mapping");
+  static_assert(NSTAGES % NPW == 0, "a slot must always be refilled by the same producer warp");
   static_assert(DYN_BYTES <= SMEM_MAX, "shared memory");
   static_assert(TILE % BS == 0 && BS % 16 == 0, "block size");
 };
@@ -185,7 +216,7 @@ struct Ctrl {                 // lives in the CTRL_BYTES area
   uint32_t meta[MAX_STAGES];  // per stage: bit j set = page j of the tile had a bad id
   uint32_t abort;
 };
-static_assert(sizeof(Ctrl) <= 256, "control block");
+static_assert(sizeof(Ctrl) <= 512, "control block");
 
 // ------------------------------------------------------------------------------------------
 // The walk over a span: pieces = (unit, tile range) in order.  Every warp runs the same walk.
@@ -321,15 +352,20 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
       m[nt][e] = m_new;
       l[nt][e] *= alpha[nt][e];
     }
+  bool moved = false;
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt)
+  for (int nt = 0; nt < NT; ++nt) moved |= (alpha[nt][0] != 1.f) | (alpha[nt][1] != 1.f);
+  if (__any_sync(0xffffffffu, moved)) {   // the running max rarely moves after the first tiles
 #pragma unroll
-    for (int jm = 0; jm < D / 16; ++jm) {
-      acc[nt][jm][0] *= alpha[nt][0];
-      acc[nt][jm][1] *= alpha[nt][1];
-      acc[nt][jm][2] *= alpha[nt][0];
-      acc[nt][jm][3] *= alpha[nt][1];
-    }
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int jm = 0; jm < D / 16; ++jm) {
+        acc[nt][jm][0] *= alpha[nt][0];
+        acc[nt][jm][1] *= alpha[nt][1];
+        acc[nt][jm][2] *= alpha[nt][0];
+        acc[nt][jm][3] *= alpha[nt][1];
+      }
+  }
 
   // ---- P = exp2(S - m), transposed into the B-operand layout.  bf16 keeps 8 bits of P, which is
   // not enough when a few tokens carry the weight (short contexts, peaked softmax), so P goes
@@ -380,7 +416,9 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
 // ------------------------------------------------------------------------------------------
 // The decode kernel
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS>
+// PROBE = true builds the page-gather ceiling: identical walk, page-id lookups and TMA ring, but
+// the consumers release every tile untouched and nothing is written.
+template <int D, int NT, int BS, bool PROBE = false>
 __global__ void __launch_bounds__(Cfg<D, NT, BS>::NTHREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
               const __grid_constant__ DecodeParams P) {
@@ -435,8 +473,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   Piece pc;
   int it = 0;   // tile counter within this CTA: tile `it` uses ring slot it % NST
 
-  if (warp == NCW) {
-    // ================= producer warp =================
+  if (warp >= NCW) {
+    // ================= producer warp(s) =================
+    const int pw = warp - NCW;
     constexpr int IDS_PER_BATCH = 32;
     constexpr int TILES_PER_BATCH = IDS_PER_BATCH / C::PAGES;
     bool any_bad = false;
@@ -455,6 +494,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           const int nb = pbase + rel * C::PAGES + IDS_PER_BATCH;
           ids_nxt = (nb + lane < npages) ? __ldg(row + nb + lane) : 0;
         }
+        if (C::NPW > 1 && it % C::NPW != pw) continue;
         const int slot = it % NST;
         const uint32_t phase = (it / NST) & 1;
         if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) {
@@ -477,8 +517,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           const bool isV = lane >= C::PAGES;
           const uint32_t dst = ring + slot * C::STAGE_BYTES + (isV ? C::KV_BYTES : 0) + j * C::PAGE_BYTES;
           const CUtensorMap* tm = isV ? &tmV : &tmK;
+          if (P.box5d) {
+            tma_load_5d(dst, tm, 0, 0, 0, pc.g, id, bar);
+          } else {
 #pragma unroll
-          for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, tm, h * 64, 0, pc.g, id, bar);
+            for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, tm, h * 64, 0, pc.g, id, bar);
+          }
         }
         any_bad |= (badmask != 0);
       }
@@ -551,7 +595,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       const uint32_t sV = sK + C::KV_BYTES;
       const uint32_t badmask = ctrl->meta[slot];
       const int n_valid = min(TILE, pc.L - t * TILE);
-      if (n_valid == TILE) {
+      if (PROBE) {
+        // ceiling probe: no math
+      } else if (n_valid == TILE) {
         compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane);
       } else {
         compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_valid, badmask, lane);
@@ -561,6 +607,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
     }
 
+    const bool complete = (pc.tb == 0 && pc.te == pc.nt);
+    const int slot_idx = piece_idx == 0 ? 0 : 1;
+    if constexpr (!PROBE) {
     // ---- merge the NCW warp states of this piece
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
@@ -594,8 +643,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
     }
     bar_consumers<NCT>();
-    const bool complete = (pc.tb == 0 && pc.te == pc.nt);
-    const int slot_idx = piece_idx == 0 ? 0 : 1;
     float* part = P.partials + (static_cast<int64_t>(cta) * 2 + slot_idx) * C::SLOT_FLOATS;
     for (int idx = ct; idx < C::HP * (D / 4); idx += NCT) {
       const int h = idx / (D / 4);
@@ -633,6 +680,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
     }
     bar_consumers<NCT>();   // scratch is reused by the next piece
+    }   // !PROBE
     if (piece_idx == 0) {
       first_unit = pc.unit;
       first_tb = pc.tb;
@@ -643,7 +691,26 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
     ++piece_idx;
   }
-  if (ct == 0) P.rec[cta] = make_int4(first_unit, first_tb, own_unit, own_slot);
+  if (ct == 0 && !PROBE) P.rec[cta] = make_int4(first_unit, first_tb, own_unit, own_slot);
+}
+
+// Read-only streaming ceiling: every thread block sums a contiguous slice with 16-byte loads.
+__global__ void __launch_bounds__(512)
+stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __restrict__ sink) {
+  uint32_t acc = 0;
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+#pragma unroll 1
+  for (; i + 3 * stride < n_vec; i += 4 * stride) {
+    const uint4 a = __ldcs(src + i), b = __ldcs(src + i + stride), c = __ldcs(src + i + 2 * stride),
+                d = __ldcs(src + i + 3 * stride);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ d.x ^ d.y ^ d.z ^ d.w;
+  }
+  for (; i < n_vec; i += stride) {
+    const uint4 a = __ldcs(src + i);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w;
+  }
+  if (acc == 0x9e3779b9u) *sink = acc;   // practically never: keeps the loads alive
 }
 
 // ------------------------------------------------------------------------------------------

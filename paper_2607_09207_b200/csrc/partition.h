@@ -1,4 +1,4 @@
-// Host partitioner: flattens the batch into a stream of 64-token tiles, unit-major
+// Host partitioner: flattens the batch into a stream of fixed-size token tiles, unit-major
 // (unit = sequence * Hkv + kv_head), and cuts the stream into n_ctas contiguous spans whose
 // lengths differ by at most one tile.  A long sequence is thereby split over as many CTAs as
 // its share of the bytes warrants, and a CTA that finishes a short sequence carries on with
@@ -8,7 +8,10 @@
 
 namespace pdattn {
 
-constexpr int kTileTokens = 64;
+#ifndef PDATTN_TILE_TOKENS
+#define PDATTN_TILE_TOKENS 64     // tokens per tile = per pipeline stage of the decode kernel
+#endif
+constexpr int kTileTokens = PDATTN_TILE_TOKENS;
 
 struct Plan {
   int64_t total_tiles;

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -17,6 +18,8 @@ using namespace pdattn;
 
 thread_local char g_cuda_err[256] = "";
 thread_local int g_last_launches = 0;
+thread_local cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
+thread_local bool g_probe_mode = false;   // set only inside pdattn_gather_probe
 
 struct Binding {
   bool set = false;
@@ -119,10 +122,11 @@ pdattn_status get_encode() {
 
 struct MapKey {
   const void* ptr;
-  int d, bs, hkv, nb;
+  int d, bs, hkv, nb, rank;
   int64_t sb, sh, st;
   bool operator==(const MapKey& o) const {
-    return ptr == o.ptr && d == o.d && bs == o.bs && hkv == o.hkv && nb == o.nb && sb == o.sb && sh == o.sh && st == o.st;
+    return ptr == o.ptr && d == o.d && bs == o.bs && hkv == o.hkv && nb == o.nb && rank == o.rank && sb == o.sb &&
+           sh == o.sh && st == o.st;
   }
 };
 struct MapCacheEntry {
@@ -133,11 +137,15 @@ struct MapCacheEntry {
 thread_local MapCacheEntry g_maps[8];
 thread_local int g_map_next = 0;
 
-// View of a cache as a 4-D tensor (dim, slot, kv head, page); one box = one page-head's
-// 64-element column block: [64, block_size, 1, 1], 128-byte swizzle, zero fill out of bounds.
-pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t sb, int64_t sh, int64_t st,
+// View of a cache as a tensor for TMA, 128-byte swizzle, zero fill out of bounds.
+//   rank 4: (dim, slot, kv head, page); one box = one 64-element column block of a page-head,
+//           [64, block_size, 1, 1]: head_dim / 64 copies per page-head.
+//   rank 5: (dim within column block, slot, column block, kv head, page); one box = a whole
+//           page-head [64, block_size, 2, 1, 1], landing in shared memory column block by column
+//           block exactly like two rank-4 boxes.  head_dim 128 only.
+pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t sb, int64_t sh, int64_t st, int rank,
                        CUtensorMap* out) {
-  MapKey key{ptr, d, bs, hkv, nb, sb, sh, st};
+  MapKey key{ptr, d, bs, hkv, nb, rank, sb, sh, st};
   for (auto& e : g_maps)
     if (e.valid && e.key == key) {
       *out = e.map;
@@ -145,18 +153,32 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
     }
   pdattn_status s = get_encode();
   if (s != PDATTN_OK) return s;
-  cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(hkv),
-                        static_cast<cuuint64_t>(nb > 0 ? nb : 1)};
-  cuuint64_t strides[3] = {static_cast<cuuint64_t>(st) * 2, static_cast<cuuint64_t>(sh) * 2,
-                           static_cast<cuuint64_t>(sb) * 2};
-  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(bs), 1, 1};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
+  const cuuint64_t nbu = static_cast<cuuint64_t>(nb > 0 ? nb : 1);
   CUtensorMap m;
-  CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r;
+  if (rank == 5) {
+    cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(d / 64),
+                          static_cast<cuuint64_t>(hkv), nbu};
+    cuuint64_t strides[4] = {static_cast<cuuint64_t>(st) * 2, 128, static_cast<cuuint64_t>(sh) * 2,
+                             static_cast<cuuint64_t>(sb) * 2};
+    cuuint32_t box[5] = {64, static_cast<cuuint32_t>(bs), static_cast<cuuint32_t>(d / 64), 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(hkv), nbu};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(st) * 2, static_cast<cuuint64_t>(sh) * 2,
+                             static_cast<cuuint64_t>(sb) * 2};
+    cuuint32_t box[4] = {64, static_cast<cuuint32_t>(bs), 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   if (r != CUDA_SUCCESS) {
-    snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+    snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled (rank %d) failed with CUresult %d", rank,
+             static_cast<int>(r));
     return PDATTN_CUDA_ERROR;
   }
   MapCacheEntry& e = g_maps[g_map_next];
@@ -180,9 +202,20 @@ pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeP
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
     done = true;
   }
+  if (g_probe_mode) {
+    auto probe = decode_kernel<D, NT, 16, true>;
+    cudaError_t pe = cudaFuncSetAttribute(probe, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
+    if (pe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", pe);
+    probe<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
+    pe = cudaGetLastError();
+    if (pe != cudaSuccess) return cuda_fail("gather probe launch", pe);
+    return PDATTN_OK;
+  }
+  if (g_prof_start) cudaEventRecord(g_prof_start, stream);
   kern<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
+  if (g_prof_stop) cudaEventRecord(g_prof_stop, stream);
   combine_kernel<D, NT><<<grid, 256, 0, stream>>>(P.rec, P.partials, P.out, grid, P.Hq, P.Hkv, P.G);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("combine_kernel launch", e);
@@ -287,13 +320,23 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     g_last_launches += 1;
   }
 
+  // One TMA op per page-head (rank-5 view) when head_dim is 128; the rank-4 view otherwise, or if
+  // the driver refuses the rank-5 encoding.
+  static const bool force4d = getenv("PDATTN_BOX4D") != nullptr;
   CUtensorMap mk, mv;
+  int rank = (a->head_dim == 128 && !force4d) ? 5 : 4;
   s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-               a->kv_head_stride, a->kv_token_stride, &mk);
+               a->kv_head_stride, a->kv_token_stride, rank, &mk);
+  if (s != PDATTN_OK && rank == 5) {
+    rank = 4;
+    s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+                 a->kv_head_stride, a->kv_token_stride, rank, &mk);
+  }
   if (s != PDATTN_OK) return s;
   s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-               a->kv_head_stride, a->kv_token_stride, &mv);
+               a->kv_head_stride, a->kv_token_stride, rank, &mv);
   if (s != PDATTN_OK) return s;
+  P.box5d = rank == 5;
 
   const bool nt2 = G > 8;
   if (a->head_dim == 128)
@@ -429,6 +472,34 @@ pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream_) {
   if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
   if (word & ERR_TIMEOUT) return PDATTN_DEVICE_TIMEOUT;
   return PDATTN_BAD_PAGE_INDEX;
+}
+
+pdattn_status pdattn_gather_probe(const pdattn_args* args, pdattn_stream_t stream) {
+  g_probe_mode = true;
+  pdattn_status s = pdattn_decode_ex(args, stream);
+  g_probe_mode = false;
+  g_last_launches = 0;
+  return s;
+}
+
+pdattn_status pdattn_stream_read_probe(const void* src, size_t bytes, void* sink, pdattn_stream_t stream) {
+  if (!src || !sink || (reinterpret_cast<uintptr_t>(src) & 15)) return PDATTN_INVALID_ARG;
+  int dev = 0;
+  DevInfo* di = nullptr;
+  pdattn_status s = device_info(&dev, &di);
+  if (s != PDATTN_OK) return s;
+  stream_read_kernel<<<di->sm_count * 4, 512, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4*>(src), bytes / 16, static_cast<uint32_t*>(sink));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("stream_read_kernel launch", e);
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_profile_events(void* start_event, void* stop_event) {
+  if ((start_event == nullptr) != (stop_event == nullptr)) return PDATTN_INVALID_ARG;
+  g_prof_start = static_cast<cudaEvent_t>(start_event);
+  g_prof_stop = static_cast<cudaEvent_t>(stop_event);
+  return PDATTN_OK;
 }
 
 int pdattn_last_launch_count(void) { return g_last_launches; }

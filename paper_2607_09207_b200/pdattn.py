@@ -29,7 +29,8 @@ DEVICE_TIMEOUT = -8
 EXPORTS = [
     "pdattn_workspace_size", "pdattn_workspace_init", "pdattn_decode_ex", "pdattn_bind", "pdattn_decode",
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
-    "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error",
+    "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
+    "pdattn_gather_probe", "pdattn_stream_read_probe",
 ]
 
 
@@ -81,6 +82,9 @@ def lib():
         L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i32),
                                        ctypes.POINTER(i64)]
         L.pdattn_check.argtypes = [vp, vp]
+        L.pdattn_profile_events.argtypes = [vp, vp]
+        L.pdattn_gather_probe.argtypes = [ctypes.POINTER(Args), vp]
+        L.pdattn_stream_read_probe.argtypes = [vp, sz, vp, vp]
         L.pdattn_last_launch_count.argtypes = []
         L.pdattn_status_string.argtypes = [i32]
         L.pdattn_status_string.restype = ctypes.c_char_p
@@ -117,7 +121,7 @@ def alloc_workspace(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size=16
 
 def decode_ex(q, k_cache, v_cache, block_table, context_lens, scale, out, workspace,
               context_lens_host: Optional[np.ndarray] = None, num_blocks: Optional[int] = None,
-              stream=None, check: bool = True) -> int:
+              stream=None, check: bool = True, probe: bool = False) -> int:
     """pdattn_decode_ex.  k_cache / v_cache: bf16 tensors indexed [page, kv_head, slot, dim] with any
     strides whose last dimension is contiguous.  Returns the status (raises unless check=False)."""
     S, Hq, d = q.shape
@@ -137,10 +141,18 @@ def decode_ex(q, k_cache, v_cache, block_table, context_lens, scale, out, worksp
     a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
     a.scale = float(scale)
     a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
-    st = lib().pdattn_decode_ex(ctypes.byref(a), _stream_ptr(stream))
+    fn = lib().pdattn_gather_probe if probe else lib().pdattn_decode_ex
+    st = fn(ctypes.byref(a), _stream_ptr(stream))
     if check and st != OK:
-        raise PdattnError(st, "pdattn_decode_ex")
+        raise PdattnError(st, "pdattn_gather_probe" if probe else "pdattn_decode_ex")
     return st
+
+
+def stream_read_probe(src: torch.Tensor, sink: torch.Tensor, stream=None):
+    st = lib().pdattn_stream_read_probe(src.data_ptr(), src.numel() * src.element_size(), sink.data_ptr(),
+                                        _stream_ptr(stream))
+    if st != OK:
+        raise PdattnError(st, "pdattn_stream_read_probe")
 
 
 def bind(max_blocks_per_seq, num_blocks, workspace, context_lens_host: Optional[np.ndarray] = None):
