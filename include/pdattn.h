@@ -135,16 +135,32 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
                                  void* workspace, size_t workspace_bytes, pdattn_stream_t stream);
 
 /*
- * The host partitioner on its own (no GPU needed): splits the batch's KV stream into n_ctas
- * contiguous spans of 64-token tiles so that long-tail sequences are spread over all SMs.
- * Units are (sequence, kv head) pairs in the order unit = s * num_kv_heads + kv_head; unit u has
- * ceil(L_s / 64) tiles.  Span c starts at tile spans[2c+1] of unit spans[2c] and holds
- * *tiles_q + (c < *tiles_r) tiles.  spans: HOST int32 [2 * n_ctas].  Returns the total tile
- * count in *total_tiles.  Depends on the context lengths only, never on page ids.
+ * The host partitioner on its own (no GPU needed).  It flattens the batch into a stream of
+ * 64-token tiles, unit-major (unit = s * num_kv_heads + kv_head; unit u has ceil(L_s / 64)
+ * tiles), and cuts it into contiguous spans so that long-tail sequences are spread over all SMs
+ * (Section 2.3: a few long responses dominate the rollout): n_static spans, one per CTA, cover
+ * the stream; with dynamic_per_cta > 0 they cover only its first three quarters and up to
+ * n_ctas * dynamic_per_cta short spans cover the rest, taken at run time by whichever CTA is free.  Span i starts at tile spans[2i+1] of unit spans[2i];
+ * static span i holds static_q + (i < static_r) tiles, dynamic span j (index n_static + j) holds
+ * dynamic_q + (j < dynamic_r).  spans: HOST int32 [2 * max_spans]; n_static + n_dynamic <=
+ * max_spans.  The plan depends on the context lengths only, never on page ids.
  */
+typedef struct {
+  int n_static, n_dynamic;
+  int static_q, static_r;
+  int dynamic_q, dynamic_r;
+  int total_tiles;
+} pdattn_plan;
 pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, int num_kv_heads,
-                               int n_ctas, int32_t* spans, int* tiles_q, int* tiles_r,
-                               int64_t* total_tiles);
+                               int n_ctas, int dynamic_per_cta, int max_spans, int32_t* spans,
+                               pdattn_plan* plan);
+
+/*
+ * Process-wide tuning of the partitioner above: at most `per_cta` run-time spans per CTA
+ * (0..8; 0 = every span is static, the default).  Results stay bit-identical from run to run
+ * for a given setting; different settings cut sequences at different tiles.
+ */
+pdattn_status pdattn_set_dynamic_spans(int per_cta);
 
 /*
  * Synchronises `stream`, reads and clears the workspace's sticky error word.

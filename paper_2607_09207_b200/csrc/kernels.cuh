@@ -31,20 +31,22 @@
 namespace pdattn {
 
 constexpr int TILE = kTileTokens;                // tokens per pipeline stage
-constexpr int MAX_PARAM_SPANS = 320;             // spans that travel in kernel parameters
-constexpr int MAX_CTAS = 592;                    // upper bound used for workspace sizing
-constexpr int MAX_STAGES = 24;
+constexpr int MAX_SPANS = 2048;                  // spans per call (static + run-time); sizes the workspace
+constexpr int MAX_PARAM_SPANS = 1536;            // spans that can travel in kernel parameters
+constexpr int SPAN_QUEUE = 32;                   // in-CTA queue of run-time span ids
+constexpr int MAX_STAGES = 12;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2 };
 
 // Workspace header (first 256 bytes of the workspace)
 struct WsHeader {
-  int32_t err;       // sticky error bits
-  int32_t tiles_q;   // written by plan_kernel
-  int32_t tiles_r;
-  int32_t pad[61];
+  int32_t err;        // sticky error bits
+  int32_t counter;    // next run-time span; zero between calls (combine_kernel resets it)
+  PlanParams plan;    // written by plan_kernel
+  int32_t pad[54];
 };
+static_assert(sizeof(WsHeader) == 256, "header size");
 
 struct DecodeParams {
   const __nv_bfloat16* q;
@@ -53,11 +55,11 @@ struct DecodeParams {
   const int32_t* context_lens;
   WsHeader* hdr;
   const int2* spans_ws;     // spans written by plan_kernel (used when use_ws_plan)
-  int4* rec;                // per-CTA record: (first_unit, first_tile, own_unit, own_slot)
-  float* partials;          // [cta][2][HP*(D+2)] fp32
+  int4* rec;                // per-span record: (first_unit, first_tile, own_unit, own_slot)
+  float* partials;          // [span][2][HP*(D+2)] fp32
   int S, Hq, Hkv, G, MB, NB;
   float scale_log2;         // scale * log2(e)
-  int tiles_q, tiles_r;
+  PlanParams plan;          // host plan (ignored when use_ws_plan)
   int use_ws_plan;
   int box5d;                // 1: the tensor maps are 5-D and one TMA op brings a whole page-head
   int2 spans[MAX_PARAM_SPANS];
@@ -215,6 +217,9 @@ struct Ctrl {                 // lives in the CTRL_BYTES area
   uint64_t empty[MAX_STAGES];
   uint32_t meta[MAX_STAGES];  // per stage: bit j set = page j of the tile had a bad id
   uint32_t abort;
+  int32_t sq_pub;             // number of run-time span ids published so far
+  int32_t sq_id[SPAN_QUEUE];  // k-th id (k >= 1) at [(k-1) % SPAN_QUEUE]; -1 = no more spans
+  int32_t sq_tag[SPAN_QUEUE]; // k, to detect an overwritten entry
 };
 static_assert(sizeof(Ctrl) <= 512, "control block");
 
@@ -414,10 +419,44 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
 }
 
 // ------------------------------------------------------------------------------------------
-// The decode kernel
+// Span sequencing inside a CTA.  Every warp walks the same sequence of spans: first the CTA's
+// static span, then run-time spans.  Lane 0 of producer warp 0 draws run-time spans from the
+// global counter (one atomic per span, issued a whole span ahead of its use) and publishes the
+// ids through a small shared-memory queue; every other warp reads them from there.
 // ------------------------------------------------------------------------------------------
-// PROBE = true builds the page-gather ceiling: identical walk, page-id lookups and TMA ring, but
-// the consumers release every tile untouched and nothing is written.
+__device__ __forceinline__ int ld_acquire_shared(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.cta.shared.b32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_shared(int32_t* p, int v) {
+  asm volatile("st.release.cta.shared.b32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+// k-th span of this CTA (k >= 1), or -1 when there is none (or the bounded wait expired).
+__device__ __forceinline__ int read_span(Ctrl* ctrl, int k, bool& aborted) {
+  if (aborted) return -1;
+  if (ld_acquire_shared(&ctrl->sq_pub) < k) {
+    const unsigned long long t0 = globaltimer_ns();
+    while (ld_acquire_shared(&ctrl->sq_pub) < k) {
+      if (*reinterpret_cast<volatile uint32_t*>(&ctrl->abort) || globaltimer_ns() - t0 > kWaitLimitNs) {
+        aborted = true;
+        return -1;
+      }
+    }
+  }
+  const int slot = (k - 1) % SPAN_QUEUE;
+  const int id = ctrl->sq_id[slot];
+  if (ctrl->sq_tag[slot] != k) {   // the queue wrapped past a reader: cannot happen while warps stay
+    aborted = true;                //  within a ring's worth of tiles of each other; fail loudly if it does
+    return -1;
+  }
+  return id;
+}
+
+// ------------------------------------------------------------------------------------------
+// The decode kernel.  PROBE = true builds the page-gather ceiling: identical span walk, page-id
+// lookups and TMA ring, but the consumers release every tile untouched and nothing is written.
+// ------------------------------------------------------------------------------------------
 template <int D, int NT, int BS, bool PROBE = false>
 __global__ void __launch_bounds__(Cfg<D, NT, BS>::NTHREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -447,31 +486,15 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       mbar_init(smem_u32(&ctrl->empty[i]), 1);
     }
     ctrl->abort = 0;
+    ctrl->sq_pub = 0;
     fence_mbar_init();
   }
   __syncthreads();
 
-  // this CTA's span
-  int unit0, tile0, ntiles;
-  {
-    int2 sp;
-    int tq, tr;
-    if (P.use_ws_plan) {
-      sp = P.spans_ws[cta];
-      tq = P.hdr->tiles_q;
-      tr = P.hdr->tiles_r;
-    } else {
-      sp = P.spans[cta];
-      tq = P.tiles_q;
-      tr = P.tiles_r;
-    }
-    unit0 = sp.x;
-    tile0 = sp.y;
-    ntiles = tq + (cta < tr ? 1 : 0);
-  }
-  Walker walk{P.context_lens, P.Hkv, P.S * P.Hkv, unit0, tile0, ntiles};
-  Piece pc;
-  int it = 0;   // tile counter within this CTA: tile `it` uses ring slot it % NST
+  const PlanParams pp = P.use_ws_plan ? P.hdr->plan : P.plan;
+  const int nunits = P.S * P.Hkv;
+  int it = 0;        // tile counter within this CTA: tile `it` uses ring slot it % NST
+  bool aborted = false;
 
   if (warp >= NCW) {
     // ================= producer warp(s) =================
@@ -479,53 +502,75 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     constexpr int IDS_PER_BATCH = 32;
     constexpr int TILES_PER_BATCH = IDS_PER_BATCH / C::PAGES;
     bool any_bad = false;
-    bool aborted = false;
-    while (!aborted && walk.next(pc)) {
-      const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
-      const int npages = (pc.L + BS - 1) / BS;
-      const int pbase = pc.tb * C::PAGES;
-      int ids_cur = (pbase + lane < npages) ? __ldg(row + pbase + lane) : 0;
-      int ids_nxt = (pbase + IDS_PER_BATCH + lane < npages) ? __ldg(row + pbase + IDS_PER_BATCH + lane) : 0;
-      for (int t = pc.tb; t < pc.te; ++t, ++it) {
-        const int rel = t - pc.tb;
-        const int k = rel % TILES_PER_BATCH;
-        if (k == 0 && rel != 0) {
-          ids_cur = ids_nxt;
-          const int nb = pbase + rel * C::PAGES + IDS_PER_BATCH;
-          ids_nxt = (nb + lane < npages) ? __ldg(row + nb + lane) : 0;
+    int span = cta;
+    for (int k = 0; span >= 0; ++k) {
+      // draw the next run-time span now; its id is only consumed after this span's tiles are issued
+      int nxt = -1;
+      if (pw == 0 && lane == 0 && pp.n_dyn > 0) {
+        const int j = atomicAdd(&P.hdr->counter, 1);
+        nxt = j < pp.n_dyn ? pp.n_static + j : -1;
+      }
+      const int2 sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
+      Walker walk{P.context_lens, P.Hkv, nunits, sp.x, sp.y, span_len(pp, span)};
+      Piece pc;
+      while (!aborted && walk.next(pc)) {
+        const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
+        const int npages = (pc.L + BS - 1) / BS;
+        const int pbase = pc.tb * C::PAGES;
+        int ids_cur = (pbase + lane < npages) ? __ldg(row + pbase + lane) : 0;
+        int ids_nxt = (pbase + IDS_PER_BATCH + lane < npages) ? __ldg(row + pbase + IDS_PER_BATCH + lane) : 0;
+        for (int t = pc.tb; t < pc.te; ++t, ++it) {
+          const int rel = t - pc.tb;
+          const int kb = rel % TILES_PER_BATCH;
+          if (kb == 0 && rel != 0) {
+            ids_cur = ids_nxt;
+            const int nb = pbase + rel * C::PAGES + IDS_PER_BATCH;
+            ids_nxt = (nb + lane < npages) ? __ldg(row + nb + lane) : 0;
+          }
+          if (C::NPW > 1 && it % C::NPW != pw) continue;
+          const int slot = it % NST;
+          const uint32_t phase = (it / NST) & 1;
+          if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) {
+            aborted = true;
+            break;
+          }
+          const int np = min(C::PAGES, npages - t * C::PAGES);
+          const int j = lane % C::PAGES;
+          int id = __shfl_sync(0xffffffffu, ids_cur, kb * C::PAGES + j);
+          const bool bad = (lane < C::PAGES) && (j < np) && (id < 0 || id >= P.NB);
+          const uint32_t badmask = __ballot_sync(0xffffffffu, bad);
+          if (id < 0 || id >= P.NB) id = P.NB;   // out-of-bounds coordinate: TMA fills zeros, nothing is read
+          const uint32_t bar = smem_u32(&ctrl->full[slot]);
+          if (lane == 0) {
+            ctrl->meta[slot] = badmask;
+            mbar_arrive_expect_tx(bar, static_cast<uint32_t>(np) * 2u * C::PAGE_BYTES);
+          }
+          __syncwarp();
+          if (lane < 2 * C::PAGES && j < np) {
+            const bool isV = lane >= C::PAGES;
+            const uint32_t dst = ring + slot * C::STAGE_BYTES + (isV ? C::KV_BYTES : 0) + j * C::PAGE_BYTES;
+            const CUtensorMap* tm = isV ? &tmV : &tmK;
+            if (P.box5d) {
+              tma_load_5d(dst, tm, 0, 0, 0, pc.g, id, bar);
+            } else {
+#pragma unroll
+              for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, tm, h * 64, 0, pc.g, id, bar);
+            }
+          }
+          any_bad |= (badmask != 0);
         }
-        if (C::NPW > 1 && it % C::NPW != pw) continue;
-        const int slot = it % NST;
-        const uint32_t phase = (it / NST) & 1;
-        if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) {
-          aborted = true;
-          break;
-        }
-        const int np = min(C::PAGES, npages - t * C::PAGES);
-        const int j = lane % C::PAGES;
-        int id = __shfl_sync(0xffffffffu, ids_cur, k * C::PAGES + j);
-        const bool bad = (lane < C::PAGES) && (j < np) && (id < 0 || id >= P.NB);
-        const uint32_t badmask = __ballot_sync(0xffffffffu, bad);
-        if (id < 0 || id >= P.NB) id = P.NB;   // out-of-bounds coordinate: TMA fills zeros, nothing is read
-        const uint32_t bar = smem_u32(&ctrl->full[slot]);
+      }
+      if (aborted) break;
+      if (pw == 0) {
         if (lane == 0) {
-          ctrl->meta[slot] = badmask;
-          mbar_arrive_expect_tx(bar, static_cast<uint32_t>(np) * 2u * C::PAGE_BYTES);
+          const int slot = k % SPAN_QUEUE;
+          ctrl->sq_id[slot] = nxt;
+          ctrl->sq_tag[slot] = k + 1;
+          st_release_shared(&ctrl->sq_pub, k + 1);
         }
         __syncwarp();
-        if (lane < 2 * C::PAGES && j < np) {
-          const bool isV = lane >= C::PAGES;
-          const uint32_t dst = ring + slot * C::STAGE_BYTES + (isV ? C::KV_BYTES : 0) + j * C::PAGE_BYTES;
-          const CUtensorMap* tm = isV ? &tmV : &tmK;
-          if (P.box5d) {
-            tma_load_5d(dst, tm, 0, 0, 0, pc.g, id, bar);
-          } else {
-#pragma unroll
-            for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, tm, h * 64, 0, pc.g, id, bar);
-          }
-        }
-        any_bad |= (badmask != 0);
       }
+      span = read_span(ctrl, k + 1, aborted);
     }
     if (lane == 0) {
       if (any_bad) atomicOr(&P.hdr->err, ERR_BAD_PAGE);
@@ -539,159 +584,173 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
   // ================= consumer warps =================
   const int ct = threadIdx.x;   // 0..NCT-1
-  // sequences with no context produce zeros
-  for (int s = cta; s < P.S; s += gridDim.x) {
-    if (__ldg(P.context_lens + s) <= 0) {
-      uint32_t* o = reinterpret_cast<uint32_t*>(P.out + static_cast<int64_t>(s) * P.Hq * D);
-      for (int i = ct; i < P.Hq * D / 2; i += NCT) o[i] = 0u;
+  if (!PROBE) {
+    // sequences with no context produce zeros
+    for (int s = cta; s < P.S; s += gridDim.x) {
+      if (__ldg(P.context_lens + s) <= 0) {
+        uint32_t* o = reinterpret_cast<uint32_t*>(P.out + static_cast<int64_t>(s) * P.Hq * D);
+        for (int i = ct; i < P.Hq * D / 2; i += NCT) o[i] = 0u;
+      }
     }
   }
-
-  int first_unit = -1, first_tb = 0, own_unit = -1, own_slot = 0, piece_idx = 0;
-  bool aborted = false;
   const int hq0 = lane >> 2;         // B-operand column (head) this lane feeds
   const int qcol = (lane & 3) * 2;
 
-  while (walk.next(pc)) {
-    // ---- packed query rows of this KV head as MMA B fragments
-    uint32_t qf[NT][D / 16][2];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int head = nt * 8 + hq0;
-      const bool live = head < P.G;
-      const uint32_t* qp = reinterpret_cast<const uint32_t*>(
-          P.q + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + (live ? head : 0)) * D);
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        qf[nt][kk][0] = live ? __ldg(qp + (kk * 16 + qcol) / 2) : 0u;
-        qf[nt][kk][1] = live ? __ldg(qp + (kk * 16 + 8 + qcol) / 2) : 0u;
-      }
-    }
-    float acc[NT][D / 16][4];
-    float m[NT][2], l[NT][2];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      m[nt][0] = m[nt][1] = NEG_INF;
-      l[nt][0] = l[nt][1] = 0.f;
-#pragma unroll
-      for (int jm = 0; jm < D / 16; ++jm) acc[nt][jm][0] = acc[nt][jm][1] = acc[nt][jm][2] = acc[nt][jm][3] = 0.f;
-    }
+  int span = cta;
+  for (int k = 0; span >= 0; ++k) {
+    const int2 sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
+    Walker walk{P.context_lens, P.Hkv, nunits, sp.x, sp.y, span_len(pp, span)};
+    Piece pc;
+    int first_unit = -1, first_tb = 0, own_unit = -1, own_slot = 0, piece_idx = 0;
 
-    for (int t = pc.tb; t < pc.te; ++t, ++it) {
-      if (it % NCW != warp) continue;
-      if (!aborted && *reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) aborted = true;
-      if (aborted) continue;
-      const int slot = it % NST;
-      const uint32_t phase = (it / NST) & 1;
-      if (!mbar_wait(smem_u32(&ctrl->full[slot]), phase)) {
-        aborted = true;
-        if (lane == 0) {
-          atomicOr(&P.hdr->err, ERR_TIMEOUT);
-          atomicExch(&ctrl->abort, 1u);
-        }
-        continue;
-      }
-      const uint32_t sK = ring + slot * C::STAGE_BYTES;
-      const uint32_t sV = sK + C::KV_BYTES;
-      const uint32_t badmask = ctrl->meta[slot];
-      const int n_valid = min(TILE, pc.L - t * TILE);
-      if (PROBE) {
-        // ceiling probe: no math
-      } else if (n_valid == TILE) {
-        compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane);
-      } else {
-        compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_valid, badmask, lane);
-        fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
-    }
-
-    const bool complete = (pc.tb == 0 && pc.te == pc.nt);
-    const int slot_idx = piece_idx == 0 ? 0 : 1;
-    if constexpr (!PROBE) {
-    // ---- merge the NCW warp states of this piece
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        float v = l[nt][e];
-        v += __shfl_xor_sync(0xffffffffu, v, 4);
-        v += __shfl_xor_sync(0xffffffffu, v, 8);
-        v += __shfl_xor_sync(0xffffffffu, v, 16);
-        l[nt][e] = v;
-      }
-    {
-      float* my = scratch + warp * C::HP * C::ACC_STRIDE;
-      const int drow = lane >> 2;
+    while (walk.next(pc)) {
+      const int w_first = it % NCW;   // warp that takes this piece's first tile
+      // ---- packed query rows of this KV head as MMA B fragments
+      uint32_t qf[NT][D / 16][2];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        const int h0 = nt * 8 + qcol;
+        const int head = nt * 8 + hq0;
+        const bool live = head < P.G;
+        const uint32_t* qp = reinterpret_cast<const uint32_t*>(
+            P.q + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + (live ? head : 0)) * D);
 #pragma unroll
-        for (int jm = 0; jm < D / 16; ++jm) {
-          my[h0 * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][0];
-          my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][1];
-          my[h0 * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][2];
-          my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][3];
-        }
-        if (lane < 4) {
-          sm_m[warp * C::HP + h0] = m[nt][0];
-          sm_m[warp * C::HP + h0 + 1] = m[nt][1];
-          sm_l[warp * C::HP + h0] = l[nt][0];
-          sm_l[warp * C::HP + h0 + 1] = l[nt][1];
+        for (int kk = 0; kk < D / 16; ++kk) {
+          qf[nt][kk][0] = live ? __ldg(qp + (kk * 16 + qcol) / 2) : 0u;
+          qf[nt][kk][1] = live ? __ldg(qp + (kk * 16 + 8 + qcol) / 2) : 0u;
         }
       }
-    }
-    bar_consumers<NCT>();
-    float* part = P.partials + (static_cast<int64_t>(cta) * 2 + slot_idx) * C::SLOT_FLOATS;
-    for (int idx = ct; idx < C::HP * (D / 4); idx += NCT) {
-      const int h = idx / (D / 4);
-      const int dq = idx % (D / 4);
-      float M = NEG_INF;
+      float acc[NT][D / 16][4];
+      float m[NT][2], l[NT][2];
 #pragma unroll
-      for (int w = 0; w < NCW; ++w) M = fmaxf(M, sm_m[w * C::HP + h]);
-      const float Mu = (M == NEG_INF) ? 0.f : M;
-      float Ls = 0.f;
-      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int nt = 0; nt < NT; ++nt) {
+        m[nt][0] = m[nt][1] = NEG_INF;
+        l[nt][0] = l[nt][1] = 0.f;
 #pragma unroll
-      for (int w = 0; w < NCW; ++w) {
-        const float f = fast_exp2(sm_m[w * C::HP + h] - Mu);
-        Ls += sm_l[w * C::HP + h] * f;
-        const float4 v = *reinterpret_cast<const float4*>(scratch + (w * C::HP + h) * C::ACC_STRIDE + dq * 4);
-        a.x += v.x * f;
-        a.y += v.y * f;
-        a.z += v.z * f;
-        a.w += v.w * f;
+        for (int jm = 0; jm < D / 16; ++jm) acc[nt][jm][0] = acc[nt][jm][1] = acc[nt][jm][2] = acc[nt][jm][3] = 0.f;
       }
-      if (complete) {
-        if (h < P.G) {
-          const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
-          uint2 o;
-          o.x = pack_bf16x2(a.x * inv, a.y * inv);
-          o.y = pack_bf16x2(a.z * inv, a.w * inv);
-          *reinterpret_cast<uint2*>(P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + h) * D + dq * 4) = o;
+
+      for (int t = pc.tb; t < pc.te; ++t, ++it) {
+        if (it % NCW != warp) continue;
+        if (!aborted && *reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) aborted = true;
+        if (aborted) continue;
+        const int slot = it % NST;
+        const uint32_t phase = (it / NST) & 1;
+        if (!mbar_wait(smem_u32(&ctrl->full[slot]), phase)) {
+          aborted = true;
+          if (lane == 0) {
+            atomicOr(&P.hdr->err, ERR_TIMEOUT);
+            atomicExch(&ctrl->abort, 1u);
+          }
+          continue;
         }
-      } else {
-        if (dq == 0) {
-          part[h] = M;
-          part[C::HP + h] = Ls;
+        const uint32_t sK = ring + slot * C::STAGE_BYTES;
+        const uint32_t sV = sK + C::KV_BYTES;
+        const uint32_t badmask = ctrl->meta[slot];
+        const int n_valid = min(TILE, pc.L - t * TILE);
+        if (PROBE) {
+          // ceiling probe: no math
+        } else if (n_valid == TILE) {
+          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane);
+        } else {
+          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_valid, badmask, lane);
+          fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
         }
-        *reinterpret_cast<float4*>(part + 2 * C::HP + h * D + dq * 4) = a;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
       }
+
+      const bool complete = (pc.tb == 0 && pc.te == pc.nt);
+      const int slot_idx = piece_idx == 0 ? 0 : 1;
+      if constexpr (!PROBE) {
+        // ---- merge the NCW warp states of this piece
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            float v = l[nt][e];
+            v += __shfl_xor_sync(0xffffffffu, v, 4);
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            l[nt][e] = v;
+          }
+        {
+          float* my = scratch + warp * C::HP * C::ACC_STRIDE;
+          const int drow = lane >> 2;
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const int h0 = nt * 8 + qcol;
+#pragma unroll
+            for (int jm = 0; jm < D / 16; ++jm) {
+              my[h0 * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][0];
+              my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][1];
+              my[h0 * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][2];
+              my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][3];
+            }
+            if (lane < 4) {
+              sm_m[warp * C::HP + h0] = m[nt][0];
+              sm_m[warp * C::HP + h0 + 1] = m[nt][1];
+              sm_l[warp * C::HP + h0] = l[nt][0];
+              sm_l[warp * C::HP + h0 + 1] = l[nt][1];
+            }
+          }
+        }
+        bar_consumers<NCT>();
+        float* part = P.partials + (static_cast<int64_t>(span) * 2 + slot_idx) * C::SLOT_FLOATS;
+        for (int idx = ct; idx < C::HP * (D / 4); idx += NCT) {
+          const int h = idx / (D / 4);
+          const int dq = idx % (D / 4);
+          float M = NEG_INF;
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) M = fmaxf(M, sm_m[w * C::HP + h]);
+          const float Mu = (M == NEG_INF) ? 0.f : M;
+          float Ls = 0.f;
+          float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+          // Sum in the order of the tiles' residue classes within the piece, not of warp numbers:
+          // which warp holds which class depends on what this CTA processed before.
+#pragma unroll
+          for (int r = 0; r < NCW; ++r) {
+            int w = w_first + r;
+            if (w >= NCW) w -= NCW;
+            const float f = fast_exp2(sm_m[w * C::HP + h] - Mu);
+            Ls += sm_l[w * C::HP + h] * f;
+            const float4 v = *reinterpret_cast<const float4*>(scratch + (w * C::HP + h) * C::ACC_STRIDE + dq * 4);
+            a.x += v.x * f;
+            a.y += v.y * f;
+            a.z += v.z * f;
+            a.w += v.w * f;
+          }
+          if (complete) {
+            if (h < P.G) {
+              const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
+              uint2 o;
+              o.x = pack_bf16x2(a.x * inv, a.y * inv);
+              o.y = pack_bf16x2(a.z * inv, a.w * inv);
+              *reinterpret_cast<uint2*>(P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + h) * D + dq * 4) = o;
+            }
+          } else {
+            if (dq == 0) {
+              part[h] = M;
+              part[C::HP + h] = Ls;
+            }
+            *reinterpret_cast<float4*>(part + 2 * C::HP + h * D + dq * 4) = a;
+          }
+        }
+        bar_consumers<NCT>();   // scratch is reused by the next piece
+      }
+      if (piece_idx == 0) {
+        first_unit = pc.unit;
+        first_tb = pc.tb;
+      }
+      if (!complete && pc.tb == 0) {
+        own_unit = pc.unit;
+        own_slot = slot_idx;
+      }
+      ++piece_idx;
     }
-    bar_consumers<NCT>();   // scratch is reused by the next piece
-    }   // !PROBE
-    if (piece_idx == 0) {
-      first_unit = pc.unit;
-      first_tb = pc.tb;
-    }
-    if (!complete && pc.tb == 0) {
-      own_unit = pc.unit;
-      own_slot = slot_idx;
-    }
-    ++piece_idx;
+    if (ct == 0 && !PROBE) P.rec[span] = make_int4(first_unit, first_tb, own_unit, own_slot);
+    span = read_span(ctrl, k + 1, aborted);
   }
-  if (ct == 0 && !PROBE) P.rec[cta] = make_int4(first_unit, first_tb, own_unit, own_slot);
+  if (aborted && lane == 0) atomicOr(&P.hdr->err, ERR_TIMEOUT);
 }
 
 // Read-only streaming ceiling: every thread block sums a contiguous slice with 16-byte loads.
@@ -714,25 +773,29 @@ stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __rest
 }
 
 // ------------------------------------------------------------------------------------------
-// Split-combine: block c merges the unit that started in CTA c's span and ran past its end.
-// The pieces live in consecutive CTAs (slot 0 of each follower), merged in ascending token
-// order:  M = max m_c;  Lsum = sum l_c 2^(m_c - M);  out = bf16( sum acc_c 2^(m_c - M) / Lsum ).
+// Split-combine: block i merges the unit that started in span i and ran past its end.  The
+// pieces live in consecutive spans (slot 0 of each follower), merged in ascending token order:
+//   M = max m_c;  Lsum = sum l_c 2^(m_c - M);  out = bf16( sum acc_c 2^(m_c - M) / Lsum ).
+// Block 0 also rearms the run-time span counter for the next call.
 // ------------------------------------------------------------------------------------------
 template <int D, int NT>
 __global__ void __launch_bounds__(256)
-combine_kernel(const int4* __restrict__ rec, const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
-               int n_ctas, int Hq, int Hkv, int G) {
+combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, const float* __restrict__ partials,
+               __nv_bfloat16* __restrict__ out, int Hq, int Hkv, int G) {
   constexpr int HP = 8 * NT;
   constexpr int SLOT_FLOATS = HP * (D + 2);
   const int c = blockIdx.x;
+  if (c == 0 && threadIdx.x == 0) hdr->counter = 0;
+  const int n_spans = n_spans_host >= 0 ? n_spans_host : hdr->plan.n_static + hdr->plan.n_dyn;
+  if (c >= n_spans) return;
   const int4 r = rec[c];
   const int unit = r.z;
   if (unit < 0) return;
-  // followers: CTAs c+1.. whose first piece continues `unit`
+  // followers: spans c+1.. whose first piece continues `unit`
   __shared__ int n_follow;
   if (threadIdx.x == 0) {
     int n = 0;
-    for (int cc = c + 1; cc < n_ctas; ++cc) {
+    for (int cc = c + 1; cc < n_spans; ++cc) {
       const int4 rr = rec[cc];
       if (rr.x != unit || rr.y <= 0) break;
       ++n;
@@ -777,10 +840,11 @@ combine_kernel(const int4* __restrict__ rec, const float* __restrict__ partials,
 // Device twin of the host partitioner (one block).  prefix: [S+1] ints of scratch.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
-plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_ctas, int32_t* __restrict__ prefix,
-            int2* __restrict__ spans, WsHeader* hdr) {
+plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_static, int n_dyn_max,
+            int32_t* __restrict__ prefix, int2* __restrict__ spans, WsHeader* hdr) {
   __shared__ int warp_sums[32];
   __shared__ int carry_s;
+  __shared__ PlanParams pp_s;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   if (tid == 0) {
     carry_s = 0;
@@ -819,17 +883,18 @@ plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_ctas
     __syncthreads();
   }
   const int total = carry_s;
-  const int tq = total / n_ctas, tr = total % n_ctas;
   if (tid == 0) {
-    hdr->tiles_q = tq;
-    hdr->tiles_r = tr;
+    pp_s = make_plan_params(total, n_static, n_dyn_max);
+    hdr->plan = pp_s;
   }
   __threadfence_block();
   __syncthreads();
-  for (int c = tid; c < n_ctas; c += 1024) {
-    const int start = c * tq + min(c, tr);
+  const PlanParams pp = pp_s;
+  const int n_spans = pp.n_static + pp.n_dyn;
+  for (int c = tid; c < n_spans; c += 1024) {
     int2 sp = make_int2(S * Hkv, 0);
-    if (start < total) {
+    const int start = span_start(pp, c);
+    if (span_len(pp, c) > 0 && start < total) {
       int lo = 0, hi = S;   // find s with prefix[s] <= start < prefix[s+1]
       while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;

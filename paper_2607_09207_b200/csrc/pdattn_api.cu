@@ -20,6 +20,7 @@ thread_local char g_cuda_err[256] = "";
 thread_local int g_last_launches = 0;
 thread_local cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 thread_local bool g_probe_mode = false;   // set only inside pdattn_gather_probe
+int g_dyn_per_cta = 0;                    // run-time spans per CTA (pdattn_set_dynamic_spans)
 
 struct Binding {
   bool set = false;
@@ -47,10 +48,10 @@ WsLayout ws_layout(int num_seqs, int G, int head_dim) {
   WsLayout w;
   w.hdr = 0;
   w.spans = 256;
-  w.rec = w.spans + align_up(static_cast<size_t>(MAX_CTAS) * sizeof(int2), 256);
-  w.prefix = w.rec + align_up(static_cast<size_t>(MAX_CTAS) * sizeof(int4), 256);
+  w.rec = w.spans + align_up(static_cast<size_t>(MAX_SPANS) * sizeof(int2), 256);
+  w.prefix = w.rec + align_up(static_cast<size_t>(MAX_SPANS) * sizeof(int4), 256);
   w.partials = w.prefix + align_up(static_cast<size_t>(num_seqs + 1) * 4, 256);
-  w.total = w.partials + align_up(static_cast<size_t>(MAX_CTAS) * 2 * slot_bytes, 256);
+  w.total = w.partials + align_up(static_cast<size_t>(MAX_SPANS) * 2 * slot_bytes, 256);
   return w;
 }
 
@@ -192,8 +193,8 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
 
 // ---- launches ------------------------------------------------------------------------------------
 template <int D, int NT>
-pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, DevInfo* di,
-                     cudaStream_t stream) {
+pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
+                     int n_spans_host, DevInfo* di, cudaStream_t stream) {
   using C = Cfg<D, NT, 16>;
   auto kern = decode_kernel<D, NT, 16>;
   bool& done = di->attr_set[D == 128][NT == 2];
@@ -209,6 +210,8 @@ pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeP
     probe<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
     pe = cudaGetLastError();
     if (pe != cudaSuccess) return cuda_fail("gather probe launch", pe);
+    pe = cudaMemsetAsync(&P.hdr->counter, 0, 4, stream);   // the combine kernel normally rearms it
+    if (pe != cudaSuccess) return cuda_fail("cudaMemsetAsync", pe);
     return PDATTN_OK;
   }
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
@@ -216,7 +219,8 @@ pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeP
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
   if (g_prof_stop) cudaEventRecord(g_prof_stop, stream);
-  combine_kernel<D, NT><<<grid, 256, 0, stream>>>(P.rec, P.partials, P.out, grid, P.Hq, P.Hkv, P.G);
+  combine_kernel<D, NT><<<combine_grid, 256, 0, stream>>>(P.hdr, n_spans_host, P.rec, P.partials, P.out, P.Hq, P.Hkv,
+                                                          P.G);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("combine_kernel launch", e);
   return PDATTN_OK;
@@ -244,13 +248,25 @@ pdattn_status pdattn_workspace_init(void* workspace, size_t workspace_bytes, pda
   return PDATTN_OK;
 }
 
+pdattn_status pdattn_set_dynamic_spans(int per_cta) {
+  if (per_cta < 0 || per_cta > kMaxDynPerCta) return PDATTN_INVALID_ARG;
+  g_dyn_per_cta = per_cta;
+  return PDATTN_OK;
+}
+
 pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, int num_kv_heads, int n_ctas,
-                               int32_t* spans, int* tiles_q, int* tiles_r, int64_t* total_tiles) {
-  Plan plan;
-  if (!plan_spans(context_lens_host, num_seqs, num_kv_heads, n_ctas, spans, &plan)) return PDATTN_INVALID_ARG;
-  if (tiles_q) *tiles_q = plan.tiles_q;
-  if (tiles_r) *tiles_r = plan.tiles_r;
-  if (total_tiles) *total_tiles = plan.total_tiles;
+                               int dynamic_per_cta, int max_spans, int32_t* spans, pdattn_plan* plan_out) {
+  if (!plan_out) return PDATTN_INVALID_ARG;
+  PlanParams plan;
+  if (!plan_spans(context_lens_host, num_seqs, num_kv_heads, n_ctas, dynamic_per_cta, max_spans, spans, &plan))
+    return PDATTN_INVALID_ARG;
+  plan_out->n_static = plan.n_static;
+  plan_out->n_dynamic = plan.n_dyn;
+  plan_out->static_q = plan.qs;
+  plan_out->static_r = plan.rs;
+  plan_out->dynamic_q = plan.qd;
+  plan_out->dynamic_r = plan.rd;
+  plan_out->total_tiles = plan.total;
   return PDATTN_OK;
 }
 
@@ -279,7 +295,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   uint8_t* ws = static_cast<uint8_t*>(a->workspace);
 
-  static_assert(sizeof(DecodeParams) + 2 * sizeof(CUtensorMap) <= 4000, "kernel parameters");
+  static_assert(sizeof(DecodeParams) + 2 * sizeof(CUtensorMap) <= 32000, "kernel parameters");
   DecodeParams P;
   P.q = static_cast<const __nv_bfloat16*>(a->q);
   P.out = static_cast<__nv_bfloat16*>(a->out);
@@ -296,28 +312,33 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   P.MB = a->max_blocks_per_seq;
   P.NB = a->num_blocks;
   P.scale_log2 = a->scale * 1.4426950408889634f;
-  P.tiles_q = P.tiles_r = 0;
   P.use_ws_plan = 0;
+  P.box5d = 0;
 
   int n_ctas = di->sm_count;
-  if (n_ctas > MAX_PARAM_SPANS) n_ctas = MAX_PARAM_SPANS;
-  int grid = n_ctas;
+  if (n_ctas > MAX_SPANS / (1 + kMaxDynPerCta)) n_ctas = MAX_SPANS / (1 + kMaxDynPerCta);
+  const int dyn_per_cta = g_dyn_per_cta;
+  int grid = n_ctas, combine_grid = 0, n_spans_host = -1;
   if (a->context_lens_host) {
-    Plan plan;
-    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, reinterpret_cast<int32_t*>(P.spans),
-                    &plan))
+    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta, MAX_PARAM_SPANS,
+                    reinterpret_cast<int32_t*>(P.spans), &P.plan))
       return PDATTN_INVALID_ARG;
-    P.tiles_q = plan.tiles_q;
-    P.tiles_r = plan.tiles_r;
-    if (plan.total_tiles < n_ctas) grid = plan.total_tiles > 0 ? static_cast<int>(plan.total_tiles) : 1;
+    if (P.plan.total < n_ctas) {          // fewer tiles than CTAs: one tile each, no empty CTAs
+      grid = P.plan.total > 0 ? P.plan.total : 1;
+    }
+    n_spans_host = P.plan.n_dyn > 0 ? P.plan.n_static + P.plan.n_dyn : grid;
+    combine_grid = n_spans_host;
   } else {
     P.use_ws_plan = 1;
-    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas,
+    memset(&P.plan, 0, sizeof P.plan);
+    const int n_dyn_max = n_ctas * dyn_per_cta;
+    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
                                          reinterpret_cast<int32_t*>(ws + wl.prefix),
                                          reinterpret_cast<int2*>(ws + wl.spans), P.hdr);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
     g_last_launches += 1;
+    combine_grid = n_ctas + n_dyn_max;
   }
 
   // One TMA op per page-head (rank-5 view) when head_dim is 128; the rank-4 view otherwise, or if
@@ -340,9 +361,11 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
 
   const bool nt2 = G > 8;
   if (a->head_dim == 128)
-    s = nt2 ? launch<128, 2>(mk, mv, P, grid, di, stream) : launch<128, 1>(mk, mv, P, grid, di, stream);
+    s = nt2 ? launch<128, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
+            : launch<128, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
   else
-    s = nt2 ? launch<64, 2>(mk, mv, P, grid, di, stream) : launch<64, 1>(mk, mv, P, grid, di, stream);
+    s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
+            : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
   if (s == PDATTN_OK) g_last_launches += 2;
   return s;
 }

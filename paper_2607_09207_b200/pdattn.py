@@ -30,7 +30,7 @@ EXPORTS = [
     "pdattn_workspace_size", "pdattn_workspace_init", "pdattn_decode_ex", "pdattn_bind", "pdattn_decode",
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
-    "pdattn_gather_probe", "pdattn_stream_read_probe",
+    "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_set_dynamic_spans",
 ]
 
 
@@ -58,6 +58,18 @@ class Args(ctypes.Structure):
     ]
 
 
+class Plan(ctypes.Structure):
+    _fields_ = [("n_static", ctypes.c_int), ("n_dynamic", ctypes.c_int), ("static_q", ctypes.c_int),
+                ("static_r", ctypes.c_int), ("dynamic_q", ctypes.c_int), ("dynamic_r", ctypes.c_int),
+                ("total_tiles", ctypes.c_int)]
+
+    def span_len(self, i: int) -> int:
+        if i < self.n_static:
+            return self.static_q + (1 if i < self.static_r else 0)
+        j = i - self.n_static
+        return self.dynamic_q + (1 if j < self.dynamic_r else 0)
+
+
 _lib = None
 
 
@@ -79,8 +91,8 @@ def lib():
         L.pdattn_host_staging_size.argtypes = [i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32,
                                          vp, sz, vp, sz, vp]
-        L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i32),
-                                       ctypes.POINTER(i64)]
+        L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(Plan)]
+        L.pdattn_set_dynamic_spans.argtypes = [i32]
         L.pdattn_check.argtypes = [vp, vp]
         L.pdattn_profile_events.argtypes = [vp, vp]
         L.pdattn_gather_probe.argtypes = [ctypes.POINTER(Args), vp]
@@ -196,16 +208,24 @@ def decode_host(q_host, block_table_host, context_lens_host, out_host, k_cache, 
     return st
 
 
-def plan_host(context_lens_host, num_kv_heads, n_ctas):
-    """pdattn_plan_host -> (spans[n_ctas,2], tiles_q, tiles_r, total_tiles).  Needs no GPU."""
+def set_dynamic_spans(per_cta: int):
+    st = lib().pdattn_set_dynamic_spans(per_cta)
+    if st != OK:
+        raise PdattnError(st, "pdattn_set_dynamic_spans")
+
+
+def plan_host(context_lens_host, num_kv_heads, n_ctas, dynamic_per_cta=0, max_spans=None):
+    """pdattn_plan_host -> (spans[n_spans, 2], Plan).  Needs no GPU."""
     lens = np.ascontiguousarray(context_lens_host, dtype=np.int32)
-    spans = np.zeros((n_ctas, 2), dtype=np.int32)
-    tq, tr, tot = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int64(0)
+    if max_spans is None:
+        max_spans = n_ctas * 9
+    spans = np.zeros((max_spans, 2), dtype=np.int32)
+    plan = Plan()
     st = lib().pdattn_plan_host(lens.ctypes.data if lens.size else None, lens.size, num_kv_heads, n_ctas,
-                                spans.ctypes.data, ctypes.byref(tq), ctypes.byref(tr), ctypes.byref(tot))
+                                dynamic_per_cta, max_spans, spans.ctypes.data, ctypes.byref(plan))
     if st != OK:
         raise PdattnError(st, "pdattn_plan_host")
-    return spans, tq.value, tr.value, tot.value
+    return spans[: plan.n_static + plan.n_dynamic].copy(), plan
 
 
 def check(workspace, stream=None) -> int:

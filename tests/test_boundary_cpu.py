@@ -93,14 +93,14 @@ def test_short_form_needs_a_binding():
     assert res == [pdattn.NOT_BOUND]
 
 
-def walk_spans(lens, Hkv, n_ctas):
-    """Re-walk the plan the way a CTA does and return the set of (unit, tile) each CTA covers."""
-    spans, tq, tr, total = pdattn.plan_host(lens, Hkv, n_ctas)
+def walk_spans(lens, Hkv, n_ctas, dyn=8):
+    """Re-walk the plan the way a CTA does and return the list of (unit, tile) each span covers."""
+    spans, plan = pdattn.plan_host(lens, Hkv, n_ctas, dynamic_per_cta=dyn)
     nt = [(int(L) + 63) // 64 if L > 0 else 0 for L in lens]
     cover = []
-    for c in range(n_ctas):
+    for c in range(len(spans)):
         unit, tb = int(spans[c, 0]), int(spans[c, 1])
-        rem = tq + (1 if c < tr else 0)
+        rem = plan.span_len(c)
         mine = []
         while rem > 0 and unit < len(lens) * Hkv:
             n = nt[unit // Hkv]
@@ -113,30 +113,39 @@ def walk_spans(lens, Hkv, n_ctas):
             unit, tb = unit + 1, 0
         assert rem == 0
         cover.append(mine)
-    return cover, total
+    return cover, plan
 
 
 @pytest.mark.parametrize("case", ["cfg1", "cfg2", "cfg5", "zeros", "short", "one"])
-@pytest.mark.parametrize("n_ctas", [1, 7, 148, 320])
-def test_partitioner_covers_every_tile_exactly_once(case, n_ctas):
+@pytest.mark.parametrize("n_ctas", [1, 7, 148])
+@pytest.mark.parametrize("dyn", [0, 8])
+def test_partitioner_covers_every_tile_exactly_once(case, n_ctas, dyn):
     lens, Hkv = {
         "cfg1": (W.config_lengths(1), 1), "cfg2": (W.config_lengths(2), 4), "cfg5": (W.config_lengths(5), 4),
         "zeros": (np.array([0, 5, 0, 0, 300, 0]), 2), "short": (np.arange(1, 40), 3), "one": (np.array([1]), 8),
     }[case]
-    cover, total = walk_spans(lens, Hkv, n_ctas)
+    cover, plan = walk_spans(lens, Hkv, n_ctas, dyn)
     want = [(s * Hkv + g, t) for s, L in enumerate(lens) for g in range(Hkv) for t in range((int(L) + 63) // 64)]
     flat = [x for mine in cover for x in mine]
-    assert total == len(want)
+    assert plan.total_tiles == len(want)
     assert flat == want                      # contiguous, ordered, nothing twice, nothing missing
-    sizes = [len(m) for m in cover]
-    assert max(sizes) - min(sizes) <= 1      # balanced to within one tile
+    assert plan.n_static == n_ctas and len(cover) == plan.n_static + plan.n_dynamic
+    st = [len(m) for m in cover[:n_ctas]]
+    assert max(st) - min(st) <= 1            # static spans balanced to within one tile
+    assert dyn > 0 or plan.n_dynamic == 0
+    if plan.n_dynamic:
+        dy = [len(m) for m in cover[n_ctas:]]
+        assert max(dy) - min(dy) <= 1 and min(dy) >= 3
+        assert plan.n_dynamic <= 8 * n_ctas
+        # static spans cover three quarters, the run-time pool one quarter
+        assert abs(sum(dy) - plan.total_tiles // 4) <= 1
 
 
 def test_partitioner_spreads_the_straggler_phase_over_all_sms():
     """8 sequences x 4 KV heads = 32 units must still occupy all 148 CTAs."""
     lens = W.config_lengths(5)
-    cover, total = walk_spans(lens, 4, 148)
-    assert all(len(m) > 0 for m in cover)
+    cover, plan = walk_spans(lens, 4, 148)
+    assert all(len(m) > 0 for m in cover[:148]) and plan.n_dynamic > 0
     splits = {}
     for c, mine in enumerate(cover):
         for u, _ in mine:
@@ -144,8 +153,21 @@ def test_partitioner_spreads_the_straggler_phase_over_all_sms():
     assert min(len(v) for v in splits.values()) >= 3
 
 
+def test_partitioner_small_batches_use_static_spans_only():
+    cover, plan = walk_spans(W.config_lengths(1), 1, 148)
+    assert plan.n_dynamic == 0 and plan.total_tiles == 8
+    assert [len(m) for m in cover] == [1] * 8 + [0] * 140
+
+
 def test_partitioner_depends_on_lengths_only():
     lens = W.config_lengths(2, num_seqs=32)
-    a = pdattn.plan_host(lens, 4, 148)
-    b = pdattn.plan_host(lens.copy(), 4, 148)
-    assert np.array_equal(a[0], b[0]) and a[1:] == b[1:]
+    a = pdattn.plan_host(lens, 4, 148, 8)
+    b = pdattn.plan_host(lens.copy(), 4, 148, 8)
+    assert np.array_equal(a[0], b[0])
+    assert [getattr(a[1], f) for f, _ in a[1]._fields_] == [getattr(b[1], f) for f, _ in b[1]._fields_]
+
+
+def test_partitioner_respects_max_spans():
+    lens = W.config_lengths(2)
+    spans, plan = pdattn.plan_host(lens, 4, 148, 8, max_spans=200)
+    assert plan.n_static == 148 and 0 < plan.n_dynamic <= 52

@@ -402,3 +402,24 @@ def test_workspace_too_small_and_misaligned_are_rejected_on_gpu():
     st = pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws[16:],
                           check=False)
     assert st == pdattn.MISALIGNED
+
+
+@pytest.fixture
+def runtime_spans():
+    pdattn.set_dynamic_spans(8)
+    yield
+    pdattn.set_dynamic_spans(0)
+
+
+@pytest.mark.parametrize("cfg,num_seqs,len_div", [(2, 48, 1), (5, 2, 2), (3, 24, 2)])
+def test_runtime_span_scheduling_is_correct_and_deterministic(runtime_spans, cfg, num_seqs, len_div):
+    """With run-time spans the CTA that processes a span varies from run to run; the output bits must not."""
+    w = W.make_config(cfg, device=DEV, num_seqs=num_seqs, len_div=len_div)
+    _, plan = pdattn.plan_host(w.context_lens_host, w.num_kv_heads, 148, dynamic_per_cta=8)
+    assert plan.n_dynamic > 0
+    out = check_against_oracle(w, f"config {cfg} with run-time spans")
+    for _ in range(4):
+        again, st = run(w)
+        assert st == pdattn.OK and torch.equal(out, again)
+    dev_plan, st = run(w, use_host_lens=False)
+    assert st == pdattn.OK and torch.equal(out, dev_plan)
