@@ -169,6 +169,33 @@ pdattn_status pdattn_set_dynamic_spans(int per_cta);
 pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream);
 
 /*
+ * Decode step for callers that cannot give the library any scratch memory and cannot let it
+ * allocate.  (The paper has no counterpart for this entry point; it is a deployment variant of
+ * pdattn_decode_ex.)  Meant for hosts where every byte of device memory was handed to the
+ * engine's KV-cache pool at start-up, so a cudaMalloc at decode time fails or fragments the pool,
+ * and for plug-in contexts whose owner forbids device allocation inside the step function.
+ *
+ * Same computation, same arguments and same results as pdattn_decode_ex, except:
+ *   - args->workspace and args->workspace_bytes are ignored.  The partial (m, l, acc) triples, the
+ *     per-span records and the error word live in a 4 MiB array built into the library image; every
+ *     GPU that loads the library holds that array until the process exits.
+ *   - Limits: num_seqs <= 65536 and the layout must fit the 4 MiB (it does for every supported
+ *     head configuration on a B200); otherwise PDATTN_WORKSPACE_TOO_SMALL is returned and
+ *     pdattn_last_cuda_error() says how many bytes were needed.  Spans are always static.
+ *   - status_out (DEVICE int32, optional): receives 0, or the error bits of this call
+ *     (1 = a used block_table entry was out of range, 2 = a bounded wait expired), on `stream`.
+ *   - The first call on a device looks up the array's device address (one-time set-up, no
+ *     allocation); make that first call before any stream capture is begun.
+ *   - All calls on a device share the one array and it keeps the previous call's contents (the
+ *     library clears the words that must start at zero).  Two calls that overlap on the GPU, from
+ *     different streams or threads, race on it: serialise them, or use pdattn_decode_ex with
+ *     separate workspaces.
+ * Calls no cudaMalloc / cudaFree and no allocating library routine.
+ */
+pdattn_status pdattn_decode_static_scratch(const pdattn_args* args, int32_t* status_out,
+                                           pdattn_stream_t stream);
+
+/*
  * Measurement aid (roofline accounting of the split-KV kernel, Appendix A.1.2's history-token
  * term being the bytes it moves): while two CUDA events are registered on this thread, every
  * decode call records `start` just before and `stop` just after the split-KV kernel on its

@@ -497,6 +497,152 @@ pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream_) {
   return PDATTN_BAD_PAGE_INDEX;
 }
 
+}  // extern "C"
+
+// ---- decode without any caller-provided or allocated scratch -----------------------------------
+// The scratch of this variant is a fixed array inside the library image.  Every GPU that loads the
+// library carries it until the process exits, and every call on a device shares it.
+#define PDATTN_STATIC_SCRATCH_BYTES (4u << 20)
+#define PDATTN_STATIC_SCRATCH_MAX_SEQS 65536
+static __device__ __align__(256) unsigned char g_static_scratch[PDATTN_STATIC_SCRATCH_BYTES];
+
+namespace {
+void* g_static_scratch_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+std::mutex g_static_scratch_mu;
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can
+// use; the device address has to be asked for, once per device, with that device current.
+pdattn_status static_scratch_address(int dev, uint8_t** out) {
+  std::lock_guard<std::mutex> lk(g_static_scratch_mu);
+  if (!g_static_scratch_ptr[dev]) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return cuda_fail("cudaGetSymbolAddress(static scratch)", e);
+    if (!p || (reinterpret_cast<uintptr_t>(p) & 255)) {
+      snprintf(g_cuda_err, sizeof g_cuda_err, "static scratch address is null or misaligned");
+      return PDATTN_CUDA_ERROR;
+    }
+    g_static_scratch_ptr[dev] = p;
+  }
+  *out = static_cast<uint8_t*>(g_static_scratch_ptr[dev]);
+  return PDATTN_OK;
+}
+}  // namespace
+
+extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int32_t* status_out,
+                                                      pdattn_stream_t stream_) {
+  g_last_launches = 0;
+  if (!a) return PDATTN_INVALID_ARG;
+  pdattn_status s = check_shape(a->num_seqs, a->num_q_heads, a->num_kv_heads, a->head_dim, a->block_size);
+  if (s != PDATTN_OK) return s;
+  if (a->num_seqs == 0) return PDATTN_OK;
+  if (!a->q || !a->k_cache || !a->v_cache || !a->out || !a->block_table || !a->context_lens) return PDATTN_INVALID_ARG;
+  if (a->max_blocks_per_seq <= 0 || a->num_blocks <= 0) return PDATTN_INVALID_ARG;
+  if (a->kv_block_stride <= 0 || a->kv_head_stride <= 0 || a->kv_token_stride < a->head_dim) return PDATTN_INVALID_ARG;
+  if ((a->kv_block_stride | a->kv_head_stride | a->kv_token_stride) % 8 != 0) return PDATTN_UNSUPPORTED;
+  auto mis = [](const void* p, size_t al) { return (reinterpret_cast<uintptr_t>(p) & (al - 1)) != 0; };
+  if (mis(a->q, 16) || mis(a->k_cache, 16) || mis(a->v_cache, 16) || mis(a->out, 16)) return PDATTN_MISALIGNED;
+
+  int dev = 0;
+  DevInfo* di = nullptr;
+  s = device_info(&dev, &di);
+  if (s != PDATTN_OK) return s;
+  int n_ctas = di->sm_count;
+  if (n_ctas > 256) n_ctas = 256;
+
+  // layout inside the static array: header | spans | records | prefix sums | partial slots
+  const int G = a->num_q_heads / a->num_kv_heads;
+  const size_t slot_bytes = static_cast<size_t>(G > 8 ? 16 : 8) * (a->head_dim + 2) * 4;
+  const size_t off_spans = 256;
+  const size_t off_rec = off_spans + align_up(static_cast<size_t>(n_ctas) * sizeof(int2), 256);
+  const size_t off_prefix = off_rec + align_up(static_cast<size_t>(n_ctas) * sizeof(int4), 256);
+  const size_t off_part = off_prefix + align_up(static_cast<size_t>(a->num_seqs + 1) * 4, 256);
+  const size_t need = off_part + align_up(static_cast<size_t>(n_ctas) * 2 * slot_bytes, 256);
+  if (a->num_seqs > PDATTN_STATIC_SCRATCH_MAX_SEQS || need > PDATTN_STATIC_SCRATCH_BYTES) {
+    snprintf(g_cuda_err, sizeof g_cuda_err,
+             "pdattn_decode_static_scratch: %d sequences need %zu bytes of scratch; the built-in array holds %u "
+             "bytes and at most %d sequences",
+             a->num_seqs, need, PDATTN_STATIC_SCRATCH_BYTES, PDATTN_STATIC_SCRATCH_MAX_SEQS);
+    return PDATTN_WORKSPACE_TOO_SMALL;
+  }
+  uint8_t* ws = nullptr;
+  s = static_scratch_address(dev, &ws);
+  if (s != PDATTN_OK) return s;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+
+  // The array still holds whatever the previous call left: the error word and the span counter
+  // must start at zero; everything else is written before it is read.
+  cudaError_t e = cudaMemsetAsync(ws, 0, 256, stream);
+  if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync(static scratch header)", e);
+
+  DecodeParams P;
+  P.q = static_cast<const __nv_bfloat16*>(a->q);
+  P.out = static_cast<__nv_bfloat16*>(a->out);
+  P.block_table = a->block_table;
+  P.context_lens = a->context_lens;
+  P.hdr = reinterpret_cast<WsHeader*>(ws);
+  P.spans_ws = reinterpret_cast<const int2*>(ws + off_spans);
+  P.rec = reinterpret_cast<int4*>(ws + off_rec);
+  P.partials = reinterpret_cast<float*>(ws + off_part);
+  P.S = a->num_seqs;
+  P.Hq = a->num_q_heads;
+  P.Hkv = a->num_kv_heads;
+  P.G = G;
+  P.MB = a->max_blocks_per_seq;
+  P.NB = a->num_blocks;
+  P.scale_log2 = a->scale * 1.4426950408889634f;
+  P.use_ws_plan = 0;
+  P.box5d = 0;
+  int grid = n_ctas, combine_grid = n_ctas, n_spans_host = -1;
+  if (a->context_lens_host) {
+    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, 0, n_ctas,
+                    reinterpret_cast<int32_t*>(P.spans), &P.plan))
+      return PDATTN_INVALID_ARG;
+    if (P.plan.total < n_ctas) grid = P.plan.total > 0 ? P.plan.total : 1;
+    n_spans_host = grid;
+    combine_grid = grid;
+  } else {
+    P.use_ws_plan = 1;
+    memset(&P.plan, 0, sizeof P.plan);
+    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas, 0,
+                                         reinterpret_cast<int32_t*>(ws + off_prefix),
+                                         reinterpret_cast<int2*>(ws + off_spans), P.hdr);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
+    g_last_launches += 1;
+  }
+  CUtensorMap mk, mv;
+  int rank = a->head_dim == 128 ? 5 : 4;
+  s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+               a->kv_head_stride, a->kv_token_stride, rank, &mk);
+  if (s != PDATTN_OK && rank == 5) {
+    rank = 4;
+    s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+                 a->kv_head_stride, a->kv_token_stride, rank, &mk);
+  }
+  if (s != PDATTN_OK) return s;
+  s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+               a->kv_head_stride, a->kv_token_stride, rank, &mv);
+  if (s != PDATTN_OK) return s;
+  P.box5d = rank == 5;
+  const bool nt2 = G > 8;
+  if (a->head_dim == 128)
+    s = nt2 ? launch<128, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
+            : launch<128, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+  else
+    s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
+            : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+  if (s != PDATTN_OK) return s;
+  g_last_launches += 2;
+  if (status_out) {
+    e = cudaMemcpyAsync(status_out, ws, 4, cudaMemcpyDeviceToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail("cudaMemcpyAsync(status_out)", e);
+  }
+  return PDATTN_OK;
+}
+
+extern "C" {
+
 pdattn_status pdattn_gather_probe(const pdattn_args* args, pdattn_stream_t stream) {
   g_probe_mode = true;
   pdattn_status s = pdattn_decode_ex(args, stream);

@@ -31,6 +31,7 @@ EXPORTS = [
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_set_dynamic_spans",
+    "pdattn_decode_static_scratch",
 ]
 
 
@@ -93,6 +94,7 @@ def lib():
                                          vp, sz, vp, sz, vp]
         L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(Plan)]
         L.pdattn_set_dynamic_spans.argtypes = [i32]
+        L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
         L.pdattn_check.argtypes = [vp, vp]
         L.pdattn_profile_events.argtypes = [vp, vp]
         L.pdattn_gather_probe.argtypes = [ctypes.POINTER(Args), vp]
@@ -157,6 +159,33 @@ def decode_ex(q, k_cache, v_cache, block_table, context_lens, scale, out, worksp
     st = fn(ctypes.byref(a), _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_gather_probe" if probe else "pdattn_decode_ex")
+    return st
+
+
+def decode_static_scratch(q, k_cache, v_cache, block_table, context_lens, scale, out,
+                          context_lens_host: Optional[np.ndarray] = None, status_out: Optional[torch.Tensor] = None,
+                          stream=None, check: bool = True) -> int:
+    """pdattn_decode_static_scratch: the decode step on the library's built-in scratch array, for callers
+    that can neither provide a workspace nor let the library allocate one.  status_out: optional int32
+    device tensor of one element that receives this call's error bits."""
+    S, Hq, d = q.shape
+    NB, Hkv, bs, _ = k_cache.shape
+    a = Args()
+    a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr()
+    a.block_table, a.context_lens = block_table.data_ptr(), context_lens.data_ptr()
+    keep = None
+    if context_lens_host is not None:
+        keep = np.ascontiguousarray(context_lens_host, dtype=np.int32)
+        a.context_lens_host = keep.ctypes.data
+    a.num_seqs, a.num_q_heads, a.num_kv_heads, a.head_dim, a.block_size = S, Hq, Hkv, d, bs
+    a.max_blocks_per_seq = block_table.shape[1] if block_table.dim() == 2 else 0
+    a.num_blocks = NB
+    a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
+    a.scale = float(scale)
+    st = lib().pdattn_decode_static_scratch(ctypes.byref(a), status_out.data_ptr() if status_out is not None else None,
+                                            _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_static_scratch")
     return st
 
 
