@@ -164,6 +164,15 @@ class Workload:
             q=self.q.to(device), k_cache=self.k_cache.to(device), v_cache=self.v_cache.to(device),
             block_table=self.block_table.to(device), context_lens=self.context_lens.to(device))
 
+    def shard(self, idx) -> "Workload":
+        """The sub-batch of the sequences in idx (a rank's share): rows of q / block_table / context_lens
+        are selected, the page pools stay whole (a rank only ever reads the pages its rows reference)."""
+        idx = np.asarray(idx, dtype=np.int64)
+        t = torch.from_numpy(idx).to(self.q.device)
+        return dataclasses.replace(
+            self, q=self.q[t].contiguous(), block_table=self.block_table[t].contiguous(),
+            context_lens=self.context_lens[t].contiguous(), context_lens_host=self.context_lens_host[idx].copy())
+
     def clone(self) -> "Workload":
         return dataclasses.replace(
             self, q=self.q.clone(), k_cache=self.k_cache.clone(), v_cache=self.v_cache.clone(),
