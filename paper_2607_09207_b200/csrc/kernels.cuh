@@ -34,7 +34,7 @@ constexpr int TILE = kTileTokens;                // tokens per pipeline stage
 constexpr int MAX_SPANS = 2048;                  // spans per call (static + run-time); sizes the workspace
 constexpr int MAX_PARAM_SPANS = 1536;            // spans that can travel in kernel parameters
 constexpr int SPAN_QUEUE = 32;                   // in-CTA queue of run-time span ids
-constexpr int MAX_STAGES = 12;
+constexpr int MAX_STAGES = 14;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2 };
@@ -121,6 +121,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
       : "memory");
 }
+// Untiled bulk copy global -> shared (16-byte aligned addresses, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
 // 5-D variant: (dim-in-half, slot, half, kv head, page)
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, int c4,
                                             uint32_t bar) {
@@ -180,34 +185,29 @@ struct Cfg {
   static constexpr int HP = 8 * NT;                    // padded query heads per KV head
   static constexpr int KSTEPS = D / 16;
   // Consumer warp w owns the tiles with index = w (mod NCW) and tile i lives in ring slot i mod
-  // NSTAGES.  NSTAGES must be a multiple of NCW: then the tile that used a slot one ring turn
-  // earlier belonged to the same warp, so a warp can never wait on a slot's next mbarrier phase
-  // while the previous one is still pending (a parity wait cannot tell those apart).
-  static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the scratch stores conflict-free
+  // NSTAGES.  NSTAGES is a multiple of NCW: then the tile that used a slot one ring turn earlier
+  // belonged to the same warp, so a warp can never wait on a slot's next mbarrier phase while the
+  // previous one is still pending (a parity wait cannot tell those apart).  Producer warps do not
+  // have that property (tile i is issued by producer i mod NPW); they check the previous user's
+  // progress word instead.
+  // There is no separate merge scratch: at the end of a piece the ring slot of the piece's last
+  // tile is kept back and the warps exchange their accumulators through it.
+  static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the parked stores conflict-free
   static constexpr int SMEM_MAX = 232448;              // 227 KB
-  static constexpr int CTRL_BYTES = 512;
-  static constexpr int fixed_bytes(int ncw) { return 1024 + ncw * HP * ACC_STRIDE * 4 + ncw * HP * 2 * 4 + CTRL_BYTES; }
-  static constexpr int stages_for(int ncw) {
-    int fit = (SMEM_MAX - fixed_bytes(ncw)) / STAGE_BYTES;
-    if (fit > MAX_STAGES) fit = MAX_STAGES;
-    return fit / ncw * ncw;
-  }
-  static constexpr int pick_ncw() {   // the requested warp count, lowered until a ring of >= NCW stages fits
-    int ncw = PDATTN_NCW;
-    while (ncw > 1 && stages_for(ncw) < ncw) --ncw;
-    return ncw;
-  }
-  static constexpr int NCW = pick_ncw();                               // consumer warps
-  static constexpr int NSTAGES = stages_for(NCW);
-  static constexpr int NCT = NCW * 32;                                 // consumer threads
-  static constexpr int NPW = (NSTAGES % PDATTN_NPW == 0) ? PDATTN_NPW : 1;   // producer warps
-  static constexpr int NTHREADS = NCT + 32 * NPW;
-  static constexpr int SCRATCH_BYTES = NCW * HP * ACC_STRIDE * 4;
+  static constexpr int CTRL_BYTES = 640;
+  static constexpr int NCW = PDATTN_NCW;                               // consumer warps
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
-  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + SCRATCH_BYTES + ML_BYTES + CTRL_BYTES;
+  static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged by producer 0
+  static constexpr int Q_BYTES = HP * D * 2;           // one slot: the packed query heads of one KV head
+  static constexpr int NSTAGES_FIT = (SMEM_MAX - 1024 - QSLOTS * Q_BYTES - ML_BYTES - CTRL_BYTES) / STAGE_BYTES;
+  static constexpr int NSTAGES = (NSTAGES_FIT > MAX_STAGES ? MAX_STAGES : NSTAGES_FIT) / NCW * NCW;
+  static constexpr int NCT = NCW * 32;                                 // consumer threads
+  static constexpr int NPW = PDATTN_NPW;                               // producer warps
+  static constexpr int NTHREADS = NCT + 32 * NPW;
+  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + QSLOTS * Q_BYTES + ML_BYTES + CTRL_BYTES;
   static constexpr int SLOT_FLOATS = HP * (D + 2);     // one partial: m[HP], l[HP], acc[HP][D]
-  static_assert(NSTAGES >= NCW && NSTAGES % NCW == 0 && NSTAGES <= MAX_STAGES, "ring/warp mapping");
-  static_assert(NSTAGES % NPW == 0, "a slot must always be refilled by the same producer warp");
+  static_assert(NSTAGES >= NCW && NSTAGES % NCW == 0, "ring/warp mapping");
+  static_assert(HP * ACC_STRIDE * 4 <= STAGE_BYTES, "a parked accumulator must fit one stage");
   static_assert(DYN_BYTES <= SMEM_MAX, "shared memory");
   static_assert(TILE % BS == 0 && BS % 16 == 0, "block size");
 };
@@ -220,8 +220,11 @@ struct Ctrl {                 // lives in the CTRL_BYTES area
   int32_t sq_pub;             // number of run-time span ids published so far
   int32_t sq_id[SPAN_QUEUE];  // k-th id (k >= 1) at [(k-1) % SPAN_QUEUE]; -1 = no more spans
   int32_t sq_tag[SPAN_QUEUE]; // k, to detect an overwritten entry
+  int32_t prod_last[4];       // per producer warp: index of the last tile it issued (-1 = none)
+  uint64_t q_full[4];         // query slot q holds the rows of piece p, p mod 4 == q
+  uint64_t q_empty[4];        // ... and every consumer warp has copied them to registers
 };
-static_assert(sizeof(Ctrl) <= 512, "control block");
+static_assert(sizeof(Ctrl) <= 640, "control block");
 
 // ------------------------------------------------------------------------------------------
 // The walk over a span: pieces = (unit, tile range) in order.  Every warp runs the same walk.
@@ -232,10 +235,15 @@ struct Piece {
 struct Walker {
   const int32_t* ctx;
   int Hkv, nunits, unit, tb, rem;
+  int pf_unit = -1, pf_L = 0;   // context length of the following unit, loaded one piece early
   __device__ __forceinline__ bool next(Piece& p) {
     while (rem > 0 && unit < nunits) {
       const int s = unit / Hkv;
-      const int L = __ldg(ctx + s);
+      const int L = (unit == pf_unit) ? pf_L : __ldg(ctx + s);
+      if (unit + 1 < nunits) {
+        pf_unit = unit + 1;
+        pf_L = __ldg(ctx + (unit + 1) / Hkv);
+      }
       const int nt = L > 0 ? (L + TILE - 1) / TILE : 0;
       if (tb >= nt) {
         ++unit;
@@ -470,8 +478,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   const uint32_t ring = raw + pad;                                        // NST stages, 1024-aligned
-  float* scratch = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);  // [NCW][HP][ACC_STRIDE]
-  float* sm_m = scratch + NCW * C::HP * C::ACC_STRIDE;                     // [NCW][HP]
+  const uint32_t qbuf = ring + NST * C::STAGE_BYTES;                       // [QSLOTS][HP][D] bf16
+  float* sm_m = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES + C::QSLOTS * C::Q_BYTES);   // [NCW][HP]
   float* sm_l = sm_m + NCW * C::HP;                                        // [NCW][HP]
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm_l + NCW * C::HP);
 
@@ -487,6 +495,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
     ctrl->abort = 0;
     ctrl->sq_pub = 0;
+    for (int i = 0; i < 4; ++i) ctrl->prod_last[i] = -1;
+    for (int i = 0; i < C::QSLOTS; ++i) {
+      mbar_init(smem_u32(&ctrl->q_full[i]), 1);
+      mbar_init(smem_u32(&ctrl->q_empty[i]), NCW);
+    }
     fence_mbar_init();
   }
   __syncthreads();
@@ -494,6 +507,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const PlanParams pp = P.use_ws_plan ? P.hdr->plan : P.plan;
   const int nunits = P.S * P.Hkv;
   int it = 0;        // tile counter within this CTA: tile `it` uses ring slot it % NST
+  int pcnt = 0;      // piece counter within this CTA: piece p's query rows use query slot p % QSLOTS
   bool aborted = false;
 
   if (warp >= NCW) {
@@ -514,6 +528,22 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       Walker walk{P.context_lens, P.Hkv, nunits, sp.x, sp.y, span_len(pp, span)};
       Piece pc;
       while (!aborted && walk.next(pc)) {
+        if (!PROBE && pw == 0) {
+          // stage this piece's packed query rows; the consumers reach the piece several tiles later
+          const int qs = pcnt % C::QSLOTS;
+          const uint32_t qphase = (pcnt / C::QSLOTS) & 1;
+          if (!mbar_wait(smem_u32(&ctrl->q_empty[qs]), qphase ^ 1u)) {
+            aborted = true;
+            break;
+          }
+          if (lane == 0) {
+            const uint32_t bytes = static_cast<uint32_t>(P.G) * D * 2;
+            const uint32_t qb = smem_u32(&ctrl->q_full[qs]);
+            mbar_arrive_expect_tx(qb, bytes);
+            bulk_load(qbuf + qs * C::Q_BYTES, P.q + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G) * D, bytes, qb);
+          }
+        }
+        ++pcnt;
         const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
         const int npages = (pc.L + BS - 1) / BS;
         const int pbase = pc.tb * C::PAGES;
@@ -530,6 +560,22 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           if (C::NPW > 1 && it % C::NPW != pw) continue;
           const int slot = it % NST;
           const uint32_t phase = (it / NST) & 1;
+          if (NST % C::NPW != 0 && it >= NST) {
+            // the slot's previous tile was issued by another producer: make sure it has been, so
+            // that the parity wait below refers to that tile's release and not to an older one
+            const int prev = it - NST;
+            const int32_t* pl = &ctrl->prod_last[prev % C::NPW];
+            if (ld_acquire_shared(pl) < prev) {
+              const unsigned long long t0 = globaltimer_ns();
+              while (ld_acquire_shared(pl) < prev) {
+                if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                  aborted = true;
+                  break;
+                }
+              }
+              if (aborted) break;
+            }
+          }
           if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) {
             aborted = true;
             break;
@@ -558,6 +604,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
           }
           any_bad |= (badmask != 0);
+          if (NST % C::NPW != 0) {
+            __syncwarp();
+            if (lane == 0) st_release_shared(&ctrl->prod_last[pw], it);
+          }
         }
       }
       if (aborted) break;
@@ -605,20 +655,40 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     while (walk.next(pc)) {
       const int w_first = it % NCW;   // warp that takes this piece's first tile
-      // ---- packed query rows of this KV head as MMA B fragments
+      // ---- packed query rows of this KV head as MMA B fragments, from the staged copy
       uint32_t qf[NT][D / 16][2];
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        const int head = nt * 8 + hq0;
-        const bool live = head < P.G;
-        const uint32_t* qp = reinterpret_cast<const uint32_t*>(
-            P.q + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + (live ? head : 0)) * D);
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          qf[nt][kk][0] = live ? __ldg(qp + (kk * 16 + qcol) / 2) : 0u;
-          qf[nt][kk][1] = live ? __ldg(qp + (kk * 16 + 8 + qcol) / 2) : 0u;
+      if constexpr (!PROBE) {
+        const int qs = pcnt % C::QSLOTS;
+        const uint32_t qphase = (pcnt / C::QSLOTS) & 1;
+        bool have_q = !aborted;
+        if (have_q && !mbar_wait(smem_u32(&ctrl->q_full[qs]), qphase)) {
+          have_q = false;
+          aborted = true;
+          if (lane == 0) {
+            atomicOr(&P.hdr->err, ERR_TIMEOUT);
+            atomicExch(&ctrl->abort, 1u);
+          }
         }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const int head = nt * 8 + hq0;
+          const bool live = have_q && head < P.G;
+          const uint32_t qa = qbuf + qs * C::Q_BYTES + (live ? head : 0) * (D * 2) + qcol * 2;
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            uint32_t v0 = 0u, v1 = 0u;
+            if (live) {
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v0) : "r"(qa + kk * 32) : "memory");
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v1) : "r"(qa + kk * 32 + 16) : "memory");
+            }
+            qf[nt][kk][0] = v0;
+            qf[nt][kk][1] = v1;
+          }
+        }
+        __syncwarp();
+        if (have_q && lane == 0) mbar_arrive(smem_u32(&ctrl->q_empty[qs]));
       }
+      ++pcnt;
       float acc[NT][D / 16][4];
       float m[NT][2], l[NT][2];
 #pragma unroll
@@ -629,6 +699,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         for (int jm = 0; jm < D / 16; ++jm) acc[nt][jm][0] = acc[nt][jm][1] = acc[nt][jm][2] = acc[nt][jm][3] = 0.f;
       }
 
+      // The slot of the piece's last tile is kept back after it has been consumed: it is where the
+      // warps exchange their accumulators for the merge.  Every other slot is released at once, so
+      // the producers keep streaming the next piece meanwhile.
+      const int n_piece = pc.te - pc.tb;              // tiles in this piece
+      const int it_last = it + n_piece - 1;           // ring index of the piece's last tile
+      const int park_slot = it_last % NST;
+      const int w_last = it_last % NCW;               // the warp that consumes it
       for (int t = pc.tb; t < pc.te; ++t, ++it) {
         if (it % NCW != warp) continue;
         if (!aborted && *reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) aborted = true;
@@ -656,13 +733,18 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
+        if ((PROBE || t != pc.te - 1) && lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
       }
 
       const bool complete = (pc.tb == 0 && pc.te == pc.nt);
       const int slot_idx = piece_idx == 0 ? 0 : 1;
       if constexpr (!PROBE) {
-        // ---- merge the NCW warp states of this piece
+        // ---- merge the warp states of this piece
+        constexpr int ACC_FLOATS = C::HP * C::ACC_STRIDE;                 // one parked accumulator
+        constexpr int WPR = C::STAGE_BYTES / (ACC_FLOATS * 4) < NCW ? C::STAGE_BYTES / (ACC_FLOATS * 4) : NCW;
+        constexpr int ROUNDS = (NCW + WPR - 1) / WPR;                     // warps are merged WPR at a time
+        int pos = warp - w_first;                      // this warp's tiles are residue class `pos` of the piece
+        if (pos < 0) pos += NCW;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -673,69 +755,103 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             v += __shfl_xor_sync(0xffffffffu, v, 16);
             l[nt][e] = v;
           }
-        {
-          float* my = scratch + warp * C::HP * C::ACC_STRIDE;
-          const int drow = lane >> 2;
+        if (lane < 4) {
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
             const int h0 = nt * 8 + qcol;
-#pragma unroll
-            for (int jm = 0; jm < D / 16; ++jm) {
-              my[h0 * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][0];
-              my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][1];
-              my[h0 * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][2];
-              my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][3];
-            }
-            if (lane < 4) {
-              sm_m[warp * C::HP + h0] = m[nt][0];
-              sm_m[warp * C::HP + h0 + 1] = m[nt][1];
-              sm_l[warp * C::HP + h0] = l[nt][0];
-              sm_l[warp * C::HP + h0 + 1] = l[nt][1];
-            }
+            sm_m[pos * C::HP + h0] = m[nt][0];
+            sm_m[pos * C::HP + h0 + 1] = m[nt][1];
+            sm_l[pos * C::HP + h0] = l[nt][0];
+            sm_l[pos * C::HP + h0 + 1] = l[nt][1];
           }
         }
-        bar_consumers<NCT>();
+        bar_consumers<NCT>();   // the last tile has been consumed: its slot is free for the exchange
+        float* park = reinterpret_cast<float*>(smem + park_slot * C::STAGE_BYTES);
+        const int n_cls = n_piece < NCW ? n_piece : NCW;   // residue classes that hold tiles
         float* part = P.partials + (static_cast<int64_t>(span) * 2 + slot_idx) * C::SLOT_FLOATS;
-        for (int idx = ct; idx < C::HP * (D / 4); idx += NCT) {
-          const int h = idx / (D / 4);
-          const int dq = idx % (D / 4);
+        constexpr int ITEMS = C::HP * (D / 4);
+        constexpr int IPT = (ITEMS + NCT - 1) / NCT;        // merge items per thread
+        float Mu_r[IPT], Ls_r[IPT], M_r[IPT];
+        float4 a_r[IPT];
+#pragma unroll
+        for (int i = 0; i < IPT; ++i) {
+          const int idx = ct + i * NCT;
+          const int h = (idx < ITEMS ? idx : 0) / (D / 4);
           float M = NEG_INF;
+          for (int c = 0; c < n_cls; ++c) M = fmaxf(M, sm_m[c * C::HP + h]);
+          M_r[i] = M;
+          Mu_r[i] = (M == NEG_INF) ? 0.f : M;
+          Ls_r[i] = 0.f;
+          a_r[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
 #pragma unroll
-          for (int w = 0; w < NCW; ++w) M = fmaxf(M, sm_m[w * C::HP + h]);
-          const float Mu = (M == NEG_INF) ? 0.f : M;
-          float Ls = 0.f;
-          float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-          // Sum in the order of the tiles' residue classes within the piece, not of warp numbers:
-          // which warp holds which class depends on what this CTA processed before.
+        for (int q = 0; q < ROUNDS; ++q) {
+          if (pos >= q * WPR && pos < (q + 1) * WPR && pos < n_cls) {
+            float* my = park + (pos - q * WPR) * ACC_FLOATS;
+            const int drow = lane >> 2;
 #pragma unroll
-          for (int r = 0; r < NCW; ++r) {
-            int w = w_first + r;
-            if (w >= NCW) w -= NCW;
-            const float f = fast_exp2(sm_m[w * C::HP + h] - Mu);
-            Ls += sm_l[w * C::HP + h] * f;
-            const float4 v = *reinterpret_cast<const float4*>(scratch + (w * C::HP + h) * C::ACC_STRIDE + dq * 4);
-            a.x += v.x * f;
-            a.y += v.y * f;
-            a.z += v.z * f;
-            a.w += v.w * f;
+            for (int nt = 0; nt < NT; ++nt) {
+              const int h0 = nt * 8 + qcol;
+#pragma unroll
+              for (int jm = 0; jm < D / 16; ++jm) {
+                my[h0 * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][0];
+                my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow] = acc[nt][jm][1];
+                my[h0 * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][2];
+                my[(h0 + 1) * C::ACC_STRIDE + jm * 16 + drow + 8] = acc[nt][jm][3];
+              }
+            }
           }
-          if (complete) {
-            if (h < P.G) {
-              const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
-              uint2 o;
-              o.x = pack_bf16x2(a.x * inv, a.y * inv);
-              o.y = pack_bf16x2(a.z * inv, a.w * inv);
-              *reinterpret_cast<uint2*>(P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + h) * D + dq * 4) = o;
+          bar_consumers<NCT>();
+          // residue classes in ascending order: the sum does not depend on which warp held which class
+#pragma unroll
+          for (int i = 0; i < IPT; ++i) {
+            const int idx = ct + i * NCT;
+            if (idx < ITEMS) {
+              const int h = idx / (D / 4);
+              const int dq = idx % (D / 4);
+              for (int c = q * WPR; c < (q + 1) * WPR && c < n_cls; ++c) {
+                const float f = fast_exp2(sm_m[c * C::HP + h] - Mu_r[i]);
+                Ls_r[i] += sm_l[c * C::HP + h] * f;
+                const float4 v =
+                    *reinterpret_cast<const float4*>(park + (c - q * WPR) * ACC_FLOATS + h * C::ACC_STRIDE + dq * 4);
+                a_r[i].x += v.x * f;
+                a_r[i].y += v.y * f;
+                a_r[i].z += v.z * f;
+                a_r[i].w += v.w * f;
+              }
             }
-          } else {
-            if (dq == 0) {
-              part[h] = M;
-              part[C::HP + h] = Ls;
+          }
+          bar_consumers<NCT>();   // everyone has read this round's accumulators
+        }
+        if (warp == w_last && !aborted) {
+          fence_proxy_async();    // our stores into the slot are ordered before the TMA write that refills it
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[park_slot]));
+        }
+#pragma unroll
+        for (int i = 0; i < IPT; ++i) {
+          const int idx = ct + i * NCT;
+          if (idx < ITEMS) {
+            const int h = idx / (D / 4);
+            const int dq = idx % (D / 4);
+            const float4 a = a_r[i];
+            if (complete) {
+              if (h < P.G) {
+                const float inv = Ls_r[i] > 0.f ? 1.f / Ls_r[i] : 0.f;
+                uint2 o;
+                o.x = pack_bf16x2(a.x * inv, a.y * inv);
+                o.y = pack_bf16x2(a.z * inv, a.w * inv);
+                *reinterpret_cast<uint2*>(P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + h) * D + dq * 4) = o;
+              }
+            } else {
+              if (dq == 0) {
+                part[h] = M_r[i];
+                part[C::HP + h] = Ls_r[i];
+              }
+              *reinterpret_cast<float4*>(part + 2 * C::HP + h * D + dq * 4) = a;
             }
-            *reinterpret_cast<float4*>(part + 2 * C::HP + h * D + dq * 4) = a;
           }
         }
-        bar_consumers<NCT>();   // scratch is reused by the next piece
       }
       if (piece_idx == 0) {
         first_unit = pc.unit;
