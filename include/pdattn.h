@@ -138,17 +138,18 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
  * The host partitioner on its own (no GPU needed).  It flattens the batch into a stream of
  * 64-token tiles, unit-major (unit = s * num_kv_heads + kv_head; unit u has ceil(L_s / 64)
  * tiles), and cuts it into contiguous spans so that long-tail sequences are spread over all SMs
- * (Section 2.3: a few long responses dominate the rollout): n_static spans, one per CTA, cover
- * the stream; with dynamic_per_cta > 0 they cover only its first three quarters and up to
- * n_ctas * dynamic_per_cta short spans cover the rest, taken at run time by whichever CTA is free.  Span i starts at tile spans[2i+1] of unit spans[2i];
- * static span i holds static_q + (i < static_r) tiles, dynamic span j (index n_static + j) holds
- * dynamic_q + (j < dynamic_r).  spans: HOST int32 [2 * max_spans]; n_static + n_dynamic <=
- * max_spans.  The plan depends on the context lengths only, never on page ids.
+ * (Section 2.3: a few long responses dominate the rollout).  Spans are balanced by cost: a unit
+ * costs its tiles plus 2 for starting it, so a CTA that walks many short sequences gets fewer
+ * tiles than one inside a long sequence.  n_static spans, one per CTA, cover the stream; with
+ * dynamic_per_cta > 0 they cover only its first three quarters (by cost) and up to n_ctas *
+ * dynamic_per_cta short spans cover the rest, taken at run time by whichever CTA is free.
+ * spans: HOST int32 [4 * (max_spans + 1)], one (unit, tile, flat, 0) entry per span plus an end
+ * marker: span i starts at tile `tile` of unit `unit`, which is tile number `flat` of the stream,
+ * and holds flat[i + 1] - flat[i] tiles (possibly none).  n_static + n_dynamic <= max_spans.
+ * The plan depends on the context lengths only, never on page ids.
  */
 typedef struct {
   int n_static, n_dynamic;
-  int static_q, static_r;
-  int dynamic_q, dynamic_r;
   int total_tiles;
 } pdattn_plan;
 pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, int num_kv_heads,

@@ -32,7 +32,7 @@ namespace pdattn {
 
 constexpr int TILE = kTileTokens;                // tokens per pipeline stage
 constexpr int MAX_SPANS = 2048;                  // spans per call (static + run-time); sizes the workspace
-constexpr int MAX_PARAM_SPANS = 1536;            // spans that can travel in kernel parameters
+constexpr int MAX_PARAM_SPANS = 768;             // spans that can travel in kernel parameters
 constexpr int SPAN_QUEUE = 32;                   // in-CTA queue of run-time span ids
 constexpr int MAX_STAGES = 14;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -54,7 +54,7 @@ struct DecodeParams {
   const int32_t* block_table;
   const int32_t* context_lens;
   WsHeader* hdr;
-  const int2* spans_ws;     // spans written by plan_kernel (used when use_ws_plan)
+  const SpanStart* spans_ws;  // spans written by plan_kernel (used when use_ws_plan)
   int4* rec;                // per-span record: (first_unit, first_tile, own_unit, own_slot)
   float* partials;          // [span][2][HP*(D+2)] fp32
   int S, Hq, Hkv, G, MB, NB;
@@ -62,7 +62,7 @@ struct DecodeParams {
   PlanParams plan;          // host plan (ignored when use_ws_plan)
   int use_ws_plan;
   int box5d;                // 1: the tensor maps are 5-D and one TMA op brings a whole page-head
-  int2 spans[MAX_PARAM_SPANS];
+  SpanStart spans[MAX_PARAM_SPANS + 1];
 };
 
 // ------------------------------------------------------------------------------------------
@@ -524,8 +524,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const int j = atomicAdd(&P.hdr->counter, 1);
         nxt = j < pp.n_dyn ? pp.n_static + j : -1;
       }
-      const int2 sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
-      Walker walk{P.context_lens, P.Hkv, nunits, sp.x, sp.y, span_len(pp, span)};
+      const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
+      const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
+      Walker walk{P.context_lens, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
       Piece pc;
       while (!aborted && walk.next(pc)) {
         if (!PROBE && pw == 0) {
@@ -648,8 +649,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
   int span = cta;
   for (int k = 0; span >= 0; ++k) {
-    const int2 sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
-    Walker walk{P.context_lens, P.Hkv, nunits, sp.x, sp.y, span_len(pp, span)};
+    const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
+    const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
+    Walker walk{P.context_lens, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
     Piece pc;
     int first_unit = -1, first_tb = 0, own_unit = -1, own_slot = 0, piece_idx = 0;
 
@@ -890,7 +892,7 @@ stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __rest
 
 // ------------------------------------------------------------------------------------------
 // Split-combine: block i merges the unit that started in span i and ran past its end.  The
-// pieces live in consecutive spans (slot 0 of each follower), merged in ascending token order:
+// pieces live in the following spans (slot 0 of each follower), merged in ascending token order:
 //   M = max m_c;  Lsum = sum l_c 2^(m_c - M);  out = bf16( sum acc_c 2^(m_c - M) / Lsum ).
 // Block 0 also rearms the run-time span counter for the next call.
 // ------------------------------------------------------------------------------------------
@@ -907,14 +909,16 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
   const int4 r = rec[c];
   const int unit = r.z;
   if (unit < 0) return;
-  // followers: spans c+1.. whose first piece continues `unit`
+  // followers: later spans whose first piece continues `unit` (spans without tiles may sit between)
   __shared__ int n_follow;
+  __shared__ int follow[MAX_SPANS];
   if (threadIdx.x == 0) {
     int n = 0;
     for (int cc = c + 1; cc < n_spans; ++cc) {
       const int4 rr = rec[cc];
+      if (rr.x < 0) continue;                 // a span that holds no tile
       if (rr.x != unit || rr.y <= 0) break;
-      ++n;
+      follow[n++] = cc;
     }
     n_follow = n;
   }
@@ -928,14 +932,14 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
     if (h >= G) continue;
     float M = NEG_INF;
     for (int p = 0; p < np; ++p) {
-      const float* part = partials + (static_cast<int64_t>(c + p) * 2 + (p == 0 ? r.w : 0)) * SLOT_FLOATS;
+      const float* part = partials + (p == 0 ? static_cast<int64_t>(c) * 2 + r.w : static_cast<int64_t>(follow[p - 1]) * 2) * SLOT_FLOATS;
       M = fmaxf(M, part[h]);
     }
     const float Mu = (M == NEG_INF) ? 0.f : M;
     float Ls = 0.f;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int p = 0; p < np; ++p) {
-      const float* part = partials + (static_cast<int64_t>(c + p) * 2 + (p == 0 ? r.w : 0)) * SLOT_FLOATS;
+      const float* part = partials + (p == 0 ? static_cast<int64_t>(c) * 2 + r.w : static_cast<int64_t>(follow[p - 1]) * 2) * SLOT_FLOATS;
       const float f = fast_exp2(part[h] - Mu);
       Ls += part[HP + h] * f;
       const float4 v = *reinterpret_cast<const float4*>(part + 2 * HP + h * D + dq * 4);
@@ -953,73 +957,96 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
 }
 
 // ------------------------------------------------------------------------------------------
-// Device twin of the host partitioner (one block).  prefix: [S+1] ints of scratch.
+// Device twin of the host partitioner (one block).  prefix: [2 * (S + 1)] ints of scratch:
+// running cost, then running tile count, per sequence.
 // ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int block_scan_1024(int v, int* warp_sums, int lane, int wid) {
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) warp_sums[wid] = x;
+  __syncthreads();
+  if (wid == 0) {
+    int w = warp_sums[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += y;
+    }
+    warp_sums[lane] = w;
+  }
+  __syncthreads();
+  const int incl = x + (wid > 0 ? warp_sums[wid - 1] : 0);
+  __syncthreads();
+  return incl;
+}
+
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_static, int n_dyn_max,
-            int32_t* __restrict__ prefix, int2* __restrict__ spans, WsHeader* hdr) {
+            int32_t* __restrict__ prefix, SpanStart* __restrict__ spans, WsHeader* hdr) {
   __shared__ int warp_sums[32];
-  __shared__ int carry_s;
+  __shared__ int carry_c, carry_t;
   __shared__ PlanParams pp_s;
+  int32_t* pcost = prefix;
+  int32_t* ptile = prefix + (S + 1);
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   if (tid == 0) {
-    carry_s = 0;
-    prefix[0] = 0;
+    carry_c = carry_t = 0;
+    pcost[0] = ptile[0] = 0;
   }
   __syncthreads();
   for (int base = 0; base < S; base += 1024) {
     const int s = base + tid;
-    int v = 0;
+    int nt = 0;
     if (s < S) {
       const int L = context_lens[s];
-      v = L > 0 ? ((L + TILE - 1) / TILE) * Hkv : 0;
+      nt = L > 0 ? (L + TILE - 1) / TILE : 0;
     }
-    int x = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= o) x += y;
-    }
-    if (lane == 31) warp_sums[wid] = x;
-    __syncthreads();
-    if (wid == 0) {
-      int w = warp_sums[lane];
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, w, o);
-        if (lane >= o) w += y;
-      }
-      warp_sums[lane] = w;
+    const int ic = block_scan_1024(static_cast<int>(seq_cost(nt, Hkv)), warp_sums, lane, wid) + carry_c;
+    const int itl = block_scan_1024(nt * Hkv, warp_sums, lane, wid) + carry_t;
+    if (s < S) {
+      pcost[s + 1] = ic;
+      ptile[s + 1] = itl;
     }
     __syncthreads();
-    const int incl = x + (wid > 0 ? warp_sums[wid - 1] : 0) + carry_s;
-    if (s < S) prefix[s + 1] = incl;
-    __syncthreads();
-    if (tid == 1023) carry_s = incl;
+    if (tid == 1023) {
+      carry_c = ic;
+      carry_t = itl;
+    }
     __syncthreads();
   }
-  const int total = carry_s;
   if (tid == 0) {
-    pp_s = make_plan_params(total, n_static, n_dyn_max);
+    pp_s = make_plan_params(carry_c, carry_t, n_static, n_dyn_max);
     hdr->plan = pp_s;
   }
   __threadfence_block();
   __syncthreads();
   const PlanParams pp = pp_s;
   const int n_spans = pp.n_static + pp.n_dyn;
-  for (int c = tid; c < n_spans; c += 1024) {
-    int2 sp = make_int2(S * Hkv, 0);
-    const int start = span_start(pp, c);
-    if (span_len(pp, c) > 0 && start < total) {
-      int lo = 0, hi = S;   // find s with prefix[s] <= start < prefix[s+1]
+  const int total_cost = static_cast<int>(pp.cost_total);
+  for (int c = tid; c <= n_spans; c += 1024) {
+    SpanStart sp;
+    sp.unit = S * Hkv;
+    sp.tile = 0;
+    sp.flat = pp.total;
+    sp.pad = 0;
+    const int x = static_cast<int>(span_cost_start(pp, c));
+    if (c < n_spans && x < total_cost) {
+      int lo = 0, hi = S;   // find s with pcost[s] <= x < pcost[s+1]
       while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (prefix[mid] <= start) lo = mid; else hi = mid;
+        if (pcost[mid] <= x) lo = mid; else hi = mid;
       }
       const int L = context_lens[lo];
       const int nt = (L + TILE - 1) / TILE;
-      const int off = start - prefix[lo];
-      sp = make_int2(lo * Hkv + off / nt, off % nt);
+      int k, tile;
+      locate_in_seq(x - pcost[lo], nt, &k, &tile);
+      sp.unit = lo * Hkv + k;
+      sp.tile = tile;
+      sp.flat = ptile[lo] + k * nt + tile;
     }
     spans[c] = sp;
   }

@@ -2,10 +2,14 @@
 //
 // The batch is flattened into a stream of fixed-size token tiles, unit-major (unit = sequence *
 // Hkv + kv_head; unit u has ceil(L_s / tile) tiles), and the stream is cut into contiguous spans:
-//   - n_static spans, one per CTA, cover the first three quarters of the stream in equal parts;
-//   - n_dyn small spans cover the rest and are handed out at run time to whichever CTA finishes
-//     first, because SMs do not all stream at the same speed.
-// A long sequence is thereby split over as many CTAs as its share of the bytes warrants, a CTA
+//   - n_static spans, one per CTA;
+//   - optionally n_dyn short spans over the last quarter of the stream, handed out at run time to
+//     whichever CTA finishes first.
+// Spans are balanced by COST, not by tile count: a unit costs its tiles plus kPieceCostTiles for
+// starting it (query rows, page-table row, merge of the warp states, output); a sweep of that
+// constant on the 7B-shaped batch put the best value at 2.  In cost coordinates unit u covers
+// [C_u, C_u + kPieceCostTiles + nt_u); a cut that falls into the start-up part moves to tile 0.
+// A long sequence is thereby split over as many CTAs as its share of the work warrants, a CTA
 // that finishes a short sequence carries on with the next one, and only span boundaries ever
 // produce partial (m, l, acc) triples.  The cut points depend on the context lengths alone, so
 // the result does not depend on which CTA takes which span.
@@ -23,54 +27,63 @@ namespace pdattn {
 #ifndef PDATTN_TILE_TOKENS
 #define PDATTN_TILE_TOKENS 64     // tokens per tile = per pipeline stage of the decode kernel
 #endif
+#ifndef PDATTN_PIECE_COST
+#define PDATTN_PIECE_COST 2       // cost of starting a unit, in tiles
+#endif
 constexpr int kTileTokens = PDATTN_TILE_TOKENS;
+constexpr int kPieceCostTiles = PDATTN_PIECE_COST;
 constexpr int kMaxDynPerCta = 8;      // at most this many run-time spans per CTA
-constexpr int kMinDynTiles = 4;       // a run-time span is never shorter than this
-constexpr int kStaticOnlyBelow = 16;  // fewer tiles per CTA than this: no run-time spans
+constexpr int kMinDynCost = 8;        // a run-time span is never cheaper than this
+constexpr int kStaticOnlyBelow = 16;  // less cost per CTA than this: no run-time spans
 
 struct PlanParams {
   int n_static, n_dyn;
-  int qs, rs;          // static span i holds qs + (i < rs) tiles
-  int qd, rd;          // run-time span j holds qd + (j < rd) tiles
-  int total_static;    // tiles covered by the static spans
-  int total;           // all tiles
+  int64_t cost_static;   // cost covered by the static spans
+  int64_t cost_total;
+  int total;             // all tiles
 };
 
-PDATTN_HD inline PlanParams make_plan_params(int64_t total_tiles, int n_static, int n_dyn_max) {
+// One span: where it starts and the index of its first tile in the flattened stream.  Span i
+// holds spans[i + 1].flat - spans[i].flat tiles, so the table has n_static + n_dyn + 1 entries.
+struct SpanStart {
+  int32_t unit, tile, flat, pad;
+};
+
+PDATTN_HD inline PlanParams make_plan_params(int64_t total_cost, int64_t total_tiles, int n_static, int n_dyn_max) {
   PlanParams p;
   p.n_static = n_static;
+  p.n_dyn = 0;
+  p.cost_total = total_cost;
+  p.cost_static = total_cost;
   p.total = static_cast<int>(total_tiles);
-  int64_t ts = total_tiles, td = 0;
-  p.n_dyn = p.qd = p.rd = 0;
-  if (n_dyn_max > 0 && total_tiles >= static_cast<int64_t>(n_static) * kStaticOnlyBelow) {
-    td = total_tiles / 4;
-    ts = total_tiles - td;
-    int64_t d = (td + n_dyn_max - 1) / n_dyn_max;
-    if (d < kMinDynTiles) d = kMinDynTiles;
-    p.n_dyn = static_cast<int>((td + d - 1) / d);
-    p.qd = static_cast<int>(td / p.n_dyn);
-    p.rd = static_cast<int>(td % p.n_dyn);
+  if (n_dyn_max > 0 && total_cost >= static_cast<int64_t>(n_static) * kStaticOnlyBelow) {
+    const int64_t cd = total_cost / 4;
+    int64_t d = (cd + n_dyn_max - 1) / n_dyn_max;
+    if (d < kMinDynCost) d = kMinDynCost;
+    p.n_dyn = static_cast<int>((cd + d - 1) / d);
+    p.cost_static = total_cost - cd;
   }
-  p.qs = static_cast<int>(ts / n_static);
-  p.rs = static_cast<int>(ts % n_static);
-  p.total_static = static_cast<int>(ts);
   return p;
 }
-PDATTN_HD inline int span_len(const PlanParams& p, int i) {
-  if (i < p.n_static) return p.qs + (i < p.rs ? 1 : 0);
+// cost coordinate at which span i begins (i == n_static + n_dyn gives the end of the stream)
+PDATTN_HD inline int64_t span_cost_start(const PlanParams& p, int i) {
+  if (i <= p.n_static) return p.cost_static * i / p.n_static;
   const int j = i - p.n_static;
-  return p.qd + (j < p.rd ? 1 : 0);
+  return p.cost_static + (p.cost_total - p.cost_static) * j / p.n_dyn;
 }
-// index of the span's first tile in the flattened stream
-PDATTN_HD inline int span_start(const PlanParams& p, int i) {
-  if (i < p.n_static) return i * p.qs + (i < p.rs ? i : p.rs);
-  const int j = i - p.n_static;
-  return p.total_static + j * p.qd + (j < p.rd ? j : p.rd);
+// cost of one sequence: Hkv units of nt tiles each
+PDATTN_HD inline int64_t seq_cost(int64_t nt, int hkv) { return nt > 0 ? (nt + kPieceCostTiles) * hkv : 0; }
+// position `r` (cost units) inside a sequence of Hkv units of nt tiles -> (unit within sequence, tile)
+PDATTN_HD inline void locate_in_seq(int64_t r, int64_t nt, int* k, int* tile) {
+  const int64_t per = nt + kPieceCostTiles;
+  *k = static_cast<int>(r / per);
+  const int64_t pos = r % per;
+  *tile = pos > kPieceCostTiles ? static_cast<int>(pos - kPieceCostTiles) : 0;
 }
 
-// spans: [2 * (n_static + n_dyn)] = (unit0, tile0) per span; at most 2 * max_spans ints are
-// written and n_dyn is lowered to fit.  Returns false on invalid arguments.
+// spans: [n_static + n_dyn + 1] entries; at most max_spans + 1 are written and n_dyn is lowered
+// to fit.  Returns false on invalid arguments.
 bool plan_spans(const int32_t* context_lens, int num_seqs, int num_kv_heads, int n_static, int dyn_per_cta,
-                int max_spans, int32_t* spans, PlanParams* plan);
+                int max_spans, SpanStart* spans, PlanParams* plan);
 
 }  // namespace pdattn

@@ -48,9 +48,9 @@ WsLayout ws_layout(int num_seqs, int G, int head_dim) {
   WsLayout w;
   w.hdr = 0;
   w.spans = 256;
-  w.rec = w.spans + align_up(static_cast<size_t>(MAX_SPANS) * sizeof(int2), 256);
+  w.rec = w.spans + align_up(static_cast<size_t>(MAX_SPANS + 1) * sizeof(SpanStart), 256);
   w.prefix = w.rec + align_up(static_cast<size_t>(MAX_SPANS) * sizeof(int4), 256);
-  w.partials = w.prefix + align_up(static_cast<size_t>(num_seqs + 1) * 4, 256);
+  w.partials = w.prefix + align_up(static_cast<size_t>(num_seqs + 1) * 8, 256);
   w.total = w.partials + align_up(static_cast<size_t>(MAX_SPANS) * 2 * slot_bytes, 256);
   return w;
 }
@@ -258,14 +258,13 @@ pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, i
                                int dynamic_per_cta, int max_spans, int32_t* spans, pdattn_plan* plan_out) {
   if (!plan_out) return PDATTN_INVALID_ARG;
   PlanParams plan;
-  if (!plan_spans(context_lens_host, num_seqs, num_kv_heads, n_ctas, dynamic_per_cta, max_spans, spans, &plan))
+  if (!spans || max_spans < n_ctas) return PDATTN_INVALID_ARG;
+  static_assert(sizeof(SpanStart) == 4 * sizeof(int32_t), "span table entries are four int32");
+  if (!plan_spans(context_lens_host, num_seqs, num_kv_heads, n_ctas, dynamic_per_cta, max_spans,
+                  reinterpret_cast<SpanStart*>(spans), &plan))
     return PDATTN_INVALID_ARG;
   plan_out->n_static = plan.n_static;
   plan_out->n_dynamic = plan.n_dyn;
-  plan_out->static_q = plan.qs;
-  plan_out->static_r = plan.rs;
-  plan_out->dynamic_q = plan.qd;
-  plan_out->dynamic_r = plan.rd;
   plan_out->total_tiles = plan.total;
   return PDATTN_OK;
 }
@@ -302,7 +301,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   P.block_table = a->block_table;
   P.context_lens = a->context_lens;
   P.hdr = reinterpret_cast<WsHeader*>(ws + wl.hdr);
-  P.spans_ws = reinterpret_cast<const int2*>(ws + wl.spans);
+  P.spans_ws = reinterpret_cast<const SpanStart*>(ws + wl.spans);
   P.rec = reinterpret_cast<int4*>(ws + wl.rec);
   P.partials = reinterpret_cast<float*>(ws + wl.partials);
   P.S = a->num_seqs;
@@ -320,13 +319,10 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   const int dyn_per_cta = g_dyn_per_cta;
   int grid = n_ctas, combine_grid = 0, n_spans_host = -1;
   if (a->context_lens_host) {
-    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta, MAX_PARAM_SPANS,
-                    reinterpret_cast<int32_t*>(P.spans), &P.plan))
+    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta, MAX_PARAM_SPANS, P.spans,
+                    &P.plan))
       return PDATTN_INVALID_ARG;
-    if (P.plan.total < n_ctas) {          // fewer tiles than CTAs: one tile each, no empty CTAs
-      grid = P.plan.total > 0 ? P.plan.total : 1;
-    }
-    n_spans_host = P.plan.n_dyn > 0 ? P.plan.n_static + P.plan.n_dyn : grid;
+    n_spans_host = P.plan.n_static + P.plan.n_dyn;
     combine_grid = n_spans_host;
   } else {
     P.use_ws_plan = 1;
@@ -334,7 +330,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     const int n_dyn_max = n_ctas * dyn_per_cta;
     plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
                                          reinterpret_cast<int32_t*>(ws + wl.prefix),
-                                         reinterpret_cast<int2*>(ws + wl.spans), P.hdr);
+                                         reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
     g_last_launches += 1;
@@ -554,9 +550,9 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   const int G = a->num_q_heads / a->num_kv_heads;
   const size_t slot_bytes = static_cast<size_t>(G > 8 ? 16 : 8) * (a->head_dim + 2) * 4;
   const size_t off_spans = 256;
-  const size_t off_rec = off_spans + align_up(static_cast<size_t>(n_ctas) * sizeof(int2), 256);
+  const size_t off_rec = off_spans + align_up(static_cast<size_t>(n_ctas + 1) * sizeof(SpanStart), 256);
   const size_t off_prefix = off_rec + align_up(static_cast<size_t>(n_ctas) * sizeof(int4), 256);
-  const size_t off_part = off_prefix + align_up(static_cast<size_t>(a->num_seqs + 1) * 4, 256);
+  const size_t off_part = off_prefix + align_up(static_cast<size_t>(a->num_seqs + 1) * 8, 256);
   const size_t need = off_part + align_up(static_cast<size_t>(n_ctas) * 2 * slot_bytes, 256);
   if (a->num_seqs > PDATTN_STATIC_SCRATCH_MAX_SEQS || need > PDATTN_STATIC_SCRATCH_BYTES) {
     snprintf(g_cuda_err, sizeof g_cuda_err,
@@ -581,7 +577,7 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   P.block_table = a->block_table;
   P.context_lens = a->context_lens;
   P.hdr = reinterpret_cast<WsHeader*>(ws);
-  P.spans_ws = reinterpret_cast<const int2*>(ws + off_spans);
+  P.spans_ws = reinterpret_cast<const SpanStart*>(ws + off_spans);
   P.rec = reinterpret_cast<int4*>(ws + off_rec);
   P.partials = reinterpret_cast<float*>(ws + off_part);
   P.S = a->num_seqs;
@@ -595,18 +591,16 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   P.box5d = 0;
   int grid = n_ctas, combine_grid = n_ctas, n_spans_host = -1;
   if (a->context_lens_host) {
-    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, 0, n_ctas,
-                    reinterpret_cast<int32_t*>(P.spans), &P.plan))
+    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, 0, n_ctas, P.spans, &P.plan))
       return PDATTN_INVALID_ARG;
-    if (P.plan.total < n_ctas) grid = P.plan.total > 0 ? P.plan.total : 1;
-    n_spans_host = grid;
-    combine_grid = grid;
+    n_spans_host = n_ctas;
+    combine_grid = n_ctas;
   } else {
     P.use_ws_plan = 1;
     memset(&P.plan, 0, sizeof P.plan);
     plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas, 0,
                                          reinterpret_cast<int32_t*>(ws + off_prefix),
-                                         reinterpret_cast<int2*>(ws + off_spans), P.hdr);
+                                         reinterpret_cast<SpanStart*>(ws + off_spans), P.hdr);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
     g_last_launches += 1;

@@ -60,15 +60,7 @@ class Args(ctypes.Structure):
 
 
 class Plan(ctypes.Structure):
-    _fields_ = [("n_static", ctypes.c_int), ("n_dynamic", ctypes.c_int), ("static_q", ctypes.c_int),
-                ("static_r", ctypes.c_int), ("dynamic_q", ctypes.c_int), ("dynamic_r", ctypes.c_int),
-                ("total_tiles", ctypes.c_int)]
-
-    def span_len(self, i: int) -> int:
-        if i < self.n_static:
-            return self.static_q + (1 if i < self.static_r else 0)
-        j = i - self.n_static
-        return self.dynamic_q + (1 if j < self.dynamic_r else 0)
+    _fields_ = [("n_static", ctypes.c_int), ("n_dynamic", ctypes.c_int), ("total_tiles", ctypes.c_int)]
 
 
 _lib = None
@@ -244,17 +236,18 @@ def set_dynamic_spans(per_cta: int):
 
 
 def plan_host(context_lens_host, num_kv_heads, n_ctas, dynamic_per_cta=0, max_spans=None):
-    """pdattn_plan_host -> (spans[n_spans, 2], Plan).  Needs no GPU."""
+    """pdattn_plan_host -> (spans[n_spans + 1, 4], Plan).  Row i is (unit, tile, flat, 0); span i holds
+    spans[i + 1, 2] - spans[i, 2] tiles.  Needs no GPU."""
     lens = np.ascontiguousarray(context_lens_host, dtype=np.int32)
     if max_spans is None:
         max_spans = n_ctas * 9
-    spans = np.zeros((max_spans, 2), dtype=np.int32)
+    spans = np.zeros((max_spans + 1, 4), dtype=np.int32)
     plan = Plan()
     st = lib().pdattn_plan_host(lens.ctypes.data if lens.size else None, lens.size, num_kv_heads, n_ctas,
                                 dynamic_per_cta, max_spans, spans.ctypes.data, ctypes.byref(plan))
     if st != OK:
         raise PdattnError(st, "pdattn_plan_host")
-    return spans[: plan.n_static + plan.n_dynamic].copy(), plan
+    return spans[: plan.n_static + plan.n_dynamic + 1].copy(), plan
 
 
 def check(workspace, stream=None) -> int:

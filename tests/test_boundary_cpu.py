@@ -93,14 +93,18 @@ def test_short_form_needs_a_binding():
     assert res == [pdattn.NOT_BOUND]
 
 
+PIECE_COST = 2     # cost of starting a unit, in tiles (the partitioner's constant)
+
+
 def walk_spans(lens, Hkv, n_ctas, dyn=8):
     """Re-walk the plan the way a CTA does and return the list of (unit, tile) each span covers."""
     spans, plan = pdattn.plan_host(lens, Hkv, n_ctas, dynamic_per_cta=dyn)
     nt = [(int(L) + 63) // 64 if L > 0 else 0 for L in lens]
     cover = []
-    for c in range(len(spans)):
+    for c in range(len(spans) - 1):
         unit, tb = int(spans[c, 0]), int(spans[c, 1])
-        rem = plan.span_len(c)
+        rem = int(spans[c + 1, 2] - spans[c, 2])
+        assert rem >= 0
         mine = []
         while rem > 0 and unit < len(lens) * Hkv:
             n = nt[unit // Hkv]
@@ -114,6 +118,11 @@ def walk_spans(lens, Hkv, n_ctas, dyn=8):
         assert rem == 0
         cover.append(mine)
     return cover, plan
+
+
+def span_cost(mine):
+    """tiles plus the start-up cost of every unit the span touches"""
+    return len(mine) + PIECE_COST * len({u for u, _ in mine})
 
 
 @pytest.mark.parametrize("case", ["cfg1", "cfg2", "cfg5", "zeros", "short", "one"])
@@ -130,15 +139,21 @@ def test_partitioner_covers_every_tile_exactly_once(case, n_ctas, dyn):
     assert plan.total_tiles == len(want)
     assert flat == want                      # contiguous, ordered, nothing twice, nothing missing
     assert plan.n_static == n_ctas and len(cover) == plan.n_static + plan.n_dynamic
-    st = [len(m) for m in cover[:n_ctas]]
-    assert max(st) - min(st) <= 1            # static spans balanced to within one tile
     assert dyn > 0 or plan.n_dynamic == 0
-    if plan.n_dynamic:
-        dy = [len(m) for m in cover[n_ctas:]]
-        assert max(dy) - min(dy) <= 1 and min(dy) >= 3
-        assert plan.n_dynamic <= 8 * n_ctas
-        # static spans cover three quarters, the run-time pool one quarter
-        assert abs(sum(dy) - plan.total_tiles // 4) <= 1
+    assert plan.n_dynamic <= 8 * n_ctas
+
+
+def test_partitioner_balances_cost_not_tiles():
+    """Config 2: CTAs inside long sequences get more tiles than CTAs that walk many short ones, and the
+    cost (tiles + 2 per unit touched) is even to within one unit's start-up plus the cut unit."""
+    lens = W.config_lengths(2)
+    cover, plan = walk_spans(lens, 4, 148, dyn=0)
+    costs = np.array([span_cost(m) for m in cover])
+    tiles = np.array([len(m) for m in cover])
+    assert costs.max() - costs.min() <= 2 * PIECE_COST + 1
+    assert tiles.max() - tiles.min() > 4
+    units = np.array([len({u for u, _ in m}) for m in cover])
+    assert np.corrcoef(units, tiles)[0, 1] < -0.8       # more units to start -> fewer tiles
 
 
 def test_partitioner_spreads_the_straggler_phase_over_all_sms():
@@ -156,7 +171,7 @@ def test_partitioner_spreads_the_straggler_phase_over_all_sms():
 def test_partitioner_small_batches_use_static_spans_only():
     cover, plan = walk_spans(W.config_lengths(1), 1, 148)
     assert plan.n_dynamic == 0 and plan.total_tiles == 8
-    assert [len(m) for m in cover] == [1] * 8 + [0] * 140
+    assert sum(len(m) for m in cover) == 8 and max(len(m) for m in cover) <= 2
 
 
 def test_partitioner_depends_on_lengths_only():
