@@ -300,6 +300,45 @@ def main():
     d2h = oh.numel() * 2
     assert pdattn.check(ws) == pdattn.OK
 
+    # ---- secondary runs (N = 1 only): bandwidth ceilings from the library's probes, the device-side
+    # planner (no host copy of the lengths) and the token-major cache layout through strides
+    extras = None
+    if world == 1:
+        def timed(fn, n=20, reps=5):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            best = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for _ in range(n):
+                    fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                best.append(a.elapsed_time(b) / n)
+            return float(np.median(best))
+
+        c = copies[0]
+        sink = torch.zeros(4, dtype=torch.int32, device=dev)
+        pool_bytes = 2 * c.k_cache.numel() * 2
+        t_stream = timed(lambda: (pdattn.stream_read_probe(c.k_cache, sink), pdattn.stream_read_probe(c.v_cache, sink)))
+        t_gather = timed(lambda: pdattn.decode_ex(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale,
+                                                  outs[0], ws, context_lens_host=c.context_lens_host, probe=True))
+        t_devplan = timed(lambda: pdattn.decode_ex(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale,
+                                                   outs[0], ws, context_lens_host=None))
+        extras = {"stream_read_gbs": pool_bytes / (t_stream * 1e-3) / 1e9,
+                  "page_gather_gbs": uniq / (t_gather * 1e-3) / 1e9,
+                  "device_plan_ms_per_step": t_devplan}
+        if uniq < (20 << 30):
+            k_nhd = c.k_cache.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            v_nhd = c.v_cache.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            extras["token_major_layout_ms_per_step"] = timed(
+                lambda: pdattn.decode_ex(c.q, k_nhd, v_nhd, c.block_table, c.context_lens, c.scale, outs[0], ws,
+                                         context_lens_host=c.context_lens_host))
+            del k_nhd, v_nhd
+        assert pdattn.check(ws) == pdattn.OK
+
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only)
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -334,6 +373,7 @@ def main():
             "gpu_launches": launches_per_step * K,
             "clocks": sampler.summary(),
             "cpu_baseline": cpu_baseline,
+            "secondary": extras,
         }
         print(json.dumps(line), flush=True)
     if dist is not None:

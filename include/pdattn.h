@@ -102,6 +102,24 @@ typedef struct {
 pdattn_status pdattn_decode_ex(const pdattn_args* args, pdattn_stream_t stream);
 
 /*
+ * KV append: the step that precedes attention in the decoding loop (Section 2.3; the cache grows by
+ * b_kv bytes per token and layer, Appendix A.1.2).  For every sequence s with t = context_lens[s]:
+ * the rows k_new[s], v_new[s] (DEVICE bf16 [num_seqs, num_kv_heads, head_dim], dense) are written to
+ * slot t % block_size of page block_table[s, t / block_size] of the caches (same strides as
+ * pdattn_args), and context_lens[s] becomes t + 1 (DEVICE, updated in place).  The page must
+ * already be in the table: page allocation stays with the caller.  A sequence whose target page id
+ * is outside [0, num_blocks), or whose table row is full, is left untouched and, if `workspace`
+ * (DEVICE, may be NULL) is given, its sticky error word is set (see pdattn_check).
+ * Followed by pdattn_decode_ex with context_lens_host = NULL, a whole decode step needs no host
+ * work that depends on the lengths.
+ */
+pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                               const int32_t* block_table, int32_t* context_lens, int num_seqs,
+                               int num_kv_heads, int head_dim, int block_size, int max_blocks_per_seq,
+                               int num_blocks, int64_t kv_block_stride, int64_t kv_head_stride,
+                               int64_t kv_token_stride, void* workspace, pdattn_stream_t stream);
+
+/*
  * Thread-local binding of the arguments the short form below does not carry.
  * context_lens_host may be NULL.  The pointers must stay valid while bound.
  */

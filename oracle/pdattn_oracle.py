@@ -140,3 +140,28 @@ def bf16_rne(x: np.ndarray) -> np.ndarray:
     for i, v in enumerate(flat):
         out[i] = L.pdattn_oracle_bf16_to_double(L.pdattn_oracle_bf16_rne(float(v)))
     return out.reshape(np.shape(x))
+
+
+def append_kv(k_cache, v_cache, block_table, context_lens, k_new, v_new):
+    """Plain definition of the KV append step on CPU tensors, in place: token t = context_lens[s] of
+    sequence s goes to slot t % bs of page block_table[s, t // bs]; then context_lens[s] = t + 1.
+    A sequence whose target page id is out of range, or whose table row is full, is skipped.
+    Returns the number of skipped sequences.  (Byte and index work: compared bit for bit.)"""
+    NB, Hkv, bs, d = k_cache.shape
+    S = k_new.shape[0]
+    MB = block_table.shape[1]
+    skipped = 0
+    for s in range(S):
+        t = int(context_lens[s])
+        if t < 0 or t // bs >= MB:
+            skipped += 1
+            continue
+        page = int(block_table[s, t // bs])
+        if page < 0 or page >= NB:
+            skipped += 1
+            continue
+        for g in range(Hkv):
+            k_cache[page, g, t % bs, :] = k_new[s, g, :]
+            v_cache[page, g, t % bs, :] = v_new[s, g, :]
+        context_lens[s] = t + 1
+    return skipped

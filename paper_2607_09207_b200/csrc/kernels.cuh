@@ -871,6 +871,43 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   if (aborted && lane == 0) atomicOr(&P.hdr->err, ERR_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------------------
+// KV append: the step on the input side of decode attention.  Block s writes the new token's K
+// and V rows of every KV head into slot L_s % bs of page block_table[s, L_s / bs] and then
+// advances context_lens[s].  One warp per KV head: lanes copy 16-byte chunks, K then V.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+append_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
+              __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
+              const int32_t* __restrict__ block_table, int32_t* __restrict__ context_lens, int Hkv, int D, int bs,
+              int MB, int NB, int64_t sb, int64_t sh, int64_t st, int32_t* err) {
+  const int s = blockIdx.x;
+  const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int L = context_lens[s];
+  __syncthreads();                       // every warp has read the old length before it is advanced
+  if (L < 0 || L / bs >= MB) {
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  const int page = block_table[static_cast<int64_t>(s) * MB + L / bs];
+  if (page < 0 || page >= NB) {          // not dereferenced; the length is left as it was
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  if (g < Hkv) {
+    const int64_t dst = page * sb + g * sh + static_cast<int64_t>(L % bs) * st;
+    const int64_t src = (static_cast<int64_t>(s) * Hkv + g) * D;
+    const int chunks = D / 8;            // 16-byte chunks per row
+    for (int c = lane; c < 2 * chunks; c += 32) {
+      const bool isV = c >= chunks;
+      const int cc = isV ? c - chunks : c;
+      const uint4 v = *reinterpret_cast<const uint4*>((isV ? v_new : k_new) + src + cc * 8);
+      *reinterpret_cast<uint4*>((isV ? v_cache : k_cache) + dst + cc * 8) = v;
+    }
+  }
+  if (threadIdx.x == 0) context_lens[s] = L + 1;
+}
+
 // Read-only streaming ceiling: every thread block sums a contiguous slice with 16-byte loads.
 __global__ void __launch_bounds__(512)
 stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __restrict__ sink) {

@@ -248,6 +248,31 @@ pdattn_status pdattn_workspace_init(void* workspace, size_t workspace_bytes, pda
   return PDATTN_OK;
 }
 
+pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                               const int32_t* block_table, int32_t* context_lens, int num_seqs, int num_kv_heads,
+                               int head_dim, int block_size, int max_blocks_per_seq, int num_blocks,
+                               int64_t kv_block_stride, int64_t kv_head_stride, int64_t kv_token_stride,
+                               void* workspace, pdattn_stream_t stream) {
+  if (num_seqs < 0 || num_kv_heads <= 0 || num_kv_heads > 16 || max_blocks_per_seq <= 0 || num_blocks <= 0)
+    return PDATTN_INVALID_ARG;
+  if (head_dim != 64 && head_dim != 128) return PDATTN_UNSUPPORTED;
+  if (block_size != 16) return PDATTN_UNSUPPORTED;
+  if (num_seqs == 0) return PDATTN_OK;
+  if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !context_lens) return PDATTN_INVALID_ARG;
+  if (kv_block_stride <= 0 || kv_head_stride <= 0 || kv_token_stride < head_dim) return PDATTN_INVALID_ARG;
+  if ((kv_block_stride | kv_head_stride | kv_token_stride) % 8 != 0) return PDATTN_UNSUPPORTED;
+  auto mis = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; };
+  if (mis(k_new) || mis(v_new) || mis(k_cache) || mis(v_cache)) return PDATTN_MISALIGNED;
+  append_kernel<<<num_seqs, 32 * num_kv_heads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+      static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache), block_table, context_lens,
+      num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks, kv_block_stride, kv_head_stride,
+      kv_token_stride, static_cast<int32_t*>(workspace));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("append_kernel launch", e);
+  return PDATTN_OK;
+}
+
 pdattn_status pdattn_set_dynamic_spans(int per_cta) {
   if (per_cta < 0 || per_cta > kMaxDynPerCta) return PDATTN_INVALID_ARG;
   g_dyn_per_cta = per_cta;

@@ -31,7 +31,7 @@ EXPORTS = [
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_set_dynamic_spans",
-    "pdattn_decode_static_scratch",
+    "pdattn_decode_static_scratch", "pdattn_append_kv",
 ]
 
 
@@ -87,6 +87,7 @@ def lib():
         L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(Plan)]
         L.pdattn_set_dynamic_spans.argtypes = [i32]
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
+        L.pdattn_append_kv.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp]
         L.pdattn_check.argtypes = [vp, vp]
         L.pdattn_profile_events.argtypes = [vp, vp]
         L.pdattn_gather_probe.argtypes = [ctypes.POINTER(Args), vp]
@@ -178,6 +179,21 @@ def decode_static_scratch(q, k_cache, v_cache, block_table, context_lens, scale,
                                             _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_decode_static_scratch")
+    return st
+
+
+def append_kv(k_new, v_new, k_cache, v_cache, block_table, context_lens, workspace=None, stream=None,
+              check: bool = True) -> int:
+    """pdattn_append_kv: write this step's K/V rows ([S, Hkv, d]) into the paged caches and advance
+    context_lens (device tensor, in place)."""
+    S, Hkv, d = k_new.shape
+    NB, _, bs, _ = k_cache.shape
+    st = lib().pdattn_append_kv(k_new.data_ptr(), v_new.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                block_table.data_ptr(), context_lens.data_ptr(), S, Hkv, d, bs, block_table.shape[1],
+                                NB, k_cache.stride(0), k_cache.stride(1), k_cache.stride(2),
+                                workspace.data_ptr() if workspace is not None else None, _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_append_kv")
     return st
 
 

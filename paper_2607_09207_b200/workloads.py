@@ -208,12 +208,15 @@ def poison_unused(w: Workload) -> None:
 
 
 def _build(name, seed, lens, Hq, Hkv, d, bs, device, *, num_blocks=None, shared_prefix_pages=0,
-           group=1, head_scales=False, poison=True, pad_blocks_to=1024, max_blocks=None) -> Workload:
+           group=1, head_scales=False, poison=True, pad_blocks_to=1024, max_blocks=None,
+           headroom_tokens=0) -> Workload:
     """lens: int array [S] of context lengths.  With shared_prefix_pages > 0 the first
-    that many pages of every run of `group` consecutive sequences are the same physical pages."""
+    that many pages of every run of `group` consecutive sequences are the same physical pages.
+    headroom_tokens: pages for that many further tokens per sequence are put in the table (a decode
+    loop appends into them); they start out poisoned like every slot nobody owns yet."""
     lens = np.asarray(lens, dtype=np.int64)
     S = len(lens)
-    pages_per_seq = (lens + bs - 1) // bs
+    pages_per_seq = (lens + headroom_tokens + bs - 1) // bs
     MB = int(max_blocks if max_blocks is not None else max(1, pages_per_seq.max() if S else 1))
     # pages needed
     need = 0
@@ -291,7 +294,7 @@ CONFIG_NAMES = {1: "tiny", 2: "7B-shaped rollout step", 3: "GRPO group sharing",
 
 
 def make_config(cfg: int, device="cpu", num_seqs: Optional[int] = None, len_div: int = 1,
-                poison: bool = True) -> Workload:
+                poison: bool = True, headroom_tokens: int = 0) -> Workload:
     """Build benchmark configuration cfg (1..5), seed cfg-1."""
     seed = cfg - 1
     lens = config_lengths(cfg, num_seqs, len_div)
@@ -299,7 +302,7 @@ def make_config(cfg: int, device="cpu", num_seqs: Optional[int] = None, len_div:
     if cfg == 1:
         return _build(name, seed, lens, 4, 1, 64, 16, device, num_blocks=64, poison=poison)
     if cfg == 2:
-        return _build(name, seed, lens, 28, 4, 128, 16, device, poison=poison)
+        return _build(name, seed, lens, 28, 4, 128, 16, device, poison=poison, headroom_tokens=headroom_tokens)
     if cfg == 3:
         pre = (1024 // len_div) // 16
         return _build(name, seed, lens, 40, 8, 128, 16, device, shared_prefix_pages=pre, group=8, poison=poison)

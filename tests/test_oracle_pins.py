@@ -253,3 +253,27 @@ def test_bf16_rounding_helper():
     # 1.00390625 = 1 + 2^-8 is a tie: rounds to even (1.0); 1.005859375 = 1 + 1.5*2^-8 rounds up
     assert got[2] == 1.0 and got[3] == 1.0078125
     np.testing.assert_array_equal(got, want)
+
+
+def test_append_then_attend_equals_the_longer_cache():
+    """Oracle append pin: take a cache of L + 1 tokens, cut the last token out (poison its slot), append
+    it back: the bits of the caches and the attention output are those of the original."""
+    lens = [16, 33, 1]                               # the appended token lands at slot 0, 1 and 1 of a page
+    full = W.make_custom([L + 1 for L in lens], Hq=4, Hkv=2, d=32, seed=26, num_blocks=16)
+    ref_out = orc.decode_workload(full)
+    cut = full.clone()
+    bt = full.block_table.numpy()
+    k_new = torch.zeros(3, 2, 32, dtype=BF16)
+    v_new = torch.zeros(3, 2, 32, dtype=BF16)
+    for s, L in enumerate(lens):
+        page, slot = bt[s, L // 16], L % 16
+        k_new[s] = full.k_cache[page, :, slot]
+        v_new[s] = full.v_cache[page, :, slot]
+        cut.k_cache[page, :, slot] = float("nan")
+        cut.v_cache[page, :, slot] = float("nan")
+    cut.context_lens = torch.tensor(lens, dtype=torch.int32)
+    assert orc.append_kv(cut.k_cache, cut.v_cache, cut.block_table, cut.context_lens, k_new, v_new) == 0
+    assert cut.context_lens.tolist() == [L + 1 for L in lens]
+    assert torch.equal(cut.k_cache.view(torch.int16), full.k_cache.view(torch.int16))
+    assert torch.equal(cut.v_cache.view(torch.int16), full.v_cache.view(torch.int16))
+    assert np.array_equal(orc.decode_workload(cut), ref_out)
