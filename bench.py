@@ -338,6 +338,8 @@ def main():
                                          context_lens_host=c.context_lens_host))
             del k_nhd, v_nhd
         assert pdattn.check(ws) == pdattn.OK
+        if args.cfg == 2 and args.num_seqs is None:
+            extras["decode_loop"] = decode_loop(pdattn, W, dev, stream)
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only)
     cpu_baseline = None
@@ -379,6 +381,48 @@ def main():
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def decode_loop(pdattn, W, dev, stream, steps=64):
+    """64 consecutive growing steps of the same batch: KV append, device-side plan, decode, combine.
+    Nothing in a step depends on host knowledge of the lengths.  The tokens read over the loop are
+    checked against the closed form of the paper's decode-history feature (Appendix A.1.2)."""
+    w = W.make_config(2, device=dev, headroom_tokens=steps + 16)
+    S = w.num_seqs
+    ws = pdattn.alloc_workspace(S, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, device=dev)
+    out = torch.empty_like(w.q)
+    k_new = W.normal_bf16(S * w.num_kv_heads * w.head_dim, 9, 100, dev).view(S, w.num_kv_heads, w.head_dim)
+    v_new = W.normal_bf16(S * w.num_kv_heads * w.head_dim, 9, 101, dev).view(S, w.num_kv_heads, w.head_dim)
+    lens0 = w.context_lens.clone()
+    tokens = torch.zeros((), dtype=torch.int64, device=dev)
+
+    def step():
+        pdattn.append_kv(k_new, v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens, workspace=ws,
+                         stream=stream)
+        pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws,
+                         context_lens_host=None, stream=stream)
+
+    # pass 1 (untimed, also the warm-up): count the tokens every step attends to
+    for _ in range(steps):
+        step()
+        tokens += w.context_lens.sum()
+    torch.cuda.synchronize()
+    want = sum(W.h_dec(int(p), steps) + steps for p in lens0.cpu().tolist())
+    assert int(tokens.item()) == want, (int(tokens.item()), want)
+    # pass 2 (timed): the same 64 steps again, nothing but the library's launches on the stream
+    w.context_lens.copy_(lens0)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(steps):
+        step()
+    b.record(stream)
+    torch.cuda.synchronize()
+    assert pdattn.check(ws) == pdattn.OK
+    assert torch.equal(w.context_lens, lens0 + steps)
+    ms = a.elapsed_time(b) / steps
+    return {"steps": steps, "ms_per_step": ms, "seq_steps_per_s": S / (ms * 1e-3),
+            "history_tokens_read": want, "launches_per_step": 4}
 
 
 def _physical_copy(w, seed):

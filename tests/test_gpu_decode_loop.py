@@ -94,3 +94,46 @@ def test_growing_decode_loop_matches_the_oracle_every_step():
     # sees p + t - 1 tokens) plus r per request in this library's (the current token is already cached)
     r = steps
     assert tokens == sum(W.h_dec(int(p), r) + r for p in L0)
+
+
+def test_a_decode_step_replays_as_a_cuda_graph():
+    """append + device-side plan + decode + combine captured once and replayed: no host work per step.
+    (The first, uncaptured calls do the one-time set-up: function attributes, driver entry points.)"""
+    w = W.make_config(2, device=DEV, num_seqs=16, len_div=4, headroom_tokens=40)
+    S = w.num_seqs
+    ws = pdattn.alloc_workspace(S, 28, 4, 128)
+    out = torch.empty_like(w.q)
+    k_new, v_new = new_rows(S, 4, 128, 0)
+    lens0 = w.context_lens.clone()
+    k0, v0 = w.k_cache.clone(), w.v_cache.clone()
+
+    def step(stream=None):
+        pdattn.append_kv(k_new, v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens, workspace=ws,
+                         stream=stream)
+        pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws,
+                         context_lens_host=None, stream=stream)
+
+    for _ in range(12):
+        step()
+    torch.cuda.synchronize()
+    eager = out.clone()
+
+    def reset():
+        w.context_lens.copy_(lens0)
+        w.k_cache.copy_(k0)
+        w.v_cache.copy_(v0)
+
+    reset()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step(stream=side)
+    torch.cuda.synchronize()
+    reset()
+    for _ in range(12):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert pdattn.check(ws) == pdattn.OK
+    assert w.context_lens.cpu().tolist() == [int(L) + 12 for L in lens0.cpu().tolist()]
+    assert torch.equal(out, eager)
