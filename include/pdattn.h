@@ -102,6 +102,27 @@ typedef struct {
 pdattn_status pdattn_decode_ex(const pdattn_args* args, pdattn_stream_t stream);
 
 /*
+ * Decode step for GRPO sample groups (Section 2.1: several responses are sampled per prompt and form
+ * a prompt-level group; Section 7.1 uses 8 per prompt).  Sequences g*group_size .. (g+1)*group_size-1
+ * form group g and share their first prefix_tiles[g] * 64 tokens: their block_table rows must hold
+ * the SAME page ids for those tokens.  The shared tiles are then streamed from HBM once per group
+ * and KV head and scored against the query rows of all samples (group_size * G rows at a time),
+ * and every sequence continues with its own pages; results equal pdattn_decode_ex's definition
+ * (within rounding: the summation order differs) and are bit-identical from run to run.
+ *   prefix_tiles      DEVICE int32 [num_seqs / group_size]; prefix_tiles_host its HOST copy.
+ *   Requirements: args->context_lens_host given; num_seqs a multiple of group_size; G <= 8 and
+ *   group_size * G <= 48; every member of group g has context_len > prefix_tiles[g] * 64
+ *   (it owns at least its current token); 0 is allowed (the group shares nothing).
+ *   args->workspace must hold pdattn_grouped_workspace_size() bytes.
+ * The caller vouches for the page ids being shared; if they are not, the group's first row is
+ * used for the shared tiles of all its members.
+ */
+pdattn_status pdattn_grouped_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                                            int block_size, size_t* device_bytes);
+pdattn_status pdattn_decode_grouped(const pdattn_args* args, int group_size, const int32_t* prefix_tiles,
+                                    const int32_t* prefix_tiles_host, pdattn_stream_t stream);
+
+/*
  * KV append: the step that precedes attention in the decoding loop (Section 2.3; the cache grows by
  * b_kv bytes per token and layer, Appendix A.1.2).  For every sequence s with t = context_lens[s]:
  * the rows k_new[s], v_new[s] (DEVICE bf16 [num_seqs, num_kv_heads, head_dim], dense) are written to

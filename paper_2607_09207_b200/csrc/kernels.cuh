@@ -53,6 +53,8 @@ struct DecodeParams {
   __nv_bfloat16* out;
   const int32_t* block_table;
   const int32_t* context_lens;
+  const int32_t* start_tiles;   // per sequence: leading tiles this call skips (null = none)
+  const float* pfx_partials;    // with start_tiles: [seq][kv head][HP*(D+2)] partial of the skipped tiles
   WsHeader* hdr;
   const SpanStart* spans_ws;  // spans written by plan_kernel (used when use_ws_plan)
   int4* rec;                // per-span record: (first_unit, first_tile, own_unit, own_slot)
@@ -231,20 +233,27 @@ static_assert(sizeof(Ctrl) <= 640, "control block");
 // ------------------------------------------------------------------------------------------
 struct Piece {
   int unit, s, g, L, nt, tb, te;
+  int t0;   // tiles of the sequence that are skipped (shared prefix handled elsewhere): tile t of the
+            // piece is tile t0 + t of the sequence
 };
 struct Walker {
   const int32_t* ctx;
+  const int32_t* start_tiles;   // per sequence, may be null (= 0)
   int Hkv, nunits, unit, tb, rem;
-  int pf_unit = -1, pf_L = 0;   // context length of the following unit, loaded one piece early
+  int pf_unit = -1, pf_L = 0, pf_t0 = 0;   // the following unit's length and start, loaded one piece early
   __device__ __forceinline__ bool next(Piece& p) {
     while (rem > 0 && unit < nunits) {
       const int s = unit / Hkv;
-      const int L = (unit == pf_unit) ? pf_L : __ldg(ctx + s);
+      const bool hit = unit == pf_unit;
+      const int L = hit ? pf_L : __ldg(ctx + s);
+      const int t0 = hit ? pf_t0 : (start_tiles ? __ldg(start_tiles + s) : 0);
       if (unit + 1 < nunits) {
         pf_unit = unit + 1;
         pf_L = __ldg(ctx + (unit + 1) / Hkv);
+        pf_t0 = start_tiles ? __ldg(start_tiles + (unit + 1) / Hkv) : 0;
       }
-      const int nt = L > 0 ? (L + TILE - 1) / TILE : 0;
+      const int nt_all = L > 0 ? (L + TILE - 1) / TILE : 0;
+      const int nt = nt_all > t0 ? nt_all - t0 : 0;
       if (tb >= nt) {
         ++unit;
         tb = 0;
@@ -255,6 +264,7 @@ struct Walker {
       p.g = unit - s * Hkv;
       p.L = L;
       p.nt = nt;
+      p.t0 = t0;
       p.tb = tb;
       p.te = min(nt, tb + rem);
       rem -= p.te - p.tb;
@@ -526,7 +536,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
       const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
       const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
-      Walker walk{P.context_lens, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
+      Walker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
       Piece pc;
       while (!aborted && walk.next(pc)) {
         if (!PROBE && pw == 0) {
@@ -547,7 +557,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         ++pcnt;
         const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
         const int npages = (pc.L + BS - 1) / BS;
-        const int pbase = pc.tb * C::PAGES;
+        const int pbase = (pc.t0 + pc.tb) * C::PAGES;
         int ids_cur = (pbase + lane < npages) ? __ldg(row + pbase + lane) : 0;
         int ids_nxt = (pbase + IDS_PER_BATCH + lane < npages) ? __ldg(row + pbase + IDS_PER_BATCH + lane) : 0;
         for (int t = pc.tb; t < pc.te; ++t, ++it) {
@@ -581,7 +591,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             aborted = true;
             break;
           }
-          const int np = min(C::PAGES, npages - t * C::PAGES);
+          const int np = min(C::PAGES, npages - (pc.t0 + t) * C::PAGES);
           const int j = lane % C::PAGES;
           int id = __shfl_sync(0xffffffffu, ids_cur, kb * C::PAGES + j);
           const bool bad = (lane < C::PAGES) && (j < np) && (id < 0 || id >= P.NB);
@@ -651,7 +661,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   for (int k = 0; span >= 0; ++k) {
     const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
     const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
-    Walker walk{P.context_lens, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
+    Walker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
     Piece pc;
     int first_unit = -1, first_tb = 0, own_unit = -1, own_slot = 0, piece_idx = 0;
 
@@ -725,7 +735,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const uint32_t sK = ring + slot * C::STAGE_BYTES;
         const uint32_t sV = sK + C::KV_BYTES;
         const uint32_t badmask = ctrl->meta[slot];
-        const int n_valid = min(TILE, pc.L - t * TILE);
+        const int n_valid = min(TILE, pc.L - (pc.t0 + t) * TILE);
         if (PROBE) {
           // ceiling probe: no math
         } else if (n_valid == TILE) {
@@ -781,10 +791,23 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           const int h = (idx < ITEMS ? idx : 0) / (D / 4);
           float M = NEG_INF;
           for (int c = 0; c < n_cls; ++c) M = fmaxf(M, sm_m[c * C::HP + h]);
+          // A unit whose leading tiles were handled elsewhere (shared prefix) and whose remaining tiles
+          // all lie in this span: fold that partial in here, first in the order, and finish the unit.
+          const float* pfx = (complete && pc.t0 > 0)
+                                 ? P.pfx_partials + (static_cast<int64_t>(pc.s) * P.Hkv + pc.g) * C::SLOT_FLOATS
+                                 : nullptr;
+          if (pfx) M = fmaxf(M, pfx[h]);
           M_r[i] = M;
           Mu_r[i] = (M == NEG_INF) ? 0.f : M;
           Ls_r[i] = 0.f;
           a_r[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (pfx && idx < ITEMS) {
+            const int dq = idx % (D / 4);
+            const float f = fast_exp2(pfx[h] - Mu_r[i]);
+            Ls_r[i] = pfx[C::HP + h] * f;
+            const float4 v = *reinterpret_cast<const float4*>(pfx + 2 * C::HP + h * D + dq * 4);
+            a_r[i] = make_float4(v.x * f, v.y * f, v.z * f, v.w * f);
+          }
         }
 #pragma unroll
         for (int q = 0; q < ROUNDS; ++q) {
@@ -872,6 +895,206 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 }
 
 // ------------------------------------------------------------------------------------------
+// Shared-prefix kernel (GRPO groups): the samples of a group share their prompt pages, so the
+// prompt's K/V tiles are streamed ONCE per (group, kv head) and scored against the query rows of
+// all samples: group_size * G rows, eight per consumer warp.  Here every consumer warp works on
+// every tile (its own rows), so there is nothing to merge across warps; at the end of a unit each
+// warp writes the (m, l, acc) partial of its rows into the per-(sequence, kv head) prefix slots,
+// which decode_kernel / combine_kernel fold into the sequence's result.  Units (group * Hkv + kv
+// head) are never cut: CTA c takes units [ranges[c].x, ranges[c].y).
+// ------------------------------------------------------------------------------------------
+constexpr int MAX_PREFIX_ROWS = 48;
+struct PrefixParams {
+  const __nv_bfloat16* q;
+  const int32_t* block_table;
+  const int32_t* prefix_tiles;   // per group
+  int32_t* start_tiles;          // per sequence, written here for the decode kernel that follows
+  float* pfx_partials;           // [seq][kv head][HP*(D+2)]
+  int32_t* err;
+  int S, Hq, Hkv, G, Gs, MB, NB;
+  float scale_log2;
+  int box5d;
+  int2 ranges[160];
+};
+
+template <int D, int BS>
+__global__ void __launch_bounds__(Cfg<D, 1, BS>::NTHREADS, 1)
+prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+              const __grid_constant__ PrefixParams P) {
+  using C = Cfg<D, 1, BS>;
+  constexpr int NST = C::NSTAGES;
+  constexpr int NCW = C::NCW;
+  static_assert(NST % C::NPW == 0, "a slot is always refilled by the same producer warp");
+  static_assert(NCW * 8 >= MAX_PREFIX_ROWS, "rows per CTA");
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;
+  const uint32_t ring = raw + pad;
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + NST * C::STAGE_BYTES);
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int cta = blockIdx.x;
+  const float NEG_INF = __int_as_float(0xff800000);
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NST; ++i) {
+      mbar_init(smem_u32(&ctrl->full[i]), 1);
+      mbar_init(smem_u32(&ctrl->empty[i]), NCW);   // every consumer warp releases every tile
+    }
+    ctrl->abort = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  // per-sequence start tiles for the decode kernel
+  for (int s = cta * blockDim.x + threadIdx.x; s < P.S; s += gridDim.x * blockDim.x)
+    P.start_tiles[s] = P.prefix_tiles[s / P.Gs];
+
+  const int2 range = P.ranges[cta];
+  int it = 0;
+  bool aborted = false;
+
+  if (warp >= NCW) {
+    // ---- producers
+    const int pw = warp - NCW;
+    bool any_bad = false;
+    for (int u = range.x; u < range.y && !aborted; ++u) {
+      const int gi = u / P.Hkv, g = u - gi * P.Hkv;
+      const int pt = __ldg(P.prefix_tiles + gi);
+      const int32_t* row = P.block_table + static_cast<int64_t>(gi) * P.Gs * P.MB;   // the group's first row
+      const int npages = pt * C::PAGES;
+      constexpr int TILES_PER_BATCH = 32 / C::PAGES;
+      int ids_cur = (lane < npages) ? __ldg(row + lane) : 0;
+      int ids_nxt = (32 + lane < npages) ? __ldg(row + 32 + lane) : 0;
+      for (int t = 0; t < pt; ++t, ++it) {
+        const int kb = t % TILES_PER_BATCH;
+        if (kb == 0 && t != 0) {
+          ids_cur = ids_nxt;
+          const int nb = t * C::PAGES + 32;
+          ids_nxt = (nb + lane < npages) ? __ldg(row + nb + lane) : 0;
+        }
+        if (C::NPW > 1 && it % C::NPW != pw) continue;
+        const int slot = it % NST;
+        const uint32_t phase = (it / NST) & 1;
+        if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) {
+          aborted = true;
+          break;
+        }
+        const int j = lane % C::PAGES;
+        int id = __shfl_sync(0xffffffffu, ids_cur, kb * C::PAGES + j);
+        const bool bad = (lane < C::PAGES) && (id < 0 || id >= P.NB);
+        const uint32_t badmask = __ballot_sync(0xffffffffu, bad);
+        if (id < 0 || id >= P.NB) id = P.NB;
+        const uint32_t bar = smem_u32(&ctrl->full[slot]);
+        if (lane == 0) {
+          ctrl->meta[slot] = badmask;
+          mbar_arrive_expect_tx(bar, static_cast<uint32_t>(C::STAGE_BYTES));
+        }
+        __syncwarp();
+        if (lane < 2 * C::PAGES) {
+          const bool isV = lane >= C::PAGES;
+          const uint32_t dst = ring + slot * C::STAGE_BYTES + (isV ? C::KV_BYTES : 0) + j * C::PAGE_BYTES;
+          const CUtensorMap* tm = isV ? &tmV : &tmK;
+          if (P.box5d) {
+            tma_load_5d(dst, tm, 0, 0, 0, g, id, bar);
+          } else {
+#pragma unroll
+            for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, tm, h * 64, 0, g, id, bar);
+          }
+        }
+        any_bad |= (badmask != 0);
+      }
+    }
+    if (lane == 0) {
+      if (any_bad) atomicOr(P.err, ERR_BAD_PAGE);
+      if (aborted) {
+        atomicOr(P.err, ERR_TIMEOUT);
+        atomicExch(&ctrl->abort, 1u);
+      }
+    }
+    return;
+  }
+
+  // ---- consumers: warp w owns query rows [8w, 8w + 8) of the group's group_size * G rows
+  const int R = P.Gs * P.G;
+  const int hq0 = lane >> 2;
+  const int qcol = (lane & 3) * 2;
+  const bool has_rows = warp * 8 < R;
+  for (int u = range.x; u < range.y; ++u) {
+    const int gi = u / P.Hkv, g = u - gi * P.Hkv;
+    const int pt = __ldg(P.prefix_tiles + gi);
+    if (pt <= 0) continue;
+    const int s0 = gi * P.Gs;
+    uint32_t qf[1][D / 16][2];
+    {
+      const int r = warp * 8 + hq0;
+      const bool live = r < R;
+      const int j = live ? r / P.G : 0, h = live ? r - j * P.G : 0;
+      const uint32_t* qp =
+          reinterpret_cast<const uint32_t*>(P.q + (static_cast<int64_t>(s0 + j) * P.Hq + g * P.G + h) * D);
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        qf[0][kk][0] = live ? __ldg(qp + (kk * 16 + qcol) / 2) : 0u;
+        qf[0][kk][1] = live ? __ldg(qp + (kk * 16 + 8 + qcol) / 2) : 0u;
+      }
+    }
+    float acc[1][D / 16][4];
+    float m[1][2] = {{NEG_INF, NEG_INF}}, l[1][2] = {{0.f, 0.f}};
+#pragma unroll
+    for (int jm = 0; jm < D / 16; ++jm) acc[0][jm][0] = acc[0][jm][1] = acc[0][jm][2] = acc[0][jm][3] = 0.f;
+    for (int t = 0; t < pt; ++t, ++it) {
+      if (!aborted && *reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) aborted = true;
+      if (aborted) continue;
+      const int slot = it % NST;
+      const uint32_t phase = (it / NST) & 1;
+      if (!mbar_wait(smem_u32(&ctrl->full[slot]), phase)) {
+        aborted = true;
+        if (lane == 0) {
+          atomicOr(P.err, ERR_TIMEOUT);
+          atomicExch(&ctrl->abort, 1u);
+        }
+        continue;
+      }
+      if (has_rows) {
+        const uint32_t sK = ring + slot * C::STAGE_BYTES;
+        compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, P.scale_log2, TILE, ctrl->meta[slot], lane);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
+    }
+    if (has_rows && !aborted) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float v = l[0][e];
+        v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        l[0][e] = v;
+      }
+      const int drow = lane >> 2;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int r = warp * 8 + qcol + e;
+        if (r < R) {
+          const int j = r / P.G, h = r - j * P.G;
+          float* slotp = P.pfx_partials + (static_cast<int64_t>(s0 + j) * P.Hkv + g) * C::SLOT_FLOATS;
+          if (lane < 4) {
+            slotp[h] = m[0][e];
+            slotp[C::HP + h] = l[0][e];
+          }
+          float* a = slotp + 2 * C::HP + h * D;
+#pragma unroll
+          for (int jm = 0; jm < D / 16; ++jm) {
+            a[jm * 16 + drow] = acc[0][jm][e];
+            a[jm * 16 + drow + 8] = acc[0][jm][2 + e];
+          }
+        }
+      }
+    }
+  }
+  if (aborted && lane == 0) atomicOr(P.err, ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------
 // KV append: the step on the input side of decode attention.  Block s writes the new token's K
 // and V rows of every KV head into slot L_s % bs of page block_table[s, L_s / bs] and then
 // advances context_lens[s].  One warp per KV head: lanes copy 16-byte chunks, K then V.
@@ -936,7 +1159,8 @@ stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __rest
 template <int D, int NT>
 __global__ void __launch_bounds__(256)
 combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, const float* __restrict__ partials,
-               __nv_bfloat16* __restrict__ out, int Hq, int Hkv, int G) {
+               __nv_bfloat16* __restrict__ out, int Hq, int Hkv, int G, const int32_t* __restrict__ start_tiles,
+               const float* __restrict__ pfx_partials) {
   constexpr int HP = 8 * NT;
   constexpr int SLOT_FLOATS = HP * (D + 2);
   const int c = blockIdx.x;
@@ -962,21 +1186,24 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
   __syncthreads();
   const int np = n_follow + 1;
   const int s = unit / Hkv, g = unit - s * Hkv;
+  // piece -1: the partial of the unit's leading tiles when those were handled elsewhere (shared prefix)
+  const int p0 = (start_tiles && start_tiles[s] > 0) ? -1 : 0;
+  auto piece = [&](int p) -> const float* {
+    if (p < 0) return pfx_partials + static_cast<int64_t>(unit) * SLOT_FLOATS;
+    return partials + (p == 0 ? static_cast<int64_t>(c) * 2 + r.w : static_cast<int64_t>(follow[p - 1]) * 2) * SLOT_FLOATS;
+  };
   const float NEG_INF = __int_as_float(0xff800000);
   for (int idx = threadIdx.x; idx < HP * (D / 4); idx += blockDim.x) {
     const int h = idx / (D / 4);
     const int dq = idx % (D / 4);
     if (h >= G) continue;
     float M = NEG_INF;
-    for (int p = 0; p < np; ++p) {
-      const float* part = partials + (p == 0 ? static_cast<int64_t>(c) * 2 + r.w : static_cast<int64_t>(follow[p - 1]) * 2) * SLOT_FLOATS;
-      M = fmaxf(M, part[h]);
-    }
+    for (int p = p0; p < np; ++p) M = fmaxf(M, piece(p)[h]);
     const float Mu = (M == NEG_INF) ? 0.f : M;
     float Ls = 0.f;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int p = 0; p < np; ++p) {
-      const float* part = partials + (p == 0 ? static_cast<int64_t>(c) * 2 + r.w : static_cast<int64_t>(follow[p - 1]) * 2) * SLOT_FLOATS;
+    for (int p = p0; p < np; ++p) {
+      const float* part = piece(p);
       const float f = fast_exp2(part[h] - Mu);
       Ls += part[HP + h] * f;
       const float4 v = *reinterpret_cast<const float4*>(part + 2 * HP + h * D + dq * 4);
@@ -1022,8 +1249,8 @@ __device__ __forceinline__ int block_scan_1024(int v, int* warp_sums, int lane, 
 }
 
 __global__ void __launch_bounds__(1024)
-plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_static, int n_dyn_max,
-            int32_t* __restrict__ prefix, SpanStart* __restrict__ spans, WsHeader* hdr) {
+plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict__ start_tiles, int S, int Hkv,
+            int n_static, int n_dyn_max, int32_t* __restrict__ prefix, SpanStart* __restrict__ spans, WsHeader* hdr) {
   __shared__ int warp_sums[32];
   __shared__ int carry_c, carry_t;
   __shared__ PlanParams pp_s;
@@ -1038,10 +1265,7 @@ plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_stat
   for (int base = 0; base < S; base += 1024) {
     const int s = base + tid;
     int nt = 0;
-    if (s < S) {
-      const int L = context_lens[s];
-      nt = L > 0 ? (L + TILE - 1) / TILE : 0;
-    }
+    if (s < S) nt = static_cast<int>(seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0));
     const int ic = block_scan_1024(static_cast<int>(seq_cost(nt, Hkv)), warp_sums, lane, wid) + carry_c;
     const int itl = block_scan_1024(nt * Hkv, warp_sums, lane, wid) + carry_t;
     if (s < S) {
@@ -1077,8 +1301,7 @@ plan_kernel(const int32_t* __restrict__ context_lens, int S, int Hkv, int n_stat
         const int mid = (lo + hi) >> 1;
         if (pcost[mid] <= x) lo = mid; else hi = mid;
       }
-      const int L = context_lens[lo];
-      const int nt = (L + TILE - 1) / TILE;
+      const int nt = static_cast<int>(seq_tiles(context_lens[lo], start_tiles ? start_tiles[lo] : 0));
       int k, tile;
       locate_in_seq(x - pcost[lo], nt, &k, &tile);
       sp.unit = lo * Hkv + k;

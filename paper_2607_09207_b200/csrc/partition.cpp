@@ -2,15 +2,14 @@
 
 namespace pdattn {
 
-bool plan_spans(const int32_t* context_lens, int num_seqs, int num_kv_heads, int n_static, int dyn_per_cta,
-                int max_spans, SpanStart* spans, PlanParams* plan) {
+bool plan_spans(const int32_t* context_lens, const int32_t* start_tiles, int num_seqs, int num_kv_heads,
+                int n_static, int dyn_per_cta, int max_spans, SpanStart* spans, PlanParams* plan) {
   if (num_seqs < 0 || num_kv_heads <= 0 || n_static <= 0 || max_spans < n_static || !spans || !plan) return false;
   if (dyn_per_cta < 0 || dyn_per_cta > kMaxDynPerCta) return false;
   if (num_seqs > 0 && !context_lens) return false;
   int64_t total = 0, cost = 0;
   for (int s = 0; s < num_seqs; ++s) {
-    const int64_t L = context_lens[s] > 0 ? context_lens[s] : 0;
-    const int64_t nt = (L + kTileTokens - 1) / kTileTokens;
+    const int64_t nt = seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0);
     total += nt * num_kv_heads;
     cost += seq_cost(nt, num_kv_heads);
   }
@@ -26,8 +25,7 @@ bool plan_spans(const int32_t* context_lens, int num_seqs, int num_kv_heads, int
   int64_t cbase = 0;   // cost coordinate of the current sequence's start
   int64_t tbase = 0;   // flattened tile index of its first tile
   for (int s = 0; s < num_seqs && c < n_spans; ++s) {
-    const int64_t L = context_lens[s] > 0 ? context_lens[s] : 0;
-    const int64_t nt = (L + kTileTokens - 1) / kTileTokens;
+    const int64_t nt = seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0);
     const int64_t sc = seq_cost(nt, num_kv_heads);
     while (c < n_spans) {
       const int64_t x = span_cost_start(p, c);

@@ -83,7 +83,14 @@ PDATTN_HD inline void locate_in_seq(int64_t r, int64_t nt, int* k, int* tile) {
 
 // spans: [n_static + n_dyn + 1] entries; at most max_spans + 1 are written and n_dyn is lowered
 // to fit.  Returns false on invalid arguments.
-bool plan_spans(const int32_t* context_lens, int num_seqs, int num_kv_heads, int n_static, int dyn_per_cta,
-                int max_spans, SpanStart* spans, PlanParams* plan);
+// start_tiles (may be null): per sequence, leading tiles that this plan leaves out.
+bool plan_spans(const int32_t* context_lens, const int32_t* start_tiles, int num_seqs, int num_kv_heads,
+                int n_static, int dyn_per_cta, int max_spans, SpanStart* spans, PlanParams* plan);
+
+// tiles of one sequence that a plan covers
+PDATTN_HD inline int64_t seq_tiles(int64_t context_len, int64_t start_tile) {
+  const int64_t all = context_len > 0 ? (context_len + kTileTokens - 1) / kTileTokens : 0;
+  return all > start_tile ? all - start_tile : 0;
+}
 
 }  // namespace pdattn

@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "../../include/pdattn.h"
 #include "kernels.cuh"
@@ -20,6 +21,14 @@ thread_local char g_cuda_err[256] = "";
 thread_local int g_last_launches = 0;
 thread_local cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 thread_local bool g_probe_mode = false;   // set only inside pdattn_gather_probe
+struct GroupedCall {                      // set only inside pdattn_decode_grouped
+  bool active = false;
+  int group_size = 0;
+  const int32_t* prefix_tiles = nullptr;        // device, per group
+  const int32_t* prefix_tiles_host = nullptr;   // host copy
+};
+thread_local GroupedCall g_grouped;
+thread_local std::vector<int32_t> g_start_tiles_host;
 int g_dyn_per_cta = 0;                    // run-time spans per CTA (pdattn_set_dynamic_spans)
 
 struct Binding {
@@ -69,6 +78,7 @@ struct DevInfo {
   bool ready = false;
   int sm_count = 0;
   bool attr_set[2][2] = {{false, false}, {false, false}};   // [D==128][NT==2]
+  bool prefix_attr_set[2] = {false, false};
 };
 constexpr int kMaxDevices = 64;
 DevInfo g_dev[kMaxDevices];
@@ -220,9 +230,28 @@ pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeP
   if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
   if (g_prof_stop) cudaEventRecord(g_prof_stop, stream);
   combine_kernel<D, NT><<<combine_grid, 256, 0, stream>>>(P.hdr, n_spans_host, P.rec, P.partials, P.out, P.Hq, P.Hkv,
-                                                          P.G);
+                                                          P.G, P.start_tiles, P.pfx_partials);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("combine_kernel launch", e);
+  return PDATTN_OK;
+}
+
+template <int D>
+pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
+                            cudaStream_t stream) {
+  using C = Cfg<D, 1, 16>;
+  const int smem = 1024 + C::NSTAGES * C::STAGE_BYTES + C::CTRL_BYTES;
+  auto kern = prefix_kernel<D, 16>;
+  bool& done = di->prefix_attr_set[D == 128];
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
+    done = true;
+  }
+  if (grid <= 0) return PDATTN_OK;
+  kern<<<grid, C::NTHREADS, smem, stream>>>(mk, mv, X);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("prefix_kernel launch", e);
   return PDATTN_OK;
 }
 
@@ -285,7 +314,7 @@ pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, i
   PlanParams plan;
   if (!spans || max_spans < n_ctas) return PDATTN_INVALID_ARG;
   static_assert(sizeof(SpanStart) == 4 * sizeof(int32_t), "span table entries are four int32");
-  if (!plan_spans(context_lens_host, num_seqs, num_kv_heads, n_ctas, dynamic_per_cta, max_spans,
+  if (!plan_spans(context_lens_host, nullptr, num_seqs, num_kv_heads, n_ctas, dynamic_per_cta, max_spans,
                   reinterpret_cast<SpanStart*>(spans), &plan))
     return PDATTN_INVALID_ARG;
   plan_out->n_static = plan.n_static;
@@ -310,7 +339,30 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     return PDATTN_MISALIGNED;
   const int G = a->num_q_heads / a->num_kv_heads;
   const WsLayout wl = ws_layout(a->num_seqs, G, a->head_dim);
-  if (a->workspace_bytes < wl.total) return PDATTN_WORKSPACE_TOO_SMALL;
+  // grouped calls keep two more arrays behind the ordinary layout
+  const bool grouped = g_grouped.active;
+  const size_t off_start = wl.total;
+  const size_t off_pfx = off_start + align_up(static_cast<size_t>(a->num_seqs) * 4, 256);
+  const size_t pfx_bytes = static_cast<size_t>(a->num_seqs) * a->num_kv_heads * (G > 8 ? 16 : 8) * (a->head_dim + 2) * 4;
+  const size_t need = grouped ? off_pfx + align_up(pfx_bytes, 256) : wl.total;
+  if (a->workspace_bytes < need) return PDATTN_WORKSPACE_TOO_SMALL;
+  const int32_t* start_tiles_host = nullptr;
+  int n_groups = 0;
+  if (grouped) {
+    const int Gs = g_grouped.group_size;
+    if (!a->context_lens_host || Gs <= 0 || a->num_seqs % Gs != 0 || G > 8 || Gs * G > MAX_PREFIX_ROWS)
+      return Gs > 0 && (G > 8 || Gs * G > MAX_PREFIX_ROWS) ? PDATTN_UNSUPPORTED : PDATTN_INVALID_ARG;
+    n_groups = a->num_seqs / Gs;
+    g_start_tiles_host.resize(a->num_seqs);
+    for (int sq = 0; sq < a->num_seqs; ++sq) {
+      const int pt = g_grouped.prefix_tiles_host[sq / Gs];
+      // every member must own at least one token past the shared tiles
+      if (pt < 0 || static_cast<int64_t>(pt) * kTileTokens >= a->context_lens_host[sq]) return PDATTN_INVALID_ARG;
+      if (static_cast<int64_t>(pt) * kTileTokens / a->block_size > a->max_blocks_per_seq) return PDATTN_INVALID_ARG;
+      g_start_tiles_host[sq] = pt;
+    }
+    start_tiles_host = g_start_tiles_host.data();
+  }
 
   int dev = 0;
   DevInfo* di = nullptr;
@@ -325,6 +377,8 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   P.out = static_cast<__nv_bfloat16*>(a->out);
   P.block_table = a->block_table;
   P.context_lens = a->context_lens;
+  P.start_tiles = nullptr;
+  P.pfx_partials = nullptr;
   P.hdr = reinterpret_cast<WsHeader*>(ws + wl.hdr);
   P.spans_ws = reinterpret_cast<const SpanStart*>(ws + wl.spans);
   P.rec = reinterpret_cast<int4*>(ws + wl.rec);
@@ -344,8 +398,8 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   const int dyn_per_cta = g_dyn_per_cta;
   int grid = n_ctas, combine_grid = 0, n_spans_host = -1;
   if (a->context_lens_host) {
-    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta, MAX_PARAM_SPANS, P.spans,
-                    &P.plan))
+    if (!plan_spans(a->context_lens_host, start_tiles_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta,
+                    MAX_PARAM_SPANS, P.spans, &P.plan))
       return PDATTN_INVALID_ARG;
     n_spans_host = P.plan.n_static + P.plan.n_dyn;
     combine_grid = n_spans_host;
@@ -353,7 +407,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     P.use_ws_plan = 1;
     memset(&P.plan, 0, sizeof P.plan);
     const int n_dyn_max = n_ctas * dyn_per_cta;
-    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
+    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, nullptr, a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
                                          reinterpret_cast<int32_t*>(ws + wl.prefix),
                                          reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr);
     cudaError_t e = cudaGetLastError();
@@ -380,6 +434,48 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   if (s != PDATTN_OK) return s;
   P.box5d = rank == 5;
 
+  if (grouped) {
+    // shared prompt tiles first: one pass per (group, kv head) for the query rows of all samples
+    PrefixParams X;
+    X.q = P.q;
+    X.block_table = a->block_table;
+    X.prefix_tiles = g_grouped.prefix_tiles;
+    X.start_tiles = reinterpret_cast<int32_t*>(ws + off_start);
+    X.pfx_partials = reinterpret_cast<float*>(ws + off_pfx);
+    X.err = &P.hdr->err;
+    X.S = a->num_seqs;
+    X.Hq = a->num_q_heads;
+    X.Hkv = a->num_kv_heads;
+    X.G = G;
+    X.Gs = g_grouped.group_size;
+    X.MB = a->max_blocks_per_seq;
+    X.NB = a->num_blocks;
+    X.scale_log2 = P.scale_log2;
+    X.box5d = P.box5d;
+    // whole units, contiguous ranges of equal tile count (to within one unit)
+    const int n_units = n_groups * a->num_kv_heads;
+    int64_t total = 0;
+    for (int gi = 0; gi < n_groups; ++gi) total += static_cast<int64_t>(g_grouped.prefix_tiles_host[gi]) * a->num_kv_heads;
+    int pgrid = n_ctas < 160 ? n_ctas : 160;
+    if (pgrid > n_units) pgrid = n_units;
+    int u = 0;
+    int64_t done = 0;
+    for (int c = 0; c < pgrid; ++c) {
+      const int64_t target = total * (c + 1) / pgrid;
+      const int u0 = u;
+      while (u < n_units && (done < target || c == pgrid - 1)) {
+        done += g_grouped.prefix_tiles_host[u / a->num_kv_heads];
+        ++u;
+      }
+      X.ranges[c] = make_int2(u0, u);
+    }
+    s = a->head_dim == 128 ? launch_prefix<128>(mk, mv, X, pgrid, di, stream) : launch_prefix<64>(mk, mv, X, pgrid, di, stream);
+    if (s != PDATTN_OK) return s;
+    g_last_launches += 1;
+    P.start_tiles = X.start_tiles;
+    P.pfx_partials = X.pfx_partials;
+  }
+
   const bool nt2 = G > 8;
   if (a->head_dim == 128)
     s = nt2 ? launch<128, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
@@ -388,6 +484,30 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
             : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
   if (s == PDATTN_OK) g_last_launches += 2;
+  return s;
+}
+
+pdattn_status pdattn_grouped_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                                            int block_size, size_t* device_bytes) {
+  if (!device_bytes) return PDATTN_INVALID_ARG;
+  pdattn_status s = check_shape(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size);
+  if (s != PDATTN_OK) return s;
+  const int G = num_q_heads / num_kv_heads;
+  const size_t base = ws_layout(num_seqs, G, head_dim).total;
+  const size_t pfx = static_cast<size_t>(num_seqs) * num_kv_heads * (G > 8 ? 16 : 8) * (head_dim + 2) * 4;
+  *device_bytes = base + align_up(static_cast<size_t>(num_seqs) * 4, 256) + align_up(pfx, 256);
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_decode_grouped(const pdattn_args* args, int group_size, const int32_t* prefix_tiles,
+                                    const int32_t* prefix_tiles_host, pdattn_stream_t stream) {
+  if (!args || !prefix_tiles || !prefix_tiles_host) return PDATTN_INVALID_ARG;
+  g_grouped.active = true;
+  g_grouped.group_size = group_size;
+  g_grouped.prefix_tiles = prefix_tiles;
+  g_grouped.prefix_tiles_host = prefix_tiles_host;
+  const pdattn_status s = pdattn_decode_ex(args, stream);
+  g_grouped = GroupedCall();
   return s;
 }
 
@@ -601,6 +721,8 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   P.out = static_cast<__nv_bfloat16*>(a->out);
   P.block_table = a->block_table;
   P.context_lens = a->context_lens;
+  P.start_tiles = nullptr;
+  P.pfx_partials = nullptr;
   P.hdr = reinterpret_cast<WsHeader*>(ws);
   P.spans_ws = reinterpret_cast<const SpanStart*>(ws + off_spans);
   P.rec = reinterpret_cast<int4*>(ws + off_rec);
@@ -616,14 +738,14 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   P.box5d = 0;
   int grid = n_ctas, combine_grid = n_ctas, n_spans_host = -1;
   if (a->context_lens_host) {
-    if (!plan_spans(a->context_lens_host, a->num_seqs, a->num_kv_heads, n_ctas, 0, n_ctas, P.spans, &P.plan))
+    if (!plan_spans(a->context_lens_host, nullptr, a->num_seqs, a->num_kv_heads, n_ctas, 0, n_ctas, P.spans, &P.plan))
       return PDATTN_INVALID_ARG;
     n_spans_host = n_ctas;
     combine_grid = n_ctas;
   } else {
     P.use_ws_plan = 1;
     memset(&P.plan, 0, sizeof P.plan);
-    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, a->num_seqs, a->num_kv_heads, n_ctas, 0,
+    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, nullptr, a->num_seqs, a->num_kv_heads, n_ctas, 0,
                                          reinterpret_cast<int32_t*>(ws + off_prefix),
                                          reinterpret_cast<SpanStart*>(ws + off_spans), P.hdr);
     e = cudaGetLastError();

@@ -32,6 +32,7 @@ EXPORTS = [
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_set_dynamic_spans",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
+    "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
 ]
 
 
@@ -87,6 +88,8 @@ def lib():
         L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(Plan)]
         L.pdattn_set_dynamic_spans.argtypes = [i32]
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
+        L.pdattn_grouped_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
+        L.pdattn_decode_grouped.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
         L.pdattn_append_kv.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp]
         L.pdattn_check.argtypes = [vp, vp]
         L.pdattn_profile_events.argtypes = [vp, vp]
@@ -179,6 +182,48 @@ def decode_static_scratch(q, k_cache, v_cache, block_table, context_lens, scale,
                                             _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_decode_static_scratch")
+    return st
+
+
+def grouped_workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size=16) -> int:
+    n = ctypes.c_size_t(0)
+    st = lib().pdattn_grouped_workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size, ctypes.byref(n))
+    if st != OK:
+        raise PdattnError(st, "pdattn_grouped_workspace_size")
+    return n.value
+
+
+def alloc_grouped_workspace(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size=16, device="cuda", stream=None):
+    n = grouped_workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    st = lib().pdattn_workspace_init(ws.data_ptr(), n, _stream_ptr(stream))
+    if st != OK:
+        raise PdattnError(st, "pdattn_workspace_init")
+    return ws
+
+
+def decode_grouped(q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, context_lens_host,
+                   group_size, prefix_tiles, prefix_tiles_host, stream=None, check: bool = True) -> int:
+    """pdattn_decode_grouped: sequences come in groups of `group_size` whose first prefix_tiles[g] * 64 tokens
+    are the same physical pages (GRPO samples of one prompt); those tiles are read once per group."""
+    S, Hq, d = q.shape
+    NB, Hkv, bs, _ = k_cache.shape
+    a = Args()
+    a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr()
+    a.block_table, a.context_lens = block_table.data_ptr(), context_lens.data_ptr()
+    lens = np.ascontiguousarray(context_lens_host, dtype=np.int32)
+    a.context_lens_host = lens.ctypes.data
+    a.num_seqs, a.num_q_heads, a.num_kv_heads, a.head_dim, a.block_size = S, Hq, Hkv, d, bs
+    a.max_blocks_per_seq = block_table.shape[1]
+    a.num_blocks = NB
+    a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
+    a.scale = float(scale)
+    a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    pth = np.ascontiguousarray(prefix_tiles_host, dtype=np.int32)
+    st = lib().pdattn_decode_grouped(ctypes.byref(a), int(group_size), prefix_tiles.data_ptr(), pth.ctypes.data,
+                                     _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_grouped")
     return st
 
 

@@ -1,0 +1,106 @@
+"""Shared-prefix (GRPO group) decode: the prompt tiles of a group are read once and scored against the
+query rows of all its samples.  The result must be the plain definition the oracle computes."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import pdattn_oracle as orc
+from paper_2607_09207_b200 import pdattn
+from paper_2607_09207_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def run_grouped(w, group, prefix_tiles_host):
+    ws = pdattn.alloc_grouped_workspace(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim)
+    pt = torch.tensor(prefix_tiles_host, dtype=torch.int32, device=DEV)
+    out = torch.empty_like(w.q)
+    pdattn.decode_grouped(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws,
+                          w.context_lens_host, group, pt, np.asarray(prefix_tiles_host, dtype=np.int32))
+    st = pdattn.check(ws)
+    return out, st
+
+
+def assert_parity(out, ref, what):
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all(), what
+    err = np.abs(got - ref)
+    bad = err > np.maximum(2e-3, 1e-2 * np.abs(ref))
+    assert not bad.any(), f"{what}: {int(bad.sum())} bad, max err {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
+
+
+def test_scaled_grpo_config_all_outputs():
+    w = W.make_config(3, device=DEV, num_seqs=32, len_div=4)          # prompt 256 tokens = 4 tiles, 4 groups of 8
+    out, st = run_grouped(w, 8, [4, 4, 4, 4])
+    assert st == pdattn.OK
+    assert_parity(out, orc.decode_workload(w.to("cpu")), "config 3 scaled, grouped")
+    again, _ = run_grouped(w, 8, [4, 4, 4, 4])
+    assert torch.equal(out, again)                                    # run to run
+    plain = pdattn.decode_workload(w)
+    assert_parity(plain, orc.decode_workload(w.to("cpu")), "config 3 scaled, plain")
+
+
+@pytest.mark.parametrize("Hq,Hkv,group", [(40, 8, 8), (28, 4, 4), (8, 2, 8), (6, 6, 3), (32, 4, 6)])
+def test_groups_with_uneven_prefixes_and_head_counts(Hq, Hkv, group):
+    """Groups that share 0, 1, 5 and 16 tiles; members only a token longer than the prefix; prefix
+    lengths that are not whole tiles in the table (only whole tiles are declared shared)."""
+    rng = np.random.default_rng(Hq * 100 + group)
+    shared_tokens = [0, 70, 330, 1024]                  # -> 0, 1, 5, 16 whole tiles
+    lens, tiles = [], []
+    for st in shared_tokens:
+        tiles.append(st // 64)
+        for j in range(group):
+            extra = 1 if j == 0 else int(rng.integers(1, 700))
+            lens.append(st + extra)
+    # build with whole shared pages = floor(shared tokens / 16)
+    w = None
+    parts = []
+    # one workload with per-group shared pages: build rows by hand
+    S = len(lens)
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=128, seed=50 + group, device=DEV, poison=False)
+    bt = w.block_table.clone()
+    for gi, st in enumerate(shared_tokens):
+        pages = st // 16
+        lead = gi * group
+        for j in range(1, group):
+            bt[lead + j, :pages] = bt[lead, :pages]
+    w = dataclasses.replace(w, block_table=bt)
+    W.poison_unused(w)
+    out, status = run_grouped(w, group, tiles)
+    assert status == pdattn.OK
+    assert_parity(out, orc.decode_workload(w.to("cpu")), f"Hq={Hq} Hkv={Hkv} group={group}")
+
+
+def test_full_size_grpo_config_sampled():
+    w = W.make_config(3, device=DEV)
+    tiles = [16] * 64
+    out, st = run_grouped(w, 8, tiles)
+    assert st == pdattn.OK
+    rng = np.random.default_rng(3)
+    L = w.context_lens_host
+    seqs = sorted(set(rng.integers(0, 512, size=5).tolist()) | {int(np.argmax(L)), int(np.argmin(L)), 0, 511})
+    pairs = np.array([(s, int(h)) for s in seqs for h in rng.choice(40, size=3, replace=False)], dtype=np.int32)
+    ref = orc.decode_workload(w.to("cpu"), pairs=pairs)
+    got = out[torch.as_tensor(pairs[:, 0], device=DEV), torch.as_tensor(pairs[:, 1], device=DEV)]
+    assert_parity(got, ref, "config 3 full, grouped")
+    again, _ = run_grouped(w, 8, tiles)
+    assert torch.equal(out, again)
+
+
+def test_grouped_rejects_what_it_cannot_do():
+    w = W.make_config(3, device=DEV, num_seqs=16, len_div=4)
+    ws = pdattn.alloc_grouped_workspace(16, 40, 8, 128)
+    pt = torch.tensor([4, 4], dtype=torch.int32, device=DEV)
+    out = torch.empty_like(w.q)
+    args = (w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws, w.context_lens_host)
+    assert pdattn.decode_grouped(*args, 8, pt, [4, 4], check=False) == pdattn.OK
+    assert pdattn.decode_grouped(*args, 5, pt, [4, 4], check=False) == pdattn.INVALID_ARG        # 16 % 5
+    assert pdattn.decode_grouped(*args, 16, pt, [4], check=False) == pdattn.UNSUPPORTED          # 16 * 5 rows > 48
+    too_long = [int(w.context_lens_host[:8].min()) // 64 + 1, 4]
+    assert pdattn.decode_grouped(*args, 8, pt, too_long, check=False) == pdattn.INVALID_ARG      # prefix >= a member
+    small = pdattn.alloc_workspace(16, 40, 8, 128)
+    a2 = args[:7] + (small,) + args[8:]
+    assert pdattn.decode_grouped(*a2, 8, pt, [4, 4], check=False) == pdattn.WORKSPACE_TOO_SMALL
