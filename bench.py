@@ -340,6 +340,17 @@ def main():
         assert pdattn.check(ws) == pdattn.OK
         if args.cfg == 2 and args.num_seqs is None:
             extras["decode_loop"] = decode_loop(pdattn, W, dev, stream)
+        if args.cfg == 3 and args.num_seqs is None:
+            # GRPO groups of 8 share their 1024-token prompt pages: read them once per group
+            gws = pdattn.alloc_grouped_workspace(S, c.num_q_heads, c.num_kv_heads, c.head_dim, device=dev)
+            pth = np.full(S // 8, 1024 // 64, dtype=np.int32)
+            ptd = torch.from_numpy(pth).to(dev)
+            t_grouped = timed(lambda: pdattn.decode_grouped(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens,
+                                                            c.scale, outs[0], gws, c.context_lens_host, 8, ptd, pth),
+                              n=10)
+            assert pdattn.check(gws) == pdattn.OK
+            extras["grouped_shared_prefix"] = {"ms_per_step": t_grouped, "seq_steps_per_s": S / (t_grouped * 1e-3),
+                                               "unique_kv_gbs": uniq / (t_grouped * 1e-3) / 1e9}
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only)
     cpu_baseline = None
