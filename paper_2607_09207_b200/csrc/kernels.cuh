@@ -903,7 +903,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 // which decode_kernel / combine_kernel fold into the sequence's result.  Units (group * Hkv + kv
 // head) are never cut: CTA c takes units [ranges[c].x, ranges[c].y).
 // ------------------------------------------------------------------------------------------
-constexpr int MAX_PREFIX_ROWS = 48;
+constexpr int MAX_PREFIX_ROWS = 8 * (PDATTN_NCW < 6 ? PDATTN_NCW : 6);   // eight query rows per consumer warp
 struct PrefixParams {
   const __nv_bfloat16* q;
   const int32_t* block_table;
