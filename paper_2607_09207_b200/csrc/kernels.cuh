@@ -204,7 +204,7 @@ struct Cfg {
   static constexpr int NSTAGES_FIT = (SMEM_MAX - 1024 - QSLOTS * Q_BYTES - ML_BYTES - CTRL_BYTES) / STAGE_BYTES;
   static constexpr int NSTAGES = (NSTAGES_FIT > MAX_STAGES ? MAX_STAGES : NSTAGES_FIT) / NCW * NCW;
   static constexpr int NCT = NCW * 32;                                 // consumer threads
-  static constexpr int NPW = PDATTN_NPW;                               // producer warps
+  static constexpr int NPW = (NT == 2 && PDATTN_NPW > 2) ? 2 : PDATTN_NPW;   // producer warps (8 warps in all for 16-row tiles: 255 registers)
   static constexpr int NTHREADS = NCT + 32 * NPW;
   static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + QSLOTS * Q_BYTES + ML_BYTES + CTRL_BYTES;
   static constexpr int SLOT_FLOATS = HP * (D + 2);     // one partial: m[HP], l[HP], acc[HP][D]

@@ -68,7 +68,7 @@ pdattn_status check_shape(int num_seqs, int Hq, int Hkv, int d, int bs) {
   if (num_seqs < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || bs <= 0) return PDATTN_INVALID_ARG;
   if (Hq % Hkv != 0) return PDATTN_INVALID_ARG;
   if (d != 64 && d != 128) return PDATTN_UNSUPPORTED;
-  if (bs != 16) return PDATTN_UNSUPPORTED;
+  if (bs != 16 && bs != 32) return PDATTN_UNSUPPORTED;
   if (Hq / Hkv > 16) return PDATTN_UNSUPPORTED;
   return PDATTN_OK;
 }
@@ -77,8 +77,9 @@ pdattn_status check_shape(int num_seqs, int Hq, int Hkv, int d, int bs) {
 struct DevInfo {
   bool ready = false;
   int sm_count = 0;
-  bool attr_set[2][2] = {{false, false}, {false, false}};   // [D==128][NT==2]
-  bool prefix_attr_set[2] = {false, false};
+  bool attr_set[2][2][2] = {};      // [D==128][NT==2][BS==32]
+  bool probe_attr_set[2][2][2] = {};
+  bool prefix_attr_set[2][2] = {};  // [D==128][BS==32]
 };
 constexpr int kMaxDevices = 64;
 DevInfo g_dev[kMaxDevices];
@@ -202,19 +203,19 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
 }
 
 // ---- launches ------------------------------------------------------------------------------------
-template <int D, int NT>
-pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
+template <int D, int NT, int BS>
+pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
                      int n_spans_host, DevInfo* di, cudaStream_t stream) {
-  using C = Cfg<D, NT, 16>;
-  auto kern = decode_kernel<D, NT, 16>;
-  bool& done = di->attr_set[D == 128][NT == 2];
+  using C = Cfg<D, NT, BS>;
+  auto kern = decode_kernel<D, NT, BS>;
+  bool& done = di->attr_set[D == 128][NT == 2][BS == 32];
   if (!done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
     done = true;
   }
   if (g_probe_mode) {
-    auto probe = decode_kernel<D, NT, 16, true>;
+    auto probe = decode_kernel<D, NT, BS, true>;
     cudaError_t pe = cudaFuncSetAttribute(probe, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
     if (pe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", pe);
     probe<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
@@ -236,13 +237,13 @@ pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeP
   return PDATTN_OK;
 }
 
-template <int D>
-pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
+template <int D, int BS>
+pdattn_status launch_prefix_bs(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
                             cudaStream_t stream) {
-  using C = Cfg<D, 1, 16>;
+  using C = Cfg<D, 1, BS>;
   const int smem = 1024 + C::NSTAGES * C::STAGE_BYTES + C::CTRL_BYTES;
-  auto kern = prefix_kernel<D, 16>;
-  bool& done = di->prefix_attr_set[D == 128];
+  auto kern = prefix_kernel<D, BS>;
+  bool& done = di->prefix_attr_set[D == 128][BS == 32];
   if (!done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
@@ -253,6 +254,21 @@ pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("prefix_kernel launch", e);
   return PDATTN_OK;
+}
+
+thread_local int g_block_size = 16;   // page size of the call being launched (set by the entry points)
+
+template <int D, int NT>
+pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
+                     int n_spans_host, DevInfo* di, cudaStream_t stream) {
+  return g_block_size == 32 ? launch_bs<D, NT, 32>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
+                            : launch_bs<D, NT, 16>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+}
+template <int D>
+pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
+                            cudaStream_t stream) {
+  return g_block_size == 32 ? launch_prefix_bs<D, 32>(mk, mv, X, grid, di, stream)
+                            : launch_prefix_bs<D, 16>(mk, mv, X, grid, di, stream);
 }
 
 }  // namespace
@@ -285,7 +301,7 @@ pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cac
   if (num_seqs < 0 || num_kv_heads <= 0 || num_kv_heads > 16 || max_blocks_per_seq <= 0 || num_blocks <= 0)
     return PDATTN_INVALID_ARG;
   if (head_dim != 64 && head_dim != 128) return PDATTN_UNSUPPORTED;
-  if (block_size != 16) return PDATTN_UNSUPPORTED;
+  if (block_size != 16 && block_size != 32) return PDATTN_UNSUPPORTED;
   if (num_seqs == 0) return PDATTN_OK;
   if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !context_lens) return PDATTN_INVALID_ARG;
   if (kv_block_stride <= 0 || kv_head_stride <= 0 || kv_token_stride < head_dim) return PDATTN_INVALID_ARG;
@@ -329,6 +345,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   pdattn_status s = check_shape(a->num_seqs, a->num_q_heads, a->num_kv_heads, a->head_dim, a->block_size);
   if (s != PDATTN_OK) return s;
   if (a->num_seqs == 0) return PDATTN_OK;
+  g_block_size = a->block_size;
   if (!a->q || !a->k_cache || !a->v_cache || !a->out || !a->block_table || !a->context_lens || !a->workspace)
     return PDATTN_INVALID_ARG;
   if (a->max_blocks_per_seq <= 0 || a->num_blocks <= 0) return PDATTN_INVALID_ARG;
@@ -677,6 +694,7 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   pdattn_status s = check_shape(a->num_seqs, a->num_q_heads, a->num_kv_heads, a->head_dim, a->block_size);
   if (s != PDATTN_OK) return s;
   if (a->num_seqs == 0) return PDATTN_OK;
+  g_block_size = a->block_size;
   if (!a->q || !a->k_cache || !a->v_cache || !a->out || !a->block_table || !a->context_lens) return PDATTN_INVALID_ARG;
   if (a->max_blocks_per_seq <= 0 || a->num_blocks <= 0) return PDATTN_INVALID_ARG;
   if (a->kv_block_stride <= 0 || a->kv_head_stride <= 0 || a->kv_token_stride < a->head_dim) return PDATTN_INVALID_ARG;

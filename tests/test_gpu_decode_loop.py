@@ -45,6 +45,21 @@ def test_append_is_bit_exact_over_page_boundaries(token_major):
     assert torch.equal(w.v_cache.cpu().view(torch.int16), ref.v_cache.view(torch.int16))
 
 
+def test_append_with_page_size_32_and_head_dim_64():
+    lens = [0, 31, 32, 33, 64]
+    w = W.make_custom(lens, Hq=4, Hkv=2, d=64, bs=32, seed=43, device=DEV, headroom_tokens=40)
+    ref = w.to("cpu")
+    ref = dataclasses.replace(ref, k_cache=ref.k_cache.clone(), v_cache=ref.v_cache.clone(),
+                              context_lens=ref.context_lens.clone())
+    for step in range(34):
+        k_new, v_new = new_rows(len(lens), 2, 64, step)
+        pdattn.append_kv(k_new, v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens)
+        assert orc.append_kv(ref.k_cache, ref.v_cache, ref.block_table, ref.context_lens, k_new.cpu(), v_new.cpu()) == 0
+    assert torch.equal(w.context_lens.cpu(), ref.context_lens)
+    assert torch.equal(w.k_cache.cpu().view(torch.int16), ref.k_cache.view(torch.int16))
+    assert torch.equal(w.v_cache.cpu().view(torch.int16), ref.v_cache.view(torch.int16))
+
+
 def test_append_skips_and_reports_bad_targets():
     w = W.make_custom([16, 5, 31], Hq=4, Hkv=2, d=64, seed=42, device=DEV, num_blocks=32, headroom_tokens=20)
     bt = w.block_table.clone()
