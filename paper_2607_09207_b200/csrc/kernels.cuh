@@ -24,6 +24,9 @@
 #ifndef PDATTN_NCW
 #define PDATTN_NCW 6
 #endif
+#ifndef PDATTN_WAIT_HINT_NS
+#define PDATTN_WAIT_HINT_NS 20000   // suspend-time hint of a waiting mbarrier poll
+#endif
 #ifndef PDATTN_NPW
 #define PDATTN_NPW 3              // producer warps (tile i is issued by producer i mod NPW)
 #endif
@@ -95,19 +98,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same with a suspend-time hint (ns): the thread may sleep in hardware until the phase
+// completes instead of spinning, which is where a waiting warp spends most of this kernel.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: false when the limit expired.
+// Bounded wait: false when the limit expired.  The clock is read once per 64 polls only.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
-  while (!mbar_try_wait(bar, parity)) {
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait_hint(bar, parity, PDATTN_WAIT_HINT_NS)) return true;
     if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
   }
-  return true;
 }
 __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1164,6 +1184,9 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
   constexpr int HP = 8 * NT;
   constexpr int SLOT_FLOATS = HP * (D + 2);
   const int c = blockIdx.x;
+  // launched as a programmatic dependent of the decode kernel: nothing of that kernel may be read
+  // before this returns (it waits for the kernel's completion and memory flush)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (c == 0 && threadIdx.x == 0) hdr->counter = 0;
   const int n_spans = n_spans_host >= 0 ? n_spans_host : hdr->plan.n_static + hdr->plan.n_dyn;
   if (c >= n_spans) return;

@@ -230,9 +230,21 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
   if (g_prof_stop) cudaEventRecord(g_prof_stop, stream);
-  combine_kernel<D, NT><<<combine_grid, 256, 0, stream>>>(P.hdr, n_spans_host, P.rec, P.partials, P.out, P.Hq, P.Hkv,
-                                                          P.G, P.start_tiles, P.pfx_partials);
-  e = cudaGetLastError();
+  // Programmatic dependent launch: the combine grid is set up while the decode kernel drains and
+  // waits (griddepcontrol.wait in the kernel) until that kernel has completed and flushed.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(combine_grid);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = (g_prof_stop == nullptr) ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, combine_kernel<D, NT>, P.hdr, n_spans_host, static_cast<const int4*>(P.rec),
+                         static_cast<const float*>(P.partials), P.out, P.Hq, P.Hkv, P.G, P.start_tiles,
+                         P.pfx_partials);
   if (e != cudaSuccess) return cuda_fail("combine_kernel launch", e);
   return PDATTN_OK;
 }
