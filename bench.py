@@ -53,6 +53,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cfg", type=int, default=2, help="BASELINE.json config index + 1 (default: the metric's config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--grouped", action="store_true",
+                    help="config 3 only: time pdattn_decode_grouped (shared prompt pages read once per group)")
     ap.add_argument("--num-seqs", type=int, default=None,
                     help="shrink the batch (profiling captures only; not the metric's workload)")
     return ap.parse_args()
@@ -193,12 +195,17 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    local = local % torch.cuda.device_count()     # ranks may share a GPU in a functional test of this script
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+        backend = os.environ.get("PDATTN_BENCH_BACKEND", "nccl")   # "gloo" when ranks share one GPU
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group(backend)
 
     K, Wm = args.steps, max(3, args.warmup)
     # ---- inputs: this rank's batch, in two physically distinct copies (pools, tables, q) so that
@@ -215,13 +222,22 @@ def main():
     S = base.num_seqs
     uniq = base.unique_kv_bytes()
     logical = base.logical_kv_bytes()
-    ws = pdattn.alloc_workspace(S, base.num_q_heads, base.num_kv_heads, base.head_dim, base.block_size, device=dev)
+    ws = pdattn.alloc_grouped_workspace(S, base.num_q_heads, base.num_kv_heads, base.head_dim, base.block_size,
+                                        device=dev)
+    grouped = args.grouped and args.cfg == 3
+    if grouped:
+        pth = np.full(S // 8, 1024 // 64, dtype=np.int32)       # 64 shared prompt pages = 16 tiles per group
+        ptd = torch.from_numpy(pth).to(dev)
     outs = [torch.empty_like(c.q) for c in copies]
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
 
     def step(i):
         c = copies[i % len(copies)]
+        if grouped:
+            pdattn.decode_grouped(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale,
+                                  outs[i % len(copies)], ws, c.context_lens_host, 8, ptd, pth, stream=stream)
+            return
         pdattn.decode_ex(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale, outs[i % len(copies)],
                          ws, context_lens_host=c.context_lens_host, stream=stream)
 
@@ -266,6 +282,9 @@ def main():
     L.pdattn_profile_events(None, None)
     torch.cuda.synchronize()
     k1_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    kernel_name = "decode_kernel"
+    if grouped:      # the prefix kernel does part of the reading: account the whole step
+        k1_ms, kernel_name = ms_step, "prefix_kernel + decode_kernel + combine_kernel (whole step)"
     peak, peak_src = measured_peak()
     achieved = uniq / (k1_ms * 1e-3) / 1e9
 
@@ -367,7 +386,8 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": CFG_DESC[args.cfg] + (f" [REDUCED to {S} seqs]" if args.num_seqs else ""),
+            "config": {"workload": CFG_DESC[args.cfg] + (f" [REDUCED to {S} seqs]" if args.num_seqs else "")
+                       + (" [grouped: shared prompt tiles read once per group]" if grouped else ""),
                        "num_seqs_per_gpu": S,
                        "unique_kv_bytes_per_step": uniq, "logical_kv_bytes_per_step": logical,
                        "l2": f"inputs ({uniq / 1e9:.2f} GB) larger than L2 and steps rotate over {len(copies)} "
@@ -380,7 +400,7 @@ def main():
             "pct_of_8tbs_nominal_step": uniq / (ms_step * 1e-3) / 8e12 * 100.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": profiled_traffic(args.cfg),
-                         "kernel": "decode_kernel", "kernel_ms": k1_ms, "peak_source": peak_src,
+                         "kernel": kernel_name, "kernel_ms": k1_ms, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": uniq,
                          "pct_of_8tbs_nominal": achieved / 8000.0 * 100.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
