@@ -203,6 +203,18 @@ pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, i
 pdattn_status pdattn_set_dynamic_spans(int per_cta);
 
 /*
+ * Process-wide choice of how the consumer warps of a CTA merge their online-softmax states at
+ * the end of a piece (a sequence's run of tiles inside one span).  1: the state is handed down a
+ * chain of warps through shared memory and no warp waits for the others, so several short pieces
+ * are in work at once.  0: all warps meet at a barrier and sum their states together; on long
+ * pieces (tens of tiles) this costs the same, on batches of short contexts one barrier round per
+ * piece.  -1 (default): 1, except for calls with run-time spans, which always use 0.  Either way
+ * the order of every sum is fixed by tile indices, so a setting's results are bit-identical from
+ * run to run and under any renumbering of the physical pages.
+ */
+pdattn_status pdattn_set_merge_mode(int mode);
+
+/*
  * Synchronises `stream`, reads and clears the workspace's sticky error word.
  * Returns PDATTN_OK, PDATTN_BAD_PAGE_INDEX or PDATTN_DEVICE_TIMEOUT.
  */

@@ -6,7 +6,9 @@
 //                    per page-head) signalled through mbarriers; the consumer warps each take whole tiles, compute
 //                    S^T = K.Q^T and O^T += V^T.P^T with bf16 tensor-core MMAs (tokens on M, the
 //                    packed GQA query heads of the KV head on N) and keep the online-softmax
-//                    running max / sum in fp32.
+//                    running max / sum in fp32.  At the end of a piece the warps' states are merged
+//                    either by handing them down a chain of warps (default, no barrier) or all at
+//                    once behind a consumer-wide barrier (template flag CHAIN).
 //   combine_kernel : merges the (m, l, acc) triples of units that a span boundary cut.
 //   plan_kernel    : device-side twin of the host partitioner for callers without host lengths.
 //
@@ -84,6 +86,9 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t count) {   // counts as `count` arrivals
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -216,7 +221,7 @@ struct Cfg {
   // tile is kept back and the warps exchange their accumulators through it.
   static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the parked stores conflict-free
   static constexpr int SMEM_MAX = 232448;              // 227 KB
-  static constexpr int CTRL_BYTES = 640;
+  static constexpr int CTRL_BYTES = 768;
   static constexpr int NCW = PDATTN_NCW;                               // consumer warps
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
   static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged by producer 0
@@ -228,6 +233,12 @@ struct Cfg {
   static constexpr int NTHREADS = NCT + 32 * NPW;
   static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + QSLOTS * Q_BYTES + ML_BYTES + CTRL_BYTES;
   static constexpr int SLOT_FLOATS = HP * (D + 2);     // one partial: m[HP], l[HP], acc[HP][D]
+  // Chained merge (decode_kernel with CHAIN): a warp's running (m, l, acc) of a piece in MMA fragment
+  // order, one float4 per lane per row: NT rows of (m0, m1, l0, l1), then acc[nt][jm] -- 512 B a row.
+  static constexpr int HANDOFF_BYTES = NT * (1 + D / 16) * 512;
+  static constexpr int HANDOFFS_FIT = (SMEM_MAX - DYN_BYTES) / HANDOFF_BYTES;
+  static constexpr int HANDOFFS = HANDOFFS_FIT > 8 ? 8 : HANDOFFS_FIT;   // pieces whose merge is under way
+  static constexpr int CHAIN_DYN_BYTES = DYN_BYTES + HANDOFFS * HANDOFF_BYTES;
   static_assert(NSTAGES >= NCW && NSTAGES % NCW == 0, "ring/warp mapping");
   static_assert(HP * ACC_STRIDE * 4 <= STAGE_BYTES, "a parked accumulator must fit one stage");
   static_assert(DYN_BYTES <= SMEM_MAX, "shared memory");
@@ -243,10 +254,12 @@ struct Ctrl {                 // lives in the CTRL_BYTES area
   int32_t sq_id[SPAN_QUEUE];  // k-th id (k >= 1) at [(k-1) % SPAN_QUEUE]; -1 = no more spans
   int32_t sq_tag[SPAN_QUEUE]; // k, to detect an overwritten entry
   int32_t prod_last[4];       // per producer warp: index of the last tile it issued (-1 = none)
-  uint64_t q_full[4];         // query slot q holds the rows of piece p, p mod 4 == q
+  uint64_t q_full[4];         // query slot q holds the rows of piece p, p mod QSLOTS == q
   uint64_t q_empty[4];        // ... and every consumer warp has copied them to registers
+  int32_t qseq[4];            // CHAIN: piece whose rows the producer last armed the query slot for
+  int32_t turn[8];            // CHAIN: hand-off slot e is waiting for class (turn % 8) of merge number (turn / 8)
 };
-static_assert(sizeof(Ctrl) <= 640, "control block");
+static_assert(sizeof(Ctrl) <= 768, "control block");
 
 // ------------------------------------------------------------------------------------------
 // The walk over a span: pieces = (unit, tile range) in order.  Every warp runs the same walk.
@@ -491,11 +504,315 @@ __device__ __forceinline__ int read_span(Ctrl* ctrl, int k, bool& aborted) {
   return id;
 }
 
+// Query slot `qs` holds the rows of piece `p`.  A parity wait alone cannot tell "piece p has landed"
+// from "the slot's previous piece has not landed yet" (two phases apart look the same), and in the
+// chained-merge variant a warp skips the pieces it holds no tile of.  The producer therefore
+// records which piece it armed the slot for (before the arming arrive, which releases the record); a
+// wait that returns while the record still names an older piece is repeated.
+template <int QSLOTS>
+__device__ __forceinline__ bool wait_q(Ctrl* ctrl, int qs, int p) {
+  const uint32_t phase = (p / QSLOTS) & 1;
+  const uint32_t bar = smem_u32(&ctrl->q_full[qs]);
+  if (!mbar_wait(bar, phase)) return false;
+  if (ld_acquire_shared(&ctrl->qseq[qs]) == p) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (ld_acquire_shared(&ctrl->qseq[qs]) == p && mbar_try_wait(bar, phase)) return true;
+    if (*reinterpret_cast<volatile uint32_t*>(&ctrl->abort) || globaltimer_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+// Bounded wait until a hand-off slot's turn word reaches `want`.
+__device__ __forceinline__ bool wait_turn(Ctrl* ctrl, int e, int want) {
+  if (ld_acquire_shared(&ctrl->turn[e]) == want) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (ld_acquire_shared(&ctrl->turn[e]) == want) return true;
+    if (*reinterpret_cast<volatile uint32_t*>(&ctrl->abort) || globaltimer_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Consumer side of decode_kernel<.., CHAIN = true>: the variant for batches of many short pieces.
+//
+// Tiles are dealt to the consumer warps exactly as in the default variant (tile i of the CTA to warp
+// i mod NCW), but the warps never meet at a barrier.  A piece of n tiles has min(n, NCW) classes
+// (class c = the tiles c, c + NCW, ... of the piece, all on one warp).  A piece with one class is
+// finished by its warp straight from registers.  Otherwise the running (m, l, acc) travels down the
+// chain of classes through a hand-off slot in shared memory: class 0 writes its state, class c
+// waits for its turn, folds the slot into its registers and writes the sum back, and the last class
+// finishes the piece.  The order of the sum is the class order, whatever the timing.  Hand-off slot
+// e serves the pieces with more than one class number e, e + HANDOFFS, ...; its turn word says
+// which class of which of those pieces may touch it next.  Warps that hold no tile of a piece skip it
+// (they do not even read its query rows), so up to NCW short pieces are in work at once.
+// ------------------------------------------------------------------------------------------
+template <int D, int NT, int BS>
+__device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanParams& pp, Ctrl* ctrl, uint32_t ring,
+                                              uint32_t qbuf, uint8_t* handoff, int warp, int lane) {
+  using C = Cfg<D, NT, BS>;
+  constexpr int NST = C::NSTAGES;
+  constexpr int NCW = C::NCW;
+  constexpr int E = C::HANDOFFS;
+  static_assert(E >= 1, "no room for a hand-off slot");
+  const float NEG_INF = __int_as_float(0xff800000);
+  const int nunits = P.S * P.Hkv;
+  const int hq0 = lane >> 2;
+  const int qcol = (lane & 3) * 2;
+  const int drow = lane >> 2;
+  bool aborted = false;
+  int it = 0, pcnt = 0, mcnt = 0;
+
+  auto fail = [&]() {
+    aborted = true;
+    if (lane == 0) {
+      atomicOr(&P.hdr->err, ERR_TIMEOUT);
+      atomicExch(&ctrl->abort, 1u);
+    }
+  };
+
+  int span = blockIdx.x;
+  for (int k = 0; span >= 0; ++k) {
+    const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
+    const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
+    Walker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
+    Piece pc;
+    int first_unit = -1, first_tb = 0, own_unit = -1, own_slot = 0, piece_idx = 0;
+
+    while (walk.next(pc)) {
+      const int n_piece = pc.te - pc.tb;
+      const int it0 = it;
+      it += n_piece;
+      const int p = pcnt++;
+      const int n_cls = n_piece < NCW ? n_piece : NCW;
+      const bool multi = n_cls > 1;
+      const int mq = mcnt;            // number of this piece among those with more than one class
+      if (multi) ++mcnt;
+      const bool complete = (pc.tb == 0 && pc.te == pc.nt);
+      const int slot_idx = piece_idx == 0 ? 0 : 1;
+      if (piece_idx == 0) {
+        first_unit = pc.unit;
+        first_tb = pc.tb;
+      }
+      if (!complete && pc.tb == 0) {
+        own_unit = pc.unit;
+        own_slot = slot_idx;
+      }
+      ++piece_idx;
+      int pos = warp - it0 % NCW;     // this warp's class in the piece
+      if (pos < 0) pos += NCW;
+      if (pos >= n_cls || aborted) continue;
+      if (*reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) {
+        aborted = true;
+        continue;
+      }
+
+      // ---- packed query rows of this KV head as MMA B fragments, from the staged copy
+      uint32_t qf[NT][D / 16][2];
+      {
+        const int qs = p % C::QSLOTS;
+        if (!wait_q<C::QSLOTS>(ctrl, qs, p)) {
+          fail();
+          continue;
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const int head = nt * 8 + hq0;
+          const bool live = head < P.G;
+          const uint32_t qa = qbuf + qs * C::Q_BYTES + (live ? head : 0) * (D * 2) + qcol * 2;
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            uint32_t v0 = 0u, v1 = 0u;
+            if (live) {
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v0) : "r"(qa + kk * 32) : "memory");
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v1) : "r"(qa + kk * 32 + 16) : "memory");
+            }
+            qf[nt][kk][0] = v0;
+            qf[nt][kk][1] = v1;
+          }
+        }
+        __syncwarp();
+        // the slot is free again once every class has its copy: class 0 also arrives for the warps
+        // that hold no tile of the piece
+        if (lane == 0) mbar_arrive_n(smem_u32(&ctrl->q_empty[qs]), pos == 0 ? NCW - n_cls + 1 : 1);
+      }
+      float acc[NT][D / 16][4];
+      float m[NT][2], l[NT][2];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        m[nt][0] = m[nt][1] = NEG_INF;
+        l[nt][0] = l[nt][1] = 0.f;
+#pragma unroll
+        for (int jm = 0; jm < D / 16; ++jm) acc[nt][jm][0] = acc[nt][jm][1] = acc[nt][jm][2] = acc[nt][jm][3] = 0.f;
+      }
+
+      // ---- this class's tiles
+      for (int its = it0 + pos; its < it0 + n_piece; its += NCW) {
+        const int slot = its % NST;
+        if (!mbar_wait(smem_u32(&ctrl->full[slot]), (its / NST) & 1)) {
+          fail();
+          break;
+        }
+        const int t = pc.tb + (its - it0);
+        const uint32_t sK = ring + slot * C::STAGE_BYTES;
+        const uint32_t sV = sK + C::KV_BYTES;
+        const uint32_t badmask = ctrl->meta[slot];
+        const int n_valid = min(TILE, pc.L - (pc.t0 + t) * TILE);
+        if (n_valid == TILE) {
+          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane);
+        } else {
+          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_valid, badmask, lane);
+          fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
+      }
+      if (aborted) continue;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          float v = l[nt][e];
+          v += __shfl_xor_sync(0xffffffffu, v, 4);
+          v += __shfl_xor_sync(0xffffffffu, v, 8);
+          v += __shfl_xor_sync(0xffffffffu, v, 16);
+          l[nt][e] = v;
+        }
+
+      // ---- the chain of classes
+      if (multi) {
+        const int e = mq % E;
+        float4* row4 = reinterpret_cast<float4*>(handoff + e * C::HANDOFF_BYTES) + lane;   // row r: row4[r * 32]
+        if (!wait_turn(ctrl, e, mq * 8 + pos)) {
+          fail();
+          continue;
+        }
+        if (pos > 0) {
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const float4 ml = row4[nt * 32];
+            const float M0 = fmaxf(ml.x, m[nt][0]), M1 = fmaxf(ml.y, m[nt][1]);
+            const float mu0 = (M0 == NEG_INF) ? 0.f : M0, mu1 = (M1 == NEG_INF) ? 0.f : M1;
+            const float fp0 = fast_exp2(ml.x - mu0), fp1 = fast_exp2(ml.y - mu1);
+            const float fo0 = fast_exp2(m[nt][0] - mu0), fo1 = fast_exp2(m[nt][1] - mu1);
+            m[nt][0] = M0;
+            m[nt][1] = M1;
+            l[nt][0] = ml.z * fp0 + l[nt][0] * fo0;
+            l[nt][1] = ml.w * fp1 + l[nt][1] * fo1;
+#pragma unroll
+            for (int jm = 0; jm < D / 16; ++jm) {
+              const float4 a = row4[(NT + nt * (D / 16) + jm) * 32];
+              acc[nt][jm][0] = a.x * fp0 + acc[nt][jm][0] * fo0;
+              acc[nt][jm][1] = a.y * fp1 + acc[nt][jm][1] * fo1;
+              acc[nt][jm][2] = a.z * fp0 + acc[nt][jm][2] * fo0;
+              acc[nt][jm][3] = a.w * fp1 + acc[nt][jm][3] * fo1;
+            }
+          }
+        }
+        if (pos < n_cls - 1) {
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            row4[nt * 32] = make_float4(m[nt][0], m[nt][1], l[nt][0], l[nt][1]);
+#pragma unroll
+            for (int jm = 0; jm < D / 16; ++jm)
+              row4[(NT + nt * (D / 16) + jm) * 32] =
+                  make_float4(acc[nt][jm][0], acc[nt][jm][1], acc[nt][jm][2], acc[nt][jm][3]);
+          }
+          __syncwarp();
+          if (lane == 0) st_release_shared(&ctrl->turn[e], mq * 8 + pos + 1);
+          continue;
+        }
+        __syncwarp();   // the last class has read the slot: it now serves merge number mq + E
+        if (lane == 0) st_release_shared(&ctrl->turn[e], (mq + E) * 8);
+      }
+
+      // ---- finish the piece from registers (one-class piece, or last class of the chain)
+      if (complete && pc.t0 > 0) {
+        // the unit's leading tiles were handled elsewhere (shared prefix): fold that partial in
+        const float* pfx = P.pfx_partials + (static_cast<int64_t>(pc.s) * P.Hkv + pc.g) * C::SLOT_FLOATS;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const int h0 = nt * 8 + qcol;
+          const float pm0 = pfx[h0], pm1 = pfx[h0 + 1];
+          const float M0 = fmaxf(pm0, m[nt][0]), M1 = fmaxf(pm1, m[nt][1]);
+          const float mu0 = (M0 == NEG_INF) ? 0.f : M0, mu1 = (M1 == NEG_INF) ? 0.f : M1;
+          const float fp0 = fast_exp2(pm0 - mu0), fp1 = fast_exp2(pm1 - mu1);
+          const float fo0 = fast_exp2(m[nt][0] - mu0), fo1 = fast_exp2(m[nt][1] - mu1);
+          m[nt][0] = M0;
+          m[nt][1] = M1;
+          l[nt][0] = pfx[C::HP + h0] * fp0 + l[nt][0] * fo0;
+          l[nt][1] = pfx[C::HP + h0 + 1] * fp1 + l[nt][1] * fo1;
+          const float* pa0 = pfx + 2 * C::HP + h0 * D + drow;
+          const float* pa1 = pa0 + D;
+#pragma unroll
+          for (int jm = 0; jm < D / 16; ++jm) {
+            acc[nt][jm][0] = pa0[jm * 16] * fp0 + acc[nt][jm][0] * fo0;
+            acc[nt][jm][1] = pa1[jm * 16] * fp1 + acc[nt][jm][1] * fo1;
+            acc[nt][jm][2] = pa0[jm * 16 + 8] * fp0 + acc[nt][jm][2] * fo0;
+            acc[nt][jm][3] = pa1[jm * 16 + 8] * fp1 + acc[nt][jm][3] * fo1;
+          }
+        }
+      }
+      if (complete) {
+        // bf16 output; neighbouring lanes swap one value so that each stores two adjacent elements
+        __nv_bfloat16* ob = P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G) * D;
+        const bool odd = drow & 1;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const float inv0 = l[nt][0] > 0.f ? 1.f / l[nt][0] : 0.f;
+          const float inv1 = l[nt][1] > 0.f ? 1.f / l[nt][1] : 0.f;
+          const int myh = nt * 8 + qcol + (odd ? 1 : 0);
+          __nv_bfloat16* orow = ob + static_cast<int64_t>(myh) * D + (drow & ~1);
+#pragma unroll
+          for (int jm = 0; jm < D / 16; ++jm) {
+            const float v0 = acc[nt][jm][0] * inv0, v1 = acc[nt][jm][1] * inv1;
+            const float v2 = acc[nt][jm][2] * inv0, v3 = acc[nt][jm][3] * inv1;
+            const float r0 = __shfl_xor_sync(0xffffffffu, odd ? v0 : v1, 4);
+            const float r1 = __shfl_xor_sync(0xffffffffu, odd ? v2 : v3, 4);
+            if (myh < P.G) {
+              *reinterpret_cast<uint32_t*>(orow + jm * 16) = odd ? pack_bf16x2(r0, v1) : pack_bf16x2(v0, r0);
+              *reinterpret_cast<uint32_t*>(orow + jm * 16 + 8) = odd ? pack_bf16x2(r1, v3) : pack_bf16x2(v2, r1);
+            }
+          }
+        }
+      } else {
+        float* part = P.partials + (static_cast<int64_t>(span) * 2 + slot_idx) * C::SLOT_FLOATS;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const int h0 = nt * 8 + qcol;
+          if (drow == 0) {
+            part[h0] = m[nt][0];
+            part[h0 + 1] = m[nt][1];
+            part[C::HP + h0] = l[nt][0];
+            part[C::HP + h0 + 1] = l[nt][1];
+          }
+          float* a0 = part + 2 * C::HP + h0 * D + drow;
+          float* a1 = a0 + D;
+#pragma unroll
+          for (int jm = 0; jm < D / 16; ++jm) {
+            a0[jm * 16] = acc[nt][jm][0];
+            a1[jm * 16] = acc[nt][jm][1];
+            a0[jm * 16 + 8] = acc[nt][jm][2];
+            a1[jm * 16 + 8] = acc[nt][jm][3];
+          }
+        }
+      }
+    }
+    if (warp == 0 && lane == 0) P.rec[span] = make_int4(first_unit, first_tb, own_unit, own_slot);
+    span = read_span(ctrl, k + 1, aborted);
+  }
+  if (aborted && lane == 0) atomicOr(&P.hdr->err, ERR_TIMEOUT);
+}
+
 // ------------------------------------------------------------------------------------------
 // The decode kernel.  PROBE = true builds the page-gather ceiling: identical span walk, page-id
 // lookups and TMA ring, but the consumers release every tile untouched and nothing is written.
+// CHAIN = true replaces the consumers' barrier-and-merge at the end of each piece by the chained
+// hand-off of consume_chain (the producers are the same).
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS, bool PROBE = false>
+template <int D, int NT, int BS, bool PROBE = false, bool CHAIN = false>
 __global__ void __launch_bounds__(Cfg<D, NT, BS>::NTHREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
               const __grid_constant__ DecodeParams P) {
@@ -529,7 +846,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     for (int i = 0; i < C::QSLOTS; ++i) {
       mbar_init(smem_u32(&ctrl->q_full[i]), 1);
       mbar_init(smem_u32(&ctrl->q_empty[i]), NCW);
+      ctrl->qseq[i] = -1;
     }
+    for (int i = 0; i < 8; ++i) ctrl->turn[i] = i * 8;   // slot i first serves merge number i, class 0
     fence_mbar_init();
   }
   __syncthreads();
@@ -570,6 +889,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           if (lane == 0) {
             const uint32_t bytes = static_cast<uint32_t>(P.G) * D * 2;
             const uint32_t qb = smem_u32(&ctrl->q_full[qs]);
+            if (CHAIN) ctrl->qseq[qs] = pcnt;
             mbar_arrive_expect_tx(qb, bytes);
             bulk_load(qbuf + qs * C::Q_BYTES, P.q + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G) * D, bytes, qb);
           }
@@ -676,6 +996,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   }
   const int hq0 = lane >> 2;         // B-operand column (head) this lane feeds
   const int qcol = (lane & 3) * 2;
+
+  if constexpr (CHAIN) {
+    consume_chain<D, NT, BS>(P, pp, ctrl, ring, qbuf,
+                             smem + NST * C::STAGE_BYTES + C::QSLOTS * C::Q_BYTES + C::ML_BYTES + C::CTRL_BYTES, warp,
+                             lane);
+    return;
+  }
 
   int span = cta;
   for (int k = 0; span >= 0; ++k) {

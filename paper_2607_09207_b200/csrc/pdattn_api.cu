@@ -30,6 +30,8 @@ struct GroupedCall {                      // set only inside pdattn_decode_group
 thread_local GroupedCall g_grouped;
 thread_local std::vector<int32_t> g_start_tiles_host;
 int g_dyn_per_cta = 0;                    // run-time spans per CTA (pdattn_set_dynamic_spans)
+int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (chained), 0 barrier, 1 chained
+thread_local bool g_use_chain = true;     // decided per call, read by the launcher
 
 struct Binding {
   bool set = false;
@@ -79,6 +81,7 @@ struct DevInfo {
   int sm_count = 0;
   bool attr_set[2][2][2] = {};      // [D==128][NT==2][BS==32]
   bool probe_attr_set[2][2][2] = {};
+  bool chain_attr_set[2][2][2] = {};
   bool prefix_attr_set[2][2] = {};  // [D==128][BS==32]
 };
 constexpr int kMaxDevices = 64;
@@ -226,7 +229,18 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
     return PDATTN_OK;
   }
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
-  kern<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
+  if (g_use_chain) {
+    auto chain = decode_kernel<D, NT, BS, false, true>;
+    bool& cdone = di->chain_attr_set[D == 128][NT == 2][BS == 32];
+    if (!cdone) {
+      cudaError_t ce = cudaFuncSetAttribute(chain, cudaFuncAttributeMaxDynamicSharedMemorySize, C::CHAIN_DYN_BYTES);
+      if (ce != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", ce);
+      cdone = true;
+    }
+    chain<<<grid, C::NTHREADS, C::CHAIN_DYN_BYTES, stream>>>(mk, mv, P);
+  } else {
+    kern<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
   if (g_prof_stop) cudaEventRecord(g_prof_stop, stream);
@@ -333,6 +347,12 @@ pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cac
 pdattn_status pdattn_set_dynamic_spans(int per_cta) {
   if (per_cta < 0 || per_cta > kMaxDynPerCta) return PDATTN_INVALID_ARG;
   g_dyn_per_cta = per_cta;
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_set_merge_mode(int mode) {
+  if (mode < -1 || mode > 1) return PDATTN_INVALID_ARG;
+  g_merge_mode = mode;
   return PDATTN_OK;
 }
 
@@ -462,6 +482,8 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
                a->kv_head_stride, a->kv_token_stride, rank, &mv);
   if (s != PDATTN_OK) return s;
   P.box5d = rank == 5;
+  // run-time spans assume warps that stay within a ring of each other: barrier merge there
+  g_use_chain = g_merge_mode != 0 && dyn_per_cta == 0;
 
   if (grouped) {
     // shared prompt tiles first: one pass per (group, kv head) for the query rows of all samples
@@ -767,6 +789,7 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   P.use_ws_plan = 0;
   P.box5d = 0;
   int grid = n_ctas, combine_grid = n_ctas, n_spans_host = -1;
+  g_use_chain = g_merge_mode != 0;
   if (a->context_lens_host) {
     if (!plan_spans(a->context_lens_host, nullptr, a->num_seqs, a->num_kv_heads, n_ctas, 0, n_ctas, P.spans, &P.plan))
       return PDATTN_INVALID_ARG;

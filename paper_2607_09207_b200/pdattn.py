@@ -31,6 +31,7 @@ EXPORTS = [
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_set_dynamic_spans",
+    "pdattn_set_merge_mode",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
 ]
@@ -87,6 +88,7 @@ def lib():
                                          vp, sz, vp, sz, vp]
         L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(Plan)]
         L.pdattn_set_dynamic_spans.argtypes = [i32]
+        L.pdattn_set_merge_mode.argtypes = [i32]
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
         L.pdattn_grouped_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_grouped.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
@@ -294,6 +296,13 @@ def set_dynamic_spans(per_cta: int):
     st = lib().pdattn_set_dynamic_spans(per_cta)
     if st != OK:
         raise PdattnError(st, "pdattn_set_dynamic_spans")
+
+
+def set_merge_mode(mode: int):
+    """-1: by piece length (default); 0: barrier merge; 1: chained merge."""
+    st = lib().pdattn_set_merge_mode(mode)
+    if st != OK:
+        raise PdattnError(st, "pdattn_set_merge_mode")
 
 
 def plan_host(context_lens_host, num_kv_heads, n_ctas, dynamic_per_cta=0, max_spans=None):

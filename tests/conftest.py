@@ -24,3 +24,28 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+# The GPU parity modules run once per merge mode of the decode kernel's consumer warps: the barrier
+# merge and the chained merge must each pass every case, whatever the library would pick by itself.
+MERGE_MODE_MODULES = ("test_gpu_parity", "test_gpu_grouped", "test_gpu_decode_loop")
+MERGE_MODES = {"barrier": 0, "chain": 1}
+
+
+def pytest_generate_tests(metafunc):
+    if metafunc.module.__name__.split(".")[-1] in MERGE_MODE_MODULES:
+        metafunc.parametrize("merge_mode", list(MERGE_MODES), indirect=True)
+
+
+@pytest.fixture(autouse=True)
+def merge_mode(request):
+    name = getattr(request, "param", None)
+    if name is None:
+        yield None
+        return
+    from paper_2607_09207_b200 import pdattn
+    pdattn.set_merge_mode(MERGE_MODES[name])
+    try:
+        yield name
+    finally:
+        pdattn.set_merge_mode(-1)

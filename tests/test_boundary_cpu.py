@@ -46,6 +46,17 @@ def test_status_strings():
     assert len(seen) == 9
 
 
+def test_tuning_setters_check_their_ranges():
+    L = pdattn.lib()
+    for mode in (-1, 0, 1):
+        assert L.pdattn_set_merge_mode(mode) == pdattn.OK
+    for mode in (-2, 2, 100):
+        assert L.pdattn_set_merge_mode(mode) == pdattn.INVALID_ARG
+    L.pdattn_set_merge_mode(-1)
+    assert L.pdattn_set_dynamic_spans(-1) == pdattn.INVALID_ARG
+    assert L.pdattn_set_dynamic_spans(0) == pdattn.OK
+
+
 def test_workspace_size_and_shape_checks():
     n = pdattn.workspace_size(256, 28, 4, 128)
     assert 0 < n < 64 << 20 and n % 256 == 0

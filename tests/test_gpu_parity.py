@@ -83,6 +83,19 @@ def test_many_short_sequences():
     check_against_oracle(W.make_custom(lens, Hq=8, Hkv=2, d=128, seed=5, device=DEV), "many short")
 
 
+@pytest.mark.parametrize("Hq,Hkv,d,bs", [(28, 4, 128, 16), (64, 4, 128, 16), (16, 2, 64, 16), (32, 2, 64, 32)])
+def test_batches_of_two_to_eleven_tile_pieces(Hq, Hkv, d, bs):
+    """Hundreds of pieces per CTA, each spread over two to six consumer warps: every hand-off slot of
+    the chained merge is reused many times, with 8- and 16-row tiles (one slot only at d = 128)."""
+    rng = np.random.default_rng(17)
+    lens = rng.integers(65, 700, size=1200)
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, bs=bs, seed=19, device=DEV)
+    out = check_against_oracle(w, f"mid-length pieces Hq={Hq} Hkv={Hkv} d={d} bs={bs}",
+                               pairs=sample_pairs(w, 600, seed=23))
+    again, st = run(w)
+    assert st == pdattn.OK and torch.equal(out, again)      # the order of every sum is fixed
+
+
 def test_single_long_sequence_is_split_over_all_sms():
     w = W.make_custom([40000], Hq=7, Hkv=1, d=128, seed=6, device=DEV)
     check_against_oracle(w, "one long sequence")
