@@ -215,6 +215,15 @@ pdattn_status pdattn_set_dynamic_spans(int per_cta);
 pdattn_status pdattn_set_merge_mode(int mode);
 
 /*
+ * Process-wide choice of the kernel that pdattn_decode_grouped runs over the shared prompt tiles.
+ * 1: the tile products run on tcgen05 tensor cores with accumulators in tensor memory (all
+ * group_size * G query rows of a group against a 64-token tile in one operand).  0: warp-level
+ * MMAs, eight rows per warp.  -1 (default): 1.  The paper has no counterpart; both compute the same
+ * partial (m, l, acc) per (sequence, KV head) and differ only in rounding order.
+ */
+pdattn_status pdattn_set_prefix_engine(int engine);
+
+/*
  * Synchronises `stream`, reads and clears the workspace's sticky error word.
  * Returns PDATTN_OK, PDATTN_BAD_PAGE_INDEX or PDATTN_DEVICE_TIMEOUT.
  */

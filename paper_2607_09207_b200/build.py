@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB = os.path.join(LIB_DIR, "libpdattn.so")
 SOURCES = ["pdattn_api.cu", "partition.cpp"]
-HEADERS = ["kernels.cuh", "partition.h", os.path.join("..", "..", "include", "pdattn.h")]
+HEADERS = ["kernels.cuh", "prefix_umma.cuh", "partition.h", os.path.join("..", "..", "include", "pdattn.h")]
 
 
 def _nvcc() -> str:

@@ -11,6 +11,7 @@
 
 #include "../../include/pdattn.h"
 #include "kernels.cuh"
+#include "prefix_umma.cuh"
 #include "partition.h"
 
 namespace {
@@ -32,6 +33,7 @@ thread_local std::vector<int32_t> g_start_tiles_host;
 int g_dyn_per_cta = 0;                    // run-time spans per CTA (pdattn_set_dynamic_spans)
 int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (chained), 0 barrier, 1 chained
 thread_local bool g_use_chain = true;     // decided per call, read by the launcher
+int g_prefix_engine = -1;                 // pdattn_set_prefix_engine: -1 default (tcgen05), 0 warp MMAs, 1 tcgen05
 
 struct Binding {
   bool set = false;
@@ -83,6 +85,7 @@ struct DevInfo {
   bool probe_attr_set[2][2][2] = {};
   bool chain_attr_set[2][2][2] = {};
   bool prefix_attr_set[2][2] = {};  // [D==128][BS==32]
+  bool prefix_umma_attr_set[2][2] = {};
 };
 constexpr int kMaxDevices = 64;
 DevInfo g_dev[kMaxDevices];
@@ -149,7 +152,7 @@ struct MapCacheEntry {
   MapKey key;
   CUtensorMap map;
 };
-thread_local MapCacheEntry g_maps[8];
+thread_local MapCacheEntry g_maps[16];
 thread_local int g_map_next = 0;
 
 // View of a cache as a tensor for TMA, 128-byte swizzle, zero fill out of bounds.
@@ -197,7 +200,7 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
     return PDATTN_CUDA_ERROR;
   }
   MapCacheEntry& e = g_maps[g_map_next];
-  g_map_next = (g_map_next + 1) % 8;
+  g_map_next = (g_map_next + 1) % 16;
   e.valid = true;
   e.key = key;
   e.map = m;
@@ -282,6 +285,24 @@ pdattn_status launch_prefix_bs(const CUtensorMap& mk, const CUtensorMap& mv, con
   return PDATTN_OK;
 }
 
+template <int D, int BS>
+pdattn_status launch_prefix_umma_bs(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
+                                    cudaStream_t stream) {
+  using C = UmmaCfg<D, BS>;
+  auto kern = prefix_umma_kernel<D, BS>;
+  bool& done = di->prefix_umma_attr_set[D == 128][BS == 32];
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
+    if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
+    done = true;
+  }
+  if (grid <= 0) return PDATTN_OK;
+  kern<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, X);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("prefix_umma_kernel launch", e);
+  return PDATTN_OK;
+}
+
 thread_local int g_block_size = 16;   // page size of the call being launched (set by the entry points)
 
 template <int D, int NT>
@@ -289,6 +310,12 @@ pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeP
                      int n_spans_host, DevInfo* di, cudaStream_t stream) {
   return g_block_size == 32 ? launch_bs<D, NT, 32>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
                             : launch_bs<D, NT, 16>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+}
+template <int D>
+pdattn_status launch_prefix_umma(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
+                                 cudaStream_t stream) {
+  return g_block_size == 32 ? launch_prefix_umma_bs<D, 32>(mk, mv, X, grid, di, stream)
+                            : launch_prefix_umma_bs<D, 16>(mk, mv, X, grid, di, stream);
 }
 template <int D>
 pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
@@ -347,6 +374,12 @@ pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cac
 pdattn_status pdattn_set_dynamic_spans(int per_cta) {
   if (per_cta < 0 || per_cta > kMaxDynPerCta) return PDATTN_INVALID_ARG;
   g_dyn_per_cta = per_cta;
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_set_prefix_engine(int engine) {
+  if (engine < -1 || engine > 1) return PDATTN_INVALID_ARG;
+  g_prefix_engine = engine;
   return PDATTN_OK;
 }
 
@@ -520,7 +553,22 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
       }
       X.ranges[c] = make_int2(u0, u);
     }
-    s = a->head_dim == 128 ? launch_prefix<128>(mk, mv, X, pgrid, di, stream) : launch_prefix<64>(mk, mv, X, pgrid, di, stream);
+    if (g_prefix_engine != 0) {
+      // tensor-memory kernel: its tiles are laid out per 64-column block, so it takes the rank-4 view
+      CUtensorMap pk = mk, pv = mv;
+      if (rank != 4) {
+        s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+                     a->kv_head_stride, a->kv_token_stride, 4, &pk);
+        if (s != PDATTN_OK) return s;
+        s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+                     a->kv_head_stride, a->kv_token_stride, 4, &pv);
+        if (s != PDATTN_OK) return s;
+      }
+      s = a->head_dim == 128 ? launch_prefix_umma<128>(pk, pv, X, pgrid, di, stream)
+                             : launch_prefix_umma<64>(pk, pv, X, pgrid, di, stream);
+    } else {
+      s = a->head_dim == 128 ? launch_prefix<128>(mk, mv, X, pgrid, di, stream) : launch_prefix<64>(mk, mv, X, pgrid, di, stream);
+    }
     if (s != PDATTN_OK) return s;
     g_last_launches += 1;
     P.start_tiles = X.start_tiles;

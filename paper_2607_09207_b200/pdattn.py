@@ -31,7 +31,7 @@ EXPORTS = [
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_set_dynamic_spans",
-    "pdattn_set_merge_mode",
+    "pdattn_set_merge_mode", "pdattn_set_prefix_engine",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
 ]
@@ -89,6 +89,7 @@ def lib():
         L.pdattn_plan_host.argtypes = [vp, i32, i32, i32, i32, i32, vp, ctypes.POINTER(Plan)]
         L.pdattn_set_dynamic_spans.argtypes = [i32]
         L.pdattn_set_merge_mode.argtypes = [i32]
+        L.pdattn_set_prefix_engine.argtypes = [i32]
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
         L.pdattn_grouped_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_grouped.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
@@ -303,6 +304,13 @@ def set_merge_mode(mode: int):
     st = lib().pdattn_set_merge_mode(mode)
     if st != OK:
         raise PdattnError(st, "pdattn_set_merge_mode")
+
+
+def set_prefix_engine(engine: int):
+    """-1: default (tcgen05); 0: warp-level MMAs; 1: tcgen05 with tensor-memory accumulators."""
+    st = lib().pdattn_set_prefix_engine(engine)
+    if st != OK:
+        raise PdattnError(st, "pdattn_set_prefix_engine")
 
 
 def plan_host(context_lens_host, num_kv_heads, n_ctas, dynamic_per_cta=0, max_spans=None):

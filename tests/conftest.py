@@ -32,9 +32,31 @@ MERGE_MODE_MODULES = ("test_gpu_parity", "test_gpu_grouped", "test_gpu_decode_lo
 MERGE_MODES = {"barrier": 0, "chain": 1}
 
 
+# ... and the grouped-decode module once per kernel for the shared prompt tiles.
+PREFIX_ENGINE_MODULES = ("test_gpu_grouped",)
+PREFIX_ENGINES = {"tcgen05": 1, "warp_mma": 0}
+
+
 def pytest_generate_tests(metafunc):
-    if metafunc.module.__name__.split(".")[-1] in MERGE_MODE_MODULES:
+    name = metafunc.module.__name__.split(".")[-1]
+    if name in MERGE_MODE_MODULES:
         metafunc.parametrize("merge_mode", list(MERGE_MODES), indirect=True)
+    if name in PREFIX_ENGINE_MODULES:
+        metafunc.parametrize("prefix_engine", list(PREFIX_ENGINES), indirect=True)
+
+
+@pytest.fixture(autouse=True)
+def prefix_engine(request):
+    name = getattr(request, "param", None)
+    if name is None:
+        yield None
+        return
+    from paper_2607_09207_b200 import pdattn
+    pdattn.set_prefix_engine(PREFIX_ENGINES[name])
+    try:
+        yield name
+    finally:
+        pdattn.set_prefix_engine(-1)
 
 
 @pytest.fixture(autouse=True)
