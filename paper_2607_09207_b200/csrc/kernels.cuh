@@ -1401,11 +1401,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
         continue;
       }
-#ifdef PDATTN_PREFIX_NOCOMPUTE
-      if (false) {
-#else
       if (has_rows) {
-#endif
         const uint32_t sK = ring + slot * C::STAGE_BYTES;
         compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, P.scale_log2, TILE, ctrl->meta[slot], lane);
       }

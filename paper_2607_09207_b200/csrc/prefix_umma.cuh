@@ -1,27 +1,32 @@
-// Shared-prefix kernel on the 5th-generation tensor cores (tcgen05, accumulators in tensor memory).
+// Shared-prefix kernel on the 5th-generation tensor cores (tcgen05, operands and accumulators in tensor memory).
 //
 // The samples of a GRPO group share their prompt pages, so the prompt's K/V tiles are streamed once
 // per (group, kv head) and scored against the query rows of all samples: R = group_size * G rows.
 // That is the one dense contraction on this path (R = 40 rows against every 64-token tile), and
 // with warp-level MMAs it is bound by shared-memory reads and the legacy tensor pipe, not by HBM.
-// Here the whole tile is one tensor-core operand:
+// Here the whole tile is one tensor-core operand (M = 128 lanes of tensor memory):
 //
-//   S[128 rows, 64 tokens]  = Q[128, d] . K^T          tcgen05.mma, A and B from shared memory
-//   O[128 rows, d]         += P[128, 64] . V[64, d]    tcgen05.mma, A = P from tensor memory
+//   S[128, 64 tokens]  = Q[128, d] . K^T          A = Q from tensor memory, B = K tile from shared memory
+//   O[128, d]         += P[128, 64] . V[64, d]    A = P from tensor memory, B = V tile from shared memory
 //
-// Rows R..127 of Q are zeros.  K and V tiles arrive by TMA exactly as in the other kernels (128-byte
-// swizzle), laid out per 64-column block as [64 tokens][128 bytes]: K is a K-major B operand of the
-// first product, V an MN-major B operand of the second, so V needs no transpose.  Row r lives in
-// tensor-memory lane (r mod 4) * 32 + r / 4, which spreads the rows over the four softmax warps (a
-// warp can only reach its own quarter of the lanes); one thread owns one row, so the online softmax
-// needs no shuffles: it loads the row's 64 scores, updates max and sum, rescales O when the max
-// moved, and stores P back to tensor memory as hi + lo bf16 (two MMAs; 8 bits of P are not enough
-// under the stated tolerance).  S and P are double buffered so the tensor cores run tile t+1's
-// scores while the softmax warps work on tile t.
+// K and V tiles arrive by TMA as in the other kernels (128-byte swizzle), laid out per 64-column block as
+// [64 tokens][128 bytes]: K is a K-major B operand of the first product, V an MN-major B operand of the
+// second, so V needs no transpose.  Query row r occupies TWO lanes, rho = (r % 2) * 32 + r / 2 and rho + 64,
+// with the same Q: both get the same scores, the first lane receives the bf16 head of P and the second
+// the bf16 rest (8 bits of P are not enough under the stated tolerance), and ONE product P.V per 16 tokens
+// yields the hi part and the lo part of O in the two lane halves while V is read once.
 //
-// Warps: 0-3 softmax (128 threads), 4 MMA issue (one elected lane; the warp also owns the tensor
-// memory allocation), 5-7 TMA producers.  Every wait is bounded; on expiry the CTA raises
-// ERR_TIMEOUT, drains its tensor-core work, frees its tensor memory and returns.
+// Eight softmax warps: warp w reaches lanes 32 * (w % 4) .. + 31 only (a hardware rule), so a row has four
+// threads -- two lanes times two halves of the tile's columns -- and each turns a quarter of the tile (16
+// tokens) into probabilities, swaps hi and lo parts with the row's other lane through shared memory and
+// stores its lane's 16 P columns.  One 128-thread barrier per tile publishes the swapped parts and the next
+// tile's quarter maxima (its scores are fetched ahead).  The reference value of the online softmax only
+// follows the running max when that grew by more than 2^8, so O in tensor memory is rarely rescaled.
+// Two MMA-issuing threads in two warps (scores; P.V), because the tensor cores take an MMA of this size
+// only about every 80-100 cycles from its issuing thread; two TMA producer warps.  Scores run two tiles
+// ahead of the softmax (two score buffers), query rows are staged a whole unit ahead (two buffers).
+// Every mbarrier wait is bounded; on expiry the CTA raises ERR_TIMEOUT, its waits fall through, the
+// issuing threads drain their tensor-core work, the tensor memory is freed and the CTA returns.
 #pragma once
 
 #include "kernels.cuh"
@@ -84,6 +89,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
@@ -110,25 +123,15 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parit
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
+    if (*reinterpret_cast<const volatile uint32_t*>(abort_flag) || globaltimer_ns() - t0 > kWaitLimitNs) return false;
 #pragma unroll 1
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait_hint(bar, parity, PDATTN_WAIT_HINT_NS)) return true;
-    if (*reinterpret_cast<const volatile uint32_t*>(abort_flag) || globaltimer_ns() - t0 > kWaitLimitNs) return false;
   }
 }
 
-
-#ifdef PDATTN_TRACE
-#define TR_DECL long long tr_t = clock64(); long long tr_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#define TR_MARK(i) { const long long tr_n = clock64(); tr_acc[i] += tr_n - tr_t; tr_t = tr_n; }
-#define TR_DUMP(base) if (blockIdx.x == 0 && lane == 0) { for (int tr_i = 0; tr_i < 8; ++tr_i) P.err[(base) + tr_i] = static_cast<int>(tr_acc[tr_i] >> 4); }
-#else
-#define TR_DECL
-#define TR_MARK(i)
-#define TR_DUMP(base)
-#endif
-
 constexpr int UMMA_ROWS = 128;              // rows of the MMA tile = tensor-memory lanes
+constexpr int UMMA_MAX_QUERY_ROWS = 64;     // query rows per unit (group_size * G): each occupies two lanes
 
 template <int D, int BS>
 struct UmmaCfg {
@@ -136,48 +139,64 @@ struct UmmaCfg {
   static constexpr int HALF_TILE_BYTES = TILE * 128;        // one block of a K or V tile: [64 tokens][128 B]
   static constexpr int KV_BYTES = HALVES * HALF_TILE_BYTES;
   static constexpr int STAGE_BYTES = 2 * KV_BYTES;          // K tile then V tile
-  static constexpr int Q_HALF_BYTES = UMMA_ROWS * 128;      // one block of Q: [128 rows][128 B]
-  static constexpr int Q_BYTES = HALVES * Q_HALF_BYTES;
   static constexpr int PAGES = TILE / BS;
   static constexpr int BOX_BYTES = BS * 128;                // one TMA box: a page-head's 64-column block
-#ifndef PDATTN_UMMA_ST64
-#define PDATTN_UMMA_ST64 12
-#endif
-  static constexpr int NSTAGES = D == 64 ? PDATTN_UMMA_ST64 : 6;
-  static constexpr int NPW = 3;                             // producer warps
-  static constexpr int MMA_WARP = 8;                        // warps 0-7: two softmax groups; 8: MMA; 9-11: producers
-  static constexpr int NTHREADS = (MMA_WARP + 1 + NPW) * 32;
+  static constexpr int NSTAGES = 6;
+  static constexpr int NPW = 2;                             // producer warps
+  static constexpr int MMA_WARP = 8;                        // warps 0-7: softmax; 8, 9: MMA issue; 10, 11: producers
+  static constexpr int NTHREADS = (MMA_WARP + 2 + NPW) * 32;
   static constexpr int CTRL_BYTES = 384;
-  static constexpr int ML_BYTES = UMMA_ROWS * 2 * 4;        // (m, l) of group 1's rows, handed to group 0
-  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + Q_BYTES + ML_BYTES + CTRL_BYTES;
+  static constexpr int XM_BYTES = 2 * 4 * 64 * 4;           // row maxima of the four column quarters, double buffered
+  static constexpr int XL_BYTES = 4 * 64 * 4;               // row sums of the four column quarters
+  static constexpr int XP_BYTES = 2 * 4 * 64 * 32;          // P halves swapped between a row's two lanes, double buffered
+  static constexpr int XO_BYTES = XP_BYTES;                 // (same memory) the lo-part rows of O as bf16, at the end of a unit
+  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + XM_BYTES + XL_BYTES + XO_BYTES + CTRL_BYTES;
   static constexpr int HP = 8;                              // heads per partial slot (G <= 8)
   static constexpr int SLOT_FLOATS = HP * (D + 2);          // same slots as decode_kernel reads
-  // tensor-memory columns: S (2 x 64), P (2 x (hi 32 + lo 32)), O (2 x D)
-  static constexpr int COL_S = 0, COL_P = 128, COL_O = 256, TMEM_COLS = 512;
+  // tensor-memory columns: Q (2 buffers x D/2), S (2 x 64), P (2 x 32), O (D)
+  static constexpr int QC = D / 2;                          // columns of a row of Q (two bf16 per column)
+  static constexpr int COL_Q = 0, COL_S = 2 * QC, COL_P = COL_S + 128, COL_O = COL_P + 64, TMEM_COLS = 512;
   static_assert(DYN_BYTES <= 232448, "shared memory");
   static_assert(NSTAGES % NPW == 0, "a slot is always refilled by the same producer warp");
-  static_assert(COL_O + 2 * D <= TMEM_COLS, "tensor memory");
+  static_assert(COL_O + D <= TMEM_COLS, "tensor memory");
 };
 
 struct UmmaCtrl {
-  uint64_t full[12], empty[12];                // ring: TMA landed / tile's MMAs done
-  uint64_t s_full[2], p_full[2], pv_done[2];    // per softmax group: scores ready / probabilities stored / O updated
-  uint64_t s_free[2];                          // ... and: the group has its scores in registers
-  uint64_t q_ready;                            // the unit's query rows are in shared memory
-  uint64_t ml_ready;                           // group 1's (m, l) of the unit are in shared memory
-  uint64_t o1_free;                            // group 0 has read group 1's accumulator of the unit
+  uint64_t full[8], empty[8];                  // ring: TMA landed / tile's MMAs done
+  uint64_t s_full[2], s_free[2];               // per score buffer: scores ready / scores are in registers
+  uint64_t p_full[2], pv_done[2];              // per probability buffer: stored / consumed and O updated
+  uint64_t q_ready[2];                         // per query buffer: the unit's query rows are in tensor memory
   uint64_t unit_done;                          // every P.V of the unit is done
-  uint64_t drained;                            // all MMAs of this CTA are done
-  uint32_t meta[12];                           // per stage: bit j set = page j of the tile had a bad id
+  uint64_t drained[2];                         // all MMAs of an issuing thread are done
+  uint32_t meta[8];                            // per stage: bit j set = page j of the tile had a bad id
   uint32_t abort;
   uint32_t tmem_base;
 };
 static_assert(sizeof(UmmaCtrl) <= 384, "control block");
 
-// Tiles alternate between two softmax groups of four warps (tile i of the CTA goes to group i & 1), each
-// with its own score / probability buffers and its own accumulator O_g, so two tiles are in work at once
-// and a group has two tile times to turn its scores into probabilities.  At the end of a unit group 0
-// merges the two states (m, l, O) and writes the partials.
+// Units of this CTA in order, skipping groups without shared tiles.
+struct UnitCursor {
+  int u, end, pt, t, i, n;   // unit, end of range, its tiles, tile in unit, tile of the CTA, unit ordinal
+  const int32_t* prefix_tiles;
+  int Hkv;
+  __device__ __forceinline__ void seek() {
+    while (u < end && (pt = __ldg(prefix_tiles + u / Hkv)) <= 0) ++u;
+  }
+  __device__ __forceinline__ bool valid() const { return u < end; }
+  __device__ __forceinline__ void next_tile() {
+    ++i;
+    if (++t == pt) {
+      t = 0;
+      ++n;
+      ++u;
+      seek();
+    }
+  }
+};
+
+// The kernel (see the head of this file for the design).  Units = (group, kv head) with shared tiles, a
+// contiguous range per CTA; the result of a unit is the partial (m, l, acc) of each of its query rows in
+// the per-(sequence, kv head) prefix slots that decode_kernel and combine_kernel fold in.
 template <int D, int BS>
 __global__ void __launch_bounds__(UmmaCfg<D, BS>::NTHREADS, 1)
 prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -189,10 +208,11 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   const uint32_t ring = raw + pad;                                  // NST stages, 1024-aligned
-  const uint32_t sQ = ring + NST * C::STAGE_BYTES;
-  uint8_t* sQ_ptr = smem + NST * C::STAGE_BYTES;
-  float2* sml = reinterpret_cast<float2*>(sQ_ptr + C::Q_BYTES);     // [128] (m, l) of group 1
-  UmmaCtrl* ctrl = reinterpret_cast<UmmaCtrl*>(sQ_ptr + C::Q_BYTES + C::ML_BYTES);
+  float* xm = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);   // [2 buffers][4 quarters][64 rows]
+  float* xl = xm + 2 * 4 * 64;                                      // [4 quarters][64 rows]
+  float* xo = xl + 4 * 64;                                          // [2 halves][64 rows][32]; also the P swap area
+  uint4* xp = reinterpret_cast<uint4*>(xo);                         // [2 buffers][4 quarters][64 rows][2]
+  UmmaCtrl* ctrl = reinterpret_cast<UmmaCtrl*>(smem + NST * C::STAGE_BYTES + C::XM_BYTES + C::XL_BYTES + C::XO_BYTES);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int cta = blockIdx.x;
@@ -205,26 +225,16 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctrl->s_full[i]), 1);
-      mbar_init(smem_u32(&ctrl->p_full[i]), 128);
+      mbar_init(smem_u32(&ctrl->s_free[i]), 256);
+      mbar_init(smem_u32(&ctrl->p_full[i]), 256);
       mbar_init(smem_u32(&ctrl->pv_done[i]), 1);
-      mbar_init(smem_u32(&ctrl->s_free[i]), 128);
+      mbar_init(smem_u32(&ctrl->q_ready[i]), 256);
     }
-    mbar_init(smem_u32(&ctrl->q_ready), 128);
-    mbar_init(smem_u32(&ctrl->ml_ready), 128);
-    mbar_init(smem_u32(&ctrl->o1_free), 128);
     mbar_init(smem_u32(&ctrl->unit_done), 1);
-    mbar_init(smem_u32(&ctrl->drained), 1);
+    mbar_init(smem_u32(&ctrl->drained[0]), 1);
+    mbar_init(smem_u32(&ctrl->drained[1]), 1);
     ctrl->abort = 0;
     fence_mbar_init();
-  }
-  if (warp < 4) {
-    // rows that hold no query stay zero for the whole kernel
-    const int lam = warp * 32 + lane;
-#pragma unroll
-    for (int h = 0; h < C::HALVES; ++h)
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(sQ_ptr + h * C::Q_HALF_BYTES + lam * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
   }
   if (warp == C::MMA_WARP) {
     tmem_alloc(smem_u32(&ctrl->tmem_base), C::TMEM_COLS);
@@ -234,7 +244,7 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tbase = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_base);
-  const uint32_t tS = tbase + C::COL_S, tP = tbase + C::COL_P, tO = tbase + C::COL_O;
+  const uint32_t tQ = tbase + C::COL_Q, tS = tbase + C::COL_S, tP = tbase + C::COL_P, tO = tbase + C::COL_O;
 
   // per-sequence start tiles for the decode kernel
   for (int s = cta * blockDim.x + threadIdx.x; s < P.S; s += gridDim.x * blockDim.x)
@@ -243,9 +253,9 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const int2 range = P.ranges[cta];
   const uint32_t* abort_flag = &ctrl->abort;
 
-  if (warp > C::MMA_WARP) {
+  if (warp > C::MMA_WARP + 1) {
     // ================= producers: tile i is issued by producer i mod NPW into slot i mod NST
-    const int pw = warp - C::MMA_WARP - 1;
+    const int pw = warp - C::MMA_WARP - 2;
     bool any_bad = false, aborted = false;
     int it = 0;
     for (int u = range.x; u < range.y && !aborted; ++u) {
@@ -298,292 +308,306 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         atomicExch(&ctrl->abort, 1u);
       }
     }
-  } else if (warp == C::MMA_WARP) {
-    // ================= MMA issue: one elected lane
+  } else if (warp >= C::MMA_WARP) {
+    // ================= MMA issue.  The tensor cores take an MMA of this size about every 80-100 cycles from
+    // the issuing thread, which runs dependent code; with sixteen and more MMAs, three commits and four waits
+    // per tile one thread would be the bottleneck of the CTA, so the score products (this warp) and the
+    // P.V products (the next warp) are issued by two threads.  They meet only through the barriers.
     if (lane == 0) {
-      constexpr uint32_t ID_S = umma_idesc(UMMA_ROWS, TILE, 0, 0);   // Q (K-major) x K tile (K-major)
-      constexpr uint32_t ID_O = umma_idesc(UMMA_ROWS, D, 0, 1);      // P (tensor memory) x V tile (MN-major)
       bool ok = true;
-      int it = 0, ucnt = 0;
-      TR_DECL
-      // Descriptors are built once; per MMA only the start-address field (16-byte units, low bits) moves.
-      // The issuing lane is a single thread running dependent code, so every instruction here is on
-      // the critical path of the whole CTA.
-      const uint64_t q_desc = umma_desc(sQ, 16, 1024);
-      const uint64_t k_desc0 = umma_desc(ring, 16, 1024);
-      const uint64_t v_desc0 = umma_desc(ring + C::KV_BYTES, C::HALF_TILE_BYTES, 1024);
-      // scores of tile i into S[i & 1]
-      auto issue_scores = [&](int i) -> bool {
-        const int slot = i % NST;
-        TR_MARK(3)
-        if (!mbar_wait_abortable(smem_u32(&ctrl->full[slot]), (i / NST) & 1, abort_flag)) return false;
-        TR_MARK(6)
-        tc_fence_after();
-        const uint64_t kd = k_desc0 + static_cast<uint64_t>(slot * (C::STAGE_BYTES >> 4));
-        const uint32_t d_s = tS + (i & 1) * 64;
-#pragma unroll
-        for (int h = 0; h < C::HALVES; ++h)
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            umma_ss(d_s, q_desc + static_cast<uint64_t>((h * C::Q_HALF_BYTES + kk * 32) >> 4),
-                    kd + static_cast<uint64_t>((h * C::HALF_TILE_BYTES + kk * 32) >> 4), ID_S, (h | kk) ? 1u : 0u);
-        tc_commit(smem_u32(&ctrl->s_full[i & 1]));
-        return true;
-      };
-      for (int u = range.x; u < range.y && ok; ++u) {
-        const int pt = __ldg(P.prefix_tiles + u / P.Hkv);
-        if (pt <= 0) continue;
-        TR_MARK(0)
-        ok = mbar_wait_abortable(smem_u32(&ctrl->q_ready), ucnt & 1, abort_flag);
-        TR_MARK(1)
-        ++ucnt;
-        for (int t = 0; t < pt && ok; ++t, ++it) {
-          const int b = it & 1;
-          if (t == 0) {   // one tile for each group to start with
-            ok = issue_scores(it);
-            if (ok && pt > 1) ok = issue_scores(it + 1);
-          }
-          // As soon as the group has tile `it`'s scores in registers, its next tile's scores are computed
-          // (while the group turns this tile's into probabilities).
-          TR_MARK(0)
-          if (ok && t + 2 < pt) {
-            ok = mbar_wait_abortable(smem_u32(&ctrl->s_free[b]), (it >> 1) & 1, abort_flag);
-            TR_MARK(2)
-            tc_fence_after();
-            if (ok) ok = issue_scores(it + 2);
-            TR_MARK(3)
-          }
-          if (!ok) break;
-          ok = mbar_wait_abortable(smem_u32(&ctrl->p_full[b]), (it >> 1) & 1, abort_flag);
-          TR_MARK(4)
+      if (warp == C::MMA_WARP) {
+        constexpr uint32_t ID_S = umma_idesc(UMMA_ROWS, TILE, 0, 0);   // Q (tensor memory) x K tile (K-major)
+        // the descriptor is built once; per MMA only the start-address field (16-byte units, low bits) moves
+        const uint64_t k_desc0 = umma_desc(ring, 16, 1024);
+        UnitCursor sc{range.x, range.y, 0, 0, 0, 0, P.prefix_tiles, P.Hkv};
+        sc.seek();
+        int slot = 0;
+        uint32_t ring_phase = 0;
+        while (sc.valid() && ok) {
+          const int b = sc.i & 1;
+          // score buffer b is free when the softmax threads have tile i - 2 in registers
+          if (sc.i >= 2) ok = mbar_wait_abortable(smem_u32(&ctrl->s_free[b]), ((sc.i - 2) >> 1) & 1, abort_flag);
+          if (ok && sc.t == 0) ok = mbar_wait_abortable(smem_u32(&ctrl->q_ready[sc.n & 1]), (sc.n >> 1) & 1, abort_flag);
+          if (ok) ok = mbar_wait_abortable(smem_u32(&ctrl->full[slot]), ring_phase, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const int slot = it % NST;
-          const uint64_t vd0 = v_desc0 + static_cast<uint64_t>(slot * (C::STAGE_BYTES >> 4));
-          const uint32_t d_o = tO + b * D, a_p = tP + b * 64;
-          const uint32_t acc0 = t >= 2 ? 1u : 0u;   // the group's first tile of the unit starts its accumulator afresh
+          const uint64_t kd = k_desc0 + static_cast<uint64_t>(slot * (C::STAGE_BYTES >> 4));
+          const uint32_t d_s = tS + b * 64, a_q = tQ + (sc.n & 1) * C::QC;
 #pragma unroll
-          for (int ks = 0; ks < TILE / 16; ++ks) {
-            const uint64_t vd = vd0 + static_cast<uint64_t>((ks * 2048) >> 4);
-            umma_ts(d_o, a_p + ks * 8, vd, ID_O, ks ? 1u : acc0);      // hi part of P
-            umma_ts(d_o, a_p + 32 + ks * 8, vd, ID_O, 1u);             // lo part of P
+          for (int h = 0; h < C::HALVES; ++h)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ts(d_s, a_q + h * 32 + kk * 8, kd + static_cast<uint64_t>((h * C::HALF_TILE_BYTES + kk * 32) >> 4),
+                      ID_S, (h | kk) ? 1u : 0u);
+          tc_commit(smem_u32(&ctrl->s_full[b]));
+          sc.next_tile();
+          if (++slot == NST) {
+            slot = 0;
+            ring_phase ^= 1u;
           }
-          TR_MARK(5)
-          tc_commit(smem_u32(&ctrl->empty[slot]));    // K and V of this tile are free again
+        }
+      } else {
+        constexpr uint32_t ID_O = umma_idesc(UMMA_ROWS, D, 0, 1);      // P (tensor memory) x V tile (MN-major)
+        const uint64_t v_desc0 = umma_desc(ring + C::KV_BYTES, C::HALF_TILE_BYTES, 1024);
+        UnitCursor pc{range.x, range.y, 0, 0, 0, 0, P.prefix_tiles, P.Hkv};
+        pc.seek();
+        int slot = 0;
+        while (pc.valid() && ok) {
+          const int b = pc.i & 1;
+          // (the tile has landed: the softmax threads saw its scores before they stored these probabilities)
+          ok = mbar_wait_abortable(smem_u32(&ctrl->p_full[b]), (pc.i >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t vd0 = v_desc0 + static_cast<uint64_t>(slot * (C::STAGE_BYTES >> 4));
+          const uint32_t a_p = tP + b * 32;
+          const uint32_t acc0 = pc.t > 0 ? 1u : 0u;   // the unit's first tile starts the accumulator afresh
+#pragma unroll
+          for (int ks = 0; ks < TILE / 16; ++ks)
+            umma_ts(tO, a_p + ks * 8, vd0 + static_cast<uint64_t>((ks * 2048) >> 4), ID_O, ks ? 1u : acc0);
+          tc_commit(smem_u32(&ctrl->empty[slot]));    // K and V of this tile are free again (its scores are long done)
           tc_commit(smem_u32(&ctrl->pv_done[b]));
-          if (t == pt - 1) tc_commit(smem_u32(&ctrl->unit_done));
-          TR_MARK(7)
+          if (pc.t == pc.pt - 1) tc_commit(smem_u32(&ctrl->unit_done));
+          pc.next_tile();
+          if (++slot == NST) slot = 0;
         }
       }
-      TR_DUMP(16)
       if (!ok) {
         atomicOr(P.err, ERR_TIMEOUT);
         atomicExch(&ctrl->abort, 1u);
       }
-      // nothing of this CTA may still be running on the tensor cores when the tensor memory goes back
-      tc_commit(smem_u32(&ctrl->drained));
-      mbar_wait(smem_u32(&ctrl->drained), 0);
+      // nothing of this thread may still be running on the tensor cores when the tensor memory goes back
+      const uint32_t dbar = smem_u32(&ctrl->drained[warp - C::MMA_WARP]);
+      tc_commit(dbar);
+      mbar_wait(dbar, 0);
     }
     __syncwarp();
   } else {
-    // ================= softmax: group wg = warp / 4 takes the tiles i with (i & 1) == wg; in each group the
-    // thread (quadrant q = warp % 4, lane) owns query row lane * 4 + q, tensor-memory lane q * 32 + lane
-    const int wg = warp >> 2;
+    // ================= softmax: warp w works on tensor-memory lanes 32 * (w % 4) .. + 31.  A query row has
+    // four threads: in its first lane (hi part of P and O) and in its second lane (lo part), each for one half
+    // of the tile's columns -- and since both lanes hold the same scores, each of the four turns only a
+    // QUARTER of the tile (16 tokens) into probabilities, then swaps with the row's other lane: hi parts
+    // go to the first lane, lo parts to the second.  No thread leaves this path early: the four meet at
+    // named barriers, so after a failed wait a thread carries on (its waits then return at once).
     const int qd = warp & 3;
-    const int lam = qd * 32 + lane;
-    const int r = lane * 4 + qd;
+    const int part = warp >> 2;           // which half of the tile's columns this thread stores P for
+    const int lh = qd >> 1;               // 0: first lane of the row (hi parts), 1: second lane (lo parts)
+    const int grp = qd & 1;               // rows 0-31 / 32-63 of the slot order: the four warps that share rows
+    const int qi = part * 2 + lh;         // quarter of the tile this thread computes: tokens qi * 16 .. + 15
+    const int rho = grp * 32 + lane;      // row slot
+    const bool is_lo = lh != 0;
+    const int r = (rho & 31) * 2 + (rho >> 5);
     const int R = P.Gs * P.G;
     const bool valid = r < R;
     const int rj = valid ? r / P.G : 0, rh = valid ? r - rj * P.G : 0;   // sample in the group, head in the KV group
     const uint32_t lane_addr = static_cast<uint32_t>(qd * 32) << 16;
-    bool ok = true;
-    auto fail = [&]() {
-      ok = false;
-      if (lane == 0) {
+    constexpr int OC = D / 2;             // columns of O per thread
+    constexpr int QCP = C::QC / 2;        // columns of Q per thread
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) {   // warp-uniform: tensor-memory accesses need the whole warp
+      if (!__all_sync(0xffffffffu, mbar_wait_abortable(smem_u32(bar), parity, abort_flag)) && lane == 0) {
         atomicOr(P.err, ERR_TIMEOUT);
         atomicExch(&ctrl->abort, 1u);
       }
     };
-    // warp-uniform wait: the tensor-memory loads and stores below need the whole warp
-    auto wait_all = [&](uint64_t* bar, uint32_t parity) {
-      return __all_sync(0xffffffffu, mbar_wait_abortable(smem_u32(bar), parity, abort_flag)) != 0;
-    };
-    // the query rows of unit u into shared memory, 128-byte swizzled like a K-major MMA operand
-    auto stage_q = [&](int u) {
+    auto row_barrier = [&]() { asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory"); };   // the four warps of these rows
+    auto all_barrier = [&]() { asm volatile("bar.sync 5, 256;" ::: "memory"); };
+    // this thread's half of its query row of unit u into query buffer n & 1 (two bf16 per column)
+    auto stage_q = [&](int u, int n) {
+      uint32_t qv[QCP];
+#pragma unroll
+      for (int c = 0; c < QCP; ++c) qv[c] = 0u;
       if (valid) {
         const int gi = u / P.Hkv, g = u - gi * P.Hkv;
         const uint4* src = reinterpret_cast<const uint4*>(
-            P.q + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hq + g * P.G + rh) * D);
+            P.q + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hq + g * P.G + rh) * D + part * (D / 2));
 #pragma unroll
-        for (int h = 0; h < C::HALVES; ++h)
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(sQ_ptr + h * C::Q_HALF_BYTES + lam * 128 + ((c ^ (lam & 7)) << 4)) =
-                __ldg(src + h * 8 + c);
+        for (int c = 0; c < QCP / 4; ++c) {
+          const uint4 v = __ldg(src + c);
+          qv[4 * c] = v.x;
+          qv[4 * c + 1] = v.y;
+          qv[4 * c + 2] = v.z;
+          qv[4 * c + 3] = v.w;
+        }
       }
-      fence_proxy_async();   // the tensor cores read these rows through the async proxy
-      mbar_arrive(smem_u32(&ctrl->q_ready));
-    };
-    auto next_unit = [&](int u) {
-      for (++u; u < range.y; ++u)
-        if (__ldg(P.prefix_tiles + u / P.Hkv) > 0) return u;
-      return -1;
+      const uint32_t dst = tQ + (n & 1) * C::QC + part * QCP + lane_addr;
+      if constexpr (QCP == 32) {
+        tmem_st32(dst, qv);
+      } else {
+        tmem_st16(dst, qv);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctrl->q_ready[n & 1]));
     };
 
-    int it = 0, ucnt = 0;
-    int u = next_unit(range.x - 1);
-    if (u >= 0 && wg == 0) stage_q(u);
-    TR_DECL
-    while (u >= 0 && ok) {
-      const int gi = u / P.Hkv, g = u - gi * P.Hkv;
-      const int pt = __ldg(P.prefix_tiles + gi);
-      float m = NEG_INF, l = 0.f;
-      bool first = true;   // this group has not had a tile of the unit yet
-      for (int t = 0; t < pt && ok; ++t, ++it) {
-        if ((it & 1) != wg) continue;
-        TR_MARK(0)
-        if (!wait_all(&ctrl->s_full[wg], (it >> 1) & 1)) {
-          fail();
-          break;
-        }
-        TR_MARK(1)
-        tc_fence_after();
-        uint32_t sa[32], sb[32];
-        tmem_ld32(tS + wg * 64 + lane_addr, sa);
-        tmem_ld32(tS + wg * 64 + 32 + lane_addr, sb);
-        tc_wait_ld();
-        tc_fence_before();
-        mbar_arrive(smem_u32(&ctrl->s_free[wg]));   // the score buffer can take this group's next tile
-        TR_MARK(2)
-        const uint32_t badmask = ctrl->meta[it % NST];
-        float mx = NEG_INF;
+    // scores of tile c.i: this thread's quarter into registers (scaled, masked) and its max into shared memory
+    uint32_t sv[16];
+    auto fetch_scores = [&](const UnitCursor& c) {
+      const int it = c.i, b = it & 1;
+      wait_all(&ctrl->s_full[b], (it >> 1) & 1);
+      tc_fence_after();
+      tmem_ld16(tS + b * 64 + qi * 16 + lane_addr, sv);
+      tc_wait_ld();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctrl->s_free[b]));   // the score buffer can take tile it + 2
+      const uint32_t badmask = ctrl->meta[it % NST];
+      float mx = NEG_INF;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          float x0 = __uint_as_float(sa[c]) * P.scale_log2, x1 = __uint_as_float(sb[c]) * P.scale_log2;
-          if (badmask) {
-            if ((badmask >> (c / BS)) & 1u) x0 = NEG_INF;
-            if ((badmask >> ((32 + c) / BS)) & 1u) x1 = NEG_INF;
-          }
-          sa[c] = __float_as_uint(x0);
-          sb[c] = __float_as_uint(x1);
-          mx = fmaxf(mx, fmaxf(x0, x1));
-        }
-        // The reference value m only follows the running max when that grew by more than 2^8: P and O may
-        // then exceed 1 by that factor (harmless in fp32 / bf16), and the pass over O in tensor memory that a
-        // new reference costs becomes rare.  (m, l, O) stay consistent, which is all the merges need.
-        const bool grow = first || mx > m + 8.f;
-        const float m_new = grow ? fmaxf(m, mx) : m;
-        const float mu = (m_new == NEG_INF) ? 0.f : m_new;
-        const float alpha = grow ? fast_exp2(m - mu) : 1.f;
-        m = m_new;
-        TR_MARK(3)
-        // this group's previous P.V must be done before its P buffers and its accumulator are touched
-        if (it >= 2 && !wait_all(&ctrl->pv_done[wg], ((it - 2) >> 1) & 1)) {
-          fail();
-          break;
-        }
-        // ... and group 0 must have read group 1's accumulator of the previous unit
-        if (wg == 1 && first && ucnt > 0 && !wait_all(&ctrl->o1_free, (ucnt - 1) & 1)) {
-          fail();
-          break;
-        }
-        tc_fence_after();
-        TR_MARK(4)
-        if (__any_sync(0xffffffffu, !first && alpha != 1.f)) {   // the running max rarely moves after the first tiles
+      for (int k = 0; k < 16; ++k) {
+        float x = __uint_as_float(sv[k]) * P.scale_log2;
+        if (badmask && ((badmask >> ((qi * 16 + k) / BS)) & 1u)) x = NEG_INF;
+        sv[k] = __float_as_uint(x);
+        mx = fmaxf(mx, x);
+      }
+      xm[(b * 4 + qi) * 64 + rho] = mx;
+    };
+
+    UnitCursor uc{range.x, range.y, 0, 0, 0, 0, P.prefix_tiles, P.Hkv};
+    uc.seek();
+    if (uc.valid()) {
+      stage_q(uc.u, 0);
+      fetch_scores(uc);
+    }
+    row_barrier();
+    float m = NEG_INF, l = 0.f;
+    // One barrier of the row's four threads per tile: it publishes this tile's swapped P parts and the NEXT
+    // tile's quarter maxima (its scores are fetched before the barrier, across unit boundaries too).
+    while (uc.valid()) {
+      const int it = uc.i, b = it & 1, t = uc.t, pt = uc.pt, n = uc.n, u = uc.u;
+      UnitCursor nx = uc;
+      nx.next_tile();
+      if (t == 0) {
+        // the next unit's query rows, a whole unit ahead (the buffer's previous unit has all its scores)
+        UnitCursor nu = uc;
+        nu.t = nu.pt - 1;
+        nu.next_tile();
+        if (nu.valid()) stage_q(nu.u, n + 1);
+        m = NEG_INF;
+        l = 0.f;
+      }
+      // the row's max over the four quarters
+      const float* xmb = xm + b * 4 * 64 + rho;
+      const float mx = fmaxf(fmaxf(xmb[0], xmb[64]), fmaxf(xmb[128], xmb[192]));
+      // The reference value m only follows the running max when that grew by more than 2^8: P and O may
+      // then exceed 1 by that factor (harmless in fp32 / bf16), and the pass over O in tensor memory that a
+      // new reference costs becomes rare.  (m, l, O) stay consistent, which is all the merges need.
+      const bool grow = t == 0 || mx > m + 8.f;
+      const float m_new = grow ? fmaxf(m, mx) : m;
+      const float mu = (m_new == NEG_INF) ? 0.f : m_new;
+      const float alpha = grow ? fast_exp2(m - mu) : 1.f;
+      m = m_new;
+      // P = exp2(S - m) as bf16 head + bf16 rest; a P column holds two tokens
+      uint32_t hi[8], lo[8];
+      float ls = 0.f;
 #pragma unroll
-          for (int q = 0; q < D / 32; ++q) {
+      for (int k = 0; k < 8; ++k) {
+        const float p0 = fast_exp2(__uint_as_float(sv[2 * k]) - mu);
+        const float p1 = fast_exp2(__uint_as_float(sv[2 * k + 1]) - mu);
+        ls += p0 + p1;
+        const uint32_t h01 = pack_bf16x2(p0, p1);
+        hi[k] = h01;
+        lo[k] = pack_bf16x2(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u));
+      }
+      l = l * alpha + ls;
+      // swap with the row's other lane: it gets the part this lane does not store
+      uint4* xpb = xp + (b * 4 * 64 + rho) * 2;
+      if (is_lo) {
+        xpb[qi * 128] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        xpb[qi * 128 + 1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+      } else {
+        xpb[qi * 128] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        xpb[qi * 128 + 1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+      }
+      if (nx.valid()) fetch_scores(nx);
+      row_barrier();
+      const uint4 g0 = xpb[(qi ^ 1) * 128], g1 = xpb[(qi ^ 1) * 128 + 1];
+      uint32_t pk[16];   // this lane's 16 P columns of the half: the first-lane quarter, then the second-lane quarter
+#pragma unroll
+      for (int k = 0; k < 8; ++k) pk[is_lo ? 8 + k : k] = is_lo ? lo[k] : hi[k];
+      pk[is_lo ? 0 : 8] = g0.x;
+      pk[is_lo ? 1 : 9] = g0.y;
+      pk[is_lo ? 2 : 10] = g0.z;
+      pk[is_lo ? 3 : 11] = g0.w;
+      pk[is_lo ? 4 : 12] = g1.x;
+      pk[is_lo ? 5 : 13] = g1.y;
+      pk[is_lo ? 6 : 14] = g1.z;
+      pk[is_lo ? 7 : 15] = g1.w;
+      // the product that read this probability buffer two tiles ago must be done
+      if (it >= 2) wait_all(&ctrl->pv_done[b], ((it - 2) >> 1) & 1);
+      if (__any_sync(0xffffffffu, t > 0 && alpha != 1.f)) {
+        // new reference: scale this thread's columns of O, once the previous tile's product is in
+        wait_all(&ctrl->pv_done[b ^ 1], ((it - 1) >> 1) & 1);
+        tc_fence_after();
+#pragma unroll
+        for (int q = 0; q < OC / 32; ++q) {
+          uint32_t o[32];
+          tmem_ld32(tO + part * OC + q * 32 + lane_addr, o);
+          tc_wait_ld();
+#pragma unroll
+          for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+          tmem_st32(tO + part * OC + q * 32 + lane_addr, o);
+        }
+      }
+      tc_fence_after();
+      tmem_st16(tP + b * 32 + part * 16 + lane_addr, pk);
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctrl->p_full[b]));
+      if (t == pt - 1) {
+        // ---- the unit's result: (m, l) and O = hi part + lo part, to the per-(sequence, KV head) prefix slot.
+        // The lo rows cross to the row's first lane through shared memory as bf16 (they are 2^-9 of O).
+        const int gi = u / P.Hkv, g = u - gi * P.Hkv;
+        wait_all(&ctrl->unit_done, n & 1);
+        tc_fence_after();
+        xl[qi * 64 + rho] = l;
+        uint32_t* xrow = reinterpret_cast<uint32_t*>(xo) + (part * 64 + rho) * (OC / 2);
+        float* slotp = P.pfx_partials + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hkv + g) * C::SLOT_FLOATS;
+        if (is_lo) {
+#pragma unroll
+          for (int q = 0; q < OC / 32; ++q) {
             uint32_t o[32];
-            tmem_ld32(tO + wg * D + q * 32 + lane_addr, o);
+            tmem_ld32(tO + part * OC + q * 32 + lane_addr, o);
             tc_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-            tmem_st32(tO + wg * D + q * 32 + lane_addr, o);
+            for (int k = 0; k < 4; ++k)
+              reinterpret_cast<uint4*>(xrow + q * 16)[k] =
+                  make_uint4(pack_bf16x2(__uint_as_float(o[8 * k]), __uint_as_float(o[8 * k + 1])),
+                             pack_bf16x2(__uint_as_float(o[8 * k + 2]), __uint_as_float(o[8 * k + 3])),
+                             pack_bf16x2(__uint_as_float(o[8 * k + 4]), __uint_as_float(o[8 * k + 5])),
+                             pack_bf16x2(__uint_as_float(o[8 * k + 6]), __uint_as_float(o[8 * k + 7])));
           }
         }
-        TR_MARK(5)
-        // P = exp2(S - m) as hi + lo bf16; column c of a P block holds tokens 2c and 2c + 1
-        float ls = 0.f;
+        all_barrier();
+        if (!is_lo) {
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t hi[16], lo[16];
+          for (int q = 0; q < OC / 32; ++q) {
+            uint32_t o[32];
+            tmem_ld32(tO + part * OC + q * 32 + lane_addr, o);
+            tc_wait_ld();
+            if (valid) {
+              float4* dst = reinterpret_cast<float4*>(slotp + 2 * C::HP + rh * D + part * OC + q * 32);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-#if defined(PDATTN_ABL) && PDATTN_ABL == 1
-            hi[c] = 0x3f803f80u; lo[c] = 0u; ls += 2.f;
-#else
-            const float p0 = fast_exp2(__uint_as_float(hf ? sb[2 * c] : sa[2 * c]) - mu);
-            const float p1 = fast_exp2(__uint_as_float(hf ? sb[2 * c + 1] : sa[2 * c + 1]) - mu);
-            ls += p0 + p1;
-            const uint32_t h01 = pack_bf16x2(p0, p1);
-            hi[c] = h01;
-            lo[c] = pack_bf16x2(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u));
-#endif
-          }
-          tmem_st16(tP + wg * 64 + hf * 16 + lane_addr, hi);
-          tmem_st16(tP + wg * 64 + 32 + hf * 16 + lane_addr, lo);
-        }
-        l = l * alpha + ls;
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(smem_u32(&ctrl->p_full[wg]));
-        TR_MARK(6)
-        first = false;
-      }
-      if (!ok) break;
-      // The group that had the unit's last tile has seen its scores: the query rows can make way for the
-      // next unit's, whose first scores then run while the epilogue below reads the accumulators.
-      const int un = next_unit(u);
-      if (((it - 1) & 1) == wg && un >= 0) stage_q(un);
-      if (wg == 1) {
-        if (first && ucnt > 0 && !wait_all(&ctrl->o1_free, (ucnt - 1) & 1)) {   // no tile here: keep in step all the same
-          fail();
-          break;
-        }
-        sml[lam] = make_float2(m, l);
-        mbar_arrive(smem_u32(&ctrl->ml_ready));
-      } else {
-        // (a barrier of its own, one phase per unit: group 0 does not follow every phase of group 1's
-        // pv_done, and a parity wait cannot tell two phases apart)
-        if (!wait_all(&ctrl->unit_done, ucnt & 1) || !wait_all(&ctrl->ml_ready, ucnt & 1)) {
-          fail();
-          break;
-        }
-        tc_fence_after();
-        const float2 ml1 = sml[lam];
-        const float M = fmaxf(m, ml1.x);
-        const float Mu = (M == NEG_INF) ? 0.f : M;
-        const bool has0 = m != NEG_INF, has1 = ml1.x != NEG_INF;   // a group without a tile holds stale data
-        const float f0 = fast_exp2(m - Mu), f1 = fast_exp2(ml1.x - Mu);
-        float* slotp = P.pfx_partials + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hkv + g) * C::SLOT_FLOATS;
-        if (valid) {
-          slotp[rh] = M;
-          slotp[C::HP + rh] = l * f0 + ml1.y * f1;
-        }
-#pragma unroll
-        for (int q = 0; q < D / 32; ++q) {
-          uint32_t o0[32], o1[32];
-          tmem_ld32(tO + q * 32 + lane_addr, o0);
-          tmem_ld32(tO + D + q * 32 + lane_addr, o1);
-          tc_wait_ld();
-          if (valid) {
-            float4* dst = reinterpret_cast<float4*>(slotp + 2 * C::HP + rh * D + q * 32);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              float v[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                v[e] = (has0 ? __uint_as_float(o0[4 * c + e]) * f0 : 0.f) + (has1 ? __uint_as_float(o1[4 * c + e]) * f1 : 0.f);
-              dst[c] = make_float4(v[0], v[1], v[2], v[3]);
+              for (int k = 0; k < 4; ++k) {
+                const uint4 w = reinterpret_cast<const uint4*>(xrow + q * 16)[k];
+                dst[2 * k] = make_float4(__uint_as_float(o[8 * k]) + __uint_as_float(w.x << 16),
+                                         __uint_as_float(o[8 * k + 1]) + __uint_as_float(w.x & 0xffff0000u),
+                                         __uint_as_float(o[8 * k + 2]) + __uint_as_float(w.y << 16),
+                                         __uint_as_float(o[8 * k + 3]) + __uint_as_float(w.y & 0xffff0000u));
+                dst[2 * k + 1] = make_float4(__uint_as_float(o[8 * k + 4]) + __uint_as_float(w.z << 16),
+                                             __uint_as_float(o[8 * k + 5]) + __uint_as_float(w.z & 0xffff0000u),
+                                             __uint_as_float(o[8 * k + 6]) + __uint_as_float(w.w << 16),
+                                             __uint_as_float(o[8 * k + 7]) + __uint_as_float(w.w & 0xffff0000u));
+              }
             }
           }
+          if (valid && part == 0) {
+            slotp[rh] = m;
+            slotp[C::HP + rh] = (xl[rho] + xl[64 + rho]) + (xl[128 + rho] + xl[192 + rho]);
+          }
         }
-        tc_fence_before();
-        mbar_arrive(smem_u32(&ctrl->o1_free));
+        all_barrier();   // the swap area is used again by the next tile
       }
-      ++ucnt;
-      u = un;
+      uc = nx;
     }
-    if (qd == 0) { TR_MARK(7) TR_DUMP(24 + wg * 8) }
   }
 
   tc_fence_before();
