@@ -53,6 +53,9 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cfg", type=int, default=2, help="BASELINE.json config index + 1 (default: the metric's config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--short-batches", action="store_true",
+                    help="also time batches of 4096 short contexts under both merge modes, and a large GRPO batch "
+                         "early in its rollout under both prefix kernels (secondary results, N = 1)")
     ap.add_argument("--grouped", action="store_true",
                     help="config 3 only: time pdattn_decode_grouped (shared prompt pages read once per group)")
     ap.add_argument("--num-seqs", type=int, default=None,
@@ -371,6 +374,9 @@ def main():
             extras["grouped_shared_prefix"] = {"ms_per_step": t_grouped, "seq_steps_per_s": S / (t_grouped * 1e-3),
                                                "unique_kv_gbs": uniq / (t_grouped * 1e-3) / 1e9}
 
+        if args.short_batches:
+            extras["short_context_batches"] = short_batches(pdattn, W, dev, timed)
+
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only)
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -415,6 +421,46 @@ def main():
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def short_batches(pdattn, W, dev, timed):
+    """Batches whose pieces are one to a few tiles long: 4096 sequences of the 7B shape under the barrier
+    and the chained merge of the decode kernel, and 512 GRPO groups of 8 (40 q / 8 KV heads) that share a
+    1024-token prompt and have generated 1..64 tokens, under both kernels for the shared tiles."""
+    res = {}
+    rng = np.random.default_rng(0)
+    for name, lens in [("4096x64", np.full(4096, 64)), ("4096x128", np.full(4096, 128)),
+                       ("4096xU[50,400]", rng.integers(50, 400, size=4096)), ("4096x512", np.full(4096, 512))]:
+        w = W.make_custom(lens, Hq=28, Hkv=4, d=128, bs=16, seed=3, device=dev, poison=False)
+        ws = pdattn.alloc_workspace(w.num_seqs, 28, 4, 128, 16, device=dev)
+        out = torch.empty_like(w.q)
+        row = {"kv_bytes": w.logical_kv_bytes()}
+        for mode, key in ((0, "barrier_merge_ms"), (1, "chained_merge_ms")):
+            pdattn.set_merge_mode(mode)
+            row[key] = timed(lambda: pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale,
+                                                      out, ws, context_lens_host=w.context_lens_host))
+        pdattn.set_merge_mode(-1)
+        assert pdattn.check(ws) == pdattn.OK
+        res[name] = row
+        del w, ws, out
+        torch.cuda.empty_cache()
+    lens = 1024 + rng.integers(1, 65, size=4096)
+    w = W.make_custom(lens, Hq=40, Hkv=8, d=128, bs=16, seed=3, device=dev, poison=False, shared_prefix_pages=64, group=8)
+    gws = pdattn.alloc_grouped_workspace(w.num_seqs, 40, 8, 128, device=dev)
+    out = torch.empty_like(w.q)
+    pth = np.full(512, 16, dtype=np.int32)
+    ptd = torch.from_numpy(pth).to(dev)
+    row = {"unique_kv_bytes": w.unique_kv_bytes(), "logical_kv_bytes": w.logical_kv_bytes()}
+    row["ungrouped_ms"] = timed(lambda: pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale,
+                                                         out, gws, context_lens_host=w.context_lens_host), n=5)
+    for eng, key in ((0, "grouped_warp_mma_ms"), (1, "grouped_tcgen05_ms")):
+        pdattn.set_prefix_engine(eng)
+        row[key] = timed(lambda: pdattn.decode_grouped(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale,
+                                                       out, gws, w.context_lens_host, 8, ptd, pth), n=10)
+    pdattn.set_prefix_engine(-1)
+    assert pdattn.check(gws) == pdattn.OK
+    res["grpo_512x8_prompt1024_resp1..64"] = row
+    return res
 
 
 def decode_loop(pdattn, W, dev, stream, steps=64):
