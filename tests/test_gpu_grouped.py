@@ -105,6 +105,41 @@ def test_full_size_grpo_config_sampled():
     assert torch.equal(out, again)
 
 
+@pytest.mark.parametrize("d", [128, 64])
+def test_grouped_with_peaked_scores_moves_the_softmax_reference(d):
+    """Score spread of about 25 in the log2 domain: the running max of a row jumps by more than 2^8 between
+    tiles again and again, so the accumulator of the shared tiles is rescaled (in tensor memory for the
+    tcgen05 kernel, which only follows the max when it grew by that much), and a few tokens carry the weight."""
+    lens = [1024 + 1 + 37 * j for j in range(16)]
+    w = W.make_custom(lens, Hq=10, Hkv=2, d=d, seed=77, device=DEV, poison=False)
+    bt = w.block_table.clone()
+    for j in range(16):
+        bt[j, :64] = bt[j - j % 8, :64]                  # two groups of 8 share 64 pages = 16 tiles
+    w = dataclasses.replace(w, block_table=bt, scale=w.scale * 16.0)
+    W.poison_unused(w)
+    out, status = run_grouped(w, 8, [16, 16])
+    assert status == pdattn.OK
+    assert_parity(out, orc.decode_workload(w.to("cpu")), f"grouped, peaked scores, d={d}")
+    again, _ = run_grouped(w, 8, [16, 16])
+    assert torch.equal(out, again)
+
+
+def test_grouped_bad_page_ids_in_the_shared_tiles_are_masked_and_reported():
+    lens = [300 + 11 * j for j in range(8)]
+    w = W.make_custom(lens, Hq=8, Hkv=2, d=128, seed=78, device=DEV, num_blocks=256, poison=False)
+    bt = w.block_table.clone()
+    for j in range(1, 8):
+        bt[j, :16] = bt[0, :16]                          # one group shares 16 pages = 4 tiles
+    bt[:, 5] = 256                                       # one past the pool, in the second shared tile
+    bt[:, 9] = -3
+    wb = dataclasses.replace(w, block_table=bt)
+    out, status = run_grouped(wb, 8, [4])
+    assert status == pdattn.BAD_PAGE_INDEX
+    ref, bad = orc.decode_workload(wb.to("cpu"), return_bad=True)
+    assert bad == 8 * 2 * 16 * 8                         # 8 rows, two pages of 16 tokens, 8 heads
+    assert_parity(out, ref, "grouped, bad pages in the shared tiles masked")
+
+
 def test_grouped_rejects_what_it_cannot_do():
     w = W.make_config(3, device=DEV, num_seqs=16, len_div=4)
     ws = pdattn.alloc_grouped_workspace(16, 40, 8, 128)
