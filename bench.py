@@ -362,6 +362,15 @@ def main():
         assert pdattn.check(ws) == pdattn.OK
         if args.cfg == 2 and args.num_seqs is None:
             extras["decode_loop"] = decode_loop(pdattn, W, dev, stream)
+            # two query tokens per sequence (a verification step of the engine): 14 rows share each KV head's tiles
+            q2 = W.normal_bf16(S * 2 * c.num_q_heads * c.head_dim, 77, 7, device=dev).view(S, 2, c.num_q_heads, c.head_dim)
+            o2 = torch.empty_like(q2)
+            mws = pdattn.alloc_multi_workspace(S, c.num_q_heads, c.num_kv_heads, c.head_dim, c.block_size, 2, device=dev)
+            t_multi = timed(lambda: pdattn.decode_multi(q2, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale,
+                                                        o2, mws, context_lens_host=c.context_lens_host))
+            assert pdattn.check(mws) == pdattn.OK
+            extras["two_query_tokens_ms_per_step"] = t_multi
+            del q2, o2, mws
         if args.cfg == 3 and args.num_seqs is None:
             # GRPO groups of 8 share their 1024-token prompt pages: read them once per group
             gws = pdattn.alloc_grouped_workspace(S, c.num_q_heads, c.num_kv_heads, c.head_dim, device=dev)

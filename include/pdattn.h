@@ -123,6 +123,25 @@ pdattn_status pdattn_decode_grouped(const pdattn_args* args, int group_size, con
                                     const int32_t* prefix_tiles_host, pdattn_stream_t stream);
 
 /*
+ * Decode step with several query tokens per sequence: the last num_query_tokens tokens of every
+ * sequence are new (their K/V are already in the cache and counted in context_lens, as the single
+ * current token is in pdattn_decode_ex), e.g. the rows of a speculative-verification or chunked step
+ * of the rollout engine (Section 2.1 only says that rollouters decode autoregressively; the paper has
+ * no counterpart for this variant).  Query token j (0 <= j < T) sits at position context_len - T + j
+ * and attends to the keys at positions <= its own (causal among the new tokens):
+ *   out[s, j, h, :] = softmax_t( scale * q[s, j, h, :] . K[t, h / G, :] ) . V[t, h / G, :],  t < context_len - (T - 1 - j)
+ * Layouts: args->q and args->out are DEVICE bf16 [num_seqs, T, num_q_heads, head_dim], dense; all else
+ * as in pdattn_decode_ex.  The T * G query rows of a KV head share its K/V tiles (read once).
+ * A query token that sees no key (context_len < T - j) gets zeros.
+ *   Requirements: T >= 1, T * G <= 16; args->workspace holds pdattn_multi_workspace_size() bytes
+ *   (pdattn_workspace_size() is enough while T * G <= 8).  T = 1 is pdattn_decode_ex.
+ *   PDATTN_UNSUPPORTED for T * G > 16.
+ */
+pdattn_status pdattn_multi_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                                          int block_size, int num_query_tokens, size_t* device_bytes);
+pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens, pdattn_stream_t stream);
+
+/*
  * KV append: the step that precedes attention in the decoding loop (Section 2.3; the cache grows by
  * b_kv bytes per token and layer, Appendix A.1.2).  For every sequence s with t = context_lens[s]:
  * the rows k_new[s], v_new[s] (DEVICE bf16 [num_seqs, num_kv_heads, head_dim], dense) are written to

@@ -104,6 +104,21 @@ def decode(q, k_cache, v_cache, block_table, context_lens, scale, pairs=None, nu
     return (out, bad.value) if return_bad else out
 
 
+def decode_multi(q, k_cache, v_cache, block_table, context_lens, scale, num_threads=None):
+    """Several query tokens per sequence, q [S, T, Hq, d]: the last T tokens of a sequence are new, and query
+    token j attends to the keys at positions up to its own, i.e. to the first L - (T - 1 - j) tokens.  Written
+    out as T plain decode steps over truncated contexts (a query token that sees no key gives zeros)."""
+    q = _cpu(q)
+    S, T, Hq, d = q.shape
+    lens = np.asarray(_cpu(context_lens).numpy(), dtype=np.int64)
+    out = np.empty((S, T, Hq, d), dtype=np.float64)
+    for j in range(T):
+        lens_j = np.maximum(lens - (T - 1 - j), 0).astype(np.int32)
+        out[:, j] = decode(q[:, j].contiguous(), k_cache, v_cache, block_table, torch.from_numpy(lens_j), scale,
+                           num_threads=num_threads)
+    return out
+
+
 def decode_workload(w, **kw):
     return decode(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, **kw)
 

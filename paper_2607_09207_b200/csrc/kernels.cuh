@@ -65,6 +65,7 @@ struct DecodeParams {
   int4* rec;                // per-span record: (first_unit, first_tile, own_unit, own_slot)
   float* partials;          // [span][2][HP*(D+2)] fp32
   int S, Hq, Hkv, G, MB, NB;
+  int T;                    // query tokens per sequence (1 = plain decode); T * G rows share a KV head's tiles
   float scale_log2;         // scale * log2(e)
   PlanParams plan;          // host plan (ignored when use_ws_plan)
   int use_ws_plan;
@@ -315,7 +316,10 @@ struct Walker {
 template <int D, int NT, int BS, bool TAIL>
 __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uint32_t (&qf)[NT][D / 16][2],
                                              float (&acc)[NT][D / 16][4], float (&m)[NT][2], float (&l)[NT][2],
-                                             float sl2, int n_valid, uint32_t badmask, int lane) {
+                                             float sl2, int n_left, uint32_t badmask, int lane,
+                                             const int (&lag)[NT][2]) {
+  // n_left: tokens of the sequence from this tile's first one on (>= TILE unless TAIL)
+  const int n_valid = n_left < TILE ? n_left : TILE;
   using C = Cfg<D, NT, BS>;
   constexpr int GROUPS = TILE / 16;     // 16-token MMA groups per tile
   const float NEG_INF = __int_as_float(0xff800000);
@@ -381,8 +385,10 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
       for (int r = 0; r < 4; ++r) {
         float v = sc[j][nt][r] * sl2;
         if (TAIL) {
+          // lag: tokens at the end of the context that this column's query token must not see (it sits
+          // that many positions before the last one; 0 for plain decode)
           const int tok = j * 16 + trow + ((r & 2) ? 8 : 0);
-          if (tok >= n_valid) v = NEG_INF;
+          if (tok >= n_left - lag[nt][r & 1]) v = NEG_INF;
         }
         if (dead_page) v = NEG_INF;
         sc[j][nt][r] = v;
@@ -562,6 +568,15 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
   const int hq0 = lane >> 2;
   const int qcol = (lane & 3) * 2;
   const int drow = lane >> 2;
+  const int R = P.G * P.T;          // query rows per unit: row = query token * G + head
+  int lag[NT][2];                   // per score column of this lane: context tokens its query token must not see
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int row = nt * 8 + qcol + e;
+      lag[nt][e] = row < R ? P.T - 1 - row / P.G : 0;
+    }
   bool aborted = false;
   int it = 0, pcnt = 0, mcnt = 0;
 
@@ -620,7 +635,7 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const int head = nt * 8 + hq0;
-          const bool live = head < P.G;
+          const bool live = head < R;
           const uint32_t qa = qbuf + qs * C::Q_BYTES + (live ? head : 0) * (D * 2) + qcol * 2;
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
@@ -659,11 +674,11 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         const uint32_t sK = ring + slot * C::STAGE_BYTES;
         const uint32_t sV = sK + C::KV_BYTES;
         const uint32_t badmask = ctrl->meta[slot];
-        const int n_valid = min(TILE, pc.L - (pc.t0 + t) * TILE);
-        if (n_valid == TILE) {
-          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane);
+        const int n_left = pc.L - (pc.t0 + t) * TILE;
+        if (n_left - (P.T - 1) >= TILE) {   // every query token sees the whole tile
+          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag);
         } else {
-          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_valid, badmask, lane);
+          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag);
           fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
         }
         __syncwarp();
@@ -757,21 +772,22 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
       }
       if (complete) {
         // bf16 output; neighbouring lanes swap one value so that each stores two adjacent elements
-        __nv_bfloat16* ob = P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G) * D;
         const bool odd = drow & 1;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const float inv0 = l[nt][0] > 0.f ? 1.f / l[nt][0] : 0.f;
           const float inv1 = l[nt][1] > 0.f ? 1.f / l[nt][1] : 0.f;
-          const int myh = nt * 8 + qcol + (odd ? 1 : 0);
-          __nv_bfloat16* orow = ob + static_cast<int64_t>(myh) * D + (drow & ~1);
+          const int myh = nt * 8 + qcol + (odd ? 1 : 0);     // row = query token * G + head
+          const int qtok = myh < R ? myh / P.G : 0;
+          __nv_bfloat16* orow = P.out + ((static_cast<int64_t>(pc.s) * P.T + qtok) * P.Hq + pc.g * P.G + (myh - qtok * P.G)) * D +
+                                (drow & ~1);
 #pragma unroll
           for (int jm = 0; jm < D / 16; ++jm) {
             const float v0 = acc[nt][jm][0] * inv0, v1 = acc[nt][jm][1] * inv1;
             const float v2 = acc[nt][jm][2] * inv0, v3 = acc[nt][jm][3] * inv1;
             const float r0 = __shfl_xor_sync(0xffffffffu, odd ? v0 : v1, 4);
             const float r1 = __shfl_xor_sync(0xffffffffu, odd ? v2 : v3, 4);
-            if (myh < P.G) {
+            if (myh < R) {
               *reinterpret_cast<uint32_t*>(orow + jm * 16) = odd ? pack_bf16x2(r0, v1) : pack_bf16x2(v0, r0);
               *reinterpret_cast<uint32_t*>(orow + jm * 16 + 8) = odd ? pack_bf16x2(r1, v3) : pack_bf16x2(v2, r1);
             }
@@ -887,11 +903,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             break;
           }
           if (lane == 0) {
+            // the G rows of each of the T query tokens, packed: row = query token * G + head
             const uint32_t bytes = static_cast<uint32_t>(P.G) * D * 2;
             const uint32_t qb = smem_u32(&ctrl->q_full[qs]);
             if (CHAIN) ctrl->qseq[qs] = pcnt;
-            mbar_arrive_expect_tx(qb, bytes);
-            bulk_load(qbuf + qs * C::Q_BYTES, P.q + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G) * D, bytes, qb);
+            mbar_arrive_expect_tx(qb, bytes * P.T);
+            for (int qt = 0; qt < P.T; ++qt)
+              bulk_load(qbuf + qs * C::Q_BYTES + qt * bytes,
+                        P.q + ((static_cast<int64_t>(pc.s) * P.T + qt) * P.Hq + pc.g * P.G) * D, bytes, qb);
           }
         }
         ++pcnt;
@@ -989,8 +1008,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     // sequences with no context produce zeros
     for (int s = cta; s < P.S; s += gridDim.x) {
       if (__ldg(P.context_lens + s) <= 0) {
-        uint32_t* o = reinterpret_cast<uint32_t*>(P.out + static_cast<int64_t>(s) * P.Hq * D);
-        for (int i = ct; i < P.Hq * D / 2; i += NCT) o[i] = 0u;
+        uint32_t* o = reinterpret_cast<uint32_t*>(P.out + static_cast<int64_t>(s) * P.T * P.Hq * D);
+        for (int i = ct; i < P.T * P.Hq * D / 2; i += NCT) o[i] = 0u;
       }
     }
   }
@@ -1003,6 +1022,16 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                              lane);
     return;
   }
+
+  const int R = P.G * P.T;          // query rows per unit: row = query token * G + head
+  int lag[NT][2];                   // per score column of this lane: context tokens its query token must not see
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int row = nt * 8 + qcol + e;
+      lag[nt][e] = row < R ? P.T - 1 - row / P.G : 0;
+    }
 
   int span = cta;
   for (int k = 0; span >= 0; ++k) {
@@ -1031,7 +1060,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const int head = nt * 8 + hq0;
-          const bool live = have_q && head < P.G;
+          const bool live = have_q && head < R;
           const uint32_t qa = qbuf + qs * C::Q_BYTES + (live ? head : 0) * (D * 2) + qcol * 2;
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
@@ -1082,13 +1111,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const uint32_t sK = ring + slot * C::STAGE_BYTES;
         const uint32_t sV = sK + C::KV_BYTES;
         const uint32_t badmask = ctrl->meta[slot];
-        const int n_valid = min(TILE, pc.L - (pc.t0 + t) * TILE);
+        const int n_left = pc.L - (pc.t0 + t) * TILE;
         if (PROBE) {
           // ceiling probe: no math
-        } else if (n_valid == TILE) {
-          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane);
+        } else if (n_left - (P.T - 1) >= TILE) {   // every query token sees the whole tile
+          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag);
         } else {
-          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_valid, badmask, lane);
+          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag);
           fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
         }
         __syncwarp();
@@ -1208,12 +1237,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             const int dq = idx % (D / 4);
             const float4 a = a_r[i];
             if (complete) {
-              if (h < P.G) {
+              if (h < R) {   // row h = query token * G + head
                 const float inv = Ls_r[i] > 0.f ? 1.f / Ls_r[i] : 0.f;
                 uint2 o;
                 o.x = pack_bf16x2(a.x * inv, a.y * inv);
                 o.y = pack_bf16x2(a.z * inv, a.w * inv);
-                *reinterpret_cast<uint2*>(P.out + (static_cast<int64_t>(pc.s) * P.Hq + pc.g * P.G + h) * D + dq * 4) = o;
+                const int qtok = h / P.G;
+                *reinterpret_cast<uint2*>(P.out + ((static_cast<int64_t>(pc.s) * P.T + qtok) * P.Hq + pc.g * P.G +
+                                                   (h - qtok * P.G)) * D + dq * 4) = o;
               }
             } else {
               if (dq == 0) {
@@ -1363,6 +1394,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
   // ---- consumers: warp w owns query rows [8w, 8w + 8) of the group's group_size * G rows
   const int R = P.Gs * P.G;
+  const int no_lag[1][2] = {{0, 0}};
   const int hq0 = lane >> 2;
   const int qcol = (lane & 3) * 2;
   const bool has_rows = warp * 8 < R;
@@ -1403,7 +1435,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
       if (has_rows) {
         const uint32_t sK = ring + slot * C::STAGE_BYTES;
-        compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, P.scale_log2, TILE, ctrl->meta[slot], lane);
+        compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, P.scale_log2, TILE, ctrl->meta[slot], lane, no_lag);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
@@ -1507,7 +1539,7 @@ template <int D, int NT>
 __global__ void __launch_bounds__(256)
 combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, const float* __restrict__ partials,
                __nv_bfloat16* __restrict__ out, int Hq, int Hkv, int G, const int32_t* __restrict__ start_tiles,
-               const float* __restrict__ pfx_partials) {
+               const float* __restrict__ pfx_partials, int T) {
   constexpr int HP = 8 * NT;
   constexpr int SLOT_FLOATS = HP * (D + 2);
   const int c = blockIdx.x;
@@ -1546,7 +1578,7 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
   for (int idx = threadIdx.x; idx < HP * (D / 4); idx += blockDim.x) {
     const int h = idx / (D / 4);
     const int dq = idx % (D / 4);
-    if (h >= G) continue;
+    if (h >= G * T) continue;   // row h = query token * G + head
     float M = NEG_INF;
     for (int p = p0; p < np; ++p) M = fmaxf(M, piece(p)[h]);
     const float Mu = (M == NEG_INF) ? 0.f : M;
@@ -1566,7 +1598,8 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
     uint2 o;
     o.x = pack_bf16x2(a.x * inv, a.y * inv);
     o.y = pack_bf16x2(a.z * inv, a.w * inv);
-    *reinterpret_cast<uint2*>(out + (static_cast<int64_t>(s) * Hq + g * G + h) * D + dq * 4) = o;
+    const int qtok = h / G;
+    *reinterpret_cast<uint2*>(out + ((static_cast<int64_t>(s) * T + qtok) * Hq + g * G + (h - qtok * G)) * D + dq * 4) = o;
   }
 }
 

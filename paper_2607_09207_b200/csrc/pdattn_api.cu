@@ -33,6 +33,7 @@ thread_local std::vector<int32_t> g_start_tiles_host;
 int g_dyn_per_cta = 0;                    // run-time spans per CTA (pdattn_set_dynamic_spans)
 int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (chained), 0 barrier, 1 chained
 thread_local bool g_use_chain = true;     // decided per call, read by the launcher
+thread_local int g_query_tokens = 1;      // query tokens per sequence of the call (pdattn_decode_multi)
 int g_prefix_engine = -1;                 // pdattn_set_prefix_engine: -1 default (tcgen05), 0 warp MMAs, 1 tcgen05
 
 struct Binding {
@@ -261,7 +262,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   cfg.numAttrs = 1;
   e = cudaLaunchKernelEx(&cfg, combine_kernel<D, NT>, P.hdr, n_spans_host, static_cast<const int4*>(P.rec),
                          static_cast<const float*>(P.partials), P.out, P.Hq, P.Hkv, P.G, P.start_tiles,
-                         P.pfx_partials);
+                         P.pfx_partials, P.T);
   if (e != cudaSuccess) return cuda_fail("combine_kernel launch", e);
   return PDATTN_OK;
 }
@@ -420,9 +421,12 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   if (mis(a->q, 16) || mis(a->k_cache, 16) || mis(a->v_cache, 16) || mis(a->out, 16) || mis(a->workspace, 256))
     return PDATTN_MISALIGNED;
   const int G = a->num_q_heads / a->num_kv_heads;
-  const WsLayout wl = ws_layout(a->num_seqs, G, a->head_dim);
-  // grouped calls keep two more arrays behind the ordinary layout
+  const int T = g_query_tokens;
   const bool grouped = g_grouped.active;
+  if (T < 1) return PDATTN_INVALID_ARG;
+  if (G * T > 16 || (T > 1 && grouped)) return PDATTN_UNSUPPORTED;
+  const WsLayout wl = ws_layout(a->num_seqs, G * T, a->head_dim);
+  // grouped calls keep two more arrays behind the ordinary layout
   const size_t off_start = wl.total;
   const size_t off_pfx = off_start + align_up(static_cast<size_t>(a->num_seqs) * 4, 256);
   const size_t pfx_bytes = static_cast<size_t>(a->num_seqs) * a->num_kv_heads * (G > 8 ? 16 : 8) * (a->head_dim + 2) * 4;
@@ -469,6 +473,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   P.Hq = a->num_q_heads;
   P.Hkv = a->num_kv_heads;
   P.G = G;
+  P.T = T;
   P.MB = a->max_blocks_per_seq;
   P.NB = a->num_blocks;
   P.scale_log2 = a->scale * 1.4426950408889634f;
@@ -575,7 +580,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     P.pfx_partials = X.pfx_partials;
   }
 
-  const bool nt2 = G > 8;
+  const bool nt2 = G * T > 8;
   if (a->head_dim == 128)
     s = nt2 ? launch<128, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
             : launch<128, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
@@ -583,6 +588,26 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
             : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
   if (s == PDATTN_OK) g_last_launches += 2;
+  return s;
+}
+
+pdattn_status pdattn_multi_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim, int block_size,
+                                          int num_query_tokens, size_t* device_bytes) {
+  if (!device_bytes) return PDATTN_INVALID_ARG;
+  pdattn_status s = check_shape(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size);
+  if (s != PDATTN_OK) return s;
+  if (num_query_tokens < 1) return PDATTN_INVALID_ARG;
+  const int G = num_q_heads / num_kv_heads;
+  if (G * num_query_tokens > 16) return PDATTN_UNSUPPORTED;
+  *device_bytes = ws_layout(num_seqs, G * num_query_tokens, head_dim).total;
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens, pdattn_stream_t stream) {
+  if (!args) return PDATTN_INVALID_ARG;
+  g_query_tokens = num_query_tokens;
+  const pdattn_status s = pdattn_decode_ex(args, stream);
+  g_query_tokens = 1;
   return s;
 }
 
@@ -831,6 +856,7 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   P.Hq = a->num_q_heads;
   P.Hkv = a->num_kv_heads;
   P.G = G;
+  P.T = 1;
   P.MB = a->max_blocks_per_seq;
   P.NB = a->num_blocks;
   P.scale_log2 = a->scale * 1.4426950408889634f;

@@ -34,6 +34,7 @@ EXPORTS = [
     "pdattn_set_merge_mode", "pdattn_set_prefix_engine",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
+    "pdattn_multi_workspace_size", "pdattn_decode_multi",
 ]
 
 
@@ -93,6 +94,8 @@ def lib():
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
         L.pdattn_grouped_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_grouped.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
+        L.pdattn_multi_workspace_size.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
+        L.pdattn_decode_multi.argtypes = [ctypes.POINTER(Args), i32, vp]
         L.pdattn_append_kv.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp]
         L.pdattn_check.argtypes = [vp, vp]
         L.pdattn_profile_events.argtypes = [vp, vp]
@@ -227,6 +230,50 @@ def decode_grouped(q, k_cache, v_cache, block_table, context_lens, scale, out, w
                                      _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_decode_grouped")
+    return st
+
+
+def multi_workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size, num_query_tokens) -> int:
+    n = ctypes.c_size_t(0)
+    st = lib().pdattn_multi_workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size,
+                                           num_query_tokens, ctypes.byref(n))
+    if st != OK:
+        raise PdattnError(st, "pdattn_multi_workspace_size")
+    return n.value
+
+
+def alloc_multi_workspace(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size, num_query_tokens,
+                          device="cuda", stream=None):
+    n = multi_workspace_size(num_seqs, num_q_heads, num_kv_heads, head_dim, block_size, num_query_tokens)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    st = lib().pdattn_workspace_init(ws.data_ptr(), n, _stream_ptr(stream))
+    if st != OK:
+        raise PdattnError(st, "pdattn_workspace_init")
+    return ws
+
+
+def decode_multi(q, k_cache, v_cache, block_table, context_lens, scale, out, workspace, context_lens_host=None,
+                 stream=None, check: bool = True) -> int:
+    """pdattn_decode_multi: q and out are [num_seqs, T, num_q_heads, head_dim]; the last T tokens of every
+    sequence are new and each attends to the keys up to its own position."""
+    S, T, Hq, d = q.shape
+    NB, Hkv, bs, _ = k_cache.shape
+    a = Args()
+    a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr()
+    a.block_table, a.context_lens = block_table.data_ptr(), context_lens.data_ptr()
+    lens = None
+    if context_lens_host is not None:
+        lens = np.ascontiguousarray(context_lens_host, dtype=np.int32)
+        a.context_lens_host = lens.ctypes.data
+    a.num_seqs, a.num_q_heads, a.num_kv_heads, a.head_dim, a.block_size = S, Hq, Hkv, d, bs
+    a.max_blocks_per_seq = block_table.shape[1]
+    a.num_blocks = NB
+    a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
+    a.scale = float(scale)
+    a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    st = lib().pdattn_decode_multi(ctypes.byref(a), int(T), _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_multi")
     return st
 
 

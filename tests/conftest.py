@@ -28,7 +28,7 @@ def pytest_collection_modifyitems(config, items):
 
 # The GPU parity modules run once per merge mode of the decode kernel's consumer warps: the barrier
 # merge and the chained merge must each pass every case, whatever the library would pick by itself.
-MERGE_MODE_MODULES = ("test_gpu_parity", "test_gpu_grouped", "test_gpu_decode_loop")
+MERGE_MODE_MODULES = ("test_gpu_parity", "test_gpu_grouped", "test_gpu_decode_loop", "test_gpu_multi_token")
 MERGE_MODES = {"barrier": 0, "chain": 1}
 
 

@@ -277,3 +277,34 @@ def test_append_then_attend_equals_the_longer_cache():
     assert torch.equal(cut.k_cache.view(torch.int16), full.k_cache.view(torch.int16))
     assert torch.equal(cut.v_cache.view(torch.int16), full.v_cache.view(torch.int16))
     assert np.array_equal(orc.decode_workload(cut), ref_out)
+
+
+def test_multi_token_queries_match_a_dense_causal_softmax():
+    """Several new tokens per sequence: textbook masked softmax on the dense gather, the mask written as a
+    matrix (query token j of T sees key t iff t <= L - T + j), against the oracle's T truncated decode steps."""
+    rng = np.random.default_rng(5)
+    for seed, (Hq, Hkv, d, T) in enumerate([(4, 2, 32, 2), (6, 2, 64, 3), (4, 1, 128, 4), (8, 8, 16, 1)]):
+        lens = [T, T + 1, 16, 17, 63, 64, 65, 130, 2]
+        w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, seed=40 + seed, num_blocks=64)
+        S = len(lens)
+        G = Hq // Hkv
+        q = W.normal_bf16(S * T * Hq * d, 900 + seed, 1).view(S, T, Hq, d)
+        got = orc.decode_multi(q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale)
+        qf = f64(q)
+        for s in range(S):
+            K, V = dense_kv(w, s)
+            L = K.shape[0]
+            mask = np.array([[t <= L - T + j for t in range(L)] for j in range(T)])
+            for h in range(Hq):
+                x = (qf[s, :, h, :] @ K[:, h // G, :].T) * float(np.float32(w.scale))      # [T, L]
+                x = np.where(mask, x, -np.inf)
+                for j in range(T):
+                    if not mask[j].any():
+                        assert not got[s, j, h].any()            # a query token that sees no key: zeros
+                        continue
+                    p = np.exp(x[j] - x[j].max())
+                    p /= p.sum()
+                    np.testing.assert_allclose(got[s, j, h], p @ V[:, h // G, :], rtol=1e-12, atol=1e-14)
+        # the last query token is the plain decode step
+        last = orc.decode(q[:, T - 1].contiguous(), w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale)
+        assert np.array_equal(got[:, T - 1], last)
