@@ -393,8 +393,12 @@ def main():
         t_probe, cores = oracle_pass(wc, min(S, 8))
         n = int(max(1, min(S, 20.0 / max(t_probe / min(S, 8), 1e-9))))
         dt, cores = oracle_pass(wc, n)
-        cpu_baseline = {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                        "sample": f"one oracle pass over the first {n} of {S} sequences ({dt:.2f} s)"}
+        passes = 1
+        while dt < 12.0 and passes < 64:            # about 10-20 s of CPU work in all
+            dt += oracle_pass(wc, n)[0]
+            passes += 1
+        cpu_baseline = {"value": n * passes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"{passes} oracle passes over the first {n} of {S} sequences ({dt:.2f} s in all)"}
 
     if rank == 0:
         line = {
