@@ -111,7 +111,8 @@ pdattn_status pdattn_decode_ex(const pdattn_args* args, pdattn_stream_t stream);
  * (within rounding: the summation order differs) and are bit-identical from run to run.
  *   prefix_tiles      DEVICE int32 [num_seqs / group_size]; prefix_tiles_host its HOST copy.
  *   Requirements: args->context_lens_host given; num_seqs a multiple of group_size; G <= 8 and
- *   group_size * G <= 48; every member of group g has context_len > prefix_tiles[g] * 64
+ *   group_size * G <= 64 (48 with pdattn_set_prefix_engine(0)), else PDATTN_UNSUPPORTED;
+ *   every member of group g has context_len > prefix_tiles[g] * 64
  *   (it owns at least its current token); 0 is allowed (the group shares nothing).
  *   args->workspace must hold pdattn_grouped_workspace_size() bytes.
  * The caller vouches for the page ids being shared; if they are not, the group's first row is

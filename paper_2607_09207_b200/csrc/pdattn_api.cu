@@ -436,8 +436,10 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   int n_groups = 0;
   if (grouped) {
     const int Gs = g_grouped.group_size;
-    if (!a->context_lens_host || Gs <= 0 || a->num_seqs % Gs != 0 || G > 8 || Gs * G > MAX_PREFIX_ROWS)
-      return Gs > 0 && (G > 8 || Gs * G > MAX_PREFIX_ROWS) ? PDATTN_UNSUPPORTED : PDATTN_INVALID_ARG;
+    // rows the kernel for the shared tiles takes per unit: 64 on tensor memory, 48 with warp MMAs
+    const int max_rows = g_prefix_engine != 0 ? UMMA_MAX_QUERY_ROWS : MAX_PREFIX_ROWS;
+    if (!a->context_lens_host || Gs <= 0 || a->num_seqs % Gs != 0 || G > 8 || Gs * G > max_rows)
+      return Gs > 0 && (G > 8 || Gs * G > max_rows) ? PDATTN_UNSUPPORTED : PDATTN_INVALID_ARG;
     n_groups = a->num_seqs / Gs;
     g_start_tiles_host.resize(a->num_seqs);
     for (int sq = 0; sq < a->num_seqs; ++sq) {

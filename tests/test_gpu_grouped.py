@@ -140,6 +140,30 @@ def test_grouped_bad_page_ids_in_the_shared_tiles_are_masked_and_reported():
     assert_parity(out, ref, "grouped, bad pages in the shared tiles masked")
 
 
+@pytest.mark.parametrize("Hq,Hkv,group,d", [(28, 4, 8, 128), (32, 4, 8, 128), (16, 2, 8, 64)])
+def test_groups_of_56_and_64_query_rows(Hq, Hkv, group, d, prefix_engine):
+    """The 7B shape (28 q / 4 KV heads) in groups of 8 is 56 rows per unit, 32 / 4 is 64: every lane pair of
+    the tensor-memory kernel is in use.  The warp-MMA kernel takes at most 48 rows and says so."""
+    rng = np.random.default_rng(group + Hq)
+    lens = [512 + int(rng.integers(1, 300)) for _ in range(2 * group)]
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, seed=90 + Hq, device=DEV, poison=False)
+    bt = w.block_table.clone()
+    for j in range(2 * group):
+        bt[j, :32] = bt[j - j % group, :32]              # each group shares 32 pages = 8 tiles
+    w = dataclasses.replace(w, block_table=bt)
+    W.poison_unused(w)
+    if prefix_engine == "warp_mma":
+        ws = pdattn.alloc_grouped_workspace(w.num_seqs, Hq, Hkv, d)
+        pt = torch.tensor([8, 8], dtype=torch.int32, device=DEV)
+        st = pdattn.decode_grouped(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale,
+                                   torch.empty_like(w.q), ws, w.context_lens_host, group, pt, [8, 8], check=False)
+        assert st == pdattn.UNSUPPORTED
+        return
+    out, status = run_grouped(w, group, [8, 8])
+    assert status == pdattn.OK
+    assert_parity(out, orc.decode_workload(w.to("cpu")), f"Hq={Hq} Hkv={Hkv} group={group} d={d}")
+
+
 def test_grouped_rejects_what_it_cannot_do():
     w = W.make_config(3, device=DEV, num_seqs=16, len_div=4)
     ws = pdattn.alloc_grouped_workspace(16, 40, 8, 128)
@@ -148,7 +172,7 @@ def test_grouped_rejects_what_it_cannot_do():
     args = (w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws, w.context_lens_host)
     assert pdattn.decode_grouped(*args, 8, pt, [4, 4], check=False) == pdattn.OK
     assert pdattn.decode_grouped(*args, 5, pt, [4, 4], check=False) == pdattn.INVALID_ARG        # 16 % 5
-    assert pdattn.decode_grouped(*args, 16, pt, [4], check=False) == pdattn.UNSUPPORTED          # 16 * 5 rows > 48
+    assert pdattn.decode_grouped(*args, 16, pt, [4], check=False) == pdattn.UNSUPPORTED          # 16 * 5 rows > 64
     too_long = [int(w.context_lens_host[:8].min()) // 64 + 1, 4]
     assert pdattn.decode_grouped(*args, 8, pt, too_long, check=False) == pdattn.INVALID_ARG      # prefix >= a member
     small = pdattn.alloc_workspace(16, 40, 8, 128)
