@@ -35,7 +35,7 @@ extern "C" {
 typedef int pdattn_status;
 #define PDATTN_OK                   0
 #define PDATTN_INVALID_ARG         (-1) /* null pointer, negative size, Hq % Hkv != 0, ...           */
-#define PDATTN_UNSUPPORTED         (-2) /* head_dim not in {64,128}, block_size not in {16,32}, G > 16, or a
+#define PDATTN_UNSUPPORTED         (-2) /* head_dim not in {64,128}, block_size not in {16,32,64}, G > 16, or a
                                            cache stride that is not a multiple of 8 elements          */
 #define PDATTN_WORKSPACE_TOO_SMALL (-3)
 #define PDATTN_MISALIGNED          (-4) /* q / k_cache / v_cache / out / workspace not 16-byte aligned */

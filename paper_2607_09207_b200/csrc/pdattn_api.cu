@@ -73,7 +73,7 @@ pdattn_status check_shape(int num_seqs, int Hq, int Hkv, int d, int bs) {
   if (num_seqs < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || bs <= 0) return PDATTN_INVALID_ARG;
   if (Hq % Hkv != 0) return PDATTN_INVALID_ARG;
   if (d != 64 && d != 128) return PDATTN_UNSUPPORTED;
-  if (bs != 16 && bs != 32) return PDATTN_UNSUPPORTED;
+  if (bs != 16 && bs != 32 && bs != 64) return PDATTN_UNSUPPORTED;
   if (Hq / Hkv > 16) return PDATTN_UNSUPPORTED;
   return PDATTN_OK;
 }
@@ -82,11 +82,11 @@ pdattn_status check_shape(int num_seqs, int Hq, int Hkv, int d, int bs) {
 struct DevInfo {
   bool ready = false;
   int sm_count = 0;
-  bool attr_set[2][2][2] = {};      // [D==128][NT==2][BS==32]
-  bool probe_attr_set[2][2][2] = {};
-  bool chain_attr_set[2][2][2] = {};
-  bool prefix_attr_set[2][2] = {};  // [D==128][BS==32]
-  bool prefix_umma_attr_set[2][2] = {};
+  bool attr_set[2][2][3] = {};      // [D==128][NT==2][page size / 32]
+  bool probe_attr_set[2][2][3] = {};
+  bool chain_attr_set[2][2][3] = {};
+  bool prefix_attr_set[2][3] = {};  // [D==128][page size / 32]
+  bool prefix_umma_attr_set[2][3] = {};
 };
 constexpr int kMaxDevices = 64;
 DevInfo g_dev[kMaxDevices];
@@ -215,7 +215,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
                      int n_spans_host, DevInfo* di, cudaStream_t stream) {
   using C = Cfg<D, NT, BS>;
   auto kern = decode_kernel<D, NT, BS>;
-  bool& done = di->attr_set[D == 128][NT == 2][BS == 32];
+  bool& done = di->attr_set[D == 128][NT == 2][BS / 32];
   if (!done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
@@ -235,7 +235,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
   if (g_use_chain) {
     auto chain = decode_kernel<D, NT, BS, false, true>;
-    bool& cdone = di->chain_attr_set[D == 128][NT == 2][BS == 32];
+    bool& cdone = di->chain_attr_set[D == 128][NT == 2][BS / 32];
     if (!cdone) {
       cudaError_t ce = cudaFuncSetAttribute(chain, cudaFuncAttributeMaxDynamicSharedMemorySize, C::CHAIN_DYN_BYTES);
       if (ce != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", ce);
@@ -273,7 +273,7 @@ pdattn_status launch_prefix_bs(const CUtensorMap& mk, const CUtensorMap& mv, con
   using C = Cfg<D, 1, BS>;
   const int smem = 1024 + C::NSTAGES * C::STAGE_BYTES + C::CTRL_BYTES;
   auto kern = prefix_kernel<D, BS>;
-  bool& done = di->prefix_attr_set[D == 128][BS == 32];
+  bool& done = di->prefix_attr_set[D == 128][BS / 32];
   if (!done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
@@ -291,7 +291,7 @@ pdattn_status launch_prefix_umma_bs(const CUtensorMap& mk, const CUtensorMap& mv
                                     cudaStream_t stream) {
   using C = UmmaCfg<D, BS>;
   auto kern = prefix_umma_kernel<D, BS>;
-  bool& done = di->prefix_umma_attr_set[D == 128][BS == 32];
+  bool& done = di->prefix_umma_attr_set[D == 128][BS / 32];
   if (!done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
@@ -309,20 +309,23 @@ thread_local int g_block_size = 16;   // page size of the call being launched (s
 template <int D, int NT>
 pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
                      int n_spans_host, DevInfo* di, cudaStream_t stream) {
-  return g_block_size == 32 ? launch_bs<D, NT, 32>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
-                            : launch_bs<D, NT, 16>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+  return g_block_size == 64   ? launch_bs<D, NT, 64>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
+         : g_block_size == 32 ? launch_bs<D, NT, 32>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
+                              : launch_bs<D, NT, 16>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
 }
 template <int D>
 pdattn_status launch_prefix_umma(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
                                  cudaStream_t stream) {
-  return g_block_size == 32 ? launch_prefix_umma_bs<D, 32>(mk, mv, X, grid, di, stream)
-                            : launch_prefix_umma_bs<D, 16>(mk, mv, X, grid, di, stream);
+  return g_block_size == 64   ? launch_prefix_umma_bs<D, 64>(mk, mv, X, grid, di, stream)
+         : g_block_size == 32 ? launch_prefix_umma_bs<D, 32>(mk, mv, X, grid, di, stream)
+                              : launch_prefix_umma_bs<D, 16>(mk, mv, X, grid, di, stream);
 }
 template <int D>
 pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
                             cudaStream_t stream) {
-  return g_block_size == 32 ? launch_prefix_bs<D, 32>(mk, mv, X, grid, di, stream)
-                            : launch_prefix_bs<D, 16>(mk, mv, X, grid, di, stream);
+  return g_block_size == 64   ? launch_prefix_bs<D, 64>(mk, mv, X, grid, di, stream)
+         : g_block_size == 32 ? launch_prefix_bs<D, 32>(mk, mv, X, grid, di, stream)
+                              : launch_prefix_bs<D, 16>(mk, mv, X, grid, di, stream);
 }
 
 }  // namespace
@@ -355,7 +358,7 @@ pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cac
   if (num_seqs < 0 || num_kv_heads <= 0 || num_kv_heads > 16 || max_blocks_per_seq <= 0 || num_blocks <= 0)
     return PDATTN_INVALID_ARG;
   if (head_dim != 64 && head_dim != 128) return PDATTN_UNSUPPORTED;
-  if (block_size != 16 && block_size != 32) return PDATTN_UNSUPPORTED;
+  if (block_size != 16 && block_size != 32 && block_size != 64) return PDATTN_UNSUPPORTED;
   if (num_seqs == 0) return PDATTN_OK;
   if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !context_lens) return PDATTN_INVALID_ARG;
   if (kv_block_stride <= 0 || kv_head_stride <= 0 || kv_token_stride < head_dim) return PDATTN_INVALID_ARG;

@@ -61,7 +61,7 @@ def test_workspace_size_and_shape_checks():
     n = pdattn.workspace_size(256, 28, 4, 128)
     assert 0 < n < 64 << 20 and n % 256 == 0
     assert pdattn.workspace_size(256, 64, 4, 128) > n          # G = 16 needs wider partial slots
-    for bad, code in [((4, 28, 4, 96, 16), pdattn.UNSUPPORTED), ((4, 28, 4, 128, 8), pdattn.UNSUPPORTED), ((4, 28, 4, 128, 64), pdattn.UNSUPPORTED),
+    for bad, code in [((4, 28, 4, 96, 16), pdattn.UNSUPPORTED), ((4, 28, 4, 128, 8), pdattn.UNSUPPORTED), ((4, 28, 4, 128, 48), pdattn.UNSUPPORTED), ((4, 28, 4, 128, 128), pdattn.UNSUPPORTED),
                       ((4, 30, 4, 128, 16), pdattn.INVALID_ARG), ((4, 68, 4, 128, 16), pdattn.UNSUPPORTED),
                       ((-1, 28, 4, 128, 16), pdattn.INVALID_ARG)]:
         with pytest.raises(pdattn.PdattnError) as e:

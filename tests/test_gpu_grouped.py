@@ -74,19 +74,21 @@ def test_groups_with_uneven_prefixes_and_head_counts(Hq, Hkv, group):
     assert_parity(out, orc.decode_workload(w.to("cpu")), f"Hq={Hq} Hkv={Hkv} group={group}")
 
 
-def test_grouped_with_page_size_32():
+@pytest.mark.parametrize("bs", [32, 64])
+def test_grouped_with_larger_pages(bs):
     lens = [200, 70, 65, 1000, 129, 500, 66, 300]
-    w = W.make_custom(lens, Hq=16, Hkv=4, d=128, bs=32, seed=61, device=DEV, poison=False)
+    w = W.make_custom(lens, Hq=16, Hkv=4, d=128, bs=bs, seed=61, device=DEV, poison=False)
     bt = w.block_table.clone()
+    n = 64 // bs
     for j in range(1, 4):
-        bt[j, :2] = bt[0, :2]                       # group 0 shares one 64-token tile (two 32-token pages)
+        bt[j, :n] = bt[0, :n]                       # group 0 shares one 64-token tile (two 32-token pages or one page)
     for j in range(5, 8):
-        bt[j, :2] = bt[4, :2]
+        bt[j, :n] = bt[4, :n]
     w = dataclasses.replace(w, block_table=bt)
     W.poison_unused(w)
     out, status = run_grouped(w, 4, [1, 1])
     assert status == pdattn.OK
-    assert_parity(out, orc.decode_workload(w.to("cpu")), "grouped, page size 32")
+    assert_parity(out, orc.decode_workload(w.to("cpu")), f"grouped, page size {bs}")
 
 
 def test_full_size_grpo_config_sampled():

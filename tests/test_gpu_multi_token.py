@@ -45,7 +45,7 @@ def reference(w, q):
 
 @pytest.mark.parametrize("host_lens", [True, False])
 @pytest.mark.parametrize("Hq,Hkv,d,bs,T", [(28, 4, 128, 16, 2), (8, 2, 128, 16, 4), (8, 2, 64, 16, 2),
-                                          (16, 4, 128, 32, 3), (3, 3, 128, 16, 16), (10, 2, 64, 32, 3)])
+                                          (16, 4, 128, 32, 3), (3, 3, 128, 16, 16), (10, 2, 64, 32, 3), (28, 4, 128, 64, 2)])
 def test_ragged_lengths_around_tile_and_page_edges(Hq, Hkv, d, bs, T, host_lens):
     """8-row and 16-row tiles, the new tokens straddling page and tile edges, sequences shorter than T
     (their first query tokens see nothing and give zeros), empty sequences."""

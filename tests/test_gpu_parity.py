@@ -438,13 +438,15 @@ def test_runtime_span_scheduling_is_correct_and_deterministic(runtime_spans, cfg
     assert st == pdattn.OK and torch.equal(out, dev_plan)
 
 
-def test_page_size_32_and_wide_gqa_groups():
-    """block_size 32 (two pages per tile) and G in 9..16 (two MMA column tiles per warp)."""
+def test_page_sizes_32_and_64_and_wide_gqa_groups():
+    """block_size 32 and 64 (two pages, one page per tile) and G in 9..16 (two MMA column tiles per warp)."""
     lens = [1, 31, 32, 33, 63, 64, 65, 100, 1000, 4097, 0, 129]
-    for (Hq, Hkv, d, bs) in [(28, 4, 128, 32), (4, 1, 64, 32), (24, 2, 128, 32), (32, 2, 128, 16), (10, 1, 64, 16)]:
+    for (Hq, Hkv, d, bs) in [(28, 4, 128, 32), (4, 1, 64, 32), (24, 2, 128, 32), (32, 2, 128, 16), (10, 1, 64, 16),
+                             (28, 4, 128, 64), (6, 2, 64, 64), (24, 2, 128, 64)]:
         w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, bs=bs, seed=200 + Hq + bs, device=DEV)
         for host in (True, False):
             check_against_oracle(w, f"bs={bs} Hq={Hq} Hkv={Hkv} d={d}", use_host_lens=host)
     w = W.make_config(2, device=DEV, num_seqs=32)
-    w32 = W.make_custom(w.context_lens_host, Hq=28, Hkv=4, d=128, bs=32, seed=77, device=DEV)
-    check_against_oracle(w32, "7B-shaped lengths, page size 32")
+    for bs in (32, 64):
+        wb = W.make_custom(w.context_lens_host, Hq=28, Hkv=4, d=128, bs=bs, seed=77, device=DEV)
+        check_against_oracle(wb, f"7B-shaped lengths, page size {bs}")
