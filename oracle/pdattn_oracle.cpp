@@ -226,4 +226,82 @@ int pdattn_oracle_merge(const double* m, const double* l, const double* acc, int
 uint16_t pdattn_oracle_bf16_rne(double x) { return double_to_bf16_rne(x); }
 double pdattn_oracle_bf16_to_double(uint16_t b) { return bf16_to_double(b); }
 
+// ---- fp8 KV cache (the per-token footprint b_kv of Appendix A.1.2 carries the cache dtype's byte size) ----
+// K and V are stored as e4m3 codes with one fp32 scale per KV head: real value = scale[g] * e4m3(code).
+// e4m3 (the finite-only 8-bit format): 1 sign bit, 4 exponent bits (bias 7), 3 mantissa bits; no infinities;
+// S.1111.111 is NaN; exponent field 0 holds the subnormals m/8 * 2^-6.
+// Layouts: k8 [num_blocks, num_kv_heads, block_size, head_dim], v8 [num_blocks, num_kv_heads, head_dim, block_size]
+// (V is kept transposed inside a page), both dense.
+double pdattn_oracle_e4m3_to_double(uint8_t b) {
+    const int sign = b >> 7, e = (b >> 3) & 15, m = b & 7;
+    if (e == 15 && m == 7) return std::numeric_limits<double>::quiet_NaN();
+    const double v = e == 0 ? std::ldexp(static_cast<double>(m), -9) : std::ldexp(static_cast<double>(8 + m), e - 10);
+    return sign ? -v : v;
+}
+
+int pdattn_oracle_decode_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, const float* k_scale,
+                             const float* v_scale, const int32_t* block_table, const int32_t* context_lens,
+                             int num_seqs, int num_q_heads, int num_kv_heads, int head_dim, int block_size,
+                             int max_blocks_per_seq, int num_blocks, float scale, double* out, int num_threads,
+                             int64_t* bad_pages) {
+    if (num_seqs < 0 || num_q_heads <= 0 || num_kv_heads <= 0 || head_dim <= 0 || block_size <= 0 ||
+        num_q_heads % num_kv_heads != 0 || max_blocks_per_seq < 0 || !out || !k_scale || !v_scale)
+        return -1;
+    const int G = num_q_heads / num_kv_heads, d = head_dim, bs = block_size;
+    for (int s = 0; s < num_seqs; ++s)
+        if ((static_cast<int64_t>(context_lens[s]) + bs - 1) / bs > max_blocks_per_seq) return -1;
+    const int64_t total = static_cast<int64_t>(num_seqs) * num_q_heads;
+    std::atomic<int64_t> next{0}, skipped{0};
+    auto worker = [&]() {
+        std::vector<double> x;
+        for (;;) {
+            const int64_t i = next.fetch_add(1);
+            if (i >= total) break;
+            const int s = static_cast<int>(i / num_q_heads), h = static_cast<int>(i % num_q_heads), g = h / G;
+            const int L = context_lens[s];
+            double* o = out + i * d;
+            for (int j = 0; j < d; ++j) o[j] = 0.0;
+            if (L <= 0) continue;
+            const uint16_t* qrow = q + i * d;
+            x.assign(static_cast<size_t>(L), 0.0);
+            double xmax = -std::numeric_limits<double>::infinity();
+            for (int t = 0; t < L; ++t) {
+                const int32_t page = block_table[static_cast<int64_t>(s) * max_blocks_per_seq + t / bs];
+                if (page < 0 || page >= num_blocks) {     // not dereferenced, left out of the softmax, counted
+                    x[t] = std::numeric_limits<double>::quiet_NaN();
+                    ++skipped;
+                    continue;
+                }
+                const uint8_t* krow = k8 + ((static_cast<int64_t>(page) * num_kv_heads + g) * bs + t % bs) * d;
+                double acc = 0.0;
+                for (int j = 0; j < d; ++j)
+                    acc += bf16_to_double(qrow[j]) * (static_cast<double>(k_scale[g]) * pdattn_oracle_e4m3_to_double(krow[j]));
+                x[t] = static_cast<double>(scale) * acc;
+                if (x[t] > xmax) xmax = x[t];
+            }
+            double Z = 0.0;
+            for (int t = 0; t < L; ++t) {
+                if (std::isnan(x[t])) continue;
+                const double w = std::exp(x[t] - xmax);
+                Z += w;
+                const int32_t page = block_table[static_cast<int64_t>(s) * max_blocks_per_seq + t / bs];
+                const uint8_t* vblk = v8 + (static_cast<int64_t>(page) * num_kv_heads + g) * d * bs;
+                for (int j = 0; j < d; ++j)
+                    o[j] += w * (static_cast<double>(v_scale[g]) * pdattn_oracle_e4m3_to_double(vblk[j * bs + t % bs]));
+            }
+            for (int j = 0; j < d; ++j) o[j] = Z > 0.0 ? o[j] / Z : 0.0;
+        }
+    };
+    const int nt = num_threads > 0 ? num_threads : 1;
+    if (nt == 1) {
+        worker();
+    } else {
+        std::vector<std::thread> pool;
+        for (int i = 0; i < nt; ++i) pool.emplace_back(worker);
+        for (auto& th : pool) th.join();
+    }
+    if (bad_pages) *bad_pages = skipped.load();
+    return 0;
+}
+
 }  // extern "C"

@@ -119,6 +119,41 @@ def decode_multi(q, k_cache, v_cache, block_table, context_lens, scale, num_thre
     return out
 
 
+def e4m3_to_double(codes) -> np.ndarray:
+    """The value of each 8-bit e4m3 code (NaN for S.1111.111)."""
+    f = lib().pdattn_oracle_e4m3_to_double
+    f.restype = ctypes.c_double
+    f.argtypes = [ctypes.c_uint8]
+    return np.array([f(int(c)) for c in np.asarray(codes, dtype=np.uint8).ravel()], dtype=np.float64)
+
+
+def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, num_threads=None, return_bad=False):
+    """fp64 attention over an fp8 (e4m3 codes) KV cache with one scale per KV head: k8 uint8
+    [pages, Hkv, block_size, d], v8 uint8 [pages, Hkv, d, block_size] (V transposed inside a page)."""
+    q = _cpu(q).contiguous()
+    k8 = _cpu(k8).contiguous()
+    v8 = _cpu(v8).contiguous()
+    bt = _cpu(block_table).to(torch.int32).contiguous()
+    lens = _cpu(context_lens).to(torch.int32).contiguous()
+    ks = _cpu(k_scale).to(torch.float32).contiguous()
+    vs = _cpu(v_scale).to(torch.float32).contiguous()
+    S, Hq, d = q.shape
+    NB, Hkv, bs, dk = k8.shape
+    assert dk == d and tuple(v8.shape) == (NB, Hkv, d, bs) and k8.dtype == torch.uint8 and v8.dtype == torch.uint8
+    out = np.empty((S, Hq, d), dtype=np.float64)
+    bad = ctypes.c_int64(0)
+    f = lib().pdattn_oracle_decode_fp8
+    f.restype = ctypes.c_int
+    f.argtypes = [ctypes.c_void_p] * 7 + [ctypes.c_int] * 7 + [ctypes.c_float, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+    nt = int(num_threads) if num_threads else host_cores()
+    rc = f(q.data_ptr(), k8.data_ptr(), v8.data_ptr(), ks.data_ptr(), vs.data_ptr(), bt.data_ptr(), lens.data_ptr(),
+           S, Hq, Hkv, d, bs, bt.shape[1] if bt.dim() == 2 else 0, NB, float(scale), out.ctypes.data, nt,
+           ctypes.addressof(bad))
+    if rc != 0:
+        raise ValueError("pdattn_oracle_decode_fp8: invalid arguments")
+    return (out, bad.value) if return_bad else out
+
+
 def decode_workload(w, **kw):
     return decode(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, **kw)
 

@@ -318,6 +318,24 @@ def make_custom(lens, Hq, Hkv, d, bs=16, seed=1234, device="cpu", **kw) -> Workl
     return _build("custom", seed, lens, Hq, Hkv, d, bs, device, **kw)
 
 
+def fp8_caches(w: "Workload", k_scale: torch.Tensor, v_scale: torch.Tensor):
+    """The workload's K/V pools as an fp8 cache: e4m3 codes (uint8) of value / scale[kv head], K as
+    [pages, Hkv, block_size, d], V transposed inside a page as [pages, Hkv, d, block_size].  NaN poison stays
+    NaN (code 0x7f).  Input preparation only: the conversion is torch's own cast."""
+    ks = k_scale.to(w.k_cache.device, torch.float32).view(1, -1, 1, 1)
+    vs = v_scale.to(w.v_cache.device, torch.float32).view(1, -1, 1, 1)
+    k8 = (w.k_cache.float() / ks).to(torch.float8_e4m3fn).view(torch.uint8).contiguous()
+    v8 = (w.v_cache.float() / vs).to(torch.float8_e4m3fn).view(torch.uint8).permute(0, 1, 3, 2).contiguous()
+    return k8, v8
+
+
+def fp8_dequantized(k8: torch.Tensor, v8: torch.Tensor):
+    """bf16 pools (ordinary layout) holding exactly the values of the e4m3 codes (scale 1)."""
+    k = k8.view(torch.float8_e4m3fn).to(torch.bfloat16)
+    v = v8.view(torch.float8_e4m3fn).to(torch.bfloat16).permute(0, 1, 3, 2).contiguous()
+    return k, v
+
+
 def balanced_shards(lens, world_size: int):
     """Split sequences over ranks, balancing the summed context length (the bytes each
     rank must read): longest-first greedy.  Returns a list of index arrays, one per rank.

@@ -308,3 +308,36 @@ def test_multi_token_queries_match_a_dense_causal_softmax():
         # the last query token is the plain decode step
         last = orc.decode(q[:, T - 1].contiguous(), w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale)
         assert np.array_equal(got[:, T - 1], last)
+
+
+def test_e4m3_table_matches_the_library_cast():
+    vals = orc.e4m3_to_double(np.arange(256))
+    ref = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(np.isnan(vals), np.isnan(ref)) and np.isnan(vals).sum() == 2
+    assert np.array_equal(vals[~np.isnan(vals)], ref[~np.isnan(ref)])
+    assert vals[0x38] == 1.0 and vals[0x7E] == 448.0 and vals[0x01] == 2.0 ** -9 and vals[0xB8] == -1.0
+
+
+def test_fp8_cache_oracle_against_the_bf16_oracle_on_the_same_values():
+    """e4m3 values are exact in bf16: with unit scales the fp8 oracle must reproduce the bf16 oracle bit for
+    bit on pools that hold the decoded values (V transposed back); scales enter as a factor on the scores
+    (K) and on the output (V)."""
+    lens = [1, 2, 15, 16, 17, 50, 0, 129]
+    for seed, (Hq, Hkv, d, bs) in enumerate([(4, 1, 64, 16), (6, 2, 128, 16), (8, 8, 32, 32)]):
+        w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, bs=bs, seed=60 + seed, num_blocks=64)
+        one = torch.ones(Hkv)
+        k8, v8 = W.fp8_caches(w, one, one)
+        kd, vd = W.fp8_dequantized(k8, v8)
+        ref = orc.decode(w.q, kd, vd, w.block_table, w.context_lens, w.scale)
+        got = orc.decode_fp8(w.q, k8, v8, one, one, w.block_table, w.context_lens, w.scale)
+        assert np.array_equal(got, ref)
+        # power-of-two scales stay exact: K scale acts like the softmax scale, V scale like a factor on the output
+        got2 = orc.decode_fp8(w.q, k8, v8, 0.5 * one, 4.0 * one, w.block_table, w.context_lens, w.scale)
+        ref2 = 4.0 * orc.decode(w.q, kd, vd, w.block_table, w.context_lens, float(np.float32(w.scale)) * 0.5)
+        np.testing.assert_allclose(got2, ref2, rtol=1e-12, atol=1e-14)
+    # per-head scales address the right KV head
+    w = W.make_custom([40, 70], Hq=4, Hkv=2, d=32, seed=70, num_blocks=16)
+    k8, v8 = W.fp8_caches(w, torch.ones(2), torch.ones(2))
+    base = orc.decode_fp8(w.q, k8, v8, torch.ones(2), torch.ones(2), w.block_table, w.context_lens, w.scale)
+    scaled = orc.decode_fp8(w.q, k8, v8, torch.ones(2), torch.tensor([1.0, 3.0]), w.block_table, w.context_lens, w.scale)
+    assert np.array_equal(scaled[:, :2], base[:, :2]) and np.allclose(scaled[:, 2:], 3.0 * base[:, 2:], rtol=1e-15)
