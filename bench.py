@@ -371,6 +371,16 @@ def main():
             assert pdattn.check(mws) == pdattn.OK
             extras["two_query_tokens_ms_per_step"] = t_multi
             del q2, o2, mws
+            # the same batch over an fp8 (e4m3, per-head scales) cache: half the bytes per history token
+            ks8 = torch.full((c.num_kv_heads,), 1.25, dtype=torch.float32, device=dev)
+            vs8 = torch.full((c.num_kv_heads,), 0.75, dtype=torch.float32, device=dev)
+            k8, v8 = W.fp8_caches(c, ks8, vs8)
+            t_fp8 = timed(lambda: pdattn.decode_fp8(c.q, k8, v8, ks8, vs8, c.block_table, c.context_lens, c.scale,
+                                                    outs[0], ws, context_lens_host=c.context_lens_host))
+            assert pdattn.check(ws) == pdattn.OK
+            extras["fp8_kv_cache"] = {"ms_per_step": t_fp8, "seq_steps_per_s": S / (t_fp8 * 1e-3),
+                                      "kv_bytes_per_step": uniq // 2, "kv_gbs": uniq / 2 / (t_fp8 * 1e-3) / 1e9}
+            del k8, v8
         if args.cfg == 3 and args.num_seqs is None:
             # GRPO groups of 8 share their 1024-token prompt pages: read them once per group
             gws = pdattn.alloc_grouped_workspace(S, c.num_q_heads, c.num_kv_heads, c.head_dim, device=dev)

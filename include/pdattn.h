@@ -143,6 +143,24 @@ pdattn_status pdattn_multi_workspace_size(int num_seqs, int num_q_heads, int num
 pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens, pdattn_stream_t stream);
 
 /*
+ * Decode step over an fp8 KV cache.  Appendix A.1.2 gives the per-token KV footprint as
+ * b_kv = 2 L H_kv d_head b_dtype / tp and the decode cost as beta_hist per history token read: with
+ * one-byte cache elements both halve.  K and V are stored as e4m3 codes (1 sign, 4 exponent, 3 mantissa
+ * bits, finite-only variant) with one fp32 scale per KV head: value = scale[kv head] * e4m3(code).
+ *   args->k_cache   DEVICE uint8 [num_blocks, num_kv_heads, block_size, head_dim]
+ *   args->v_cache   DEVICE uint8 [num_blocks, num_kv_heads, head_dim, block_size]   (V transposed inside a page)
+ *   k_scale, v_scale  DEVICE fp32 [num_kv_heads]
+ * Both pools dense (the stride fields of args are ignored); everything else as in pdattn_decode_ex,
+ * including the treatment of bad page ids and of slots past the end (any code, NaN codes too).
+ * The codes are widened exactly; q is rounded to fp16 for the products (values below 2^-14 lose bits) and
+ * the softmax weights to fp16 (11 bits), accumulation in fp32; out is bf16.
+ *   Requirements: head_dim 128, block_size 16 (else PDATTN_UNSUPPORTED); not combined with
+ *   pdattn_decode_grouped / pdattn_decode_multi.  Workspace as for pdattn_decode_ex.
+ */
+pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, const float* v_scale,
+                                pdattn_stream_t stream);
+
+/*
  * KV append: the step that precedes attention in the decoding loop (Section 2.3; the cache grows by
  * b_kv bytes per token and layer, Appendix A.1.2).  For every sequence s with t = context_lens[s]:
  * the rows k_new[s], v_new[s] (DEVICE bf16 [num_seqs, num_kv_heads, head_dim], dense) are written to

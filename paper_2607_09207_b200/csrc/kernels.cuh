@@ -66,6 +66,8 @@ struct DecodeParams {
   float* partials;          // [span][2][HP*(D+2)] fp32
   int S, Hq, Hkv, G, MB, NB;
   int T;                    // query tokens per sequence (1 = plain decode); T * G rows share a KV head's tiles
+  const float* k_scale;     // fp8 cache only: per KV head, value = scale * e4m3 code
+  const float* v_scale;
   float scale_log2;         // scale * log2(e)
   PlanParams plan;          // host plan (ignored when use_ws_plan)
   int use_ws_plan;
@@ -180,6 +182,24 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// two e4m3 codes (low 16 bits of v) to two fp16 values: exact
+__device__ __forceinline__ uint32_t cvt_e4m3x2_f16x2(uint32_t v) {
+  uint32_t r;
+  const unsigned short h = static_cast<unsigned short>(v);
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(h));
+  return r;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   uint32_t y;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
@@ -202,13 +222,13 @@ __device__ __forceinline__ void bar_consumers() {   // named barrier 1: the NCT 
 // ------------------------------------------------------------------------------------------
 // Shared-memory plan
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS>
+template <int D, int NT, int BS, int EB = 2>   // EB: bytes per cache element (2 = bf16, 1 = fp8 codes)
 struct Cfg {
   static constexpr int PAGES = TILE / BS;              // pages per tile
-  static constexpr int HALVES = D / 64;                // 128-byte column blocks per row
+  static constexpr int HALVES = D * EB / 128;          // 128-byte column blocks per row
   static constexpr int HALF_BYTES = BS * 128;          // one TMA box: BS rows x 128 bytes
-  static constexpr int PAGE_BYTES = BS * D * 2;
-  static constexpr int KV_BYTES = TILE * D * 2;
+  static constexpr int PAGE_BYTES = BS * D * EB;
+  static constexpr int KV_BYTES = TILE * D * EB;
   static constexpr int STAGE_BYTES = 2 * KV_BYTES;     // K tile then V tile
   static constexpr int HP = 8 * NT;                    // padded query heads per KV head
   static constexpr int KSTEPS = D / 16;
@@ -476,6 +496,174 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
 }
 
 // ------------------------------------------------------------------------------------------
+// One 64-token tile on one warp, fp8 cache (e4m3 codes; head_dim 128, 16-token pages).
+// K tile: [64 tokens][128 B] (one code per element, 128-byte swizzle); V tile: per page [128 d][16 tokens]
+// (V is stored transposed inside a page).  The codes are widened to fp16 in registers (exact) and both
+// products run as fp16 MMAs; Q arrives as fp16 fragments and P is rounded to fp16 (11 bits, one term).
+// ldmatrix moves 16-bit units, i.e. PAIRS of codes, so a lane receives four consecutive elements of
+// the contraction dimension where the MMA fragment wants two plus two eight further on.  Both
+// products therefore run with the contraction index permuted inside every block of 16:
+//     k = 2t + i  <->  element 4t + i,     k = 2t + 8 + i  <->  element 4t + 2 + i      (t < 4, i < 2)
+// For S^T = K.Q^T the index is the head dimension and the Q fragments are loaded in the same order.
+// For O^T = V^T.P^T it is the token: P's rows must come in that order, which they do when row rho of
+// the score MMA holds token pi(rho) of its 16-token group -- a matter of the row addresses handed to
+// ldmatrix for K.
+// ------------------------------------------------------------------------------------------
+template <int NT, bool TAIL>
+__device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const uint32_t (&qf)[NT][8][2],
+                                                float (&acc)[NT][8][4], float (&m)[NT][2], float (&l)[NT][2],
+                                                float sl2, int n_left, uint32_t badmask, int lane,
+                                                const int (&lag)[NT][2]) {
+  constexpr int GROUPS = TILE / 16;
+  const float NEG_INF = __int_as_float(0xff800000);
+  const int n_valid = n_left < TILE ? n_left : TILE;
+  const int l8 = lane & 7;
+  const int mi = lane >> 3;
+  // K: matrices (rows 0-7, chunk c), (rows 8-15, c), (rows 0-7, c+1), (rows 8-15, c+1); row rho <-> token pi(rho)
+  const int rho = l8 + 8 * (mi & 1);
+  const int k_tok = ((rho & 7) >> 1) * 4 + (rho & 1) + (rho >> 3) * 2;
+  const int k_csel = mi >> 1;
+  // V^T: matrices (d rows 0-7 of block jm), (8-15 of jm), (0-7 of jm+1), (8-15 of jm+1)
+  const int v_drow = (mi >> 1) * 16 + (mi & 1) * 8 + l8;
+
+  float sc[GROUPS][NT][4];
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) sc[j][nt][0] = sc[j][nt][1] = sc[j][nt][2] = sc[j][nt][3] = 0.f;
+    if (!TAIL || j * 16 < n_valid) {
+      const int tok = j * 16 + k_tok;
+      const uint32_t base = sK + tok * 128;
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const int ch = (cc * 2 + k_csel) ^ (tok & 7);
+        uint32_t r[4];
+        ldsm_x4(r, base + (ch << 4));
+        {
+          const uint32_t a[4] = {cvt_e4m3x2_f16x2(r[0]), cvt_e4m3x2_f16x2(r[1]), cvt_e4m3x2_f16x2(r[0] >> 16),
+                                 cvt_e4m3x2_f16x2(r[1] >> 16)};
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) mma_f16(sc[j][nt], a, qf[nt][cc * 2][0], qf[nt][cc * 2][1]);
+        }
+        {
+          const uint32_t a[4] = {cvt_e4m3x2_f16x2(r[2]), cvt_e4m3x2_f16x2(r[3]), cvt_e4m3x2_f16x2(r[2] >> 16),
+                                 cvt_e4m3x2_f16x2(r[3] >> 16)};
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) mma_f16(sc[j][nt], a, qf[nt][cc * 2 + 1][0], qf[nt][cc * 2 + 1][1]);
+        }
+      }
+    }
+  }
+
+  // ---- scale, mask: score rows g and g + 8 of a group hold tokens pi(g) and pi(g) + 2
+  const int trow = lane >> 2;
+  const int tok0 = (trow >> 1) * 4 + (trow & 1);
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j) {
+    bool dead_page = false;
+    if (badmask) dead_page = (badmask >> j) & 1u;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        float v = sc[j][nt][r] * sl2;
+        if (TAIL) {
+          const int tok = j * 16 + tok0 + ((r & 2) ? 2 : 0);
+          if (tok >= n_left - lag[nt][r & 1]) v = NEG_INF;
+        }
+        if (dead_page) v = NEG_INF;
+        sc[j][nt][r] = v;
+      }
+  }
+
+  // ---- online softmax (as in compute_tile)
+  float alpha[NT][2], muse[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      float mx = NEG_INF;
+#pragma unroll
+      for (int j = 0; j < GROUPS; ++j) mx = fmaxf(mx, fmaxf(sc[j][nt][e], sc[j][nt][e + 2]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+      const float m_new = fmaxf(m[nt][e], mx);
+      const float mu = (m_new == NEG_INF) ? 0.f : m_new;
+      alpha[nt][e] = fast_exp2(m[nt][e] - mu);
+      muse[nt][e] = mu;
+      m[nt][e] = m_new;
+      l[nt][e] *= alpha[nt][e];
+    }
+  bool moved = false;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) moved |= (alpha[nt][0] != 1.f) | (alpha[nt][1] != 1.f);
+  if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int jm = 0; jm < 8; ++jm) {
+        acc[nt][jm][0] *= alpha[nt][0];
+        acc[nt][jm][1] *= alpha[nt][1];
+        acc[nt][jm][2] *= alpha[nt][0];
+        acc[nt][jm][3] *= alpha[nt][1];
+      }
+  }
+
+  // ---- P = exp2(S - m) as fp16, transposed into the B-operand layout
+  uint32_t pb[GROUPS][NT][2];
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float p0 = fast_exp2(sc[j][nt][0] - muse[nt][0]);
+      const float p1 = fast_exp2(sc[j][nt][1] - muse[nt][1]);
+      const float p2 = fast_exp2(sc[j][nt][2] - muse[nt][0]);
+      const float p3 = fast_exp2(sc[j][nt][3] - muse[nt][1]);
+      l[nt][0] += p0 + p2;
+      l[nt][1] += p1 + p3;
+      pb[j][nt][0] = movmatrix_trans(pack_f16x2(p0, p1));
+      pb[j][nt][1] = movmatrix_trans(pack_f16x2(p2, p3));
+    }
+
+  // ---- O^T += V^T . P^T : [128] x [8*NT heads], one page (16 tokens) per MMA step
+#pragma unroll
+  for (int j = 0; j < GROUPS; ++j) {
+    if (!TAIL || j * 16 < n_valid) {
+      // codes of tokens past the end may be anything (NaN codes too) while their P is 0: blank them
+      uint32_t keep_mask = 0xffffffffu;
+      if (TAIL) {
+        const int keep = n_valid - (j * 16 + (lane & 3) * 4);   // of this lane's four tokens
+        keep_mask = keep >= 4 ? 0xffffffffu : (keep <= 0 ? 0u : ((1u << (8 * keep)) - 1u));
+      }
+#pragma unroll
+      for (int jp = 0; jp < 4; ++jp) {
+        uint32_t r[4];
+        ldsm_x4(r, sV + j * 2048 + (jp * 32 + v_drow) * 16);
+        if (TAIL) {
+          r[0] &= keep_mask;
+          r[1] &= keep_mask;
+          r[2] &= keep_mask;
+          r[3] &= keep_mask;
+        }
+        {
+          const uint32_t a[4] = {cvt_e4m3x2_f16x2(r[0]), cvt_e4m3x2_f16x2(r[1]), cvt_e4m3x2_f16x2(r[0] >> 16),
+                                 cvt_e4m3x2_f16x2(r[1] >> 16)};
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) mma_f16(acc[nt][jp * 2], a, pb[j][nt][0], pb[j][nt][1]);
+        }
+        {
+          const uint32_t a[4] = {cvt_e4m3x2_f16x2(r[2]), cvt_e4m3x2_f16x2(r[3]), cvt_e4m3x2_f16x2(r[2] >> 16),
+                                 cvt_e4m3x2_f16x2(r[3] >> 16)};
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) mma_f16(acc[nt][jp * 2 + 1], a, pb[j][nt][0], pb[j][nt][1]);
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Span sequencing inside a CTA.  Every warp walks the same sequence of spans: first the CTA's
 // static span, then run-time spans.  Lane 0 of producer warp 0 draws run-time spans from the
 // global counter (one atomic per span, issued a whole span ahead of its use) and publishes the
@@ -555,10 +743,11 @@ __device__ __forceinline__ bool wait_turn(Ctrl* ctrl, int e, int want) {
 // which class of which of those pieces may touch it next.  Warps that hold no tile of a piece skip it
 // (they do not even read its query rows), so up to NCW short pieces are in work at once.
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS>
+template <int D, int NT, int BS, int EB>
 __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanParams& pp, Ctrl* ctrl, uint32_t ring,
                                               uint32_t qbuf, uint8_t* handoff, int warp, int lane) {
-  using C = Cfg<D, NT, BS>;
+  using C = Cfg<D, NT, BS, EB>;
+  static_assert(EB == 2 || (EB == 1 && D == 128 && BS == 16), "the fp8 cache path is built for head_dim 128, 16-token pages");
   constexpr int NST = C::NSTAGES;
   constexpr int NCW = C::NCW;
   constexpr int E = C::HANDOFFS;
@@ -636,16 +825,28 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         for (int nt = 0; nt < NT; ++nt) {
           const int head = nt * 8 + hq0;
           const bool live = head < R;
-          const uint32_t qa = qbuf + qs * C::Q_BYTES + (live ? head : 0) * (D * 2) + qcol * 2;
+          if constexpr (EB == 2) {
+            const uint32_t qa = qbuf + qs * C::Q_BYTES + (live ? head : 0) * (D * 2) + qcol * 2;
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            uint32_t v0 = 0u, v1 = 0u;
-            if (live) {
-              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v0) : "r"(qa + kk * 32) : "memory");
-              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v1) : "r"(qa + kk * 32 + 16) : "memory");
+            for (int kk = 0; kk < D / 16; ++kk) {
+              uint32_t v0 = 0u, v1 = 0u;
+              if (live) {
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v0) : "r"(qa + kk * 32) : "memory");
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v1) : "r"(qa + kk * 32 + 16) : "memory");
+              }
+              qf[nt][kk][0] = v0;
+              qf[nt][kk][1] = v1;
             }
-            qf[nt][kk][0] = v0;
-            qf[nt][kk][1] = v1;
+          } else {
+            // fp16 fragments in the permuted order of compute_tile_f8: four consecutive elements per lane
+            const uint32_t qa = qbuf + qs * C::Q_BYTES + (live ? head : 0) * (D * 2) + qcol * 4;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              uint32_t v0 = 0u, v1 = 0u;
+              if (live) asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v0), "=r"(v1) : "r"(qa + kk * 32) : "memory");
+              qf[nt][kk][0] = pack_f16x2(__uint_as_float(v0 << 16), __uint_as_float(v0 & 0xffff0000u));
+              qf[nt][kk][1] = pack_f16x2(__uint_as_float(v1 << 16), __uint_as_float(v1 & 0xffff0000u));
+            }
           }
         }
         __syncwarp();
@@ -663,6 +864,9 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         for (int jm = 0; jm < D / 16; ++jm) acc[nt][jm][0] = acc[nt][jm][1] = acc[nt][jm][2] = acc[nt][jm][3] = 0.f;
       }
 
+      // fp8 cache: the K scale of this KV head joins the softmax scale
+      const float sl2 = EB == 1 ? P.scale_log2 * __ldg(P.k_scale + pc.g) : P.scale_log2;
+      (void)sl2;
       // ---- this class's tiles
       for (int its = it0 + pos; its < it0 + n_piece; its += NCW) {
         const int slot = its % NST;
@@ -675,16 +879,37 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         const uint32_t sV = sK + C::KV_BYTES;
         const uint32_t badmask = ctrl->meta[slot];
         const int n_left = pc.L - (pc.t0 + t) * TILE;
-        if (n_left - (P.T - 1) >= TILE) {   // every query token sees the whole tile
-          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag);
+        if constexpr (EB == 2) {
+          if (n_left - (P.T - 1) >= TILE) {   // every query token sees the whole tile
+            compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag);
+          } else {
+            compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag);
+            fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
+          }
         } else {
-          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag);
-          fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
+          if (n_left - (P.T - 1) >= TILE) {
+            compute_tile_f8<NT, false>(sK, sV, qf, acc, m, l, sl2, TILE, badmask, lane, lag);
+          } else {
+            compute_tile_f8<NT, true>(sK, sV, qf, acc, m, l, sl2, n_left, badmask, lane, lag);
+          }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
       }
       if (aborted) continue;
+      if constexpr (EB == 1) {
+        // the V scale of this KV head, once per piece: the accumulator is linear in V
+        const float vs = __ldg(P.v_scale + pc.g);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int jm = 0; jm < D / 16; ++jm) {
+            acc[nt][jm][0] *= vs;
+            acc[nt][jm][1] *= vs;
+            acc[nt][jm][2] *= vs;
+            acc[nt][jm][3] *= vs;
+          }
+      }
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -828,11 +1053,12 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
 // CHAIN = true replaces the consumers' barrier-and-merge at the end of each piece by the chained
 // hand-off of consume_chain (the producers are the same).
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS, bool PROBE = false, bool CHAIN = false>
-__global__ void __launch_bounds__(Cfg<D, NT, BS>::NTHREADS, 1)
+template <int D, int NT, int BS, bool PROBE = false, bool CHAIN = false, int EB = 2>
+__global__ void __launch_bounds__(Cfg<D, NT, BS, EB>::NTHREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
               const __grid_constant__ DecodeParams P) {
-  using C = Cfg<D, NT, BS>;
+  using C = Cfg<D, NT, BS, EB>;
+  static_assert(EB == 2 || CHAIN, "the fp8 cache path uses the chained merge");
   constexpr int NST = C::NSTAGES;
   constexpr int NCW = C::NCW;
   constexpr int NCT = C::NCT;
@@ -1017,7 +1243,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const int qcol = (lane & 3) * 2;
 
   if constexpr (CHAIN) {
-    consume_chain<D, NT, BS>(P, pp, ctrl, ring, qbuf,
+    consume_chain<D, NT, BS, EB>(P, pp, ctrl, ring, qbuf,
                              smem + NST * C::STAGE_BYTES + C::QSLOTS * C::Q_BYTES + C::ML_BYTES + C::CTRL_BYTES, warp,
                              lane);
     return;

@@ -33,6 +33,12 @@ thread_local std::vector<int32_t> g_start_tiles_host;
 int g_dyn_per_cta = 0;                    // run-time spans per CTA (pdattn_set_dynamic_spans)
 int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (chained), 0 barrier, 1 chained
 thread_local bool g_use_chain = true;     // decided per call, read by the launcher
+struct Fp8Call {
+  bool active = false;
+  const float* k_scale = nullptr;
+  const float* v_scale = nullptr;
+};
+thread_local Fp8Call g_fp8;               // set by pdattn_decode_fp8 around the common path
 thread_local int g_query_tokens = 1;      // query tokens per sequence of the call (pdattn_decode_multi)
 int g_prefix_engine = -1;                 // pdattn_set_prefix_engine: -1 default (tcgen05), 0 warp MMAs, 1 tcgen05
 
@@ -85,6 +91,7 @@ struct DevInfo {
   bool attr_set[2][2][3] = {};      // [D==128][NT==2][page size / 32]
   bool probe_attr_set[2][2][3] = {};
   bool chain_attr_set[2][2][3] = {};
+  bool fp8_attr_set[2] = {};        // [NT==2]
   bool prefix_attr_set[2][3] = {};  // [D==128][page size / 32]
   bool prefix_umma_attr_set[2][3] = {};
 };
@@ -139,6 +146,8 @@ pdattn_status get_encode() {
   return PDATTN_OK;
 }
 
+constexpr int kMapK8 = 81, kMapV8 = 82;   // "ranks" of the two fp8 views in make_map
+
 struct MapKey {
   const void* ptr;
   int d, bs, hkv, nb, rank;
@@ -175,7 +184,28 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
   const cuuint64_t nbu = static_cast<cuuint64_t>(nb > 0 ? nb : 1);
   CUtensorMap m;
   CUresult r;
-  if (rank == 5) {
+  if (rank == kMapK8) {
+    // fp8 K pool [pages, kv heads, slots, d] of one-byte codes: one box = a page-head, [d, block_size, 1, 1]
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(hkv), nbu};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(bs) * d,
+                             static_cast<cuuint64_t>(hkv) * bs * d};
+    cuuint32_t box[4] = {static_cast<cuuint32_t>(d), static_cast<cuuint32_t>(bs), 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (rank == kMapV8) {
+    // fp8 V pool [pages, kv heads, d, slots] (transposed inside a page): one box = a page-head,
+    // [block_size, d, 1, 1], rows of block_size bytes, no swizzle
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(hkv), nbu};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(d) * bs,
+                             static_cast<cuuint64_t>(hkv) * d * bs};
+    cuuint32_t box[4] = {static_cast<cuuint32_t>(bs), static_cast<cuuint32_t>(d), 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (rank == 5) {
     cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(d / 64),
                           static_cast<cuuint64_t>(hkv), nbu};
     cuuint64_t strides[4] = {static_cast<cuuint64_t>(st) * 2, 128, static_cast<cuuint64_t>(sh) * 2,
@@ -233,7 +263,21 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
     return PDATTN_OK;
   }
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
-  if (g_use_chain) {
+  if (g_fp8.active) {
+    if constexpr (D == 128 && BS == 16) {
+      using C8 = Cfg<D, NT, BS, 1>;
+      auto k8 = decode_kernel<D, NT, BS, false, true, 1>;
+      bool& fdone = di->fp8_attr_set[NT == 2];
+      if (!fdone) {
+        cudaError_t fe = cudaFuncSetAttribute(k8, cudaFuncAttributeMaxDynamicSharedMemorySize, C8::CHAIN_DYN_BYTES);
+        if (fe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", fe);
+        fdone = true;
+      }
+      k8<<<grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream>>>(mk, mv, P);
+    } else {
+      return PDATTN_UNSUPPORTED;
+    }
+  } else if (g_use_chain) {
     auto chain = decode_kernel<D, NT, BS, false, true>;
     bool& cdone = di->chain_attr_set[D == 128][NT == 2][BS / 32];
     if (!cdone) {
@@ -428,6 +472,8 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   const bool grouped = g_grouped.active;
   if (T < 1) return PDATTN_INVALID_ARG;
   if (G * T > 16 || (T > 1 && grouped)) return PDATTN_UNSUPPORTED;
+  const bool fp8 = g_fp8.active;
+  if (fp8 && (a->head_dim != 128 || a->block_size != 16 || T != 1 || grouped || g_probe_mode)) return PDATTN_UNSUPPORTED;
   const WsLayout wl = ws_layout(a->num_seqs, G * T, a->head_dim);
   // grouped calls keep two more arrays behind the ordinary layout
   const size_t off_start = wl.total;
@@ -484,6 +530,8 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   P.scale_log2 = a->scale * 1.4426950408889634f;
   P.use_ws_plan = 0;
   P.box5d = 0;
+  P.k_scale = fp8 ? g_fp8.k_scale : nullptr;
+  P.v_scale = fp8 ? g_fp8.v_scale : nullptr;
 
   int n_ctas = di->sm_count;
   if (n_ctas > MAX_SPANS / (1 + kMaxDynPerCta)) n_ctas = MAX_SPANS / (1 + kMaxDynPerCta);
@@ -513,6 +561,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   static const bool force4d = getenv("PDATTN_BOX4D") != nullptr;
   CUtensorMap mk, mv;
   int rank = (a->head_dim == 128 && !force4d) ? 5 : 4;
+  if (fp8) rank = kMapK8;
   s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
                a->kv_head_stride, a->kv_token_stride, rank, &mk);
   if (s != PDATTN_OK && rank == 5) {
@@ -522,7 +571,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   }
   if (s != PDATTN_OK) return s;
   s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-               a->kv_head_stride, a->kv_token_stride, rank, &mv);
+               a->kv_head_stride, a->kv_token_stride, fp8 ? kMapV8 : rank, &mv);
   if (s != PDATTN_OK) return s;
   P.box5d = rank == 5;
   // run-time spans assume warps that stay within a ring of each other: barrier merge there
@@ -613,6 +662,22 @@ pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens,
   g_query_tokens = num_query_tokens;
   const pdattn_status s = pdattn_decode_ex(args, stream);
   g_query_tokens = 1;
+  return s;
+}
+
+pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, const float* v_scale,
+                                pdattn_stream_t stream) {
+  if (!args || !k_scale || !v_scale) return PDATTN_INVALID_ARG;
+  pdattn_args a = *args;
+  // dense pools of one-byte codes; the stride fields are not used by this variant
+  a.kv_token_stride = a.head_dim;
+  a.kv_head_stride = static_cast<int64_t>(a.block_size) * a.head_dim;
+  a.kv_block_stride = static_cast<int64_t>(a.num_kv_heads) * a.block_size * a.head_dim;
+  g_fp8.active = true;
+  g_fp8.k_scale = k_scale;
+  g_fp8.v_scale = v_scale;
+  const pdattn_status s = pdattn_decode_ex(&a, stream);
+  g_fp8 = Fp8Call{};
   return s;
 }
 

@@ -34,7 +34,7 @@ EXPORTS = [
     "pdattn_set_merge_mode", "pdattn_set_prefix_engine",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
-    "pdattn_multi_workspace_size", "pdattn_decode_multi",
+    "pdattn_multi_workspace_size", "pdattn_decode_multi", "pdattn_decode_fp8",
 ]
 
 
@@ -96,6 +96,7 @@ def lib():
         L.pdattn_decode_grouped.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
         L.pdattn_multi_workspace_size.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_multi.argtypes = [ctypes.POINTER(Args), i32, vp]
+        L.pdattn_decode_fp8.argtypes = [ctypes.POINTER(Args), vp, vp, vp]
         L.pdattn_append_kv.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp]
         L.pdattn_check.argtypes = [vp, vp]
         L.pdattn_profile_events.argtypes = [vp, vp]
@@ -274,6 +275,33 @@ def decode_multi(q, k_cache, v_cache, block_table, context_lens, scale, out, wor
     st = lib().pdattn_decode_multi(ctypes.byref(a), int(T), _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_decode_multi")
+    return st
+
+
+def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, out, workspace,
+               context_lens_host=None, stream=None, check: bool = True) -> int:
+    """pdattn_decode_fp8: k8 uint8 [pages, Hkv, block_size, d], v8 uint8 [pages, Hkv, d, block_size] (e4m3 codes),
+    k_scale / v_scale fp32 [Hkv] on the device."""
+    S, Hq, d = q.shape
+    NB, Hkv, bs, _ = k8.shape
+    assert k8.dtype == torch.uint8 and v8.dtype == torch.uint8 and tuple(v8.shape) == (NB, Hkv, d, bs)
+    assert k8.is_contiguous() and v8.is_contiguous() and k_scale.dtype == torch.float32 and v_scale.dtype == torch.float32
+    a = Args()
+    a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k8.data_ptr(), v8.data_ptr(), out.data_ptr()
+    a.block_table, a.context_lens = block_table.data_ptr(), context_lens.data_ptr()
+    lens = None
+    if context_lens_host is not None:
+        lens = np.ascontiguousarray(context_lens_host, dtype=np.int32)
+        a.context_lens_host = lens.ctypes.data
+    a.num_seqs, a.num_q_heads, a.num_kv_heads, a.head_dim, a.block_size = S, Hq, Hkv, d, bs
+    a.max_blocks_per_seq = block_table.shape[1]
+    a.num_blocks = NB
+    a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = Hkv * bs * d, bs * d, d
+    a.scale = float(scale)
+    a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    st = lib().pdattn_decode_fp8(ctypes.byref(a), k_scale.data_ptr(), v_scale.data_ptr(), _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_fp8")
     return st
 
 

@@ -1,0 +1,126 @@
+"""GPU parity of pdattn_decode_fp8 (e4m3 KV cache with per-head scales) against the fp64 oracle of the same
+cache.  Tolerance as everywhere: |gpu - ref| <= max(2e-3, 1e-2 * |ref|), nothing NaN/Inf.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import pdattn_oracle as orc
+from paper_2607_09207_b200 import pdattn
+from paper_2607_09207_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def scales(Hkv, seed):
+    rng = np.random.default_rng(seed)
+    ks = torch.tensor(rng.uniform(0.5, 2.0, size=Hkv), dtype=torch.float32, device=DEV)
+    vs = torch.tensor(rng.uniform(0.5, 2.0, size=Hkv), dtype=torch.float32, device=DEV)
+    return ks, vs
+
+
+def run_fp8(w, k8, v8, ks, vs, host_lens=True, ws=None):
+    if ws is None:
+        ws = pdattn.alloc_workspace(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size)
+    out = torch.full_like(w.q, float("nan"))
+    pdattn.decode_fp8(w.q, k8, v8, ks, vs, w.block_table, w.context_lens, w.scale, out, ws,
+                      context_lens_host=w.context_lens_host if host_lens else None)
+    return out, pdattn.check(ws)
+
+
+def assert_parity(out, ref, what):
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    err = np.abs(got - ref)
+    bad = err > np.maximum(2e-3, 1e-2 * np.abs(ref))
+    assert not bad.any(), (f"{what}: {int(bad.sum())} of {bad.size} elements out of tolerance; "
+                           f"max abs err {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}")
+
+
+def reference(w, k8, v8, ks, vs, **kw):
+    return orc.decode_fp8(w.q.cpu(), k8.cpu(), v8.cpu(), ks.cpu(), vs.cpu(), w.block_table.cpu(), w.context_lens.cpu(),
+                          w.scale, **kw)
+
+
+@pytest.mark.parametrize("host_lens", [True, False])
+@pytest.mark.parametrize("Hq,Hkv", [(28, 4), (8, 2), (64, 4), (5, 5), (12, 1)])
+def test_ragged_lengths_and_head_groupings(Hq, Hkv, host_lens):
+    """8- and 16-row tiles, contexts around page and tile edges, NaN codes in every unused slot."""
+    lens = [1, 2, 3, 4, 5, 15, 16, 17, 31, 33, 47, 49, 63, 64, 65, 127, 129, 191, 193, 255, 257, 1000, 0, 4097, 577]
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=128, seed=400 + Hq, device=DEV)       # unused slots poisoned
+    ks, vs = scales(Hkv, Hq)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    out, st = run_fp8(w, k8, v8, ks, vs, host_lens)
+    assert st == pdattn.OK
+    assert_parity(out, reference(w, k8, v8, ks, vs), f"fp8 Hq={Hq} Hkv={Hkv}")
+
+
+def test_scaled_rollout_config_and_run_to_run_bits():
+    w = W.make_config(2, device=DEV, num_seqs=24, len_div=2)
+    ks, vs = scales(4, 1)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    out, st = run_fp8(w, k8, v8, ks, vs)
+    assert st == pdattn.OK
+    assert_parity(out, reference(w, k8, v8, ks, vs), "fp8 config 2 scaled")
+    again, _ = run_fp8(w, k8, v8, ks, vs)
+    assert torch.equal(out, again)
+
+
+def test_single_long_sequence_and_peaked_scores():
+    w = W.make_custom([30000], Hq=7, Hkv=1, d=128, seed=41, device=DEV)
+    ks, vs = scales(1, 2)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    out, st = run_fp8(w, k8, v8, ks, vs)
+    assert st == pdattn.OK
+    assert_parity(out, reference(w, k8, v8, ks, vs), "fp8 one long sequence")
+    wp = dataclasses.replace(W.make_custom([700, 130, 64], Hq=8, Hkv=2, d=128, seed=42, device=DEV), scale=0.7)
+    ks, vs = scales(2, 3)
+    k8, v8 = W.fp8_caches(wp, ks, vs)
+    out, st = run_fp8(wp, k8, v8, ks, vs)
+    assert st == pdattn.OK
+    assert_parity(out, reference(wp, k8, v8, ks, vs), "fp8 peaked softmax")
+
+
+def test_context_len_one_returns_the_scaled_code_value():
+    w = W.make_custom([1, 1, 1], Hq=4, Hkv=2, d=128, seed=43, device=DEV)
+    ks = torch.ones(2, device=DEV)
+    vs = torch.tensor([1.0, 0.25], device=DEV)                 # exact factors
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    out, st = run_fp8(w, k8, v8, ks, vs)
+    assert st == pdattn.OK
+    ref = reference(w, k8, v8, ks, vs)
+    assert np.array_equal(out.float().cpu().numpy().astype(np.float64), ref)        # e4m3 values are exact in bf16
+
+
+def test_out_of_range_page_ids_are_masked_and_reported():
+    w = W.make_custom([200, 48], Hq=8, Hkv=2, d=128, seed=44, device=DEV, num_blocks=64, poison=False)
+    ks, vs = scales(2, 4)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    bt = w.block_table.clone()
+    bt[0, 3] = 64
+    bt[1, 1] = -5
+    wb = dataclasses.replace(w, block_table=bt)
+    out, st = run_fp8(wb, k8, v8, ks, vs)
+    assert st == pdattn.BAD_PAGE_INDEX
+    ref, bad = reference(wb, k8, v8, ks, vs, return_bad=True)
+    assert bad == 2 * 16 * 8
+    assert_parity(out, ref, "fp8 bad pages masked")
+
+
+def test_rejects_what_it_cannot_do():
+    w = W.make_custom([100], Hq=4, Hkv=2, d=64, seed=45, device=DEV)
+    ks, vs = scales(2, 5)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    ws = pdattn.alloc_workspace(1, 4, 2, 64)
+    out = torch.empty_like(w.q)
+    args = (w.block_table, w.context_lens, w.scale, out, ws)
+    assert pdattn.decode_fp8(w.q, k8, v8, ks, vs, *args, check=False) == pdattn.UNSUPPORTED       # head_dim 64
+    w32 = W.make_custom([100], Hq=4, Hkv=2, d=128, bs=32, seed=46, device=DEV)
+    k8, v8 = W.fp8_caches(w32, ks, vs)
+    ws = pdattn.alloc_workspace(1, 4, 2, 128, 32)
+    assert pdattn.decode_fp8(w32.q, k8, v8, ks, vs, w32.block_table, w32.context_lens, w32.scale,
+                             torch.empty_like(w32.q), ws, check=False) == pdattn.UNSUPPORTED        # 32-token pages
+    assert pdattn.lib().pdattn_decode_fp8(None, None, None, None) == pdattn.INVALID_ARG
