@@ -161,6 +161,19 @@ pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, c
                                 pdattn_stream_t stream);
 
 /*
+ * KV append into the fp8 cache of pdattn_decode_fp8 (same layouts): the rows k_new[s], v_new[s] (DEVICE
+ * bf16 [num_seqs, num_kv_heads, head_dim]) are divided by their KV head's scale, rounded to e4m3 (nearest
+ * even; magnitudes beyond the largest finite code 448 saturate to it) and written at position
+ * context_lens[s], which then becomes context_lens[s] + 1.  Page rules and error reporting as in
+ * pdattn_append_kv.  head_dim 128, block_size 16.
+ */
+pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                   const float* k_scale, const float* v_scale, const int32_t* block_table,
+                                   int32_t* context_lens, int num_seqs, int num_kv_heads, int head_dim,
+                                   int block_size, int max_blocks_per_seq, int num_blocks, void* workspace,
+                                   pdattn_stream_t stream);
+
+/*
  * KV append: the step that precedes attention in the decoding loop (Section 2.3; the cache grows by
  * b_kv bytes per token and layer, Appendix A.1.2).  For every sequence s with t = context_lens[s]:
  * the rows k_new[s], v_new[s] (DEVICE bf16 [num_seqs, num_kv_heads, head_dim], dense) are written to

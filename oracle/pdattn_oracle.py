@@ -127,6 +127,45 @@ def e4m3_to_double(codes) -> np.ndarray:
     return np.array([f(int(c)) for c in np.asarray(codes, dtype=np.uint8).ravel()], dtype=np.float64)
 
 
+def e4m3_encode(x) -> np.ndarray:
+    """Nearest e4m3 code of each fp32 value, ties to the even code, magnitudes beyond the largest finite value
+    (448) saturating to it, NaN to 0x7f.  Brute force over the table of code values."""
+    x = np.asarray(x, dtype=np.float32)
+    mags = e4m3_to_double(np.arange(0x7f))                      # 0 .. 448, increasing with the code
+    a = np.abs(x.astype(np.float64)).ravel()
+    hi = np.clip(np.searchsorted(mags, a, side="left"), 1, 0x7e)
+    lo = hi - 1
+    d_lo, d_hi = a - mags[lo], mags[hi] - a
+    code = np.where(d_lo < d_hi, lo, np.where(d_hi < d_lo, hi, np.where(lo % 2 == 0, lo, hi)))
+    code = np.where(a >= mags[0x7e], 0x7e, code).astype(np.uint8)
+    code = np.where(np.isnan(a), 0x7f, code).astype(np.uint8)
+    sign = (np.signbit(x).ravel() & ~np.isnan(a)).astype(np.uint8) << 7
+    return (code | sign).reshape(x.shape)
+
+
+def append_kv_fp8(k8, v8, k_scale, v_scale, block_table, context_lens, k_new, v_new) -> int:
+    """The fp8 KV append on the CPU, in place: codes of k_new / scale and v_new / scale (fp32 division, as the
+    quantised code is decided in that precision) at position context_lens[s]; returns the number of sequences
+    left untouched because of a bad page id or a full table row."""
+    NB, Hkv, bs, d = k8.shape
+    bt = block_table.numpy()
+    lens = context_lens.numpy()
+    kq = e4m3_encode(k_new.float().numpy() / k_scale.float().numpy().reshape(1, -1, 1))
+    vq = e4m3_encode(v_new.float().numpy() / v_scale.float().numpy().reshape(1, -1, 1))
+    k8n, v8n = k8.numpy(), v8.numpy()
+    skipped = 0
+    for s in range(len(lens)):
+        L = int(lens[s])
+        if L < 0 or L // bs >= bt.shape[1] or not (0 <= bt[s, L // bs] < NB):
+            skipped += 1
+            continue
+        page = int(bt[s, L // bs])
+        k8n[page, :, L % bs, :] = kq[s]
+        v8n[page, :, :, L % bs] = vq[s]
+        lens[s] = L + 1
+    return skipped
+
+
 def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, num_threads=None, return_bad=False):
     """fp64 attention over an fp8 (e4m3 codes) KV cache with one scale per KV head: k8 uint8
     [pages, Hkv, block_size, d], v8 uint8 [pages, Hkv, d, block_size] (V transposed inside a page)."""

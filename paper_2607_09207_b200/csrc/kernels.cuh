@@ -243,7 +243,10 @@ struct Cfg {
   static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the parked stores conflict-free
   static constexpr int SMEM_MAX = 232448;              // 227 KB
   static constexpr int CTRL_BYTES = 768;
-  static constexpr int NCW = PDATTN_NCW;                               // consumer warps
+#ifndef PDATTN_NCW_F8
+#define PDATTN_NCW_F8 PDATTN_NCW
+#endif
+  static constexpr int NCW = (EB == 1 && NT == 1) ? PDATTN_NCW_F8 : PDATTN_NCW;   // consumer warps
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
   static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged by producer 0
   static constexpr int Q_BYTES = HP * D * 2;           // one slot: the packed query heads of one KV head
@@ -1753,6 +1756,50 @@ stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __rest
     acc ^= a.x ^ a.y ^ a.z ^ a.w;
   }
   if (acc == 0x9e3779b9u) *sink = acc;   // practically never: keeps the loads alive
+}
+
+// ------------------------------------------------------------------------------------------
+// KV append into an fp8 cache: the new token's K and V rows (bf16) are divided by the KV head's scale,
+// rounded to e4m3 (nearest even, saturating to the largest finite code) and written as codes: K as a
+// row of the page [slot][d], V as a column of the transposed page [d][slot].  One block per sequence,
+// one warp per KV head.  Same rules as append_kernel for bad pages and full rows.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+append_fp8_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
+                  uint8_t* __restrict__ k8, uint8_t* __restrict__ v8, const float* __restrict__ k_scale,
+                  const float* __restrict__ v_scale, const int32_t* __restrict__ block_table,
+                  int32_t* __restrict__ context_lens, int Hkv, int D, int bs, int MB, int NB, int32_t* err) {
+  const int s = blockIdx.x;
+  const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int L = context_lens[s];
+  __syncthreads();                       // every warp has read the old length before it is advanced
+  if (L < 0 || L / bs >= MB) {
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  const int page = block_table[static_cast<int64_t>(s) * MB + L / bs];
+  if (page < 0 || page >= NB) {
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  if (g < Hkv) {
+    const int slot = L % bs;
+    const float sk = k_scale[g], sv = v_scale[g];   // true divisions below: the code is decided in fp32
+    const int64_t src = (static_cast<int64_t>(s) * Hkv + g) * D;
+    uint8_t* kp = k8 + ((static_cast<int64_t>(page) * Hkv + g) * bs + slot) * D;
+    uint8_t* vp = v8 + (static_cast<int64_t>(page) * Hkv + g) * D * bs + slot;
+    for (int j = lane * 2; j < D; j += 64) {
+      const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(k_new + src + j));
+      const float2 vf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(v_new + src + j));
+      unsigned short kc, vc;
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(kc) : "f"(__fdiv_rn(kf.y, sk)), "f"(__fdiv_rn(kf.x, sk)));
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(vc) : "f"(__fdiv_rn(vf.y, sv)), "f"(__fdiv_rn(vf.x, sv)));
+      *reinterpret_cast<unsigned short*>(kp + j) = kc;
+      vp[static_cast<int64_t>(j) * bs] = static_cast<uint8_t>(vc & 0xff);
+      vp[static_cast<int64_t>(j + 1) * bs] = static_cast<uint8_t>(vc >> 8);
+    }
+  }
+  if (threadIdx.x == 0) context_lens[s] = L + 1;
 }
 
 // ------------------------------------------------------------------------------------------

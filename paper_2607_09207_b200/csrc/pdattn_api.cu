@@ -425,6 +425,28 @@ pdattn_status pdattn_set_dynamic_spans(int per_cta) {
   return PDATTN_OK;
 }
 
+pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                   const float* k_scale, const float* v_scale, const int32_t* block_table,
+                                   int32_t* context_lens, int num_seqs, int num_kv_heads, int head_dim,
+                                   int block_size, int max_blocks_per_seq, int num_blocks, void* workspace,
+                                   pdattn_stream_t stream) {
+  if (num_seqs < 0 || num_kv_heads <= 0 || num_kv_heads > 16 || max_blocks_per_seq <= 0 || num_blocks <= 0)
+    return PDATTN_INVALID_ARG;
+  if (head_dim != 128 || block_size != 16) return PDATTN_UNSUPPORTED;
+  if (num_seqs == 0) return PDATTN_OK;
+  if (!k_new || !v_new || !k_cache || !v_cache || !k_scale || !v_scale || !block_table || !context_lens)
+    return PDATTN_INVALID_ARG;
+  auto mis = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; };
+  if (mis(k_new) || mis(v_new) || mis(k_cache) || mis(v_cache)) return PDATTN_MISALIGNED;
+  append_fp8_kernel<<<num_seqs, 32 * num_kv_heads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+      static_cast<uint8_t*>(k_cache), static_cast<uint8_t*>(v_cache), k_scale, v_scale, block_table, context_lens,
+      num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks, static_cast<int32_t*>(workspace));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("append_fp8_kernel launch", e);
+  return PDATTN_OK;
+}
+
 pdattn_status pdattn_set_prefix_engine(int engine) {
   if (engine < -1 || engine > 1) return PDATTN_INVALID_ARG;
   g_prefix_engine = engine;

@@ -34,7 +34,7 @@ EXPORTS = [
     "pdattn_set_merge_mode", "pdattn_set_prefix_engine",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
-    "pdattn_multi_workspace_size", "pdattn_decode_multi", "pdattn_decode_fp8",
+    "pdattn_multi_workspace_size", "pdattn_decode_multi", "pdattn_decode_fp8", "pdattn_append_kv_fp8",
 ]
 
 
@@ -97,6 +97,7 @@ def lib():
         L.pdattn_multi_workspace_size.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_multi.argtypes = [ctypes.POINTER(Args), i32, vp]
         L.pdattn_decode_fp8.argtypes = [ctypes.POINTER(Args), vp, vp, vp]
+        L.pdattn_append_kv_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
         L.pdattn_append_kv.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp]
         L.pdattn_check.argtypes = [vp, vp]
         L.pdattn_profile_events.argtypes = [vp, vp]
@@ -302,6 +303,20 @@ def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, ou
     st = lib().pdattn_decode_fp8(ctypes.byref(a), k_scale.data_ptr(), v_scale.data_ptr(), _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_decode_fp8")
+    return st
+
+
+def append_kv_fp8(k_new, v_new, k8, v8, k_scale, v_scale, block_table, context_lens, workspace=None, stream=None,
+                  check: bool = True) -> int:
+    """pdattn_append_kv_fp8: quantise the new K/V rows into the fp8 cache and advance context_lens (device, in place)."""
+    S, Hkv, d = k_new.shape
+    NB, _, bs, _ = k8.shape
+    st = lib().pdattn_append_kv_fp8(k_new.data_ptr(), v_new.data_ptr(), k8.data_ptr(), v8.data_ptr(), k_scale.data_ptr(),
+                                    v_scale.data_ptr(), block_table.data_ptr(), context_lens.data_ptr(), S, Hkv, d, bs,
+                                    block_table.shape[1], NB, workspace.data_ptr() if workspace is not None else None,
+                                    _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_append_kv_fp8")
     return st
 
 

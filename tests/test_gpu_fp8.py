@@ -124,3 +124,35 @@ def test_rejects_what_it_cannot_do():
     assert pdattn.decode_fp8(w32.q, k8, v8, ks, vs, w32.block_table, w32.context_lens, w32.scale,
                              torch.empty_like(w32.q), ws, check=False) == pdattn.UNSUPPORTED        # 32-token pages
     assert pdattn.lib().pdattn_decode_fp8(None, None, None, None) == pdattn.INVALID_ARG
+
+
+def test_append_writes_the_same_codes_as_the_oracle_and_decode_follows():
+    """A growing loop on the fp8 cache: quantising append (codes bit-exact against the CPU), then a decode step."""
+    lens = [0, 1, 15, 16, 17, 63, 64, 300]
+    steps = 35
+    w = W.make_custom(lens, Hq=8, Hkv=2, d=128, seed=47, device=DEV, headroom_tokens=steps + 5, poison=False)
+    ks, vs = scales(2, 6)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    ck8, cv8 = k8.cpu().clone(), v8.cpu().clone()
+    clens = w.context_lens.cpu().clone()
+    dlens = w.context_lens.clone()
+    ws = pdattn.alloc_workspace(len(lens), 8, 2, 128)
+    for step in range(steps):
+        k_new = W.normal_bf16(len(lens) * 2 * 128, 500 + step, 3, device=DEV).view(len(lens), 2, 128)
+        v_new = W.normal_bf16(len(lens) * 2 * 128, 500 + step, 4, device=DEV).view(len(lens), 2, 128)
+        pdattn.append_kv_fp8(k_new, v_new, k8, v8, ks, vs, w.block_table, dlens, ws)
+        assert orc.append_kv_fp8(ck8, cv8, ks.cpu(), vs.cpu(), w.block_table.cpu(), clens, k_new.cpu(), v_new.cpu()) == 0
+    assert pdattn.check(ws) == pdattn.OK
+    assert torch.equal(dlens.cpu(), clens)
+    assert torch.equal(k8.cpu(), ck8) and torch.equal(v8.cpu(), cv8)
+    wl = dataclasses.replace(w, context_lens=dlens, context_lens_host=clens.numpy().astype(np.int32))
+    out, st = run_fp8(wl, k8, v8, ks, vs, host_lens=False, ws=ws)
+    assert st == pdattn.OK
+    assert_parity(out, orc.decode_fp8(w.q.cpu(), ck8, cv8, ks.cpu(), vs.cpu(), w.block_table.cpu(), clens, w.scale),
+                  "fp8 decode after appends")
+    # a full table row and a bad page id leave the sequence untouched and are reported
+    bt = w.block_table.clone()
+    bt[0, int(clens[0]) // 16] = -1
+    pdattn.append_kv_fp8(k_new, v_new, k8, v8, ks, vs, bt, dlens, ws)
+    assert pdattn.check(ws) == pdattn.BAD_PAGE_INDEX
+    assert int(dlens[0]) == int(clens[0]) and int(dlens[1]) == int(clens[1]) + 1

@@ -341,3 +341,20 @@ def test_fp8_cache_oracle_against_the_bf16_oracle_on_the_same_values():
     base = orc.decode_fp8(w.q, k8, v8, torch.ones(2), torch.ones(2), w.block_table, w.context_lens, w.scale)
     scaled = orc.decode_fp8(w.q, k8, v8, torch.ones(2), torch.tensor([1.0, 3.0]), w.block_table, w.context_lens, w.scale)
     assert np.array_equal(scaled[:, :2], base[:, :2]) and np.allclose(scaled[:, 2:], 3.0 * base[:, 2:], rtol=1e-15)
+
+
+def test_e4m3_encoder_matches_the_library_cast_and_round_trips():
+    rng = np.random.default_rng(9)
+    x = np.concatenate([rng.normal(size=20000) * 3, rng.uniform(-448, 448, size=20000), rng.normal(size=5000) * 1e-2,
+                        orc.e4m3_to_double(np.arange(0x7f)), [0.0, -0.0, 447.9, 448.0, 464.0, 1e9, -1e9]]).astype(np.float32)
+    got = orc.e4m3_encode(x)
+    inr = np.abs(x) <= 448
+    ref = torch.from_numpy(x[inr]).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(got[inr], ref)
+    assert np.all(got[~inr] & 0x7f == 0x7e)                                   # saturation to the largest finite code
+    codes = np.delete(np.arange(256, dtype=np.uint8), [0x7f, 0xff])
+    vals = orc.e4m3_to_double(codes).astype(np.float32)
+    back = orc.e4m3_encode(vals)
+    assert np.array_equal(back[codes != 0x80], codes[codes != 0x80]) and back[codes == 0x80][0] in (0x00, 0x80)
+    # a tie goes to the even code: 17 lies halfway between 16 (code 0x58) and 18 (0x59)
+    assert orc.e4m3_encode(np.array([17.0, 19.0], dtype=np.float32)).tolist() == [0x58, 0x5a]
