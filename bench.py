@@ -53,6 +53,9 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cfg", type=int, default=2, help="BASELINE.json config index + 1 (default: the metric's config)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fp8", action="store_true",
+                    help="time pdattn_decode_fp8 over an e4m3 copy of the same pools (half the KV bytes per step) "
+                         "instead of the bf16 step; head_dim 128 configurations only")
     ap.add_argument("--short-batches", action="store_true",
                     help="also time batches of 4096 short contexts under both merge modes, and a large GRPO batch "
                          "early in its rollout under both prefix kernels (secondary results, N = 1)")
@@ -234,9 +237,21 @@ def main():
     outs = [torch.empty_like(c.q) for c in copies]
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
+    fp8 = None
+    if args.fp8:
+        ks8 = torch.full((base.num_kv_heads,), 1.25, dtype=torch.float32, device=dev)
+        vs8 = torch.full((base.num_kv_heads,), 0.75, dtype=torch.float32, device=dev)
+        fp8 = [W.fp8_caches(c, ks8, vs8) for c in copies]
+        uniq //= 2
+        logical //= 2
 
     def step(i):
         c = copies[i % len(copies)]
+        if fp8 is not None:
+            k8, v8 = fp8[i % len(copies)]
+            pdattn.decode_fp8(c.q, k8, v8, ks8, vs8, c.block_table, c.context_lens, c.scale, outs[i % len(copies)], ws,
+                              context_lens_host=c.context_lens_host, stream=stream)
+            return
         if grouped:
             pdattn.decode_grouped(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale,
                                   outs[i % len(copies)], ws, c.context_lens_host, 8, ptd, pth, stream=stream)
@@ -325,7 +340,9 @@ def main():
     # ---- secondary runs (N = 1 only): bandwidth ceilings from the library's probes, the device-side
     # planner (no host copy of the lengths) and the token-major cache layout through strides
     extras = None
-    if world == 1:
+    if world == 1 and fp8 is not None:
+        extras = {"note": "fp8 run: e2e and the secondary results are not taken (they describe the bf16 step)"}
+    elif world == 1:
         def timed(fn, n=20, reps=5):
             for _ in range(3):
                 fn()
@@ -414,9 +431,10 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
+            "dtype": "bf16" if fp8 is None else "e4m3 cache, fp16 products, fp32 accumulate", "data": "synthetic",
             "config": {"workload": CFG_DESC[args.cfg] + (f" [REDUCED to {S} seqs]" if args.num_seqs else "")
-                       + (" [grouped: shared prompt tiles read once per group]" if grouped else ""),
+                       + (" [grouped: shared prompt tiles read once per group]" if grouped else "")
+                       + (" [fp8 KV cache: e4m3 codes, one scale per KV head]" if fp8 is not None else ""),
                        "num_seqs_per_gpu": S,
                        "unique_kv_bytes_per_step": uniq, "logical_kv_bytes_per_step": logical,
                        "l2": f"inputs ({uniq / 1e9:.2f} GB) larger than L2 and steps rotate over {len(copies)} "
@@ -428,12 +446,13 @@ def main():
             "beta_hist_s_per_token_per_layer": base.kv_bytes_per_token() / (uniq / (ms_step * 1e-3)),
             "pct_of_8tbs_nominal_step": uniq / (ms_step * 1e-3) / 8e12 * 100.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": profiled_traffic(args.cfg),
+                         "frac": achieved / peak, "traffic": None if fp8 is not None else profiled_traffic(args.cfg),
                          "kernel": kernel_name, "kernel_ms": k1_ms, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": uniq,
                          "pct_of_8tbs_nominal": achieved / 8000.0 * 100.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": ke, "note": "q/block_table/context_lens from pinned host memory, out read back "
+                    "steps": ke, "note": ("bf16 step (pdattn_decode_host has no fp8 form); " if fp8 is not None else "")
+                                         + "q/block_table/context_lens from pinned host memory, out read back "
                                          "and the stream synchronised every step; KV pools are resident state"},
             "gpu_launches": launches_per_step * K,
             "clocks": sampler.summary(),

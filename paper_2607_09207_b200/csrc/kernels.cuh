@@ -243,10 +243,7 @@ struct Cfg {
   static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the parked stores conflict-free
   static constexpr int SMEM_MAX = 232448;              // 227 KB
   static constexpr int CTRL_BYTES = 768;
-#ifndef PDATTN_NCW_F8
-#define PDATTN_NCW_F8 PDATTN_NCW
-#endif
-  static constexpr int NCW = (EB == 1 && NT == 1) ? PDATTN_NCW_F8 : PDATTN_NCW;   // consumer warps
+  static constexpr int NCW = PDATTN_NCW;                               // consumer warps
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
   static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged by producer 0
   static constexpr int Q_BYTES = HP * D * 2;           // one slot: the packed query heads of one KV head

@@ -195,12 +195,13 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else if (rank == kMapV8) {
-    // fp8 V pool [pages, kv heads, d, slots] (transposed inside a page): one box = a page-head,
-    // [block_size, d, 1, 1], rows of block_size bytes, no swizzle
-    cuuint64_t dims[4] = {static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(hkv), nbu};
-    cuuint64_t strides[3] = {static_cast<cuuint64_t>(bs), static_cast<cuuint64_t>(d) * bs,
-                             static_cast<cuuint64_t>(hkv) * d * bs};
-    cuuint32_t box[4] = {static_cast<cuuint32_t>(bs), static_cast<cuuint32_t>(d), 1, 1};
+    // fp8 V pool [pages, kv heads, d, slots] (transposed inside a page): a page-head is d * block_size
+    // contiguous bytes and lands in shared memory in the same order, so it is described as rows of 256
+    // bytes (8 requests per box; rows of block_size bytes would be 128), no swizzle
+    const cuuint64_t rows = static_cast<cuuint64_t>(d) * bs / 256;
+    cuuint64_t dims[4] = {256, rows, static_cast<cuuint64_t>(hkv), nbu};
+    cuuint64_t strides[3] = {256, static_cast<cuuint64_t>(d) * bs, static_cast<cuuint64_t>(hkv) * d * bs};
+    cuuint32_t box[4] = {256, static_cast<cuuint32_t>(rows), 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
