@@ -156,3 +156,21 @@ def test_append_writes_the_same_codes_as_the_oracle_and_decode_follows():
     pdattn.append_kv_fp8(k_new, v_new, k8, v8, ks, vs, bt, dlens, ws)
     assert pdattn.check(ws) == pdattn.BAD_PAGE_INDEX
     assert int(dlens[0]) == int(clens[0]) and int(dlens[1]) == int(clens[1]) + 1
+
+
+def test_page_permutation_and_plan_source_leave_the_bits_unchanged():
+    w = W.make_custom([100, 33, 256, 5000, 777], Hq=28, Hkv=4, d=128, seed=48, device=DEV, num_blocks=512)
+    ks, vs = scales(4, 7)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    ref, st = run_fp8(w, k8, v8, ks, vs)
+    assert st == pdattn.OK
+    perm = torch.from_numpy(np.random.default_rng(3).permutation(512)).to(DEV)
+    inv = torch.argsort(perm)
+    bt = w.block_table.clone().long()
+    valid = bt >= 0
+    bt[valid] = perm[bt[valid]]
+    w2 = dataclasses.replace(w, block_table=bt.to(torch.int32))
+    out, st = run_fp8(w2, k8[inv].contiguous(), v8[inv].contiguous(), ks, vs)
+    assert st == pdattn.OK and torch.equal(ref, out)
+    dev_plan, st = run_fp8(w, k8, v8, ks, vs, host_lens=False)          # spans computed on the device
+    assert st == pdattn.OK and torch.equal(ref, dev_plan)
