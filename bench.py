@@ -443,7 +443,8 @@ def main():
             "hbm_tbs_step": uniq / (ms_step * 1e-3) / 1e12 * 1.0,
             # coefficient of the paper's decode-history term for ONE layer of this shape: seconds per
             # history token read = per-layer KV bytes per token / achieved bytes per second
-            "beta_hist_s_per_token_per_layer": base.kv_bytes_per_token() / (uniq / (ms_step * 1e-3)),
+            "beta_hist_s_per_token_per_layer": base.kv_bytes_per_token() / (2 if fp8 is not None else 1)
+                                               / (uniq / (ms_step * 1e-3)),
             "pct_of_8tbs_nominal_step": uniq / (ms_step * 1e-3) / 8e12 * 100.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": None if fp8 is not None else profiled_traffic(args.cfg),
