@@ -154,7 +154,7 @@ pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens,
  * including the treatment of bad page ids and of slots past the end (any code, NaN codes too).
  * The codes are widened exactly; q is rounded to fp16 for the products (values below 2^-14 lose bits) and
  * the softmax weights to fp16 (11 bits), accumulation in fp32; out is bf16.
- *   Requirements: head_dim 128, block_size 16 (else PDATTN_UNSUPPORTED); not combined with
+ *   Requirements: head_dim 128 (else PDATTN_UNSUPPORTED; every page size of pdattn_decode_ex); not combined with
  *   pdattn_decode_grouped / pdattn_decode_multi.  Workspace as for pdattn_decode_ex.
  */
 pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, const float* v_scale,
@@ -165,7 +165,7 @@ pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, c
  * bf16 [num_seqs, num_kv_heads, head_dim]) are divided by their KV head's scale, rounded to e4m3 (nearest
  * even; magnitudes beyond the largest finite code 448 saturate to it) and written at position
  * context_lens[s], which then becomes context_lens[s] + 1.  Page rules and error reporting as in
- * pdattn_append_kv.  head_dim 128, block_size 16.
+ * pdattn_append_kv.  head_dim 128.
  */
 pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                    const float* k_scale, const float* v_scale, const int32_t* block_table,

@@ -496,9 +496,10 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
 }
 
 // ------------------------------------------------------------------------------------------
-// One 64-token tile on one warp, fp8 cache (e4m3 codes; head_dim 128, 16-token pages).
-// K tile: [64 tokens][128 B] (one code per element, 128-byte swizzle); V tile: per page [128 d][16 tokens]
-// (V is stored transposed inside a page).  The codes are widened to fp16 in registers (exact) and both
+// One 64-token tile on one warp, fp8 cache (e4m3 codes; head_dim 128).
+// K tile: [64 tokens][128 B] (one code per element, 128-byte swizzle); V tile: per page [128 d][BS tokens]
+// (V is stored transposed inside a page; with pages of 32 or 64 tokens the 16-byte rows that ldmatrix
+// reads lie 32 or 64 bytes apart and collide two or four ways in the banks).  The codes are widened to fp16 in registers (exact) and both
 // products run as fp16 MMAs; Q arrives as fp16 fragments and P is rounded to fp16 (11 bits, one term).
 // ldmatrix moves 16-bit units, i.e. PAIRS of codes, so a lane receives four consecutive elements of
 // the contraction dimension where the MMA fragment wants two plus two eight further on.  Both
@@ -509,7 +510,7 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
 // the score MMA holds token pi(rho) of its 16-token group -- a matter of the row addresses handed to
 // ldmatrix for K.
 // ------------------------------------------------------------------------------------------
-template <int NT, bool TAIL>
+template <int NT, int BS, bool TAIL>
 __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const uint32_t (&qf)[NT][8][2],
                                                 float (&acc)[NT][8][4], float (&m)[NT][2], float (&l)[NT][2],
                                                 float sl2, int n_left, uint32_t badmask, int lane,
@@ -561,7 +562,7 @@ __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const 
 #pragma unroll
   for (int j = 0; j < GROUPS; ++j) {
     bool dead_page = false;
-    if (badmask) dead_page = (badmask >> j) & 1u;
+    if (badmask) dead_page = (badmask >> ((j * 16) / BS)) & 1u;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -626,7 +627,7 @@ __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const 
       pb[j][nt][1] = movmatrix_trans(pack_f16x2(p2, p3));
     }
 
-  // ---- O^T += V^T . P^T : [128] x [8*NT heads], one page (16 tokens) per MMA step
+  // ---- O^T += V^T . P^T : [128] x [8*NT heads], 16 tokens of a page per MMA step
 #pragma unroll
   for (int j = 0; j < GROUPS; ++j) {
     if (!TAIL || j * 16 < n_valid) {
@@ -639,7 +640,7 @@ __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const 
 #pragma unroll
       for (int jp = 0; jp < 4; ++jp) {
         uint32_t r[4];
-        ldsm_x4(r, sV + j * 2048 + (jp * 32 + v_drow) * 16);
+        ldsm_x4(r, sV + ((j * 16) / BS) * (128 * BS) + (jp * 32 + v_drow) * BS + (j * 16) % BS);
         if (TAIL) {
           r[0] &= keep_mask;
           r[1] &= keep_mask;
@@ -747,7 +748,7 @@ template <int D, int NT, int BS, int EB>
 __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanParams& pp, Ctrl* ctrl, uint32_t ring,
                                               uint32_t qbuf, uint8_t* handoff, int warp, int lane) {
   using C = Cfg<D, NT, BS, EB>;
-  static_assert(EB == 2 || (EB == 1 && D == 128 && BS == 16), "the fp8 cache path is built for head_dim 128, 16-token pages");
+  static_assert(EB == 2 || (EB == 1 && D == 128), "the fp8 cache path is built for head_dim 128");
   constexpr int NST = C::NSTAGES;
   constexpr int NCW = C::NCW;
   constexpr int E = C::HANDOFFS;
@@ -888,9 +889,9 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
           }
         } else {
           if (n_left - (P.T - 1) >= TILE) {
-            compute_tile_f8<NT, false>(sK, sV, qf, acc, m, l, sl2, TILE, badmask, lane, lag);
+            compute_tile_f8<NT, BS, false>(sK, sV, qf, acc, m, l, sl2, TILE, badmask, lane, lag);
           } else {
-            compute_tile_f8<NT, true>(sK, sV, qf, acc, m, l, sl2, n_left, badmask, lane, lag);
+            compute_tile_f8<NT, BS, true>(sK, sV, qf, acc, m, l, sl2, n_left, badmask, lane, lag);
           }
         }
         __syncwarp();

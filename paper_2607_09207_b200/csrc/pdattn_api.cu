@@ -91,7 +91,7 @@ struct DevInfo {
   bool attr_set[2][2][3] = {};      // [D==128][NT==2][page size / 32]
   bool probe_attr_set[2][2][3] = {};
   bool chain_attr_set[2][2][3] = {};
-  bool fp8_attr_set[2] = {};        // [NT==2]
+  bool fp8_attr_set[2][3] = {};     // [NT==2][page size / 32]
   bool prefix_attr_set[2][3] = {};  // [D==128][page size / 32]
   bool prefix_umma_attr_set[2][3] = {};
 };
@@ -265,10 +265,10 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   }
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
   if (g_fp8.active) {
-    if constexpr (D == 128 && BS == 16) {
+    if constexpr (D == 128) {
       using C8 = Cfg<D, NT, BS, 1>;
       auto k8 = decode_kernel<D, NT, BS, false, true, 1>;
-      bool& fdone = di->fp8_attr_set[NT == 2];
+      bool& fdone = di->fp8_attr_set[NT == 2][BS / 32];
       if (!fdone) {
         cudaError_t fe = cudaFuncSetAttribute(k8, cudaFuncAttributeMaxDynamicSharedMemorySize, C8::CHAIN_DYN_BYTES);
         if (fe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", fe);
@@ -433,7 +433,7 @@ pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k
                                    pdattn_stream_t stream) {
   if (num_seqs < 0 || num_kv_heads <= 0 || num_kv_heads > 16 || max_blocks_per_seq <= 0 || num_blocks <= 0)
     return PDATTN_INVALID_ARG;
-  if (head_dim != 128 || block_size != 16) return PDATTN_UNSUPPORTED;
+  if (head_dim != 128 || (block_size != 16 && block_size != 32 && block_size != 64)) return PDATTN_UNSUPPORTED;
   if (num_seqs == 0) return PDATTN_OK;
   if (!k_new || !v_new || !k_cache || !v_cache || !k_scale || !v_scale || !block_table || !context_lens)
     return PDATTN_INVALID_ARG;
@@ -496,7 +496,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   if (T < 1) return PDATTN_INVALID_ARG;
   if (G * T > 16 || (T > 1 && grouped)) return PDATTN_UNSUPPORTED;
   const bool fp8 = g_fp8.active;
-  if (fp8 && (a->head_dim != 128 || a->block_size != 16 || T != 1 || grouped || g_probe_mode)) return PDATTN_UNSUPPORTED;
+  if (fp8 && (a->head_dim != 128 || T != 1 || grouped || g_probe_mode)) return PDATTN_UNSUPPORTED;
   const WsLayout wl = ws_layout(a->num_seqs, G * T, a->head_dim);
   // grouped calls keep two more arrays behind the ordinary layout
   const size_t off_start = wl.total;

@@ -58,6 +58,19 @@ def test_ragged_lengths_and_head_groupings(Hq, Hkv, host_lens):
     assert_parity(out, reference(w, k8, v8, ks, vs), f"fp8 Hq={Hq} Hkv={Hkv}")
 
 
+@pytest.mark.parametrize("bs", [32, 64])
+@pytest.mark.parametrize("Hq,Hkv", [(28, 4), (32, 2)])
+def test_larger_pages(Hq, Hkv, bs):
+    lens = [1, 15, 16, 17, 31, 32, 33, 63, 64, 65, 100, 127, 129, 1000, 0, 4097]
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=128, bs=bs, seed=420 + bs, device=DEV)
+    ks, vs = scales(Hkv, bs)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    for host in (True, False):
+        out, st = run_fp8(w, k8, v8, ks, vs, host)
+        assert st == pdattn.OK
+        assert_parity(out, reference(w, k8, v8, ks, vs), f"fp8 page size {bs} Hq={Hq} Hkv={Hkv}")
+
+
 def test_scaled_rollout_config_and_run_to_run_bits():
     w = W.make_config(2, device=DEV, num_seqs=24, len_div=2)
     ks, vs = scales(4, 1)
@@ -118,25 +131,21 @@ def test_rejects_what_it_cannot_do():
     out = torch.empty_like(w.q)
     args = (w.block_table, w.context_lens, w.scale, out, ws)
     assert pdattn.decode_fp8(w.q, k8, v8, ks, vs, *args, check=False) == pdattn.UNSUPPORTED       # head_dim 64
-    w32 = W.make_custom([100], Hq=4, Hkv=2, d=128, bs=32, seed=46, device=DEV)
-    k8, v8 = W.fp8_caches(w32, ks, vs)
-    ws = pdattn.alloc_workspace(1, 4, 2, 128, 32)
-    assert pdattn.decode_fp8(w32.q, k8, v8, ks, vs, w32.block_table, w32.context_lens, w32.scale,
-                             torch.empty_like(w32.q), ws, check=False) == pdattn.UNSUPPORTED        # 32-token pages
     assert pdattn.lib().pdattn_decode_fp8(None, None, None, None) == pdattn.INVALID_ARG
 
 
-def test_append_writes_the_same_codes_as_the_oracle_and_decode_follows():
+@pytest.mark.parametrize("bs", [16, 32])
+def test_append_writes_the_same_codes_as_the_oracle_and_decode_follows(bs):
     """A growing loop on the fp8 cache: quantising append (codes bit-exact against the CPU), then a decode step."""
     lens = [0, 1, 15, 16, 17, 63, 64, 300]
     steps = 35
-    w = W.make_custom(lens, Hq=8, Hkv=2, d=128, seed=47, device=DEV, headroom_tokens=steps + 5, poison=False)
+    w = W.make_custom(lens, Hq=8, Hkv=2, d=128, bs=bs, seed=47, device=DEV, headroom_tokens=steps + 5, poison=False)
     ks, vs = scales(2, 6)
     k8, v8 = W.fp8_caches(w, ks, vs)
     ck8, cv8 = k8.cpu().clone(), v8.cpu().clone()
     clens = w.context_lens.cpu().clone()
     dlens = w.context_lens.clone()
-    ws = pdattn.alloc_workspace(len(lens), 8, 2, 128)
+    ws = pdattn.alloc_workspace(len(lens), 8, 2, 128, bs)
     for step in range(steps):
         k_new = W.normal_bf16(len(lens) * 2 * 128, 500 + step, 3, device=DEV).view(len(lens), 2, 128)
         v_new = W.normal_bf16(len(lens) * 2 * 128, 500 + step, 4, device=DEV).view(len(lens), 2, 128)
@@ -152,7 +161,7 @@ def test_append_writes_the_same_codes_as_the_oracle_and_decode_follows():
                   "fp8 decode after appends")
     # a full table row and a bad page id leave the sequence untouched and are reported
     bt = w.block_table.clone()
-    bt[0, int(clens[0]) // 16] = -1
+    bt[0, int(clens[0]) // bs] = -1
     pdattn.append_kv_fp8(k_new, v_new, k8, v8, ks, vs, bt, dlens, ws)
     assert pdattn.check(ws) == pdattn.BAD_PAGE_INDEX
     assert int(dlens[0]) == int(clens[0]) and int(dlens[1]) == int(clens[1]) + 1
