@@ -155,10 +155,14 @@ pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens,
  * The codes are widened exactly; q is rounded to fp16 for the products (values below 2^-14 lose bits) and
  * the softmax weights to fp16 (11 bits), accumulation in fp32; out is bf16.
  *   Requirements: head_dim 128 (else PDATTN_UNSUPPORTED; every page size of pdattn_decode_ex); not combined with
- *   pdattn_decode_grouped / pdattn_decode_multi.  Workspace as for pdattn_decode_ex.
+ *   pdattn_decode_grouped.  Workspace as for pdattn_decode_ex.
  */
 pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, const float* v_scale,
                                 pdattn_stream_t stream);
+/* The same with num_query_tokens new tokens per sequence: pdattn_decode_multi's definition and layouts
+ * (q, out [num_seqs, T, num_q_heads, head_dim]; T * G <= 16; pdattn_multi_workspace_size) over the fp8 cache. */
+pdattn_status pdattn_decode_fp8_multi(const pdattn_args* args, int num_query_tokens, const float* k_scale,
+                                      const float* v_scale, pdattn_stream_t stream);
 
 /*
  * KV append into the fp8 cache of pdattn_decode_fp8 (same layouts): the rows k_new[s], v_new[s] (DEVICE

@@ -193,6 +193,19 @@ def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, nu
     return (out, bad.value) if return_bad else out
 
 
+def decode_fp8_multi(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, num_threads=None):
+    """decode_multi's definition over the fp8 cache: T plain fp8 decode steps over truncated contexts."""
+    q = _cpu(q)
+    S, T, Hq, d = q.shape
+    lens = np.asarray(_cpu(context_lens).numpy(), dtype=np.int64)
+    out = np.empty((S, T, Hq, d), dtype=np.float64)
+    for j in range(T):
+        lens_j = torch.from_numpy(np.maximum(lens - (T - 1 - j), 0).astype(np.int32))
+        out[:, j] = decode_fp8(q[:, j].contiguous(), k8, v8, k_scale, v_scale, block_table, lens_j, scale,
+                               num_threads=num_threads)
+    return out
+
+
 def decode_workload(w, **kw):
     return decode(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, **kw)
 

@@ -496,7 +496,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
   if (T < 1) return PDATTN_INVALID_ARG;
   if (G * T > 16 || (T > 1 && grouped)) return PDATTN_UNSUPPORTED;
   const bool fp8 = g_fp8.active;
-  if (fp8 && (a->head_dim != 128 || T != 1 || grouped || g_probe_mode)) return PDATTN_UNSUPPORTED;
+  if (fp8 && (a->head_dim != 128 || grouped || g_probe_mode)) return PDATTN_UNSUPPORTED;
   const WsLayout wl = ws_layout(a->num_seqs, G * T, a->head_dim);
   // grouped calls keep two more arrays behind the ordinary layout
   const size_t off_start = wl.total;
@@ -701,6 +701,14 @@ pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, c
   g_fp8.v_scale = v_scale;
   const pdattn_status s = pdattn_decode_ex(&a, stream);
   g_fp8 = Fp8Call{};
+  return s;
+}
+
+pdattn_status pdattn_decode_fp8_multi(const pdattn_args* args, int num_query_tokens, const float* k_scale,
+                                      const float* v_scale, pdattn_stream_t stream) {
+  g_query_tokens = num_query_tokens;
+  const pdattn_status s = pdattn_decode_fp8(args, k_scale, v_scale, stream);
+  g_query_tokens = 1;
   return s;
 }
 

@@ -34,7 +34,7 @@ EXPORTS = [
     "pdattn_set_merge_mode", "pdattn_set_prefix_engine",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
-    "pdattn_multi_workspace_size", "pdattn_decode_multi", "pdattn_decode_fp8", "pdattn_append_kv_fp8",
+    "pdattn_multi_workspace_size", "pdattn_decode_multi", "pdattn_decode_fp8", "pdattn_append_kv_fp8", "pdattn_decode_fp8_multi",
 ]
 
 
@@ -97,6 +97,7 @@ def lib():
         L.pdattn_multi_workspace_size.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_multi.argtypes = [ctypes.POINTER(Args), i32, vp]
         L.pdattn_decode_fp8.argtypes = [ctypes.POINTER(Args), vp, vp, vp]
+        L.pdattn_decode_fp8_multi.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
         L.pdattn_append_kv_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
         L.pdattn_append_kv.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp]
         L.pdattn_check.argtypes = [vp, vp]
@@ -283,7 +284,8 @@ def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, ou
                context_lens_host=None, stream=None, check: bool = True) -> int:
     """pdattn_decode_fp8: k8 uint8 [pages, Hkv, block_size, d], v8 uint8 [pages, Hkv, d, block_size] (e4m3 codes),
     k_scale / v_scale fp32 [Hkv] on the device."""
-    S, Hq, d = q.shape
+    T = q.shape[1] if q.dim() == 4 else 0          # [S, T, Hq, d]: several new tokens per sequence
+    S, Hq, d = q.shape[0], q.shape[-2], q.shape[-1]
     NB, Hkv, bs, _ = k8.shape
     assert k8.dtype == torch.uint8 and v8.dtype == torch.uint8 and tuple(v8.shape) == (NB, Hkv, d, bs)
     assert k8.is_contiguous() and v8.is_contiguous() and k_scale.dtype == torch.float32 and v_scale.dtype == torch.float32
@@ -300,7 +302,10 @@ def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, ou
     a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = Hkv * bs * d, bs * d, d
     a.scale = float(scale)
     a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
-    st = lib().pdattn_decode_fp8(ctypes.byref(a), k_scale.data_ptr(), v_scale.data_ptr(), _stream_ptr(stream))
+    if T:
+        st = lib().pdattn_decode_fp8_multi(ctypes.byref(a), T, k_scale.data_ptr(), v_scale.data_ptr(), _stream_ptr(stream))
+    else:
+        st = lib().pdattn_decode_fp8(ctypes.byref(a), k_scale.data_ptr(), v_scale.data_ptr(), _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_decode_fp8")
     return st

@@ -183,3 +183,21 @@ def test_page_permutation_and_plan_source_leave_the_bits_unchanged():
     assert st == pdattn.OK and torch.equal(ref, out)
     dev_plan, st = run_fp8(w, k8, v8, ks, vs, host_lens=False)          # spans computed on the device
     assert st == pdattn.OK and torch.equal(ref, dev_plan)
+
+
+@pytest.mark.parametrize("Hq,Hkv,T,bs", [(28, 4, 2, 16), (8, 2, 4, 16), (8, 2, 2, 32)])
+def test_several_query_tokens_over_the_fp8_cache(Hq, Hkv, T, bs):
+    lens = [T, T + 1, 15, 16, 17, 63, 64, 65, 66, 67, 127, 128, 129, 130, 131, 255, 257, 1000, 0, 2, 64 * 9 + 2]
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=128, bs=bs, seed=430 + T, device=DEV)
+    ks, vs = scales(Hkv, 10 + T)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    S = len(lens)
+    q = W.normal_bf16(S * T * Hq * 128, 21, 7, device=DEV).view(S, T, Hq, 128)
+    ws = pdattn.alloc_multi_workspace(S, Hq, Hkv, 128, bs, T)
+    out = torch.full_like(q, float("nan"))
+    pdattn.decode_fp8(q, k8, v8, ks, vs, w.block_table, w.context_lens, w.scale, out, ws,
+                      context_lens_host=w.context_lens_host)
+    assert pdattn.check(ws) == pdattn.OK
+    ref = orc.decode_fp8_multi(q.cpu(), k8.cpu(), v8.cpu(), ks.cpu(), vs.cpu(), w.block_table.cpu(),
+                               w.context_lens.cpu(), w.scale)
+    assert_parity(out, ref, f"fp8, T={T}, Hq={Hq} Hkv={Hkv} bs={bs}")
