@@ -10,7 +10,8 @@ CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB = os.path.join(LIB_DIR, "libpdattn.so")
 SOURCES = ["pdattn_api.cu", "partition.cpp"]
-HEADERS = ["kernels.cuh", "prefix_umma.cuh", "partition.h", os.path.join("..", "..", "include", "pdattn.h")]
+HEADERS = ["kernels.cuh", "common.cuh", "tile_bf16.cuh", "tile_fp8.cuh", "decode.cuh", "prefix_mma.cuh",
+           "prefix_umma.cuh", "aux_kernels.cuh", "partition.h", os.path.join("..", "..", "include", "pdattn.h")]
 
 
 def _nvcc() -> str:

@@ -1,0 +1,274 @@
+// KV append (bf16 and fp8), stream-read probe, combine of cut units, device-side planner.
+#pragma once
+
+#include "common.cuh"
+
+namespace pdattn {
+
+// ------------------------------------------------------------------------------------------
+// KV append: the step on the input side of decode attention.  Block s writes the new token's K
+// and V rows of every KV head into slot L_s % bs of page block_table[s, L_s / bs] and then
+// advances context_lens[s].  One warp per KV head: lanes copy 16-byte chunks, K then V.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+append_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
+              __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
+              const int32_t* __restrict__ block_table, int32_t* __restrict__ context_lens, int Hkv, int D, int bs,
+              int MB, int NB, int64_t sb, int64_t sh, int64_t st, int32_t* err) {
+  const int s = blockIdx.x;
+  const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int L = context_lens[s];
+  __syncthreads();                       // every warp has read the old length before it is advanced
+  if (L < 0 || L / bs >= MB) {
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  const int page = block_table[static_cast<int64_t>(s) * MB + L / bs];
+  if (page < 0 || page >= NB) {          // not dereferenced; the length is left as it was
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  if (g < Hkv) {
+    const int64_t dst = page * sb + g * sh + static_cast<int64_t>(L % bs) * st;
+    const int64_t src = (static_cast<int64_t>(s) * Hkv + g) * D;
+    const int chunks = D / 8;            // 16-byte chunks per row
+    for (int c = lane; c < 2 * chunks; c += 32) {
+      const bool isV = c >= chunks;
+      const int cc = isV ? c - chunks : c;
+      const uint4 v = *reinterpret_cast<const uint4*>((isV ? v_new : k_new) + src + cc * 8);
+      *reinterpret_cast<uint4*>((isV ? v_cache : k_cache) + dst + cc * 8) = v;
+    }
+  }
+  if (threadIdx.x == 0) context_lens[s] = L + 1;
+}
+
+// Read-only streaming ceiling: every thread block sums a contiguous slice with 16-byte loads.
+__global__ void __launch_bounds__(512)
+stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __restrict__ sink) {
+  uint32_t acc = 0;
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+#pragma unroll 1
+  for (; i + 3 * stride < n_vec; i += 4 * stride) {
+    const uint4 a = __ldcs(src + i), b = __ldcs(src + i + stride), c = __ldcs(src + i + 2 * stride),
+                d = __ldcs(src + i + 3 * stride);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ d.x ^ d.y ^ d.z ^ d.w;
+  }
+  for (; i < n_vec; i += stride) {
+    const uint4 a = __ldcs(src + i);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w;
+  }
+  if (acc == 0x9e3779b9u) *sink = acc;   // practically never: keeps the loads alive
+}
+
+// ------------------------------------------------------------------------------------------
+// KV append into an fp8 cache: the new token's K and V rows (bf16) are divided by the KV head's scale,
+// rounded to e4m3 (nearest even, saturating to the largest finite code) and written as codes: K as a
+// row of the page [slot][d], V as a column of the transposed page [d][slot].  One block per sequence,
+// one warp per KV head.  Same rules as append_kernel for bad pages and full rows.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+append_fp8_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
+                  uint8_t* __restrict__ k8, uint8_t* __restrict__ v8, const float* __restrict__ k_scale,
+                  const float* __restrict__ v_scale, const int32_t* __restrict__ block_table,
+                  int32_t* __restrict__ context_lens, int Hkv, int D, int bs, int MB, int NB, int32_t* err) {
+  const int s = blockIdx.x;
+  const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int L = context_lens[s];
+  __syncthreads();                       // every warp has read the old length before it is advanced
+  if (L < 0 || L / bs >= MB) {
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  const int page = block_table[static_cast<int64_t>(s) * MB + L / bs];
+  if (page < 0 || page >= NB) {
+    if (threadIdx.x == 0 && err) atomicOr(err, ERR_BAD_PAGE);
+    return;
+  }
+  if (g < Hkv) {
+    const int slot = L % bs;
+    const float sk = k_scale[g], sv = v_scale[g];   // true divisions below: the code is decided in fp32
+    const int64_t src = (static_cast<int64_t>(s) * Hkv + g) * D;
+    uint8_t* kp = k8 + ((static_cast<int64_t>(page) * Hkv + g) * bs + slot) * D;
+    uint8_t* vp = v8 + (static_cast<int64_t>(page) * Hkv + g) * D * bs + slot;
+    for (int j = lane * 2; j < D; j += 64) {
+      const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(k_new + src + j));
+      const float2 vf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(v_new + src + j));
+      unsigned short kc, vc;
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(kc) : "f"(__fdiv_rn(kf.y, sk)), "f"(__fdiv_rn(kf.x, sk)));
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(vc) : "f"(__fdiv_rn(vf.y, sv)), "f"(__fdiv_rn(vf.x, sv)));
+      *reinterpret_cast<unsigned short*>(kp + j) = kc;
+      vp[static_cast<int64_t>(j) * bs] = static_cast<uint8_t>(vc & 0xff);
+      vp[static_cast<int64_t>(j + 1) * bs] = static_cast<uint8_t>(vc >> 8);
+    }
+  }
+  if (threadIdx.x == 0) context_lens[s] = L + 1;
+}
+
+// ------------------------------------------------------------------------------------------
+// Split-combine: block i merges the unit that started in span i and ran past its end.  The
+// pieces live in the following spans (slot 0 of each follower), merged in ascending token order:
+//   M = max m_c;  Lsum = sum l_c 2^(m_c - M);  out = bf16( sum acc_c 2^(m_c - M) / Lsum ).
+// Block 0 also rearms the run-time span counter for the next call.
+// ------------------------------------------------------------------------------------------
+template <int D, int NT>
+__global__ void __launch_bounds__(256)
+combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, const float* __restrict__ partials,
+               __nv_bfloat16* __restrict__ out, int Hq, int Hkv, int G, const int32_t* __restrict__ start_tiles,
+               const float* __restrict__ pfx_partials, int T) {
+  constexpr int HP = 8 * NT;
+  constexpr int SLOT_FLOATS = HP * (D + 2);
+  const int c = blockIdx.x;
+  // launched as a programmatic dependent of the decode kernel: nothing of that kernel may be read
+  // before this returns (it waits for the kernel's completion and memory flush)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (c == 0 && threadIdx.x == 0) hdr->counter = 0;
+  const int n_spans = n_spans_host >= 0 ? n_spans_host : hdr->plan.n_static + hdr->plan.n_dyn;
+  if (c >= n_spans) return;
+  const int4 r = rec[c];
+  const int unit = r.z;
+  if (unit < 0) return;
+  // followers: later spans whose first piece continues `unit` (spans without tiles may sit between)
+  __shared__ int n_follow;
+  __shared__ int follow[MAX_SPANS];
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int cc = c + 1; cc < n_spans; ++cc) {
+      const int4 rr = rec[cc];
+      if (rr.x < 0) continue;                 // a span that holds no tile
+      if (rr.x != unit || rr.y <= 0) break;
+      follow[n++] = cc;
+    }
+    n_follow = n;
+  }
+  __syncthreads();
+  const int np = n_follow + 1;
+  const int s = unit / Hkv, g = unit - s * Hkv;
+  // piece -1: the partial of the unit's leading tiles when those were handled elsewhere (shared prefix)
+  const int p0 = (start_tiles && start_tiles[s] > 0) ? -1 : 0;
+  auto piece = [&](int p) -> const float* {
+    if (p < 0) return pfx_partials + static_cast<int64_t>(unit) * SLOT_FLOATS;
+    return partials + (p == 0 ? static_cast<int64_t>(c) * 2 + r.w : static_cast<int64_t>(follow[p - 1]) * 2) * SLOT_FLOATS;
+  };
+  const float NEG_INF = __int_as_float(0xff800000);
+  for (int idx = threadIdx.x; idx < HP * (D / 4); idx += blockDim.x) {
+    const int h = idx / (D / 4);
+    const int dq = idx % (D / 4);
+    if (h >= G * T) continue;   // row h = query token * G + head
+    float M = NEG_INF;
+    for (int p = p0; p < np; ++p) M = fmaxf(M, piece(p)[h]);
+    const float Mu = (M == NEG_INF) ? 0.f : M;
+    float Ls = 0.f;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = p0; p < np; ++p) {
+      const float* part = piece(p);
+      const float f = fast_exp2(part[h] - Mu);
+      Ls += part[HP + h] * f;
+      const float4 v = *reinterpret_cast<const float4*>(part + 2 * HP + h * D + dq * 4);
+      a.x += v.x * f;
+      a.y += v.y * f;
+      a.z += v.z * f;
+      a.w += v.w * f;
+    }
+    const float inv = Ls > 0.f ? 1.f / Ls : 0.f;
+    uint2 o;
+    o.x = pack_bf16x2(a.x * inv, a.y * inv);
+    o.y = pack_bf16x2(a.z * inv, a.w * inv);
+    const int qtok = h / G;
+    *reinterpret_cast<uint2*>(out + ((static_cast<int64_t>(s) * T + qtok) * Hq + g * G + (h - qtok * G)) * D + dq * 4) = o;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Device twin of the host partitioner (one block).  prefix: [2 * (S + 1)] ints of scratch:
+// running cost, then running tile count, per sequence.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int block_scan_1024(int v, int* warp_sums, int lane, int wid) {
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) warp_sums[wid] = x;
+  __syncthreads();
+  if (wid == 0) {
+    int w = warp_sums[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += y;
+    }
+    warp_sums[lane] = w;
+  }
+  __syncthreads();
+  const int incl = x + (wid > 0 ? warp_sums[wid - 1] : 0);
+  __syncthreads();
+  return incl;
+}
+
+__global__ void __launch_bounds__(1024)
+plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict__ start_tiles, int S, int Hkv,
+            int n_static, int n_dyn_max, int32_t* __restrict__ prefix, SpanStart* __restrict__ spans, WsHeader* hdr) {
+  __shared__ int warp_sums[32];
+  __shared__ int carry_c, carry_t;
+  __shared__ PlanParams pp_s;
+  int32_t* pcost = prefix;
+  int32_t* ptile = prefix + (S + 1);
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) {
+    carry_c = carry_t = 0;
+    pcost[0] = ptile[0] = 0;
+  }
+  __syncthreads();
+  for (int base = 0; base < S; base += 1024) {
+    const int s = base + tid;
+    int nt = 0;
+    if (s < S) nt = static_cast<int>(seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0));
+    const int ic = block_scan_1024(static_cast<int>(seq_cost(nt, Hkv)), warp_sums, lane, wid) + carry_c;
+    const int itl = block_scan_1024(nt * Hkv, warp_sums, lane, wid) + carry_t;
+    if (s < S) {
+      pcost[s + 1] = ic;
+      ptile[s + 1] = itl;
+    }
+    __syncthreads();
+    if (tid == 1023) {
+      carry_c = ic;
+      carry_t = itl;
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    pp_s = make_plan_params(carry_c, carry_t, n_static, n_dyn_max);
+    hdr->plan = pp_s;
+  }
+  __threadfence_block();
+  __syncthreads();
+  const PlanParams pp = pp_s;
+  const int n_spans = pp.n_static + pp.n_dyn;
+  const int total_cost = static_cast<int>(pp.cost_total);
+  for (int c = tid; c <= n_spans; c += 1024) {
+    SpanStart sp;
+    sp.unit = S * Hkv;
+    sp.tile = 0;
+    sp.flat = pp.total;
+    sp.pad = 0;
+    const int x = static_cast<int>(span_cost_start(pp, c));
+    if (c < n_spans && x < total_cost) {
+      int lo = 0, hi = S;   // find s with pcost[s] <= x < pcost[s+1]
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pcost[mid] <= x) lo = mid; else hi = mid;
+      }
+      const int nt = static_cast<int>(seq_tiles(context_lens[lo], start_tiles ? start_tiles[lo] : 0));
+      int k, tile;
+      locate_in_seq(x - pcost[lo], nt, &k, &tile);
+      sp.unit = lo * Hkv + k;
+      sp.tile = tile;
+      sp.flat = ptile[lo] + k * nt + tile;
+    }
+    spans[c] = sp;
+  }
+}
+
+}  // namespace pdattn
