@@ -330,6 +330,15 @@ pdattn_status pdattn_profile_events(void* start_event, void* stop_event);
 pdattn_status pdattn_gather_probe(const pdattn_args* args, pdattn_stream_t stream);
 pdattn_status pdattn_stream_read_probe(const void* src, size_t bytes, void* sink, pdattn_stream_t stream);
 
+/*
+ * Self-test of the kernels' failure path (no paper counterpart).  Every wait inside the kernels is bounded:
+ * when a wait expires, the CTA sets the DEVICE_TIMEOUT bit of the workspace's error word and returns.
+ * This call enqueues one warp that waits, for at most limit_us microseconds (1 .. 1,000,000), on a barrier
+ * that nothing arrives on; afterwards pdattn_check(workspace) returns PDATTN_DEVICE_TIMEOUT once, and the
+ * context and the workspace remain usable.
+ */
+pdattn_status pdattn_wait_limit_probe(void* workspace, int limit_us, pdattn_stream_t stream);
+
 /* Number of kernels the last pdattn_decode_ex on this thread launched (2 or 3). */
 int pdattn_last_launch_count(void);
 

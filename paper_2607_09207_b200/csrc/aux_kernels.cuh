@@ -271,4 +271,28 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever arrive on, with the
+// given limit, and reports the expiry through the workspace's sticky error word exactly as the kernels
+// do.  The context stays usable: the kernel returns normally.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32)
+wait_limit_probe_kernel(int32_t* err, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+  const uint32_t b = smem_u32(&bar);
+  bool done = mbar_try_wait(b, 0);
+  const unsigned long long t0 = globaltimer_ns();
+  while (!done) {
+    if (globaltimer_ns() - t0 > limit_ns) break;
+#pragma unroll 1
+    for (int i = 0; i < 16 && !done; ++i) done = mbar_try_wait_hint(b, 0, 1000);
+  }
+  if (!done && threadIdx.x == 0) atomicOr(err, ERR_TIMEOUT);
+}
+
 }  // namespace pdattn

@@ -1020,6 +1020,15 @@ pdattn_status pdattn_gather_probe(const pdattn_args* args, pdattn_stream_t strea
   return s;
 }
 
+pdattn_status pdattn_wait_limit_probe(void* workspace, int limit_us, pdattn_stream_t stream) {
+  if (!workspace || limit_us < 1 || limit_us > 1000000) return PDATTN_INVALID_ARG;
+  wait_limit_probe_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      &static_cast<WsHeader*>(workspace)->err, static_cast<unsigned long long>(limit_us) * 1000ull);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail("wait_limit_probe_kernel launch", e);
+  return PDATTN_OK;
+}
+
 pdattn_status pdattn_stream_read_probe(const void* src, size_t bytes, void* sink, pdattn_stream_t stream) {
   if (!src || !sink || (reinterpret_cast<uintptr_t>(src) & 15)) return PDATTN_INVALID_ARG;
   int dev = 0;

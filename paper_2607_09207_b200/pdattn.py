@@ -30,7 +30,7 @@ EXPORTS = [
     "pdattn_workspace_size", "pdattn_workspace_init", "pdattn_decode_ex", "pdattn_bind", "pdattn_decode",
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
-    "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_set_dynamic_spans",
+    "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_wait_limit_probe", "pdattn_set_dynamic_spans",
     "pdattn_set_merge_mode", "pdattn_set_prefix_engine",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
@@ -104,6 +104,7 @@ def lib():
         L.pdattn_profile_events.argtypes = [vp, vp]
         L.pdattn_gather_probe.argtypes = [ctypes.POINTER(Args), vp]
         L.pdattn_stream_read_probe.argtypes = [vp, sz, vp, vp]
+        L.pdattn_wait_limit_probe.argtypes = [vp, i32, vp]
         L.pdattn_last_launch_count.argtypes = []
         L.pdattn_status_string.argtypes = [i32]
         L.pdattn_status_string.restype = ctypes.c_char_p
@@ -406,6 +407,11 @@ def set_prefix_engine(engine: int):
     st = lib().pdattn_set_prefix_engine(engine)
     if st != OK:
         raise PdattnError(st, "pdattn_set_prefix_engine")
+
+
+def wait_limit_probe(workspace, limit_us: int, stream=None) -> int:
+    """One warp waits limit_us microseconds on a barrier nothing arrives on, then raises the timeout bit."""
+    return lib().pdattn_wait_limit_probe(workspace.data_ptr(), int(limit_us), _stream_ptr(stream))
 
 
 def plan_host(context_lens_host, num_kv_heads, n_ctas, dynamic_per_cta=0, max_spans=None):

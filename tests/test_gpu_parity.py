@@ -450,3 +450,23 @@ def test_page_sizes_32_and_64_and_wide_gqa_groups():
     for bs in (32, 64):
         wb = W.make_custom(w.context_lens_host, Hq=28, Hkv=4, d=128, bs=bs, seed=77, device=DEV)
         check_against_oracle(wb, f"7B-shaped lengths, page size {bs}")
+
+
+def test_an_expired_wait_is_reported_and_leaves_the_context_usable():
+    """Failure path without a fault: a wait that nothing satisfies runs into its limit (2 ms here), the
+    kernel sets the timeout bit and returns; the check reports it once; the next decode step is fine."""
+    w = W.make_config(1, device=DEV)
+    ws = pdattn.alloc_workspace(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim)
+    ref, st = run(w, ws=ws)
+    assert st == pdattn.OK
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    assert pdattn.wait_limit_probe(ws, 2000) == pdattn.OK
+    t1.record()
+    assert pdattn.check(ws) == pdattn.DEVICE_TIMEOUT
+    assert 1.5 < t0.elapsed_time(t1) < 200.0                       # it waited about its limit, not forever
+    assert pdattn.check(ws) == pdattn.OK                           # the word is sticky until read, then clear
+    out, st = run(w, ws=ws)
+    assert st == pdattn.OK and torch.equal(out, ref)
+    assert pdattn.wait_limit_probe(ws, 0) == pdattn.INVALID_ARG
