@@ -4,7 +4,7 @@ kernel) over one rollout batch, through the C ABI.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--cfg 2]
 
-Workload: benchmark configs[1], the 7B-shaped rollout step (256 sequences, 28 q heads / 4 KV
+Workload: the benchmark's second configuration, the 7B-shaped rollout step (256 sequences, 28 q heads / 4 KV
 heads, head_dim 128, page size 16, context = 512-token prompt + lognormal response), synthetic and
 seeded.  With N > 1 (torchrun, one rank per GPU) every rank runs its own batch of that shape
 (sequences are independent: no collective on the data path) and the value is the sum over ranks
@@ -51,7 +51,7 @@ def parse():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cfg", type=int, default=2, help="BASELINE.json config index + 1 (default: the metric's config)")
+    ap.add_argument("--cfg", type=int, default=2, help="benchmark configuration, 1-based (default 2: the one the metric is quoted on)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--fp8", action="store_true",
                     help="time pdattn_decode_fp8 over an e4m3 copy of the same pools (half the KV bytes per step) "
