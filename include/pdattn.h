@@ -251,9 +251,11 @@ pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, i
                                pdattn_plan* plan);
 
 /*
- * Process-wide tuning of the partitioner above: at most `per_cta` run-time spans per CTA
- * (0..8; 0 = every span is static, the default).  Results stay bit-identical from run to run
- * for a given setting; different settings cut sequences at different tiles.
+ * Process-wide tuning of the partitioner above: at most `per_cta` run-time spans per CTA (0..8; 0 = every
+ * span is static).  -1 (default): 4 when the batch has at least 4 units (sequence x KV head) per CTA, else 0 --
+ * run-time spans even out the finishing times of the CTAs when there are many units, and only lengthen
+ * the merge of cut sequences when there are few long ones.  Results stay bit-identical from run to run for
+ * a given setting and batch shape; different settings cut sequences at different tiles.
  */
 pdattn_status pdattn_set_dynamic_spans(int per_cta);
 

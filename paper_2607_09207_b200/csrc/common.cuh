@@ -348,8 +348,8 @@ __device__ __forceinline__ int read_span(Ctrl* ctrl, int k, bool& aborted) {
   }
   const int slot = (k - 1) % SPAN_QUEUE;
   const int id = ctrl->sq_id[slot];
-  if (ctrl->sq_tag[slot] != k) {   // the queue wrapped past a reader: cannot happen while warps stay
-    aborted = true;                //  within a ring's worth of tiles of each other; fail loudly if it does
+  if (ctrl->sq_tag[slot] != k) {   // the queue wrapped past a reader: cannot happen while a CTA draws fewer
+    aborted = true;                //  run-time spans than the queue has entries; fail loudly if it does
     return -1;
   }
   return id;

@@ -30,7 +30,9 @@ struct GroupedCall {                      // set only inside pdattn_decode_group
 };
 thread_local GroupedCall g_grouped;
 thread_local std::vector<int32_t> g_start_tiles_host;
-int g_dyn_per_cta = 0;                    // run-time spans per CTA (pdattn_set_dynamic_spans)
+int g_dyn_per_cta = -1;                   // run-time spans per CTA (pdattn_set_dynamic_spans); -1: by batch shape
+constexpr int kAutoDynPerCta = 4;         // ... then this many when the batch has at least kAutoDynUnits units per CTA
+constexpr int kAutoDynUnits = 4;
 int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (chained), 0 barrier, 1 chained
 thread_local bool g_use_chain = true;     // decided per call, read by the launcher
 struct Fp8Call {
@@ -421,7 +423,7 @@ pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cac
 }
 
 pdattn_status pdattn_set_dynamic_spans(int per_cta) {
-  if (per_cta < 0 || per_cta > kMaxDynPerCta) return PDATTN_INVALID_ARG;
+  if (per_cta < -1 || per_cta > kMaxDynPerCta) return PDATTN_INVALID_ARG;
   g_dyn_per_cta = per_cta;
   return PDATTN_OK;
 }
@@ -558,7 +560,12 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
 
   int n_ctas = di->sm_count;
   if (n_ctas > MAX_SPANS / (1 + kMaxDynPerCta)) n_ctas = MAX_SPANS / (1 + kMaxDynPerCta);
-  const int dyn_per_cta = g_dyn_per_cta;
+  // Run-time spans even out the CTAs' finishing times when there are many units; with few long sequences
+  // they only lengthen the chains the combine kernel walks.  The choice depends on the batch shape alone.
+  const int dyn_per_cta = g_dyn_per_cta >= 0 ? g_dyn_per_cta
+                          : (static_cast<int64_t>(a->num_seqs) * a->num_kv_heads >= static_cast<int64_t>(kAutoDynUnits) * n_ctas
+                                 ? kAutoDynPerCta
+                                 : 0);
   int grid = n_ctas, combine_grid = 0, n_spans_host = -1;
   if (a->context_lens_host) {
     if (!plan_spans(a->context_lens_host, start_tiles_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta,
@@ -597,8 +604,7 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
                a->kv_head_stride, a->kv_token_stride, fp8 ? kMapV8 : rank, &mv);
   if (s != PDATTN_OK) return s;
   P.box5d = rank == 5;
-  // run-time spans assume warps that stay within a ring of each other: barrier merge there
-  g_use_chain = g_merge_mode != 0 && dyn_per_cta == 0;
+  g_use_chain = g_merge_mode != 0;
 
   if (grouped) {
     // shared prompt tiles first: one pass per (group, kv head) for the query rows of all samples

@@ -53,8 +53,10 @@ def test_tuning_setters_check_their_ranges():
     for mode in (-2, 2, 100):
         assert L.pdattn_set_merge_mode(mode) == pdattn.INVALID_ARG
     L.pdattn_set_merge_mode(-1)
-    assert L.pdattn_set_dynamic_spans(-1) == pdattn.INVALID_ARG
+    assert L.pdattn_set_dynamic_spans(-2) == pdattn.INVALID_ARG
+    assert L.pdattn_set_dynamic_spans(9) == pdattn.INVALID_ARG
     assert L.pdattn_set_dynamic_spans(0) == pdattn.OK
+    assert L.pdattn_set_dynamic_spans(-1) == pdattn.OK
 
 
 def test_workspace_size_and_shape_checks():

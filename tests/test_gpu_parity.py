@@ -421,7 +421,7 @@ def test_workspace_too_small_and_misaligned_are_rejected_on_gpu():
 def runtime_spans():
     pdattn.set_dynamic_spans(8)
     yield
-    pdattn.set_dynamic_spans(0)
+    pdattn.set_dynamic_spans(-1)
 
 
 @pytest.mark.parametrize("cfg,num_seqs,len_div", [(2, 48, 1), (5, 2, 2), (3, 24, 2)])
@@ -470,3 +470,15 @@ def test_an_expired_wait_is_reported_and_leaves_the_context_usable():
     out, st = run(w, ws=ws)
     assert st == pdattn.OK and torch.equal(out, ref)
     assert pdattn.wait_limit_probe(ws, 0) == pdattn.INVALID_ARG
+
+
+@pytest.mark.parametrize("per_cta", [0, 2])
+def test_full_config2_with_a_fixed_number_of_runtime_spans(per_cta):
+    """The default picks the number of run-time spans from the batch shape (4 per CTA here); static spans only
+    and another count must give the same attention within tolerance (the cuts differ, so not the same bits)."""
+    w = W.make_config(2, device=DEV)
+    pdattn.set_dynamic_spans(per_cta)
+    try:
+        check_against_oracle(w, f"config 2, {per_cta} run-time spans per CTA", pairs=sample_pairs(w, 24, seed=31))
+    finally:
+        pdattn.set_dynamic_spans(-1)
