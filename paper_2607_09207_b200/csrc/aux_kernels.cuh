@@ -128,18 +128,42 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
   const int4 r = rec[c];
   const int unit = r.z;
   if (unit < 0) return;
-  // followers: later spans whose first piece continues `unit` (spans without tiles may sit between)
-  __shared__ int n_follow;
+  // followers: later spans whose first piece continues `unit` (spans without tiles may sit between).
+  // The block looks at blockDim.x span records at a time instead of walking them one dependent load after
+  // the other: a long sequence can be cut by hundreds of spans.
+  __shared__ int n_follow, first_break;
   __shared__ int follow[MAX_SPANS];
-  if (threadIdx.x == 0) {
-    int n = 0;
-    for (int cc = c + 1; cc < n_spans; ++cc) {
-      const int4 rr = rec[cc];
-      if (rr.x < 0) continue;                 // a span that holds no tile
-      if (rr.x != unit || rr.y <= 0) break;
-      follow[n++] = cc;
+  if (threadIdx.x == 0) n_follow = 0;
+  for (int base = c + 1; base < n_spans; base += blockDim.x) {
+    if (threadIdx.x == 0) first_break = blockDim.x;
+    __syncthreads();
+    const int cc = base + threadIdx.x;
+    int4 rr = make_int4(-1, 0, 0, 0);
+    if (cc < n_spans) rr = rec[cc];
+    const bool past_end = cc >= n_spans;
+    const bool empty = !past_end && rr.x < 0;                      // a span that holds no tile
+    const bool cont = !past_end && rr.x == unit && rr.y > 0;       // its first piece continues the unit
+    if (past_end || (!empty && !cont)) atomicMin(&first_break, static_cast<int>(threadIdx.x));
+    __syncthreads();
+    const int fb = first_break;
+    // compact the continuing spans below the break, in order
+    const bool take = cont && static_cast<int>(threadIdx.x) < fb;
+    const int lane_id = threadIdx.x & 31, warp_id = threadIdx.x >> 5;
+    __shared__ int warp_count[32];
+    const uint32_t bal = __ballot_sync(0xffffffffu, take);
+    if (lane_id == 0) warp_count[warp_id] = __popc(bal);
+    __syncthreads();
+    int before = n_follow;
+    for (int w = 0; w < warp_id; ++w) before += warp_count[w];
+    if (take) follow[before + __popc(bal & ((1u << lane_id) - 1u))] = cc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int tot = 0;
+      for (int w = 0; w < static_cast<int>(blockDim.x) / 32; ++w) tot += warp_count[w];
+      n_follow += tot;
     }
-    n_follow = n;
+    __syncthreads();
+    if (fb < static_cast<int>(blockDim.x)) break;
   }
   __syncthreads();
   const int np = n_follow + 1;
@@ -156,10 +180,12 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
     const int dq = idx % (D / 4);
     if (h >= G * T) continue;   // row h = query token * G + head
     float M = NEG_INF;
-    for (int p = p0; p < np; ++p) M = fmaxf(M, piece(p)[h]);
+#pragma unroll 8
+    for (int p = p0; p < np; ++p) M = fmaxf(M, piece(p)[h]);   // independent loads: many in flight
     const float Mu = (M == NEG_INF) ? 0.f : M;
     float Ls = 0.f;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
     for (int p = p0; p < np; ++p) {
       const float* part = piece(p);
       const float f = fast_exp2(part[h] - Mu);
