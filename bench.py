@@ -453,8 +453,10 @@ def main():
                          "pct_of_8tbs_nominal": achieved / 8000.0 * 100.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": ke, "note": ("bf16 step (pdattn_decode_host has no fp8 form); " if fp8 is not None else "")
-                                         + "q/block_table/context_lens from pinned host memory, out read back "
-                                         "and the stream synchronised every step; KV pools are resident state"},
+                                         + "q/block_table/context_lens in pinned host memory, out in pinned host memory "
+                                         "and the stream synchronised every step: block_table and context_lens are "
+                                         "copied, q rows are fetched and out rows written over the bus by the kernels "
+                                         "themselves (same bytes, off the critical path); KV pools are resident state"},
             "gpu_launches": launches_per_step * K,
             "clocks": sampler.summary(),
             "cpu_baseline": cpu_baseline,

@@ -217,7 +217,12 @@ pdattn_status pdattn_decode(const void* q, const void* k_cache, const void* v_ca
  * pdattn_decode_ex (host partitioner on context_lens_host = the given lengths), copies `out`
  * back.  All on `stream`; the caller synchronises.  The KV pools are resident device state.
  * staging: DEVICE, >= pdattn_host_staging_size() bytes, 256-byte aligned.
+ * When q_host and out_host are both pinned, mapped host memory (cudaHostAlloc / cudaHostRegister; 16-byte
+ * aligned) the kernels read q and write out in place over the bus instead of through the two copies --
+ * same results bit for bit; out_host is complete once `stream` has been synchronised.
+ * pdattn_set_host_zero_copy(0) always takes the copies; -1 (default) and 1: in place when possible.
  */
+pdattn_status pdattn_set_host_zero_copy(int mode);
 pdattn_status pdattn_host_staging_size(int num_seqs, int num_q_heads, int head_dim,
                                        int max_blocks_per_seq, size_t* device_bytes);
 pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_host,

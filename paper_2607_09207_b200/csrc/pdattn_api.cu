@@ -42,6 +42,7 @@ struct Fp8Call {
 };
 thread_local Fp8Call g_fp8;               // set by pdattn_decode_fp8 around the common path
 thread_local int g_query_tokens = 1;      // query tokens per sequence of the call (pdattn_decode_multi)
+int g_host_zero_copy = -1;                // pdattn_set_host_zero_copy: -1 default (when possible), 0 never, 1 as -1
 int g_prefix_engine = -1;                 // pdattn_set_prefix_engine: -1 default (tcgen05), 0 warp MMAs, 1 tcgen05
 
 struct Binding {
@@ -794,6 +795,22 @@ pdattn_status pdattn_host_staging_size(int num_seqs, int num_q_heads, int head_d
   return PDATTN_OK;
 }
 
+pdattn_status pdattn_set_host_zero_copy(int mode) {
+  if (mode < -1 || mode > 1) return PDATTN_INVALID_ARG;
+  g_host_zero_copy = mode;
+  return PDATTN_OK;
+}
+
+// The device-side address of pinned, mapped host memory (null for pageable or unknown memory).
+static void* mapped_host_pointer(const void* p) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_host,
                                  const int32_t* context_lens_host, void* out_host, const void* k_cache,
                                  const void* v_cache, int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
@@ -816,8 +833,21 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
   void* out_dev = st + align_up(q_bytes, 256);
   void* bt_dev = st + 2 * align_up(q_bytes, 256);
   void* len_dev = st + 2 * align_up(q_bytes, 256) + align_up(t_bytes, 256);
+  // q is read once and out written once per step: when both are pinned and mapped the kernels use them
+  // in place (query rows arrive by bulk copy a few units ahead of their use, output rows are posted
+  // writes), which takes both transfers out of the step's critical path
+  bool in_place = false;
+  if (g_host_zero_copy != 0) {
+    void* qm = mapped_host_pointer(q_host);
+    void* om = mapped_host_pointer(out_host);
+    if (qm && om && !(reinterpret_cast<uintptr_t>(qm) & 15) && !(reinterpret_cast<uintptr_t>(om) & 15)) {
+      q_dev = qm;
+      out_dev = om;
+      in_place = true;
+    }
+  }
   cudaError_t e;
-  if ((e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+  if (!in_place && (e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
     return cuda_fail("cudaMemcpyAsync(q)", e);
   if ((e = cudaMemcpyAsync(bt_dev, block_table_host, t_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
     return cuda_fail("cudaMemcpyAsync(block_table)", e);
@@ -847,7 +877,7 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
   a.workspace_bytes = workspace_bytes;
   s = pdattn_decode_ex(&a, stream_);
   if (s != PDATTN_OK) return s;
-  if ((e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+  if (!in_place && (e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
     return cuda_fail("cudaMemcpyAsync(out)", e);
   return PDATTN_OK;
 }

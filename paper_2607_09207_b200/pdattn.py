@@ -31,7 +31,7 @@ EXPORTS = [
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_wait_limit_probe", "pdattn_set_dynamic_spans",
-    "pdattn_set_merge_mode", "pdattn_set_prefix_engine",
+    "pdattn_set_merge_mode", "pdattn_set_prefix_engine", "pdattn_set_host_zero_copy",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
     "pdattn_multi_workspace_size", "pdattn_decode_multi", "pdattn_decode_fp8", "pdattn_append_kv_fp8", "pdattn_decode_fp8_multi",
@@ -91,6 +91,7 @@ def lib():
         L.pdattn_set_dynamic_spans.argtypes = [i32]
         L.pdattn_set_merge_mode.argtypes = [i32]
         L.pdattn_set_prefix_engine.argtypes = [i32]
+        L.pdattn_set_host_zero_copy.argtypes = [i32]
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
         L.pdattn_grouped_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_grouped.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
@@ -407,6 +408,13 @@ def set_prefix_engine(engine: int):
     st = lib().pdattn_set_prefix_engine(engine)
     if st != OK:
         raise PdattnError(st, "pdattn_set_prefix_engine")
+
+
+def set_host_zero_copy(mode: int):
+    """-1 / 1: decode_host uses pinned, mapped q and out in place; 0: always through the staging copies."""
+    st = lib().pdattn_set_host_zero_copy(mode)
+    if st != OK:
+        raise PdattnError(st, "pdattn_set_host_zero_copy")
 
 
 def wait_limit_probe(workspace, limit_us: int, stream=None) -> int:

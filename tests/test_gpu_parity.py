@@ -400,9 +400,20 @@ def test_short_form_with_binding_and_host_buffer_form():
     oh = torch.empty_like(qh).pin_memory()
     staging = torch.empty(pdattn.host_staging_size(w.num_seqs, 28, 128, w.max_blocks_per_seq), dtype=torch.uint8,
                           device=DEV)
-    pdattn.decode_host(qh, bth, lh, oh, w.k_cache, w.v_cache, w.scale, staging, ws)
-    torch.cuda.synchronize()
-    assert torch.equal(ref.cpu(), oh)
+    try:
+        for mode in (0, 1):     # through the staging copies; pinned q and out used in place by the kernels
+            pdattn.set_host_zero_copy(mode)
+            oh.fill_(float("nan"))
+            pdattn.decode_host(qh, bth, lh, oh, w.k_cache, w.v_cache, w.scale, staging, ws)
+            torch.cuda.synchronize()
+            assert pdattn.check(ws) == pdattn.OK and torch.equal(ref.cpu(), oh)
+        # pageable q and out: the in-place form does not apply and the copies are taken
+        qp, op = w.q.cpu(), torch.full_like(w.q.cpu(), float("nan"))
+        pdattn.decode_host(qp, bth, lh, op, w.k_cache, w.v_cache, w.scale, staging, ws)
+        torch.cuda.synchronize()
+        assert pdattn.check(ws) == pdattn.OK and torch.equal(ref.cpu(), op)
+    finally:
+        pdattn.set_host_zero_copy(-1)
 
 
 def test_workspace_too_small_and_misaligned_are_rejected_on_gpu():
