@@ -17,6 +17,7 @@ append_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __re
               int MB, int NB, int64_t sb, int64_t sh, int64_t st, int32_t* err) {
   const int s = blockIdx.x;
   const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // a programmatic dependent of the kernel before it on the stream
   const int L = context_lens[s];
   __syncthreads();                       // every warp has read the old length before it is advanced
   if (L < 0 || L / bs >= MB) {
@@ -74,6 +75,7 @@ append_fp8_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* 
                   int32_t* __restrict__ context_lens, int Hkv, int D, int bs, int MB, int NB, int32_t* err) {
   const int s = blockIdx.x;
   const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // a programmatic dependent of the kernel before it on the stream
   const int L = context_lens[s];
   __syncthreads();                       // every warp has read the old length before it is advanced
   if (L < 0 || L / bs >= MB) {
@@ -242,6 +244,9 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
   int32_t* pcost = prefix;
   int32_t* ptile = prefix + (S + 1);
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  // launched as a programmatic dependent of whatever precedes it on the stream (the KV append in a decode
+  // loop): nothing may be read or written before that kernel has completed and flushed
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid == 0) {
     carry_c = carry_t = 0;
     pcost[0] = ptile[0] = 0;

@@ -244,6 +244,24 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
 }
 
 // ---- launches ------------------------------------------------------------------------------------
+// Launch that may begin while the kernel before it on the stream drains (programmatic dependent launch); the
+// kernel itself waits (griddepcontrol.wait) before it touches global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, bool dependent,
+                             Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <int D, int NT, int BS>
 pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
                      int n_spans_host, DevInfo* di, cudaStream_t stream) {
@@ -266,6 +284,8 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
     if (pe != cudaSuccess) return cuda_fail("cudaMemsetAsync", pe);
     return PDATTN_OK;
   }
+  // behind a device-side plan the kernel starts while plan_kernel runs (and waits for it inside)
+  const bool after_plan = P.use_ws_plan && g_prof_start == nullptr;
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
   if (g_fp8.active) {
     if constexpr (D == 128) {
@@ -277,7 +297,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
         if (fe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", fe);
         fdone = true;
       }
-      k8<<<grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream>>>(mk, mv, P);
+      launch_dependent(k8, grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream, after_plan, mk, mv, P);
     } else {
       return PDATTN_UNSUPPORTED;
     }
@@ -289,9 +309,9 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
       if (ce != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", ce);
       cdone = true;
     }
-    chain<<<grid, C::NTHREADS, C::CHAIN_DYN_BYTES, stream>>>(mk, mv, P);
+    launch_dependent(chain, grid, C::NTHREADS, C::CHAIN_DYN_BYTES, stream, after_plan, mk, mv, P);
   } else {
-    kern<<<grid, C::NTHREADS, C::DYN_BYTES, stream>>>(mk, mv, P);
+    launch_dependent(kern, grid, C::NTHREADS, C::DYN_BYTES, stream, after_plan, mk, mv, P);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
@@ -413,12 +433,12 @@ pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cac
   if ((kv_block_stride | kv_head_stride | kv_token_stride) % 8 != 0) return PDATTN_UNSUPPORTED;
   auto mis = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; };
   if (mis(k_new) || mis(v_new) || mis(k_cache) || mis(v_cache)) return PDATTN_MISALIGNED;
-  append_kernel<<<num_seqs, 32 * num_kv_heads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+  cudaError_t e = launch_dependent(
+      append_kernel, num_seqs, 32 * num_kv_heads, 0, reinterpret_cast<cudaStream_t>(stream), true,
       static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
       static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache), block_table, context_lens,
       num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks, kv_block_stride, kv_head_stride,
       kv_token_stride, static_cast<int32_t*>(workspace));
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("append_kernel launch", e);
   return PDATTN_OK;
 }
@@ -442,11 +462,11 @@ pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k
     return PDATTN_INVALID_ARG;
   auto mis = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; };
   if (mis(k_new) || mis(v_new) || mis(k_cache) || mis(v_cache)) return PDATTN_MISALIGNED;
-  append_fp8_kernel<<<num_seqs, 32 * num_kv_heads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+  cudaError_t e = launch_dependent(
+      append_fp8_kernel, num_seqs, 32 * num_kv_heads, 0, reinterpret_cast<cudaStream_t>(stream), true,
       static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
       static_cast<uint8_t*>(k_cache), static_cast<uint8_t*>(v_cache), k_scale, v_scale, block_table, context_lens,
       num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks, static_cast<int32_t*>(workspace));
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("append_fp8_kernel launch", e);
   return PDATTN_OK;
 }
@@ -578,10 +598,10 @@ pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
     P.use_ws_plan = 1;
     memset(&P.plan, 0, sizeof P.plan);
     const int n_dyn_max = n_ctas * dyn_per_cta;
-    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, nullptr, a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
-                                         reinterpret_cast<int32_t*>(ws + wl.prefix),
-                                         reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_dependent(plan_kernel, 1, 1024, 0, stream, true, a->context_lens,
+                                     static_cast<const int32_t*>(nullptr), a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
+                                     reinterpret_cast<int32_t*>(ws + wl.prefix),
+                                     reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr);
     if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
     g_last_launches += 1;
     combine_grid = n_ctas + n_dyn_max;
@@ -1009,10 +1029,9 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   } else {
     P.use_ws_plan = 1;
     memset(&P.plan, 0, sizeof P.plan);
-    plan_kernel<<<1, 1024, 0, stream>>>(a->context_lens, nullptr, a->num_seqs, a->num_kv_heads, n_ctas, 0,
-                                         reinterpret_cast<int32_t*>(ws + off_prefix),
-                                         reinterpret_cast<SpanStart*>(ws + off_spans), P.hdr);
-    e = cudaGetLastError();
+    e = launch_dependent(plan_kernel, 1, 1024, 0, stream, true, a->context_lens, static_cast<const int32_t*>(nullptr),
+                         a->num_seqs, a->num_kv_heads, n_ctas, 0, reinterpret_cast<int32_t*>(ws + off_prefix),
+                         reinterpret_cast<SpanStart*>(ws + off_spans), P.hdr);
     if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
     g_last_launches += 1;
   }
