@@ -379,9 +379,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   }
   __syncthreads();
 
-  // With a device-side plan this kernel is a programmatic dependent of plan_kernel: its set-up above runs
-  // while that kernel works; nothing in global memory is touched before it has completed and flushed.
-  if (P.use_ws_plan) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // This kernel is launched as a programmatic dependent of whatever precedes it on the stream (plan_kernel
+  // with a device-side plan, else the previous step's last kernel): its set-up above runs while that kernel
+  // drains; nothing in global memory is touched before it has completed and flushed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const PlanParams pp = P.use_ws_plan ? P.hdr->plan : P.plan;
   const int nunits = P.S * P.Hkv;
   int it = 0;        // tile counter within this CTA: tile `it` uses ring slot it % NST

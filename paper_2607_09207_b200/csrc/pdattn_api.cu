@@ -284,8 +284,8 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
     if (pe != cudaSuccess) return cuda_fail("cudaMemsetAsync", pe);
     return PDATTN_OK;
   }
-  // behind a device-side plan the kernel starts while plan_kernel runs (and waits for it inside)
-  const bool after_plan = P.use_ws_plan && g_prof_start == nullptr;
+  // the kernel may be set up while its predecessor on the stream drains (and waits for it inside)
+  const bool dependent = g_prof_start == nullptr;
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
   if (g_fp8.active) {
     if constexpr (D == 128) {
@@ -297,7 +297,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
         if (fe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", fe);
         fdone = true;
       }
-      launch_dependent(k8, grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream, after_plan, mk, mv, P);
+      launch_dependent(k8, grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream, dependent, mk, mv, P);
     } else {
       return PDATTN_UNSUPPORTED;
     }
@@ -309,9 +309,9 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
       if (ce != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", ce);
       cdone = true;
     }
-    launch_dependent(chain, grid, C::NTHREADS, C::CHAIN_DYN_BYTES, stream, after_plan, mk, mv, P);
+    launch_dependent(chain, grid, C::NTHREADS, C::CHAIN_DYN_BYTES, stream, dependent, mk, mv, P);
   } else {
-    launch_dependent(kern, grid, C::NTHREADS, C::DYN_BYTES, stream, after_plan, mk, mv, P);
+    launch_dependent(kern, grid, C::NTHREADS, C::DYN_BYTES, stream, dependent, mk, mv, P);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("decode_kernel launch", e);
