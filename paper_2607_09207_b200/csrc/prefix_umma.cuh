@@ -16,18 +16,25 @@
 // the bf16 rest (8 bits of P are not enough under the stated tolerance), and ONE product P.V per 16 tokens
 // yields the hi part and the lo part of O in the two lane halves while V is read once.
 //
-// Eight softmax warps: warp w reaches lanes 32 * (w % 4) .. + 31 only (a hardware rule), so a row has four
-// threads -- two lanes times two halves of the tile's columns -- and each turns a quarter of the tile (16
-// tokens) into probabilities, swaps hi and lo parts with the row's other lane through shared memory and
-// stores its lane's 16 P columns.  One 128-thread barrier per tile publishes the swapped parts and the next
-// tile's quarter maxima (its scores are fetched ahead).  The reference value of the online softmax only
-// follows the running max when that grew by more than 2^8, so O in tensor memory is rarely rescaled.
+// Eight softmax warps in two teams of four.  Team tm takes the tiles whose number has parity tm and owns a
+// score buffer, a probability buffer, an accumulator O_tm and a running (m, l) per row, so inside a unit the
+// teams never wait for each other and their per-tile chains (barrier wait, tensor-memory load, exponentials,
+// tensor-memory store, arrive) overlap; their states are merged at the end of the unit.  Warp w reaches lanes
+// 32 * (w % 4) .. + 31 only (a hardware rule); the thread in a row's first lane and the one in its second lane
+// both read the row's 64 scores and compute its 64 probabilities (nothing is exchanged inside a tile); the
+// first keeps the bf16 heads, the second the rests (both by truncation: no conversion instructions).  The
+// scores stay unscaled: the scale enters through the exponent's multiply-add, its sign through the staged Q.
+// The reference value of the online softmax only follows the running max when that grew by more than 2^8,
+// so O in tensor memory is rarely rescaled.
 // Two MMA-issuing threads in two warps (scores; P.V), because the tensor cores take an MMA of this size
 // only about every 80-100 cycles from its issuing thread; two TMA producer warps.  Scores run two tiles
-// ahead of the softmax (two score buffers), query rows are staged a whole unit ahead (two buffers).
+// ahead of the softmax (one buffer per team); the next unit's query rows are staged by the team that
+// meets the unit's last tile, as soon as that tile's scores (the last use of the query buffer) are there.
 // Every mbarrier wait is bounded; on expiry the CTA raises ERR_TIMEOUT, its waits fall through, the
 // issuing threads drain their tensor-core work, the tensor memory is freed and the CTA returns.
 #pragma once
+
+#include <type_traits>
 
 #include "kernels.cuh"
 
@@ -146,26 +153,25 @@ struct UmmaCfg {
   static constexpr int MMA_WARP = 8;                        // warps 0-7: softmax; 8, 9: MMA issue; 10, 11: producers
   static constexpr int NTHREADS = (MMA_WARP + 2 + NPW) * 32;
   static constexpr int CTRL_BYTES = 384;
-  static constexpr int XM_BYTES = 2 * 4 * 64 * 4;           // row maxima of the four column quarters, double buffered
-  static constexpr int XL_BYTES = 4 * 64 * 4;               // row sums of the four column quarters
-  static constexpr int XP_BYTES = 2 * 4 * 64 * 32;          // P halves swapped between a row's two lanes, double buffered
-  static constexpr int XO_BYTES = XP_BYTES;                 // (same memory) the lo-part rows of O as bf16, at the end of a unit
-  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + XM_BYTES + XL_BYTES + XO_BYTES + CTRL_BYTES;
+  static constexpr int XS_BYTES = 4 * 64 * 4;               // the teams' (m, l) per row, at the end of a unit
+  static constexpr int XO_BYTES = 64 * 32 * (4 + 2 + 2);    // 32 columns of the other three parts of a row of O
+  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + XS_BYTES + XO_BYTES + CTRL_BYTES;
   static constexpr int HP = 8;                              // heads per partial slot (G <= 8)
   static constexpr int SLOT_FLOATS = HP * (D + 2);          // same slots as decode_kernel reads
-  // tensor-memory columns: Q (2 buffers x D/2), S (2 x 64), P (2 x 32), O (D)
+  // tensor-memory columns: Q (D/2), S (2 x 64), P (2 x 32), O (2 x D): one score buffer, probability buffer and
+  // accumulator per softmax team
   static constexpr int QC = D / 2;                          // columns of a row of Q (two bf16 per column)
-  static constexpr int COL_Q = 0, COL_S = 2 * QC, COL_P = COL_S + 128, COL_O = COL_P + 64, TMEM_COLS = 512;
+  static constexpr int COL_Q = 0, COL_S = QC, COL_P = COL_S + 128, COL_O = COL_P + 64, TMEM_COLS = 512;
   static_assert(DYN_BYTES <= 232448, "shared memory");
   static_assert(NSTAGES % NPW == 0, "a slot is always refilled by the same producer warp");
-  static_assert(COL_O + D <= TMEM_COLS, "tensor memory");
+  static_assert(COL_O + 2 * D <= TMEM_COLS, "tensor memory");
 };
 
 struct UmmaCtrl {
   uint64_t full[8], empty[8];                  // ring: TMA landed / tile's MMAs done
   uint64_t s_full[2], s_free[2];               // per score buffer: scores ready / scores are in registers
   uint64_t p_full[2], pv_done[2];              // per probability buffer: stored / consumed and O updated
-  uint64_t q_ready[2];                         // per query buffer: the unit's query rows are in tensor memory
+  uint64_t q_ready;                            // the unit's query rows are in tensor memory
   uint64_t unit_done;                          // every P.V of the unit is done
   uint64_t drained[2];                         // all MMAs of an issuing thread are done
   uint32_t meta[8];                            // per stage: bit j set = page j of the tile had a bad id
@@ -208,11 +214,9 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   const uint32_t ring = raw + pad;                                  // NST stages, 1024-aligned
-  float* xm = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);   // [2 buffers][4 quarters][64 rows]
-  float* xl = xm + 2 * 4 * 64;                                      // [4 quarters][64 rows]
-  float* xo = xl + 4 * 64;                                          // [2 halves][64 rows][32]; also the P swap area
-  uint4* xp = reinterpret_cast<uint4*>(xo);                         // [2 buffers][4 quarters][64 rows][2]
-  UmmaCtrl* ctrl = reinterpret_cast<UmmaCtrl*>(smem + NST * C::STAGE_BYTES + C::XM_BYTES + C::XL_BYTES + C::XO_BYTES);
+  float* xs = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);   // [m | l][2 teams][64 rows]
+  float* xo = xs + 4 * 64;                                          // the unit-end exchange of O, 16 KB
+  UmmaCtrl* ctrl = reinterpret_cast<UmmaCtrl*>(smem + NST * C::STAGE_BYTES + C::XS_BYTES + C::XO_BYTES);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int cta = blockIdx.x;
@@ -225,11 +229,11 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctrl->s_full[i]), 1);
-      mbar_init(smem_u32(&ctrl->s_free[i]), 256);
-      mbar_init(smem_u32(&ctrl->p_full[i]), 256);
+      mbar_init(smem_u32(&ctrl->s_free[i]), 128);
+      mbar_init(smem_u32(&ctrl->p_full[i]), 128);
       mbar_init(smem_u32(&ctrl->pv_done[i]), 1);
-      mbar_init(smem_u32(&ctrl->q_ready[i]), 256);
     }
+    mbar_init(smem_u32(&ctrl->q_ready), 128);
     mbar_init(smem_u32(&ctrl->unit_done), 1);
     mbar_init(smem_u32(&ctrl->drained[0]), 1);
     mbar_init(smem_u32(&ctrl->drained[1]), 1);
@@ -327,12 +331,12 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           const int b = sc.i & 1;
           // score buffer b is free when the softmax threads have tile i - 2 in registers
           if (sc.i >= 2) ok = mbar_wait_abortable(smem_u32(&ctrl->s_free[b]), ((sc.i - 2) >> 1) & 1, abort_flag);
-          if (ok && sc.t == 0) ok = mbar_wait_abortable(smem_u32(&ctrl->q_ready[sc.n & 1]), (sc.n >> 1) & 1, abort_flag);
+          if (ok && sc.t == 0) ok = mbar_wait_abortable(smem_u32(&ctrl->q_ready), sc.n & 1, abort_flag);
           if (ok) ok = mbar_wait_abortable(smem_u32(&ctrl->full[slot]), ring_phase, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint64_t kd = k_desc0 + static_cast<uint64_t>(slot * (C::STAGE_BYTES >> 4));
-          const uint32_t d_s = tS + b * 64, a_q = tQ + (sc.n & 1) * C::QC;
+          const uint32_t d_s = tS + b * 64, a_q = tQ;
 #pragma unroll
           for (int h = 0; h < C::HALVES; ++h)
 #pragma unroll
@@ -360,10 +364,10 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           tc_fence_after();
           const uint64_t vd0 = v_desc0 + static_cast<uint64_t>(slot * (C::STAGE_BYTES >> 4));
           const uint32_t a_p = tP + b * 32;
-          const uint32_t acc0 = pc.t > 0 ? 1u : 0u;   // the unit's first tile starts the accumulator afresh
+          const uint32_t acc0 = pc.t > 1 ? 1u : 0u;   // a team's first tile of the unit starts its accumulator afresh
 #pragma unroll
           for (int ks = 0; ks < TILE / 16; ++ks)
-            umma_ts(tO, a_p + ks * 8, vd0 + static_cast<uint64_t>((ks * 2048) >> 4), ID_O, ks ? 1u : acc0);
+            umma_ts(tO + b * D, a_p + ks * 8, vd0 + static_cast<uint64_t>((ks * 2048) >> 4), ID_O, ks ? 1u : acc0);
           tc_commit(smem_u32(&ctrl->empty[slot]));    // K and V of this tile are free again (its scores are long done)
           tc_commit(smem_u32(&ctrl->pv_done[b]));
           if (pc.t == pc.pt - 1) tc_commit(smem_u32(&ctrl->unit_done));
@@ -382,231 +386,244 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     }
     __syncwarp();
   } else {
-    // ================= softmax: warp w works on tensor-memory lanes 32 * (w % 4) .. + 31.  A query row has
-    // four threads: in its first lane (hi part of P and O) and in its second lane (lo part), each for one half
-    // of the tile's columns -- and since both lanes hold the same scores, each of the four turns only a
-    // QUARTER of the tile (16 tokens) into probabilities, then swaps with the row's other lane: hi parts
-    // go to the first lane, lo parts to the second.  No thread leaves this path early: the four meet at
-    // named barriers, so after a failed wait a thread carries on (its waits then return at once).
+    // ================= softmax: two teams of four warps; team tm works on the tiles with (tile number & 1) == tm,
+    // with its own score buffer, probability buffer, accumulator O_tm and running (m, l) per row, so the two
+    // teams never wait for each other inside a unit and their per-tile chains of latencies (barrier wait,
+    // tensor-memory load, exponentials, tensor-memory store, arrive) overlap.  Warp w reaches tensor-memory
+    // lanes 32 * (w % 4) .. + 31; a row's first lane takes the bf16 heads of P, its second lane the rests, and
+    // both compute the row's 64 probabilities themselves from the same scores (no exchange inside a tile).
+    // The teams' states are merged at the end of a unit.  No thread leaves this path early: all meet at the
+    // unit's barriers, so after a failed wait a thread carries on (its waits then return at once).
     const int qd = warp & 3;
-    const int part = warp >> 2;           // which half of the tile's columns this thread stores P for
-    const int lh = qd >> 1;               // 0: first lane of the row (hi parts), 1: second lane (lo parts)
-    const int grp = qd & 1;               // rows 0-31 / 32-63 of the slot order: the four warps that share rows
-    const int qi = part * 2 + lh;         // quarter of the tile this thread computes: tokens qi * 16 .. + 15
-    const int rho = grp * 32 + lane;      // row slot
-    const bool is_lo = lh != 0;
+    const int tm = warp >> 2;             // team
+    const bool is_lo = (qd >> 1) != 0;    // second lane of the row: rests of P, lo part of O
+    const int rho = (qd & 1) * 32 + lane; // row slot
     const int r = (rho & 31) * 2 + (rho >> 5);
     const int R = P.Gs * P.G;
     const bool valid = r < R;
     const int rj = valid ? r / P.G : 0, rh = valid ? r - rj * P.G : 0;   // sample in the group, head in the KV group
     const uint32_t lane_addr = static_cast<uint32_t>(qd * 32) << 16;
-    constexpr int OC = D / 2;             // columns of O per thread
-    constexpr int QCP = C::QC / 2;        // columns of Q per thread
+    const uint32_t tOt = tO + tm * D;     // this team's accumulator
+    // the scores stay unscaled in registers (the scale is applied inside the exponent's multiply-add), so it
+    // must not be negative: its sign goes into the staged query rows
+    const float sc = fabsf(P.scale_log2);
+    const uint32_t qflip = P.scale_log2 < 0.f ? 0x80008000u : 0u;
     auto wait_all = [&](uint64_t* bar, uint32_t parity) {   // warp-uniform: tensor-memory accesses need the whole warp
       if (!__all_sync(0xffffffffu, mbar_wait_abortable(smem_u32(bar), parity, abort_flag)) && lane == 0) {
         atomicOr(P.err, ERR_TIMEOUT);
         atomicExch(&ctrl->abort, 1u);
       }
     };
-    auto row_barrier = [&]() { asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory"); };   // the four warps of these rows
     auto all_barrier = [&]() { asm volatile("bar.sync 5, 256;" ::: "memory"); };
-    // this thread's half of its query row of unit u into query buffer n & 1 (two bf16 per column)
+    auto q_row = [&](int u) {
+      const int gi = u / P.Hkv, g = u - gi * P.Hkv;
+      return P.q + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hq + g * P.G + rh) * D;
+    };
+    // this thread's query row of unit u into the (single) query buffer, two bf16 per column; the caller knows
+    // that every score product of the buffer's previous unit is done
     auto stage_q = [&](int u, int n) {
-      uint32_t qv[QCP];
 #pragma unroll
-      for (int c = 0; c < QCP; ++c) qv[c] = 0u;
-      if (valid) {
-        const int gi = u / P.Hkv, g = u - gi * P.Hkv;
-        const uint4* src = reinterpret_cast<const uint4*>(
-            P.q + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hq + g * P.G + rh) * D + part * (D / 2));
+      for (int c0 = 0; c0 < C::QC; c0 += 32) {
+        uint32_t qv[32];
 #pragma unroll
-        for (int c = 0; c < QCP / 4; ++c) {
-          const uint4 v = __ldg(src + c);
-          qv[4 * c] = v.x;
-          qv[4 * c + 1] = v.y;
-          qv[4 * c + 2] = v.z;
-          qv[4 * c + 3] = v.w;
+        for (int c = 0; c < 32; ++c) qv[c] = 0u;
+        if (valid) {
+          const uint4* src = reinterpret_cast<const uint4*>(q_row(u) + 2 * c0);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 v = __ldg(src + c);
+            qv[4 * c] = v.x ^ qflip;
+            qv[4 * c + 1] = v.y ^ qflip;
+            qv[4 * c + 2] = v.z ^ qflip;
+            qv[4 * c + 3] = v.w ^ qflip;
+          }
         }
-      }
-      const uint32_t dst = tQ + (n & 1) * C::QC + part * QCP + lane_addr;
-      if constexpr (QCP == 32) {
-        tmem_st32(dst, qv);
-      } else {
-        tmem_st16(dst, qv);
+        tmem_st32(tQ + c0 + lane_addr, qv);
       }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(smem_u32(&ctrl->q_ready[n & 1]));
-    };
-
-    // scores of tile c.i: this thread's quarter into registers (scaled, masked) and its max into shared memory
-    uint32_t sv[16];
-    auto fetch_scores = [&](const UnitCursor& c) {
-      const int it = c.i, b = it & 1;
-      wait_all(&ctrl->s_full[b], (it >> 1) & 1);
-      tc_fence_after();
-      tmem_ld16(tS + b * 64 + qi * 16 + lane_addr, sv);
-      tc_wait_ld();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&ctrl->s_free[b]));   // the score buffer can take tile it + 2
-      const uint32_t badmask = ctrl->meta[it % NST];
-      float mx = NEG_INF;
-#pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        float x = __uint_as_float(sv[k]) * P.scale_log2;
-        if (badmask && ((badmask >> ((qi * 16 + k) / BS)) & 1u)) x = NEG_INF;
-        sv[k] = __float_as_uint(x);
-        mx = fmaxf(mx, x);
-      }
-      xm[(b * 4 + qi) * 64 + rho] = mx;
+      mbar_arrive(smem_u32(&ctrl->q_ready));
+      (void)n;
     };
 
     UnitCursor uc{range.x, range.y, 0, 0, 0, 0, P.prefix_tiles, P.Hkv};
     uc.seek();
-    if (uc.valid()) {
-      stage_q(uc.u, 0);
-      fetch_scores(uc);
-    }
-    row_barrier();
+    if (uc.valid() && tm == 0) stage_q(uc.u, 0);
     float m = NEG_INF, l = 0.f;
-    // One barrier of the row's four threads per tile: it publishes this tile's swapped P parts and the NEXT
-    // tile's quarter maxima (its scores are fetched before the barrier, across unit boundaries too).
     while (uc.valid()) {
-      const int it = uc.i, b = it & 1, t = uc.t, pt = uc.pt, n = uc.n, u = uc.u;
-      UnitCursor nx = uc;
-      nx.next_tile();
-      if (t == 0) {
-        // the next unit's query rows, a whole unit ahead (the buffer's previous unit has all its scores)
-        UnitCursor nu = uc;
-        nu.t = nu.pt - 1;
-        nu.next_tile();
-        if (nu.valid()) stage_q(nu.u, n + 1);
-        m = NEG_INF;
-        l = 0.f;
-      }
-      // the row's max over the four quarters
-      const float* xmb = xm + b * 4 * 64 + rho;
-      const float mx = fmaxf(fmaxf(xmb[0], xmb[64]), fmaxf(xmb[128], xmb[192]));
-      // The reference value m only follows the running max when that grew by more than 2^8: P and O may
-      // then exceed 1 by that factor (harmless in fp32 / bf16), and the pass over O in tensor memory that a
-      // new reference costs becomes rare.  (m, l, O) stay consistent, which is all the merges need.
-      const bool grow = t == 0 || mx > m + 8.f;
-      const float m_new = grow ? fmaxf(m, mx) : m;
-      const float mu = (m_new == NEG_INF) ? 0.f : m_new;
-      const float alpha = grow ? fast_exp2(m - mu) : 1.f;
-      m = m_new;
-      // P = exp2(S - m) as bf16 head + bf16 rest; a P column holds two tokens
-      uint32_t hi[8], lo[8];
-      float ls = 0.f;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const float p0 = fast_exp2(__uint_as_float(sv[2 * k]) - mu);
-        const float p1 = fast_exp2(__uint_as_float(sv[2 * k + 1]) - mu);
-        ls += p0 + p1;
-        const uint32_t h01 = pack_bf16x2(p0, p1);
-        hi[k] = h01;
-        lo[k] = pack_bf16x2(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u));
-      }
-      l = l * alpha + ls;
-      // swap with the row's other lane: it gets the part this lane does not store
-      uint4* xpb = xp + (b * 4 * 64 + rho) * 2;
-      if (is_lo) {
-        xpb[qi * 128] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        xpb[qi * 128 + 1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-      } else {
-        xpb[qi * 128] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        xpb[qi * 128 + 1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-      }
-      if (nx.valid()) fetch_scores(nx);
-      row_barrier();
-      const uint4 g0 = xpb[(qi ^ 1) * 128], g1 = xpb[(qi ^ 1) * 128 + 1];
-      uint32_t pk[16];   // this lane's 16 P columns of the half: the first-lane quarter, then the second-lane quarter
-#pragma unroll
-      for (int k = 0; k < 8; ++k) pk[is_lo ? 8 + k : k] = is_lo ? lo[k] : hi[k];
-      pk[is_lo ? 0 : 8] = g0.x;
-      pk[is_lo ? 1 : 9] = g0.y;
-      pk[is_lo ? 2 : 10] = g0.z;
-      pk[is_lo ? 3 : 11] = g0.w;
-      pk[is_lo ? 4 : 12] = g1.x;
-      pk[is_lo ? 5 : 13] = g1.y;
-      pk[is_lo ? 6 : 14] = g1.z;
-      pk[is_lo ? 7 : 15] = g1.w;
-      // the product that read this probability buffer two tiles ago must be done
-      if (it >= 2) wait_all(&ctrl->pv_done[b], ((it - 2) >> 1) & 1);
-      if (__any_sync(0xffffffffu, t > 0 && alpha != 1.f)) {
-        // new reference: scale this thread's columns of O, once the previous tile's product is in
-        wait_all(&ctrl->pv_done[b ^ 1], ((it - 1) >> 1) & 1);
-        tc_fence_after();
-#pragma unroll
-        for (int q = 0; q < OC / 32; ++q) {
-          uint32_t o[32];
-          tmem_ld32(tO + part * OC + q * 32 + lane_addr, o);
-          tc_wait_ld();
-#pragma unroll
-          for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-          tmem_st32(tO + part * OC + q * 32 + lane_addr, o);
+      const int it = uc.i, t = uc.t, pt = uc.pt, n = uc.n, u = uc.u;
+      UnitCursor nu = uc;      // where the cursor goes after this tile
+      nu.next_tile();
+      const bool last = t == pt - 1;
+      if ((it & 1) == tm) {
+        if (t < 2) {           // this team's first tile of the unit
+          m = NEG_INF;
+          l = 0.f;
         }
-      }
-      tc_fence_after();
-      tmem_st16(tP + b * 32 + part * 16 + lane_addr, pk);
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&ctrl->p_full[b]));
-      if (t == pt - 1) {
-        // ---- the unit's result: (m, l) and O = hi part + lo part, to the per-(sequence, KV head) prefix slot.
-        // The lo rows cross to the row's first lane through shared memory as bf16 (they are 2^-9 of O).
-        const int gi = u / P.Hkv, g = u - gi * P.Hkv;
-        wait_all(&ctrl->unit_done, n & 1);
+        if (last && nu.valid() && valid)   // the next unit's query row towards L2 (it is staged after this tile's scores)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(q_row(nu.u) + (is_lo ? D / 2 : 0)));
+        uint32_t sv[64];
+        wait_all(&ctrl->s_full[tm], (it >> 1) & 1);
         tc_fence_after();
-        xl[qi * 64 + rho] = l;
-        uint32_t* xrow = reinterpret_cast<uint32_t*>(xo) + (part * 64 + rho) * (OC / 2);
-        float* slotp = P.pfx_partials + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hkv + g) * C::SLOT_FLOATS;
-        if (is_lo) {
+        tmem_ld32(tS + tm * 64 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(sv));
+        tmem_ld32(tS + tm * 64 + 32 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(sv + 32));
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&ctrl->s_free[tm]));   // the score buffer can take tile it + 2
+        const uint32_t badmask = ctrl->meta[it % NST];
+        if (badmask) {
 #pragma unroll
-          for (int q = 0; q < OC / 32; ++q) {
+          for (int k = 0; k < 64; ++k)
+            if ((badmask >> (k / BS)) & 1u) sv[k] = __float_as_uint(NEG_INF);
+        }
+        // the row max of the raw scores, four independent chains of three-input max (the scale is not negative:
+        // its sign went into the staged query rows)
+        float m4[4] = {NEG_INF, NEG_INF, NEG_INF, NEG_INF};
+#pragma unroll
+        for (int k = 0; k < 64; k += 2)
+          m4[(k >> 1) & 3] = max3(m4[(k >> 1) & 3], __uint_as_float(sv[k]), __uint_as_float(sv[k + 1]));
+        const float mr = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        const float mx = (mr == NEG_INF) ? NEG_INF : mr * sc;
+        // The reference value m only follows the running max when that grew by more than 2^8: P and O may
+        // then exceed 1 by that factor (harmless in fp32 / bf16), and the pass over O in tensor memory that a
+        // new reference costs becomes rare.  (m, l, O) stay consistent, which is all the merges need.
+        const bool grow = t < 2 || mx > m + 8.f;
+        const float m_new = grow ? fmaxf(m, mx) : m;
+        const float mu = (m_new == NEG_INF) ? 0.f : m_new;
+        const float alpha = grow ? fast_exp2(m - mu) : 1.f;
+        m = m_new;
+        // P = exp2(S * scale - m), split by truncation into a bf16 head (the row's first lane) and the bf16 head
+        // of what is left (its second lane): 16 bits of P between them, and no conversion instructions.  A P
+        // column holds two tokens.  The row sum is taken in the first lane only.
+        uint32_t pk[32];
+        float ls = 0.f, ls1 = 0.f;
+        auto probabilities = [&](auto masked) {
+          auto prob = [&](int k) {
+            const float x = __uint_as_float(sv[k]);
+            const float p = fast_exp2(fmaf(x, sc, -mu));
+            if constexpr (decltype(masked)::value) return (x == NEG_INF) ? 0.f : p;   // (a zero scale would turn the mask into NaN)
+            return p;
+          };
+          if (!is_lo) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+              const float p0 = prob(2 * k), p1 = prob(2 * k + 1);
+              ls += p0;
+              ls1 += p1;
+              pk[k] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+              const float p0 = prob(2 * k), p1 = prob(2 * k + 1);
+              const float r0 = p0 - __uint_as_float(__float_as_uint(p0) & 0xffff0000u);
+              const float r1 = p1 - __uint_as_float(__float_as_uint(p1) & 0xffff0000u);
+              pk[k] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+            }
+          }
+        };
+        if (badmask) {
+          probabilities(std::true_type{});
+        } else {
+          probabilities(std::false_type{});
+        }
+        l = l * alpha + (ls + ls1);
+        // the product that read this team's probability buffer two tiles ago must be done (it is also the
+        // latest product into this team's accumulator)
+        if (it >= 2) wait_all(&ctrl->pv_done[tm], ((it - 2) >> 1) & 1);
+        if (__any_sync(0xffffffffu, t >= 2 && alpha != 1.f)) {
+          // new reference: scale this lane's row of O
+          tc_fence_after();
+#pragma unroll
+          for (int q = 0; q < D / 32; ++q) {
             uint32_t o[32];
-            tmem_ld32(tO + part * OC + q * 32 + lane_addr, o);
+            tmem_ld32(tOt + q * 32 + lane_addr, o);
             tc_wait_ld();
 #pragma unroll
+            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+            tmem_st32(tOt + q * 32 + lane_addr, o);
+          }
+        }
+        tc_fence_after();
+        tmem_st32(tP + tm * 32 + lane_addr, pk);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&ctrl->p_full[tm]));
+        // every score product of this unit is done (this tile's scores were the last): the query buffer is free
+        if (last && nu.valid()) stage_q(nu.u, n + 1);
+      }
+      if (last) {
+        // ---- the unit's result.  Four threads hold parts of a row: (team 0 | team 1) x (hi lane | lo lane), each
+        // with its team's reference max.  They cross through shared memory, 32 columns at a time, already
+        // scaled to the common reference; the first team's hi lane adds them up and writes the prefix slot.
+        const int gi = u / P.Hkv, g = u - gi * P.Hkv;
+        const bool mine = pt >= 2 || ((it & 1) == tm);     // a one-tile unit leaves the other team without a state
+        wait_all(&ctrl->unit_done, n & 1);
+        tc_fence_after();
+        if (!is_lo) {
+          xs[tm * 64 + rho] = mine ? m : NEG_INF;
+          xs[128 + tm * 64 + rho] = mine ? l : 0.f;
+        }
+        all_barrier();
+        const float m0 = xs[rho], m1 = xs[64 + rho];
+        const float mt = fmaxf(m0, m1);
+        const float mtu = (mt == NEG_INF) ? 0.f : mt;
+        const float f = mine ? fast_exp2((tm ? m1 : m0) - mtu) : 0.f;     // (exp2(-inf) = 0 for a team without tiles)
+        const float lt = xs[128 + rho] * fast_exp2(m0 - mtu) + xs[192 + rho] * fast_exp2(m1 - mtu);
+        float* slotp = P.pfx_partials + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hkv + g) * C::SLOT_FLOATS;
+        // exchange area per round: [team 1 hi: 64 rows x 32 fp32][team 0 lo: 64 x 32 bf16][team 1 lo: 64 x 32 bf16]
+        float4* x_hi = reinterpret_cast<float4*>(xo) + rho * 8;
+        uint4* x_lo = reinterpret_cast<uint4*>(xo + 64 * 32) + (tm * 64 + rho) * 4;
+#pragma unroll 1
+        for (int q = 0; q < D / 32; ++q) {
+          uint32_t o[32];
+          tmem_ld32(tOt + q * 32 + lane_addr, o);   // (whole warps only: a row without a state drops what it read)
+          tc_wait_ld();
+#pragma unroll
+          for (int k = 0; k < 32; ++k) o[k] = (f != 0.f) ? __float_as_uint(__uint_as_float(o[k]) * f) : 0u;
+          if (is_lo) {
+#pragma unroll
             for (int k = 0; k < 4; ++k)
-              reinterpret_cast<uint4*>(xrow + q * 16)[k] =
+              x_lo[k ^ (rho & 3)] =
                   make_uint4(pack_bf16x2(__uint_as_float(o[8 * k]), __uint_as_float(o[8 * k + 1])),
                              pack_bf16x2(__uint_as_float(o[8 * k + 2]), __uint_as_float(o[8 * k + 3])),
                              pack_bf16x2(__uint_as_float(o[8 * k + 4]), __uint_as_float(o[8 * k + 5])),
                              pack_bf16x2(__uint_as_float(o[8 * k + 6]), __uint_as_float(o[8 * k + 7])));
+          } else if (tm == 1) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              x_hi[k ^ (rho & 7)] = make_float4(__uint_as_float(o[4 * k]), __uint_as_float(o[4 * k + 1]),
+                                               __uint_as_float(o[4 * k + 2]), __uint_as_float(o[4 * k + 3]));
           }
-        }
-        all_barrier();
-        if (!is_lo) {
+          all_barrier();
+          if (!is_lo && tm == 0 && valid) {
+            float4* dst = reinterpret_cast<float4*>(slotp + 2 * C::HP + rh * D + q * 32);
+            const uint4* lo0 = reinterpret_cast<const uint4*>(xo + 64 * 32) + rho * 4;
+            const uint4* lo1 = lo0 + 64 * 4;
 #pragma unroll
-          for (int q = 0; q < OC / 32; ++q) {
-            uint32_t o[32];
-            tmem_ld32(tO + part * OC + q * 32 + lane_addr, o);
-            tc_wait_ld();
-            if (valid) {
-              float4* dst = reinterpret_cast<float4*>(slotp + 2 * C::HP + rh * D + part * OC + q * 32);
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const uint4 w = reinterpret_cast<const uint4*>(xrow + q * 16)[k];
-                dst[2 * k] = make_float4(__uint_as_float(o[8 * k]) + __uint_as_float(w.x << 16),
-                                         __uint_as_float(o[8 * k + 1]) + __uint_as_float(w.x & 0xffff0000u),
-                                         __uint_as_float(o[8 * k + 2]) + __uint_as_float(w.y << 16),
-                                         __uint_as_float(o[8 * k + 3]) + __uint_as_float(w.y & 0xffff0000u));
-                dst[2 * k + 1] = make_float4(__uint_as_float(o[8 * k + 4]) + __uint_as_float(w.z << 16),
-                                             __uint_as_float(o[8 * k + 5]) + __uint_as_float(w.z & 0xffff0000u),
-                                             __uint_as_float(o[8 * k + 6]) + __uint_as_float(w.w << 16),
-                                             __uint_as_float(o[8 * k + 7]) + __uint_as_float(w.w & 0xffff0000u));
-              }
+            for (int k = 0; k < 4; ++k) {
+              const uint4 a = lo0[k ^ (rho & 3)], bq = lo1[k ^ (rho & 3)];
+              const float4 h0 = x_hi[(2 * k) ^ (rho & 7)], h1 = x_hi[(2 * k + 1) ^ (rho & 7)];
+              dst[2 * k] = make_float4(
+                  __uint_as_float(o[8 * k]) + h0.x + (__uint_as_float(a.x << 16) + __uint_as_float(bq.x << 16)),
+                  __uint_as_float(o[8 * k + 1]) + h0.y + (__uint_as_float(a.x & 0xffff0000u) + __uint_as_float(bq.x & 0xffff0000u)),
+                  __uint_as_float(o[8 * k + 2]) + h0.z + (__uint_as_float(a.y << 16) + __uint_as_float(bq.y << 16)),
+                  __uint_as_float(o[8 * k + 3]) + h0.w + (__uint_as_float(a.y & 0xffff0000u) + __uint_as_float(bq.y & 0xffff0000u)));
+              dst[2 * k + 1] = make_float4(
+                  __uint_as_float(o[8 * k + 4]) + h1.x + (__uint_as_float(a.z << 16) + __uint_as_float(bq.z << 16)),
+                  __uint_as_float(o[8 * k + 5]) + h1.y + (__uint_as_float(a.z & 0xffff0000u) + __uint_as_float(bq.z & 0xffff0000u)),
+                  __uint_as_float(o[8 * k + 6]) + h1.z + (__uint_as_float(a.w << 16) + __uint_as_float(bq.w << 16)),
+                  __uint_as_float(o[8 * k + 7]) + h1.w + (__uint_as_float(a.w & 0xffff0000u) + __uint_as_float(bq.w & 0xffff0000u)));
+            }
+            if (q == 0) {
+              slotp[rh] = mt;
+              slotp[C::HP + rh] = lt;
             }
           }
-          if (valid && part == 0) {
-            slotp[rh] = m;
-            slotp[C::HP + rh] = (xl[rho] + xl[64 + rho]) + (xl[128 + rho] + xl[192 + rho]);
-          }
+          all_barrier();   // the exchange area is used again
         }
-        all_barrier();   // the swap area is used again by the next tile
       }
-      uc = nx;
+      uc = nu;
     }
   }
 

@@ -74,6 +74,23 @@ def test_groups_with_uneven_prefixes_and_head_counts(Hq, Hkv, group):
     assert_parity(out, orc.decode_workload(w.to("cpu")), f"Hq={Hq} Hkv={Hkv} group={group}")
 
 
+@pytest.mark.parametrize("factor", [-1.0, 0.0, -4.0])
+def test_grouped_with_negative_and_zero_scale(factor):
+    """A negative scale turns the row max into a min of the raw scores (the tcgen05 kernel keeps raw scores and
+    moves the sign into the staged query rows); a zero scale gives uniform weights."""
+    lens = [640 + 3, 640 + 200, 640 + 64, 640 + 1, 128 + 5, 128 + 77, 128 + 300, 128 + 31]
+    w = W.make_custom(lens, Hq=28, Hkv=4, d=128, seed=77, device=DEV, poison=False)
+    bt = w.block_table.clone()
+    for lead, pages in ((0, 40), (4, 8)):
+        for j in range(1, 4):
+            bt[lead + j, :pages] = bt[lead, :pages]
+    w = dataclasses.replace(w, block_table=bt, scale=w.scale * factor)
+    W.poison_unused(w)
+    out, status = run_grouped(w, 4, [10, 2])
+    assert status == pdattn.OK
+    assert_parity(out, orc.decode_workload(w.to("cpu")), f"scale factor {factor}")
+
+
 @pytest.mark.parametrize("bs", [32, 64])
 def test_grouped_with_larger_pages(bs):
     lens = [200, 70, 65, 1000, 129, 500, 66, 300]
