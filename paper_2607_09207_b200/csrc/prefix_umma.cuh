@@ -154,7 +154,7 @@ struct UmmaCfg {
   static constexpr int NTHREADS = (MMA_WARP + 2 + NPW) * 32;
   static constexpr int CTRL_BYTES = 384;
   static constexpr int XS_BYTES = 4 * 64 * 4;               // the teams' (m, l) per row, at the end of a unit
-  static constexpr int XO_BYTES = 64 * 32 * (4 + 2 + 2);    // 32 columns of the other three parts of a row of O
+  static constexpr int XO_BYTES = 64 * D * 2;               // the second lanes' rows of O as bf16, at the end of a unit
   static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + XS_BYTES + XO_BYTES + CTRL_BYTES;
   static constexpr int HP = 8;                              // heads per partial slot (G <= 8)
   static constexpr int SLOT_FLOATS = HP * (D + 2);          // same slots as decode_kernel reads
@@ -215,7 +215,7 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   uint8_t* smem = smem_raw + pad;
   const uint32_t ring = raw + pad;                                  // NST stages, 1024-aligned
   float* xs = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);   // [m | l][2 teams][64 rows]
-  float* xo = xs + 4 * 64;                                          // the unit-end exchange of O, 16 KB
+  float* xo = xs + 4 * 64;                                          // [64 rows][D] bf16
   UmmaCtrl* ctrl = reinterpret_cast<UmmaCtrl*>(smem + NST * C::STAGE_BYTES + C::XS_BYTES + C::XO_BYTES);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -406,7 +406,9 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     const uint32_t tOt = tO + tm * D;     // this team's accumulator
     // the scores stay unscaled in registers (the scale is applied inside the exponent's multiply-add), so it
     // must not be negative: its sign goes into the staged query rows
-    const float sc = fabsf(P.scale_log2);
+    // (never exactly zero, so that a masked score, minus infinity, stays that under the multiply-add; a scale this
+    // small gives the same probabilities as zero)
+    const float sc = fmaxf(fabsf(P.scale_log2), 1e-30f);
     const uint32_t qflip = P.scale_log2 < 0.f ? 0x80008000u : 0u;
     auto wait_all = [&](uint64_t* bar, uint32_t parity) {   // warp-uniform: tensor-memory accesses need the whole warp
       if (!__all_sync(0xffffffffu, mbar_wait_abortable(smem_u32(bar), parity, abort_flag)) && lane == 0) {
@@ -422,24 +424,22 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     // this thread's query row of unit u into the (single) query buffer, two bf16 per column; the caller knows
     // that every score product of the buffer's previous unit is done
     auto stage_q = [&](int u, int n) {
+      uint32_t qv[C::QC];      // all loads first: under this kernel's own traffic even an L2 hit takes about a microsecond
 #pragma unroll
-      for (int c0 = 0; c0 < C::QC; c0 += 32) {
-        uint32_t qv[32];
+      for (int c = 0; c < C::QC; ++c) qv[c] = 0u;
+      if (valid) {
+        const uint4* src = reinterpret_cast<const uint4*>(q_row(u));
 #pragma unroll
-        for (int c = 0; c < 32; ++c) qv[c] = 0u;
-        if (valid) {
-          const uint4* src = reinterpret_cast<const uint4*>(q_row(u) + 2 * c0);
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint4 v = __ldg(src + c);
-            qv[4 * c] = v.x ^ qflip;
-            qv[4 * c + 1] = v.y ^ qflip;
-            qv[4 * c + 2] = v.z ^ qflip;
-            qv[4 * c + 3] = v.w ^ qflip;
-          }
+        for (int c = 0; c < C::QC / 4; ++c) {
+          const uint4 v = __ldg(src + c);
+          qv[4 * c] = v.x ^ qflip;
+          qv[4 * c + 1] = v.y ^ qflip;
+          qv[4 * c + 2] = v.z ^ qflip;
+          qv[4 * c + 3] = v.w ^ qflip;
         }
-        tmem_st32(tQ + c0 + lane_addr, qv);
       }
+#pragma unroll
+      for (int c0 = 0; c0 < C::QC; c0 += 32) tmem_st32(tQ + c0 + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(qv + c0));
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(smem_u32(&ctrl->q_ready));
@@ -459,9 +459,13 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         if (t < 2) {           // this team's first tile of the unit
           m = NEG_INF;
           l = 0.f;
+          // the next unit's query rows towards L2, a whole unit before they are staged (under this kernel's own
+          // traffic a load from DRAM takes several tiles' time)
+          UnitCursor fu = uc;
+          fu.t = pt - 1;
+          fu.next_tile();
+          if (fu.valid() && valid) asm volatile("prefetch.global.L2 [%0];" ::"l"(q_row(fu.u) + (is_lo ? D / 2 : 0)));
         }
-        if (last && nu.valid() && valid)   // the next unit's query row towards L2 (it is staged after this tile's scores)
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(q_row(nu.u) + (is_lo ? D / 2 : 0)));
         uint32_t sv[64];
         wait_all(&ctrl->s_full[tm], (it >> 1) & 1);
         tc_fence_after();
@@ -497,44 +501,33 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         // column holds two tokens.  The row sum is taken in the first lane only.
         uint32_t pk[32];
         float ls = 0.f, ls1 = 0.f;
-        auto probabilities = [&](auto masked) {
-          auto prob = [&](int k) {
-            const float x = __uint_as_float(sv[k]);
-            const float p = fast_exp2(fmaf(x, sc, -mu));
-            if constexpr (decltype(masked)::value) return (x == NEG_INF) ? 0.f : p;   // (a zero scale would turn the mask into NaN)
-            return p;
-          };
-          if (!is_lo) {
+        if (!is_lo) {
 #pragma unroll
-            for (int k = 0; k < 32; ++k) {
-              const float p0 = prob(2 * k), p1 = prob(2 * k + 1);
-              ls += p0;
-              ls1 += p1;
-              pk[k] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
-            }
-          } else {
-#pragma unroll
-            for (int k = 0; k < 32; ++k) {
-              const float p0 = prob(2 * k), p1 = prob(2 * k + 1);
-              const float r0 = p0 - __uint_as_float(__float_as_uint(p0) & 0xffff0000u);
-              const float r1 = p1 - __uint_as_float(__float_as_uint(p1) & 0xffff0000u);
-              pk[k] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
-            }
+          for (int k = 0; k < 32; ++k) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * k]), sc, -mu));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * k + 1]), sc, -mu));
+            ls += p0;
+            ls1 += p1;
+            pk[k] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
           }
-        };
-        if (badmask) {
-          probabilities(std::true_type{});
         } else {
-          probabilities(std::false_type{});
+#pragma unroll
+          for (int k = 0; k < 32; ++k) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * k]), sc, -mu));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * k + 1]), sc, -mu));
+            const float r0 = p0 - __uint_as_float(__float_as_uint(p0) & 0xffff0000u);
+            const float r1 = p1 - __uint_as_float(__float_as_uint(p1) & 0xffff0000u);
+            pk[k] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+          }
         }
         l = l * alpha + (ls + ls1);
         // the product that read this team's probability buffer two tiles ago must be done (it is also the
         // latest product into this team's accumulator)
         if (it >= 2) wait_all(&ctrl->pv_done[tm], ((it - 2) >> 1) & 1);
         if (__any_sync(0xffffffffu, t >= 2 && alpha != 1.f)) {
-          // new reference: scale this lane's row of O
+          // new reference: scale this lane's row of O (rare: kept small rather than fast)
           tc_fence_after();
-#pragma unroll
+#pragma unroll 1
           for (int q = 0; q < D / 32; ++q) {
             uint32_t o[32];
             tmem_ld32(tOt + q * 32 + lane_addr, o);
@@ -549,15 +542,21 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(smem_u32(&ctrl->p_full[tm]));
-        // every score product of this unit is done (this tile's scores were the last): the query buffer is free
-        if (last && nu.valid()) stage_q(nu.u, n + 1);
       }
       if (last) {
-        // ---- the unit's result.  Four threads hold parts of a row: (team 0 | team 1) x (hi lane | lo lane), each
-        // with its team's reference max.  They cross through shared memory, 32 columns at a time, already
-        // scaled to the common reference; the first team's hi lane adds them up and writes the prefix slot.
+        // ---- the unit's result.  Four threads hold parts of a row: (team 0 | team 1) x (first lane | second lane),
+        // each team with its own reference max.  A thread reaches both teams' accumulators in its own lane, so
+        // only the second lanes' sums cross lanes (through shared memory, as bf16: they are 2^-8 of the first
+        // lanes').  Each team takes half of the columns.
         const int gi = u / P.Hkv, g = u - gi * P.Hkv;
-        const bool mine = pt >= 2 || ((it & 1) == tm);     // a one-tile unit leaves the other team without a state
+        const bool owner = (it & 1) == tm;
+        if (!owner && nu.valid()) {
+          // The team without the last tile has time now: it stages the next unit's query rows, once the last
+          // tile's scores -- the last use of the query buffer -- are complete (it only observes that barrier).
+          wait_all(&ctrl->s_full[tm ^ 1], (it >> 1) & 1);
+          stage_q(nu.u, n + 1);
+        }
+        const bool mine = pt >= 2 || owner;     // a one-tile unit leaves the other team without a state
         wait_all(&ctrl->unit_done, n & 1);
         tc_fence_after();
         if (!is_lo) {
@@ -568,60 +567,52 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         const float m0 = xs[rho], m1 = xs[64 + rho];
         const float mt = fmaxf(m0, m1);
         const float mtu = (mt == NEG_INF) ? 0.f : mt;
-        const float f = mine ? fast_exp2((tm ? m1 : m0) - mtu) : 0.f;     // (exp2(-inf) = 0 for a team without tiles)
-        const float lt = xs[128 + rho] * fast_exp2(m0 - mtu) + xs[192 + rho] * fast_exp2(m1 - mtu);
-        float* slotp = P.pfx_partials + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hkv + g) * C::SLOT_FLOATS;
-        // exchange area per round: [team 1 hi: 64 rows x 32 fp32][team 0 lo: 64 x 32 bf16][team 1 lo: 64 x 32 bf16]
-        float4* x_hi = reinterpret_cast<float4*>(xo) + rho * 8;
-        uint4* x_lo = reinterpret_cast<uint4*>(xo + 64 * 32) + (tm * 64 + rho) * 4;
-#pragma unroll 1
-        for (int q = 0; q < D / 32; ++q) {
-          uint32_t o[32];
-          tmem_ld32(tOt + q * 32 + lane_addr, o);   // (whole warps only: a row without a state drops what it read)
+        const float f0 = fast_exp2(m0 - mtu), f1 = fast_exp2(m1 - mtu);   // 0 for a team without a state
+        const int c0 = tm * (D / 2);
+        uint4* xrow = reinterpret_cast<uint4*>(xo) + rho * (D / 8);       // a row of bf16: D / 8 chunks of 16 bytes
+        auto combined = [&](int q, float (&v)[32]) {   // columns c0 + 32 q .. + 31 of this lane, both teams, common reference
+          uint32_t a[32], bb[32];
+          tmem_ld32(tO + c0 + q * 32 + lane_addr, a);
+          tmem_ld32(tO + D + c0 + q * 32 + lane_addr, bb);
           tc_wait_ld();
 #pragma unroll
-          for (int k = 0; k < 32; ++k) o[k] = (f != 0.f) ? __float_as_uint(__uint_as_float(o[k]) * f) : 0u;
-          if (is_lo) {
+          for (int k = 0; k < 32; ++k)   // (an accumulator without a state may hold anything)
+            v[k] = (f0 != 0.f ? __uint_as_float(a[k]) * f0 : 0.f) + (f1 != 0.f ? __uint_as_float(bb[k]) * f1 : 0.f);
+        };
+        float v[D / 64][32];
+#pragma unroll
+        for (int q = 0; q < D / 64; ++q) combined(q, v[q]);
+        if (is_lo) {
+#pragma unroll
+          for (int q = 0; q < D / 64; ++q)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              x_lo[k ^ (rho & 3)] =
-                  make_uint4(pack_bf16x2(__uint_as_float(o[8 * k]), __uint_as_float(o[8 * k + 1])),
-                             pack_bf16x2(__uint_as_float(o[8 * k + 2]), __uint_as_float(o[8 * k + 3])),
-                             pack_bf16x2(__uint_as_float(o[8 * k + 4]), __uint_as_float(o[8 * k + 5])),
-                             pack_bf16x2(__uint_as_float(o[8 * k + 6]), __uint_as_float(o[8 * k + 7])));
-          } else if (tm == 1) {
+              xrow[((c0 + q * 32) / 8 + k) ^ (rho & (D / 8 - 1))] =
+                  make_uint4(pack_bf16x2(v[q][8 * k], v[q][8 * k + 1]), pack_bf16x2(v[q][8 * k + 2], v[q][8 * k + 3]),
+                             pack_bf16x2(v[q][8 * k + 4], v[q][8 * k + 5]), pack_bf16x2(v[q][8 * k + 6], v[q][8 * k + 7]));
+        }
+        all_barrier();
+        if (!is_lo && valid) {
+          float* slotp = P.pfx_partials + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hkv + g) * C::SLOT_FLOATS;
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-              x_hi[k ^ (rho & 7)] = make_float4(__uint_as_float(o[4 * k]), __uint_as_float(o[4 * k + 1]),
-                                               __uint_as_float(o[4 * k + 2]), __uint_as_float(o[4 * k + 3]));
-          }
-          all_barrier();
-          if (!is_lo && tm == 0 && valid) {
-            float4* dst = reinterpret_cast<float4*>(slotp + 2 * C::HP + rh * D + q * 32);
-            const uint4* lo0 = reinterpret_cast<const uint4*>(xo + 64 * 32) + rho * 4;
-            const uint4* lo1 = lo0 + 64 * 4;
+          for (int q = 0; q < D / 64; ++q) {
+            float4* dst = reinterpret_cast<float4*>(slotp + 2 * C::HP + rh * D + c0 + q * 32);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              const uint4 a = lo0[k ^ (rho & 3)], bq = lo1[k ^ (rho & 3)];
-              const float4 h0 = x_hi[(2 * k) ^ (rho & 7)], h1 = x_hi[(2 * k + 1) ^ (rho & 7)];
-              dst[2 * k] = make_float4(
-                  __uint_as_float(o[8 * k]) + h0.x + (__uint_as_float(a.x << 16) + __uint_as_float(bq.x << 16)),
-                  __uint_as_float(o[8 * k + 1]) + h0.y + (__uint_as_float(a.x & 0xffff0000u) + __uint_as_float(bq.x & 0xffff0000u)),
-                  __uint_as_float(o[8 * k + 2]) + h0.z + (__uint_as_float(a.y << 16) + __uint_as_float(bq.y << 16)),
-                  __uint_as_float(o[8 * k + 3]) + h0.w + (__uint_as_float(a.y & 0xffff0000u) + __uint_as_float(bq.y & 0xffff0000u)));
-              dst[2 * k + 1] = make_float4(
-                  __uint_as_float(o[8 * k + 4]) + h1.x + (__uint_as_float(a.z << 16) + __uint_as_float(bq.z << 16)),
-                  __uint_as_float(o[8 * k + 5]) + h1.y + (__uint_as_float(a.z & 0xffff0000u) + __uint_as_float(bq.z & 0xffff0000u)),
-                  __uint_as_float(o[8 * k + 6]) + h1.z + (__uint_as_float(a.w << 16) + __uint_as_float(bq.w << 16)),
-                  __uint_as_float(o[8 * k + 7]) + h1.w + (__uint_as_float(a.w & 0xffff0000u) + __uint_as_float(bq.w & 0xffff0000u)));
-            }
-            if (q == 0) {
-              slotp[rh] = mt;
-              slotp[C::HP + rh] = lt;
+              const uint4 w = xrow[((c0 + q * 32) / 8 + k) ^ (rho & (D / 8 - 1))];
+              dst[2 * k] = make_float4(v[q][8 * k] + __uint_as_float(w.x << 16), v[q][8 * k + 1] + __uint_as_float(w.x & 0xffff0000u),
+                                       v[q][8 * k + 2] + __uint_as_float(w.y << 16), v[q][8 * k + 3] + __uint_as_float(w.y & 0xffff0000u));
+              dst[2 * k + 1] = make_float4(v[q][8 * k + 4] + __uint_as_float(w.z << 16), v[q][8 * k + 5] + __uint_as_float(w.z & 0xffff0000u),
+                                           v[q][8 * k + 6] + __uint_as_float(w.w << 16), v[q][8 * k + 7] + __uint_as_float(w.w & 0xffff0000u));
             }
           }
-          all_barrier();   // the exchange area is used again
+          if (tm == 0) {
+            slotp[rh] = mt;
+            slotp[C::HP + rh] = xs[128 + rho] * f0 + xs[192 + rho] * f1;
+          }
         }
+        // (no barrier here: the next unit's writes to these areas come after its first barrier, which every
+        // thread reaches only after the reads above)
       }
       uc = nu;
     }
