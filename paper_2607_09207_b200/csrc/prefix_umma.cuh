@@ -21,9 +21,11 @@
 // teams never wait for each other and their per-tile chains (barrier wait, tensor-memory load, exponentials,
 // tensor-memory store, arrive) overlap; their states are merged at the end of the unit.  Warp w reaches lanes
 // 32 * (w % 4) .. + 31 only (a hardware rule); the thread in a row's first lane and the one in its second lane
-// both read the row's 64 scores and compute its 64 probabilities (nothing is exchanged inside a tile); the
-// first keeps the bf16 heads, the second the rests (both by truncation: no conversion instructions).  The
-// scores stay unscaled: the scale enters through the exponent's multiply-add, its sign through the staged Q.
+// both read the row's 64 scores and take the max themselves; each computes half of the row's exponentials and
+// hands the other the part that lane stores (64 bytes each way through shared memory, one barrier of the
+// team's four warps per tile); the first lane keeps the bf16 heads, the second the rests (both by
+// truncation: no conversion instructions).  The scores stay unscaled: the scale enters through the exponent's
+// multiply-add, its sign through the staged Q.
 // The reference value of the online softmax only follows the running max when that grew by more than 2^8,
 // so O in tensor memory is rarely rescaled.
 // Two MMA-issuing threads in two warps (scores; P.V), because the tensor cores take an MMA of this size
@@ -153,9 +155,10 @@ struct UmmaCfg {
   static constexpr int MMA_WARP = 8;                        // warps 0-7: softmax; 8, 9: MMA issue; 10, 11: producers
   static constexpr int NTHREADS = (MMA_WARP + 2 + NPW) * 32;
   static constexpr int CTRL_BYTES = 384;
-  static constexpr int XS_BYTES = 4 * 64 * 4;               // the teams' (m, l) per row, at the end of a unit
+  static constexpr int XS_BYTES = 6 * 64 * 4;               // the teams' m and the four partial row sums, at the end of a unit
+  static constexpr int XP_BYTES = 2 * 64 * 128;             // per team and row: the parts of P the row's two lanes hand each other
   static constexpr int XO_BYTES = 64 * D * 2;               // the second lanes' rows of O as bf16, at the end of a unit
-  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + XS_BYTES + XO_BYTES + CTRL_BYTES;
+  static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + XS_BYTES + XO_BYTES + XP_BYTES + CTRL_BYTES;
   static constexpr int HP = 8;                              // heads per partial slot (G <= 8)
   static constexpr int SLOT_FLOATS = HP * (D + 2);          // same slots as decode_kernel reads
   // tensor-memory columns: Q (D/2), S (2 x 64), P (2 x 32), O (2 x D): one score buffer, probability buffer and
@@ -214,9 +217,10 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   const uint32_t ring = raw + pad;                                  // NST stages, 1024-aligned
-  float* xs = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);   // [m | l][2 teams][64 rows]
-  float* xo = xs + 4 * 64;                                          // [64 rows][D] bf16
-  UmmaCtrl* ctrl = reinterpret_cast<UmmaCtrl*>(smem + NST * C::STAGE_BYTES + C::XS_BYTES + C::XO_BYTES);
+  float* xs = reinterpret_cast<float*>(smem + NST * C::STAGE_BYTES);   // [m | l first lanes | l second lanes][2 teams][64 rows]
+  float* xo = xs + 6 * 64;                                          // [64 rows][D] bf16
+  uint4* xp = reinterpret_cast<uint4*>(smem + NST * C::STAGE_BYTES + C::XS_BYTES + C::XO_BYTES);   // [2 teams][64 rows][8]
+  UmmaCtrl* ctrl = reinterpret_cast<UmmaCtrl*>(smem + NST * C::STAGE_BYTES + C::XS_BYTES + C::XO_BYTES + C::XP_BYTES);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int cta = blockIdx.x;
@@ -417,6 +421,7 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
       }
     };
     auto all_barrier = [&]() { asm volatile("bar.sync 5, 256;" ::: "memory"); };
+    auto team_barrier = [&]() { asm volatile("bar.sync %0, 128;" ::"r"(1 + tm) : "memory"); };
     auto q_row = [&](int u) {
       const int gi = u / P.Hkv, g = u - gi * P.Hkv;
       return P.q + (static_cast<int64_t>(gi * P.Gs + rj) * P.Hq + g * P.G + rh) * D;
@@ -496,34 +501,60 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         const float mu = (m_new == NEG_INF) ? 0.f : m_new;
         const float alpha = grow ? fast_exp2(m - mu) : 1.f;
         m = m_new;
-        // P = exp2(S * scale - m), split by truncation into a bf16 head (the row's first lane) and the bf16 head
-        // of what is left (its second lane): 16 bits of P between them, and no conversion instructions.  A P
-        // column holds two tokens.  The row sum is taken in the first lane only.
+        // the product that read this team's probability buffer two tiles ago must be done; it is also the
+        // latest product into this team's accumulator, and every thread of the team stored those probabilities
+        // after it had read the exchange area below, which is therefore free again
+        if (it >= 2) wait_all(&ctrl->pv_done[tm], ((it - 2) >> 1) & 1);
+        // P = exp2(S * scale - m), split by truncation into a bf16 head (the row's first lane stores the heads)
+        // and the bf16 head of what is left (its second lane stores those rests): 16 bits of P between them, and
+        // no conversion instructions.  Each lane computes half of the row's exponentials -- the first lane tokens
+        // 0-31, the second 32-63 -- and hands the other lane the part that lane stores, 64 bytes each way through
+        // shared memory behind a barrier of the team's four warps.  A P column holds two tokens.
         uint32_t pk[32];
         float ls = 0.f, ls1 = 0.f;
+        uint4* xq = xp + (tm * 64 + rho) * 8;      // this row's eight 16-byte chunks: rests of tokens 0-31, heads of 32-63
+        auto head_and_rest = [&](int k0, int k, uint32_t& head, uint32_t& rest) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sv[k0 + 2 * k]), sc, -mu));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sv[k0 + 2 * k + 1]), sc, -mu));
+          ls += p0;
+          ls1 += p1;
+          const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+          head = __byte_perm(b0, b1, 0x7632);
+          const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+          rest = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+        };
         if (!is_lo) {
+          uint32_t give[16];
 #pragma unroll
-          for (int k = 0; k < 32; ++k) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * k]), sc, -mu));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * k + 1]), sc, -mu));
-            ls += p0;
-            ls1 += p1;
-            pk[k] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
+          for (int k = 0; k < 16; ++k) head_and_rest(0, k, pk[k], give[k]);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) xq[c ^ (rho & 7)] = make_uint4(give[4 * c], give[4 * c + 1], give[4 * c + 2], give[4 * c + 3]);
+          team_barrier();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint4 w = xq[(4 + c) ^ (rho & 7)];
+            pk[16 + 4 * c] = w.x;
+            pk[16 + 4 * c + 1] = w.y;
+            pk[16 + 4 * c + 2] = w.z;
+            pk[16 + 4 * c + 3] = w.w;
           }
         } else {
+          uint32_t give[16];
 #pragma unroll
-          for (int k = 0; k < 32; ++k) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * k]), sc, -mu));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * k + 1]), sc, -mu));
-            const float r0 = p0 - __uint_as_float(__float_as_uint(p0) & 0xffff0000u);
-            const float r1 = p1 - __uint_as_float(__float_as_uint(p1) & 0xffff0000u);
-            pk[k] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+          for (int k = 0; k < 16; ++k) head_and_rest(32, k, give[k], pk[16 + k]);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) xq[(4 + c) ^ (rho & 7)] = make_uint4(give[4 * c], give[4 * c + 1], give[4 * c + 2], give[4 * c + 3]);
+          team_barrier();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint4 w = xq[c ^ (rho & 7)];
+            pk[4 * c] = w.x;
+            pk[4 * c + 1] = w.y;
+            pk[4 * c + 2] = w.z;
+            pk[4 * c + 3] = w.w;
           }
         }
-        l = l * alpha + (ls + ls1);
-        // the product that read this team's probability buffer two tiles ago must be done (it is also the
-        // latest product into this team's accumulator)
-        if (it >= 2) wait_all(&ctrl->pv_done[tm], ((it - 2) >> 1) & 1);
+        l = l * alpha + (ls + ls1);     // this lane's half of the row sum
         if (__any_sync(0xffffffffu, t >= 2 && alpha != 1.f)) {
           // new reference: scale this lane's row of O (rare: kept small rather than fast)
           tc_fence_after();
@@ -559,10 +590,8 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         const bool mine = pt >= 2 || owner;     // a one-tile unit leaves the other team without a state
         wait_all(&ctrl->unit_done, n & 1);
         tc_fence_after();
-        if (!is_lo) {
-          xs[tm * 64 + rho] = mine ? m : NEG_INF;
-          xs[128 + tm * 64 + rho] = mine ? l : 0.f;
-        }
+        if (!is_lo) xs[tm * 64 + rho] = mine ? m : NEG_INF;
+        xs[128 + (is_lo ? 128 : 0) + tm * 64 + rho] = mine ? l : 0.f;
         all_barrier();
         const float m0 = xs[rho], m1 = xs[64 + rho];
         const float mt = fmaxf(m0, m1);
@@ -608,7 +637,7 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           }
           if (tm == 0) {
             slotp[rh] = mt;
-            slotp[C::HP + rh] = xs[128 + rho] * f0 + xs[192 + rho] * f1;
+            slotp[C::HP + rh] = (xs[128 + rho] + xs[256 + rho]) * f0 + (xs[192 + rho] + xs[320 + rho]) * f1;
           }
         }
         // (no barrier here: the next unit's writes to these areas come after its first barrier, which every
