@@ -111,7 +111,9 @@ pdattn_status pdattn_decode_ex(const pdattn_args* args, pdattn_stream_t stream);
  * (within rounding: the summation order differs) and are bit-identical from run to run.
  *   prefix_tiles      DEVICE int32 [num_seqs / group_size]; prefix_tiles_host its HOST copy.
  *   Requirements: args->context_lens_host given; num_seqs a multiple of group_size; G <= 8 and
- *   group_size * G <= 64 (48 with pdattn_set_prefix_engine(0)), else PDATTN_UNSUPPORTED;
+ *   group_size * G <= 64 (48 with pdattn_set_prefix_engine(0)), else PDATTN_UNSUPPORTED -- a larger
+ *   group is passed as several groups of a divisor of its size with the same prefix_tiles entry (its
+ *   shared tiles are then read once per part);
  *   every member of group g has context_len > prefix_tiles[g] * 64
  *   (it owns at least its current token); 0 is allowed (the group shares nothing).
  *   args->workspace must hold pdattn_grouped_workspace_size() bytes.

@@ -91,6 +91,25 @@ def test_grouped_with_negative_and_zero_scale(factor):
     assert_parity(out, orc.decode_workload(w.to("cpu")), f"scale factor {factor}")
 
 
+def test_a_group_of_sixteen_passed_as_smaller_groups(prefix_engine):
+    """Sixteen samples of one prompt are more query rows than a unit holds (16 * 7 = 112 > 64): the caller passes
+    them as groups of eight (of four for the warp-MMA kernel, which takes 48 rows) with the same number of
+    shared tiles."""
+    rng = np.random.default_rng(5)
+    lens = [768 + int(x) for x in rng.integers(1, 500, size=32)]
+    w = W.make_custom(lens, Hq=28, Hkv=4, d=128, seed=81, device=DEV, poison=False)
+    bt = w.block_table.clone()
+    for lead in (0, 16):
+        for j in range(1, 16):
+            bt[lead + j, :48] = bt[lead, :48]
+    w = dataclasses.replace(w, block_table=bt)
+    W.poison_unused(w)
+    part = 4 if prefix_engine == "warp_mma" else 8
+    out, status = run_grouped(w, part, [12] * (32 // part))
+    assert status == pdattn.OK
+    assert_parity(out, orc.decode_workload(w.to("cpu")), "two prompts x sixteen samples")
+
+
 @pytest.mark.parametrize("bs", [32, 64])
 def test_grouped_with_larger_pages(bs):
     lens = [200, 70, 65, 1000, 129, 500, 66, 300]
