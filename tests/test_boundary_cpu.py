@@ -39,6 +39,24 @@ def test_library_exports_every_declared_symbol():
     assert set(pdattn.EXPORTS) <= set(syms)
 
 
+def test_header_and_library_from_plain_c(tmp_path):
+    """The public header parses as C99 (no C++ in it), the symbols link, and the entry points that need no GPU
+    behave as documented when called from C."""
+    import shutil
+    import subprocess
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        pytest.skip("no C compiler")
+    exe = str(tmp_path / "abi_check")
+    lib_dir = os.path.dirname(pd_build.LIB)
+    subprocess.check_call([cc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                           os.path.join(ROOT, "tests", "c", "abi_check.c"), "-o", exe, "-L", lib_dir, "-lpdattn",
+                           "-Wl,-rpath," + lib_dir])
+    out = subprocess.run([exe], capture_output=True, text=True, timeout=60)
+    assert out.returncode == 0, out.stdout + out.stderr
+    assert "abi_check: ok" in out.stdout
+
+
 def test_status_strings():
     L = pdattn.lib()
     assert L.pdattn_status_string(0) == b"ok"
