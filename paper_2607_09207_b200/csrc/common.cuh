@@ -237,7 +237,7 @@ struct Cfg {
   // tile is kept back and the warps exchange their accumulators through it.
   static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the parked stores conflict-free
   static constexpr int SMEM_MAX = 232448;              // 227 KB
-  static constexpr int CTRL_BYTES = 768;
+  static constexpr int CTRL_BYTES = 1024;
   static constexpr int NCW = PDATTN_NCW;                               // consumer warps
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
   static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged by producer 0
@@ -262,8 +262,10 @@ struct Cfg {
 };
 
 struct Ctrl {                 // lives in the CTRL_BYTES area
-  uint64_t full[MAX_STAGES];
-  uint64_t empty[MAX_STAGES];
+  uint64_t full[MAX_STAGES];    // the stage's tile has landed (with split halves: its K half)
+  uint64_t empty[MAX_STAGES];   // ... and has been consumed
+  uint64_t full_v[MAX_STAGES];  // split halves only: the V half, filled and released on its own
+  uint64_t empty_v[MAX_STAGES];
   uint32_t meta[MAX_STAGES];  // per stage: bit j set = page j of the tile had a bad id
   uint32_t abort;
   int32_t sq_pub;             // number of run-time span ids published so far
@@ -275,7 +277,7 @@ struct Ctrl {                 // lives in the CTRL_BYTES area
   int32_t qseq[4];            // CHAIN: piece whose rows the producer last armed the query slot for
   int32_t turn[8];            // CHAIN: hand-off slot e is waiting for class (turn % 8) of merge number (turn / 8)
 };
-static_assert(sizeof(Ctrl) <= 768, "control block");
+static_assert(sizeof(Ctrl) <= 1024, "control block");
 
 // ------------------------------------------------------------------------------------------
 // The walk over a span: pieces = (unit, tile range) in order.  Every warp runs the same walk.

@@ -164,12 +164,25 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         const uint32_t badmask = ctrl->meta[slot];
         const int n_left = pc.L - (pc.t0 + t) * TILE;
         if constexpr (EB == 2) {
+          // split stage halves: the K half goes back to the producers as soon as the scores are computed, and
+          // the V half is waited for only when the probabilities are ready
+          auto after_k = [&]() {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
+          };
+          auto before_v = [&]() {
+            if (!mbar_wait(smem_u32(&ctrl->full_v[slot]), (its / NST) & 1)) fail();
+          };
           if (n_left - (P.T - 1) >= TILE) {   // every query token sees the whole tile
-            compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag);
+            compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag, after_k, before_v);
           } else {
-            compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag);
+            compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag, after_k, before_v);
             fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
           }
+          if (aborted) break;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty_v[slot]));
+          continue;
         } else {
           if (n_left - (P.T - 1) >= TILE) {
             compute_tile_f8<NT, BS, false>(sK, sV, qf, acc, m, l, sl2, TILE, badmask, lane, lag);
@@ -365,6 +378,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     for (int i = 0; i < NST; ++i) {
       mbar_init(smem_u32(&ctrl->full[i]), 1);
       mbar_init(smem_u32(&ctrl->empty[i]), 1);
+      mbar_init(smem_u32(&ctrl->full_v[i]), 1);
+      mbar_init(smem_u32(&ctrl->empty_v[i]), 1);
     }
     ctrl->abort = 0;
     ctrl->sq_pub = 0;
@@ -389,6 +404,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   int pcnt = 0;      // piece counter within this CTA: piece p's query rows use query slot p % QSLOTS
   bool aborted = false;
 
+  // split stage halves: only where the consumers use them (chained merge over the bf16 cache)
+  constexpr bool SPLIT = CHAIN && EB == 2 && !PROBE;
   if (warp >= NCW) {
     // ================= producer warp(s) =================
     const int pw = warp - NCW;
@@ -470,6 +487,41 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           const bool bad = (lane < C::PAGES) && (j < np) && (id < 0 || id >= P.NB);
           const uint32_t badmask = __ballot_sync(0xffffffffu, bad);
           if (id < 0 || id >= P.NB) id = P.NB;   // out-of-bounds coordinate: TMA fills zeros, nothing is read
+          if constexpr (SPLIT) {
+            // K half and V half of the stage under their own barriers: the consumers hand the K half back
+            // after the scores and the V half after the products
+            const uint32_t bar_k = smem_u32(&ctrl->full[slot]);
+            if (lane == 0) {
+              ctrl->meta[slot] = badmask;
+              mbar_arrive_expect_tx(bar_k, static_cast<uint32_t>(np) * C::PAGE_BYTES);
+            }
+            __syncwarp();
+            if (lane < C::PAGES && j < np) {
+              const uint32_t dst = ring + slot * C::STAGE_BYTES + j * C::PAGE_BYTES;
+              if (P.box5d) {
+                tma_load_5d(dst, &tmK, 0, 0, 0, pc.g, id, bar_k);
+              } else {
+#pragma unroll
+                for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, &tmK, h * 64, 0, pc.g, id, bar_k);
+              }
+            }
+            if (!mbar_wait(smem_u32(&ctrl->empty_v[slot]), phase ^ 1u)) {
+              aborted = true;
+              break;
+            }
+            const uint32_t bar_v = smem_u32(&ctrl->full_v[slot]);
+            if (lane == 0) mbar_arrive_expect_tx(bar_v, static_cast<uint32_t>(np) * C::PAGE_BYTES);
+            __syncwarp();
+            if (lane < C::PAGES && j < np) {
+              const uint32_t dst = ring + slot * C::STAGE_BYTES + C::KV_BYTES + j * C::PAGE_BYTES;
+              if (P.box5d) {
+                tma_load_5d(dst, &tmV, 0, 0, 0, pc.g, id, bar_v);
+              } else {
+#pragma unroll
+                for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, &tmV, h * 64, 0, pc.g, id, bar_v);
+              }
+            }
+          } else {
           const uint32_t bar = smem_u32(&ctrl->full[slot]);
           if (lane == 0) {
             ctrl->meta[slot] = badmask;
@@ -486,6 +538,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
               for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, tm, h * 64, 0, pc.g, id, bar);
             }
+          }
           }
           any_bad |= (badmask != 0);
           if (NST % C::NPW != 0) {
@@ -629,9 +682,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         if (PROBE) {
           // ceiling probe: no math
         } else if (n_left - (P.T - 1) >= TILE) {   // every query token sees the whole tile
-          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag);
+          compute_tile<D, NT, BS, false>(sK, sV, qf, acc, m, l, P.scale_log2, TILE, badmask, lane, lag, [] {}, [] {});
         } else {
-          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag);
+          compute_tile<D, NT, BS, true>(sK, sV, qf, acc, m, l, P.scale_log2, n_left, badmask, lane, lag, [] {}, [] {});
           fence_proxy_async();   // our zero-fill stores must be ordered before the next TMA write
         }
         __syncwarp();

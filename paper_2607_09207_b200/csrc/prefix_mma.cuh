@@ -169,7 +169,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
       if (has_rows) {
         const uint32_t sK = ring + slot * C::STAGE_BYTES;
-        compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, P.scale_log2, TILE, ctrl->meta[slot], lane, no_lag);
+        compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, P.scale_log2, TILE, ctrl->meta[slot], lane, no_lag, [] {}, [] {});
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));

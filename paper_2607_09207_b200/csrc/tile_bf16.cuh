@@ -8,11 +8,13 @@ namespace pdattn {
 // ------------------------------------------------------------------------------------------
 // One 64-token tile on one warp
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS, bool TAIL>
+// after_k() is called right after the last read of the K tile, before_v() right before the first access to the V
+// tile (with split stage halves the caller releases K in the one and waits for V in the other).
+template <int D, int NT, int BS, bool TAIL, class AfterK, class BeforeV>
 __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uint32_t (&qf)[NT][D / 16][2],
                                              float (&acc)[NT][D / 16][4], float (&m)[NT][2], float (&l)[NT][2],
                                              float sl2, int n_left, uint32_t badmask, int lane,
-                                             const int (&lag)[NT][2]) {
+                                             const int (&lag)[NT][2], AfterK after_k, BeforeV before_v) {
   // n_left: tokens of the sequence from this tile's first one on (>= TILE unless TAIL)
   const int n_valid = n_left < TILE ? n_left : TILE;
   using C = Cfg<D, NT, BS>;
@@ -28,23 +30,6 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
   // V (A operand = V^T via .trans): matrices (tok 0-7,c), (tok 0-7,c+1), (tok 8-15,c), (tok 8-15,c+1)
   const int v_row = l8 + 8 * (mi >> 1);
   const int v_csel = mi & 1;
-
-  if (TAIL) {
-    // Zero the V rows past the last valid token inside its 16-token group: P is 0 there, but
-    // 0 * NaN would still poison the accumulator.
-    const int g_last = (n_valid - 1) >> 4;
-    const int r_beg = n_valid - (g_last << 4);   // 1..16
-    const int nrows = 16 - r_beg;
-    const int tok0 = (g_last << 4) + r_beg;
-    for (int idx = lane; idx < nrows * (D / 8); idx += 32) {
-      const int tok = tok0 + idx / (D / 8);
-      const int ch = idx % (D / 8);
-      const int page = tok / BS, row = tok % BS;
-      const uint32_t a = sV + page * C::PAGE_BYTES + (ch >> 3) * C::HALF_BYTES + row * 128 + ((ch & 7) << 4);
-      asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
-    }
-    __syncwarp();
-  }
 
   // ---- S^T = K . Q^T : [64 tokens] x [8*NT heads]
   float sc[GROUPS][NT][4];
@@ -67,6 +52,8 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
       }
     }
   }
+
+  after_k();
 
   // ---- scale, mask
   const int trow = lane >> 2;
@@ -146,6 +133,24 @@ __device__ __forceinline__ void compute_tile(uint32_t sK, uint32_t sV, const uin
       pl[j][nt][0] = movmatrix_trans(l01);
       pl[j][nt][1] = movmatrix_trans(l23);
     }
+
+  before_v();
+  if (TAIL) {
+    // Zero the V rows past the last valid token inside its 16-token group: P is 0 there, but
+    // 0 * NaN would still poison the accumulator.
+    const int g_last = (n_valid - 1) >> 4;
+    const int r_beg = n_valid - (g_last << 4);   // 1..16
+    const int nrows = 16 - r_beg;
+    const int tok0 = (g_last << 4) + r_beg;
+    for (int idx = lane; idx < nrows * (D / 8); idx += 32) {
+      const int tok = tok0 + idx / (D / 8);
+      const int ch = idx % (D / 8);
+      const int page = tok / BS, row = tok % BS;
+      const uint32_t a = sV + page * C::PAGE_BYTES + (ch >> 3) * C::HALF_BYTES + row * 128 + ((ch & 7) << 4);
+      asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+    }
+    __syncwarp();
+  }
 
   // ---- O^T += V^T . P^T : [D] x [8*NT heads], K = 64 tokens
 #pragma unroll
