@@ -17,10 +17,14 @@
 // Pins (tests/test_oracle_pins.py): L = 1 returns V exactly; equal keys / zero scale / zero q
 // return the mean of V; page permutation leaves the bits unchanged; dense brute force on tiny
 // inputs; L = 2 sigmoid closed form; dominant key; score-shift invariance; convex-hull bound
-// and linearity in V; split/merge identity; fp64 library softmax-matmul on an identity table.
+// and linearity in V; split/merge identity; fp64 library softmax-matmul on an identity table;
+// the (sequence, head) pair list against the rows of the full output; the fp8 variants against
+// the bf16 path on the decoded values and a dense masked softmax.
 //
 // Out-of-range block_table entries (id < 0 or id >= num_blocks) inside a sequence's used range
-// are not dereferenced: their tokens are left out of the softmax and counted in *bad_pages.
+// are not dereferenced: their tokens are left out of the softmax (an explicit mask, not a marker
+// value in the scores) and counted in *bad_pages.  Valid inputs are finite; a NaN that reaches a
+// live slot all the same propagates to that head's output.
 
 #include <atomic>
 #include <cmath>
@@ -72,18 +76,21 @@ struct Problem {
     double scale;
 };
 
-// Scores x_t = scale * <q, k_t> for t in [t0, t1); entries of bad pages become NaN markers (skipped).
+// Scores x_t = scale * <q, k_t> for t in [t0, t1).  live[t - t0] = 0 marks a token whose page id is out
+// of range: its score is never computed and it is left out of the softmax.  A NaN that the arithmetic
+// itself produces in a live slot stays in x and propagates to the output.
 // Returns number of tokens skipped because their page id is out of range.
-int64_t scores(const Problem& P, int s, int h, int t0, int t1, std::vector<double>& x) {
+int64_t scores(const Problem& P, int s, int h, int t0, int t1, std::vector<double>& x, std::vector<char>& live) {
     const int G = P.Hq / P.Hkv;
     const int g = h / G;
     const uint16_t* qrow = P.q + (static_cast<int64_t>(s) * P.Hq + h) * P.d;
     int64_t skipped = 0;
     x.assign(static_cast<size_t>(t1 - t0), 0.0);
+    live.assign(static_cast<size_t>(t1 - t0), 1);
     for (int t = t0; t < t1; ++t) {
         int32_t page = P.block_table[static_cast<int64_t>(s) * P.MB + t / P.bs];
         if (page < 0 || page >= P.NB) {
-            x[t - t0] = std::numeric_limits<double>::quiet_NaN();
+            live[t - t0] = 0;
             ++skipped;
             continue;
         }
@@ -101,15 +108,21 @@ int64_t partial(const Problem& P, int s, int h, int t0, int t1, double* m_out, d
     const int G = P.Hq / P.Hkv;
     const int g = h / G;
     std::vector<double> x;
-    int64_t skipped = scores(P, s, h, t0, t1, x);
+    std::vector<char> live;
+    int64_t skipped = scores(P, s, h, t0, t1, x, live);
+    // max over the live scores; a NaN among them makes the max (and with it every weight) NaN
     double m = -std::numeric_limits<double>::infinity();
-    for (double xv : x)
-        if (!std::isnan(xv) && xv > m) m = xv;
+    for (int t = t0; t < t1; ++t) {
+        if (!live[t - t0]) continue;
+        const double xv = x[t - t0];
+        if (std::isnan(xv) || xv > m) m = xv;
+        if (std::isnan(m)) break;
+    }
     double l = 0.0;
     for (int j = 0; j < P.d; ++j) acc[j] = 0.0;
     for (int t = t0; t < t1; ++t) {
+        if (!live[t - t0]) continue;
         double xv = x[t - t0];
-        if (std::isnan(xv)) continue;
         double w = std::exp(xv - m);
         l += w;
         int32_t page = P.block_table[static_cast<int64_t>(s) * P.MB + t / P.bs];
@@ -130,7 +143,7 @@ int64_t one_output(const Problem& P, int s, int h, double* out) {
     }
     double m, l;
     int64_t skipped = partial(P, s, h, 0, L, &m, &l, out);
-    if (l > 0.0) {
+    if (l > 0.0 || std::isnan(l)) {
         for (int j = 0; j < P.d; ++j) out[j] /= l;
     } else {
         for (int j = 0; j < P.d; ++j) out[j] = 0.0;   // every token sat in a bad page
@@ -213,12 +226,12 @@ int pdattn_oracle_merge(const double* m, const double* l, const double* acc, int
     double Lsum = 0.0;
     for (int j = 0; j < head_dim; ++j) out[j] = 0.0;
     for (int c = 0; c < n; ++c) {
-        if (!(l[c] > 0.0)) continue;
+        if (!(l[c] > 0.0) && !std::isnan(l[c])) continue;   // an empty partial; a NaN one propagates
         double f = std::exp(m[c] - M);
         Lsum += l[c] * f;
         for (int j = 0; j < head_dim; ++j) out[j] += acc[static_cast<int64_t>(c) * head_dim + j] * f;
     }
-    if (Lsum > 0.0)
+    if (Lsum > 0.0 || std::isnan(Lsum))
         for (int j = 0; j < head_dim; ++j) out[j] /= Lsum;
     return 0;
 }
@@ -254,6 +267,7 @@ int pdattn_oracle_decode_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t
     std::atomic<int64_t> next{0}, skipped{0};
     auto worker = [&]() {
         std::vector<double> x;
+        std::vector<char> live;
         for (;;) {
             const int64_t i = next.fetch_add(1);
             if (i >= total) break;
@@ -264,11 +278,12 @@ int pdattn_oracle_decode_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t
             if (L <= 0) continue;
             const uint16_t* qrow = q + i * d;
             x.assign(static_cast<size_t>(L), 0.0);
+            live.assign(static_cast<size_t>(L), 1);
             double xmax = -std::numeric_limits<double>::infinity();
             for (int t = 0; t < L; ++t) {
                 const int32_t page = block_table[static_cast<int64_t>(s) * max_blocks_per_seq + t / bs];
                 if (page < 0 || page >= num_blocks) {     // not dereferenced, left out of the softmax, counted
-                    x[t] = std::numeric_limits<double>::quiet_NaN();
+                    live[t] = 0;
                     ++skipped;
                     continue;
                 }
@@ -277,11 +292,11 @@ int pdattn_oracle_decode_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t
                 for (int j = 0; j < d; ++j)
                     acc += bf16_to_double(qrow[j]) * (static_cast<double>(k_scale[g]) * pdattn_oracle_e4m3_to_double(krow[j]));
                 x[t] = static_cast<double>(scale) * acc;
-                if (x[t] > xmax) xmax = x[t];
+                if (std::isnan(x[t]) || x[t] > xmax) xmax = x[t];   // a NaN score of a live slot propagates
             }
             double Z = 0.0;
             for (int t = 0; t < L; ++t) {
-                if (std::isnan(x[t])) continue;
+                if (!live[t]) continue;
                 const double w = std::exp(x[t] - xmax);
                 Z += w;
                 const int32_t page = block_table[static_cast<int64_t>(s) * max_blocks_per_seq + t / bs];
@@ -289,7 +304,7 @@ int pdattn_oracle_decode_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t
                 for (int j = 0; j < d; ++j)
                     o[j] += w * (static_cast<double>(v_scale[g]) * pdattn_oracle_e4m3_to_double(vblk[j * bs + t % bs]));
             }
-            for (int j = 0; j < d; ++j) o[j] = Z > 0.0 ? o[j] / Z : 0.0;
+            for (int j = 0; j < d; ++j) o[j] = (Z > 0.0 || std::isnan(Z)) ? o[j] / Z : 0.0;
         }
     };
     const int nt = num_threads > 0 ? num_threads : 1;

@@ -358,3 +358,122 @@ def test_e4m3_encoder_matches_the_library_cast_and_round_trips():
     assert np.array_equal(back[codes != 0x80], codes[codes != 0x80]) and back[codes == 0x80][0] in (0x00, 0x80)
     # a tie goes to the even code: 17 lies halfway between 16 (code 0x58) and 18 (0x59)
     assert orc.e4m3_encode(np.array([17.0, 19.0], dtype=np.float32)).tolist() == [0x58, 0x5a]
+
+
+def test_pair_list_equals_the_rows_of_the_full_output():
+    """decode(pairs=P) must return, row by row, exactly what the full output holds at (seq, head) = P[i]: an
+    off-by-one in the pair indexing, a swapped (head, seq) order, an output row written at the pair's own
+    index instead of its position in the list, or a stale row for a repeated pair would all show."""
+    w = W.make_custom([1, 17, 100, 0, 256, 33, 64], Hq=6, Hkv=2, d=32, seed=81, num_blocks=64)
+    full = orc.decode_workload(w)
+    pairs = np.array([[4, 5], [0, 0], [6, 3], [1, 2], [4, 5], [3, 1], [2, 4], [6, 0], [1, 2], [5, 5]], dtype=np.int32)
+    for nt in (1, 3):
+        got = orc.decode_workload(w, pairs=pairs, num_threads=nt)
+        assert got.shape == (len(pairs), 32)
+        for i, (s, h) in enumerate(pairs):
+            assert np.array_equal(got[i], full[s, h]), (i, s, h)
+    # pairs of a sequence with a bad page count their own skipped tokens only
+    bt = w.block_table.clone()
+    bt[2, 3] = -7                                       # tokens 48..63 of sequence 2
+    w.block_table = bt
+    _, bad = orc.decode_workload(w, pairs=np.array([[2, 0], [2, 5], [4, 1]]), return_bad=True)
+    assert bad == 2 * 16
+
+
+def test_fp8_append_then_attend_equals_the_longer_cache():
+    """fp8 append pin: take an fp8 cache of L + 1 tokens, lift the last token's decoded values times the scale
+    out, poison its slot in K (a row) and in the transposed V page (a column), append it back.  The code bytes
+    of both pools must be those of the original: a V column written as a row, a slot/dim swap, the wrong page,
+    a scale applied the wrong way round or a length not advanced would all show.  Then the skip rules."""
+    lens = [16, 33, 1, 47]                            # the appended token lands at slot 0, 1, 1 and 15
+    bs, Hkv, d = 16, 2, 32
+    full = W.make_custom([L + 1 for L in lens], Hq=4, Hkv=Hkv, d=d, bs=bs, seed=82, num_blocks=16)
+    ks, vs = torch.tensor([0.5, 2.0]), torch.tensor([4.0, 0.25])          # powers of two: value = scale * code exactly
+    k8, v8 = W.fp8_caches(full, ks, vs)
+    ref_out = orc.decode_fp8(full.q, k8, v8, ks, vs, full.block_table, full.context_lens, full.scale)
+    k8c, v8c = k8.clone(), v8.clone()
+    bt = full.block_table.numpy()
+    k_new = torch.zeros(len(lens), Hkv, d, dtype=BF16)
+    v_new = torch.zeros(len(lens), Hkv, d, dtype=BF16)
+    kval = orc.e4m3_to_double(k8.numpy()).reshape(k8.shape)               # [page, head, slot, dim]
+    vval = orc.e4m3_to_double(v8.numpy()).reshape(v8.shape)               # [page, head, dim, slot]
+    for s, L in enumerate(lens):
+        page, slot = int(bt[s, L // bs]), L % bs
+        k_new[s] = torch.from_numpy(kval[page, :, slot, :] * ks.numpy()[:, None]).to(BF16)
+        v_new[s] = torch.from_numpy(vval[page, :, :, slot] * vs.numpy()[:, None]).to(BF16)
+        k8c[page, :, slot, :] = 0x7f
+        v8c[page, :, :, slot] = 0x7f
+    assert not torch.equal(k8c, k8) and not torch.equal(v8c, v8)
+    cl = torch.tensor(lens, dtype=torch.int32)
+    assert orc.append_kv_fp8(k8c, v8c, ks, vs, full.block_table, cl, k_new, v_new) == 0
+    assert cl.tolist() == [L + 1 for L in lens]
+    assert torch.equal(k8c, k8) and torch.equal(v8c, v8)
+    assert np.array_equal(orc.decode_fp8(full.q, k8c, v8c, ks, vs, full.block_table, cl, full.scale), ref_out)
+    # skip rules: a bad page id and a full table row leave pools and length untouched and are counted
+    bt2 = full.block_table.clone()
+    cl2 = torch.tensor([5, 5, 5, 5], dtype=torch.int32)
+    bt2[1, 0] = 99
+    bt2[2, 0] = -1
+    before_k, before_v = k8c.clone(), v8c.clone()
+    MB = bt2.shape[1]
+    cl2[3] = MB * bs                                   # row full
+    skipped = orc.append_kv_fp8(k8c, v8c, ks, vs, bt2, cl2, k_new, v_new)
+    assert skipped == 3 and cl2.tolist() == [6, 5, 5, MB * bs]
+    page0 = int(bt2[0, 0])
+    changed_k = (k8c != before_k).any(dim=(1, 2, 3)).nonzero().flatten().tolist()
+    changed_v = (v8c != before_v).any(dim=(1, 2, 3)).nonzero().flatten().tolist()
+    assert set(changed_k) <= {page0} and set(changed_v) <= {page0}
+    assert torch.equal(k8c[page0, :, 5, :], torch.from_numpy(orc.e4m3_encode(
+        k_new[0].float().numpy() / ks.numpy()[:, None])))
+    assert torch.equal(v8c[page0, :, :, 5], torch.from_numpy(orc.e4m3_encode(
+        v_new[0].float().numpy() / vs.numpy()[:, None])))
+
+
+def test_fp8_multi_token_queries_match_a_dense_causal_softmax():
+    """decode_fp8_multi against a textbook masked softmax on the decoded values (scale * code), the mask written
+    as a matrix: a wrong truncation per query token, a transposed V page or a scale on the wrong operand shows."""
+    for seed, (Hq, Hkv, d, bs, T) in enumerate([(4, 2, 32, 16, 2), (6, 2, 64, 32, 3), (4, 1, 128, 16, 4)]):
+        lens = [T, T + 1, 16, 17, 63, 64, 65, 130, 2]
+        w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, bs=bs, seed=90 + seed, num_blocks=64)
+        S, G = len(lens), Hq // Hkv
+        ks = torch.linspace(0.5, 1.5, Hkv)
+        vs = torch.linspace(2.0, 0.75, Hkv)
+        k8, v8 = W.fp8_caches(w, ks, vs)
+        q = W.normal_bf16(S * T * Hq * d, 950 + seed, 1).view(S, T, Hq, d)
+        got = orc.decode_fp8_multi(q, k8, v8, ks, vs, w.block_table, w.context_lens, w.scale)
+        kval = orc.e4m3_to_double(k8.numpy()).reshape(k8.shape) * ks.double().numpy()[None, :, None, None]
+        vval = orc.e4m3_to_double(v8.numpy()).reshape(v8.shape) * vs.double().numpy()[None, :, None, None]
+        bt = w.block_table.numpy()
+        qf = f64(q)
+        for s in range(S):
+            L = lens[s]
+            K = np.stack([kval[bt[s, t // bs], :, t % bs, :] for t in range(L)])      # [L, Hkv, d]
+            V = np.stack([vval[bt[s, t // bs], :, :, t % bs] for t in range(L)])      # [L, Hkv, d]
+            mask = np.array([[t <= L - T + j for t in range(L)] for j in range(T)])
+            for h in range(Hq):
+                x = (qf[s, :, h, :] @ K[:, h // G, :].T) * float(np.float32(w.scale))
+                x = np.where(mask, x, -np.inf)
+                for j in range(T):
+                    if not mask[j].any():
+                        assert not got[s, j, h].any()
+                        continue
+                    p = np.exp(x[j] - x[j].max())
+                    p /= p.sum()
+                    np.testing.assert_allclose(got[s, j, h], p @ V[:, h // G, :], rtol=1e-12, atol=1e-14)
+
+
+def test_a_nan_in_a_live_slot_propagates_while_a_bad_page_is_masked():
+    """The bad-page rule is a mask, not a marker value: a NaN key in a slot the sequence owns must reach that KV
+    head's outputs (and only those), in the bf16 path, the pair path and the fp8 path."""
+    w = W.make_custom([40, 20], Hq=4, Hkv=2, d=32, seed=83, num_blocks=16, poison=False)
+    bt = w.block_table.numpy()
+    w.k_cache[int(bt[0, 1]), 1, 3, 5] = float("nan")            # token 19 of sequence 0, KV head 1
+    out = orc.decode_workload(w)
+    assert np.isnan(out[0, 2:]).all() and np.isfinite(out[0, :2]).all() and np.isfinite(out[1]).all()
+    got = orc.decode_workload(w, pairs=np.array([[0, 3], [0, 0]]))
+    assert np.isnan(got[0]).all() and np.isfinite(got[1]).all()
+    one = torch.ones(2)
+    k8, v8 = W.fp8_caches(w, one, one)
+    assert k8[int(bt[0, 1]), 1, 3, 5] == 0x7f
+    out8 = orc.decode_fp8(w.q, k8, v8, one, one, w.block_table, w.context_lens, w.scale)
+    assert np.isnan(out8[0, 2:]).all() and np.isfinite(out8[0, :2]).all() and np.isfinite(out8[1]).all()
