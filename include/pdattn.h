@@ -20,7 +20,10 @@
  *     memory.  All memory is caller-owned; the library never allocates, frees or keeps device
  *     memory, creates no streams, and synchronises only where stated.
  *   - Work is enqueued on `stream`; outputs are valid once the stream reaches that point.
- *   - The only state is the thread-local binding made by pdattn_bind().
+ *   - State.  Per thread: the binding made by pdattn_bind(), the events of pdattn_profile_events(), the
+ *     launch count and the text of the last CUDA failure.  Process-wide: the four tuning settings
+ *     pdattn_set_dynamic_spans / _merge_mode / _prefix_engine / _host_zero_copy (plain ints; set them
+ *     before the threads that decode start, not concurrently with a call).
  */
 #ifndef PDATTN_H_
 #define PDATTN_H_
@@ -38,7 +41,8 @@ typedef int pdattn_status;
 #define PDATTN_UNSUPPORTED         (-2) /* head_dim not in {64,128}, block_size not in {16,32,64}, G > 16, or a
                                            cache stride that is not a multiple of 8 elements          */
 #define PDATTN_WORKSPACE_TOO_SMALL (-3)
-#define PDATTN_MISALIGNED          (-4) /* q / k_cache / v_cache / out / workspace not 16-byte aligned */
+#define PDATTN_MISALIGNED          (-4) /* q / k_cache / v_cache / out not 16-byte aligned, or workspace /
+                                           staging not 256-byte aligned                              */
 #define PDATTN_NOT_BOUND           (-5) /* pdattn_decode() without pdattn_bind() on this thread       */
 #define PDATTN_CUDA_ERROR          (-6) /* a CUDA call failed; text in pdattn_last_cuda_error()       */
 #define PDATTN_BAD_PAGE_INDEX      (-7) /* reported by pdattn_check(): a used block_table entry was
@@ -50,7 +54,9 @@ typedef struct CUstream_st* pdattn_stream_t; /* a cudaStream_t */
 
 /*
  * Size of the scratch area a decode call needs (the partial (m, l, acc) triples of split
- * sequences, the per-CTA work spans and one sticky error word).  max_context_len is accepted
+ * sequences, the per-CTA work spans and one sticky error word).  Splitting exists because of the
+ * length skew of rollout batches (Section 2.3: a few long responses dominate the decoding time), so
+ * the size depends on the head shape and the SM count, not on the context lengths.  max_context_len is accepted
  * for forward compatibility and does not change the result today.  pinned_host_bytes (optional)
  * receives 0: no pinned staging is needed.
  */
@@ -73,7 +79,7 @@ typedef struct {
   void* out;                        /* DEVICE bf16 [num_seqs, num_q_heads, head_dim], dense          */
   const int32_t* block_table;       /* DEVICE int32 [num_seqs, max_blocks_per_seq], row-major.        */
                                     /*   Entries at or past ceil(L_s/block_size) are never read.      */
-  const int32_t* context_lens;      /* DEVICE int32 [num_seqs]                                        */
+  const int32_t* context_lens;      /* DEVICE int32 [num_seqs]; L_s <= max_blocks_per_seq * block_size */
   const int32_t* context_lens_host; /* HOST copy of context_lens for the host partitioner, or NULL:   */
                                     /*   then a small planning kernel runs on the device instead.      */
                                     /*   Read during the call only.  Must equal the device array.      */
@@ -95,6 +101,10 @@ typedef struct {
  *     and do not influence `out`.
  *   - A used block_table entry outside [0, num_blocks) is not dereferenced: its tokens are left
  *     out of the softmax and the workspace's sticky error word is set (see pdattn_check).
+ *   - A context length beyond max_blocks_per_seq * block_size (more tokens than the table row can
+ *     describe) is refused with PDATTN_INVALID_ARG when context_lens_host is given.  Without the host
+ *     copy the entries past the row's end are never read: those tokens are treated like a bad page
+ *     (left out, error word set).
  *   - The result is a pure function of the logical inputs: bit-identical from run to run, under
  *     any renumbering of physical pages, and for shared versus privately copied prefix pages.
  *   - Two calls that share a workspace must not overlap on the GPU.
@@ -198,15 +208,19 @@ pdattn_status pdattn_append_kv(const void* k_new, const void* v_new, void* k_cac
                                int64_t kv_token_stride, void* workspace, pdattn_stream_t stream);
 
 /*
- * Thread-local binding of the arguments the short form below does not carry.
- * context_lens_host may be NULL.  The pointers must stay valid while bound.
+ * Thread-local binding of the arguments the short form below does not carry: the block table's row
+ * stride and the pool size (the paged cache of Appendix A.1.2's b_kv bytes per token), the workspace,
+ * and the optional host copy of the lengths.  context_lens_host may be NULL.  The pointers must stay
+ * valid while bound.  (No pinned-host arguments: the library needs no pinned staging.)
  */
 pdattn_status pdattn_bind(int max_blocks_per_seq, int num_blocks, void* workspace,
                           size_t workspace_bytes, const int32_t* context_lens_host);
 
 /*
- * Short form: dense caches [num_blocks, num_kv_heads, block_size, head_dim]; everything else as
- * pdattn_decode_ex with the values bound on this thread.
+ * Short form of the decode step (the attention part of the rollout's decoding loop, Section 2.1 and
+ * Section 2.3, with the arguments of the problem statement): dense caches
+ * [num_blocks, num_kv_heads, block_size, head_dim]; everything else as pdattn_decode_ex with the values
+ * bound on this thread.  PDATTN_NOT_BOUND without a binding.
  */
 pdattn_status pdattn_decode(const void* q, const void* k_cache, const void* v_cache,
                             const int32_t* block_table, const int32_t* context_lens,
@@ -272,9 +286,9 @@ pdattn_status pdattn_set_dynamic_spans(int per_cta);
  * chain of warps through shared memory and no warp waits for the others, so several short pieces
  * are in work at once.  0: all warps meet at a barrier and sum their states together; on long
  * pieces (tens of tiles) this costs the same, on batches of short contexts one barrier round per
- * piece.  -1 (default): 1, except for calls with run-time spans, which always use 0.  Either way
- * the order of every sum is fixed by tile indices, so a setting's results are bit-identical from
- * run to run and under any renumbering of the physical pages.
+ * piece.  -1 (default): 1, with static and with run-time spans alike.  Either way the order of every
+ * sum is fixed by tile indices, so a setting's results are bit-identical from run to run and under any
+ * renumbering of the physical pages.
  */
 pdattn_status pdattn_set_merge_mode(int mode);
 
@@ -288,8 +302,10 @@ pdattn_status pdattn_set_merge_mode(int mode);
 pdattn_status pdattn_set_prefix_engine(int engine);
 
 /*
- * Synchronises `stream`, reads and clears the workspace's sticky error word.
- * Returns PDATTN_OK, PDATTN_BAD_PAGE_INDEX or PDATTN_DEVICE_TIMEOUT.
+ * Error report of the decode steps enqueued so far (no paper counterpart; the rollout loop of Section 2.3
+ * would call it once per step or less).  Synchronises `stream`, reads and clears the workspace's sticky
+ * error word (hence a non-const pointer).  Returns PDATTN_OK, PDATTN_BAD_PAGE_INDEX or
+ * PDATTN_DEVICE_TIMEOUT.  workspace: DEVICE.
  */
 pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream);
 
@@ -310,7 +326,8 @@ pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream);
  *   - status_out (DEVICE int32, optional): receives 0, or the error bits of this call
  *     (1 = a used block_table entry was out of range, 2 = a bounded wait expired), on `stream`.
  *   - The first call on a device looks up the array's device address (one-time set-up, no
- *     allocation); make that first call before any stream capture is begun.
+ *     allocation); make that first call before any stream capture is begun.  The address is cached
+ *     per device for the life of the process and does not survive a cudaDeviceReset.
  *   - All calls on a device share the one array and it keeps the previous call's contents (the
  *     library clears the words that must start at zero).  Two calls that overlap on the GPU, from
  *     different streams or threads, race on it: serialise them, or use pdattn_decode_ex with
@@ -351,6 +368,7 @@ pdattn_status pdattn_wait_limit_probe(void* workspace, int limit_us, pdattn_stre
 /* Number of kernels the last pdattn_decode_ex on this thread launched (2 or 3). */
 int pdattn_last_launch_count(void);
 
+/* Fixed English text for a status code (no paper counterpart); never NULL, never freed. */
 const char* pdattn_status_string(pdattn_status status);
 const char* pdattn_last_cuda_error(void); /* thread-local text of the last CUDA failure */
 

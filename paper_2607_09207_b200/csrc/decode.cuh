@@ -448,15 +448,17 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
         const int npages = (pc.L + BS - 1) / BS;
         const int pbase = (pc.t0 + pc.tb) * C::PAGES;
-        int ids_cur = (pbase + lane < npages) ? __ldg(row + pbase + lane) : 0;
-        int ids_nxt = (pbase + IDS_PER_BATCH + lane < npages) ? __ldg(row + pbase + IDS_PER_BATCH + lane) : 0;
+        // A context length beyond what the table row can describe: the entries past the row's end are not
+        // read (they belong to the next row, or lie past the allocation); their tokens count as a bad page.
+        auto page_id = [&](int idx) { return idx < npages ? (idx < P.MB ? __ldg(row + idx) : -1) : 0; };
+        int ids_cur = page_id(pbase + lane);
+        int ids_nxt = page_id(pbase + IDS_PER_BATCH + lane);
         for (int t = pc.tb; t < pc.te; ++t, ++it) {
           const int rel = t - pc.tb;
           const int kb = rel % TILES_PER_BATCH;
           if (kb == 0 && rel != 0) {
             ids_cur = ids_nxt;
-            const int nb = pbase + rel * C::PAGES + IDS_PER_BATCH;
-            ids_nxt = (nb + lane < npages) ? __ldg(row + nb + lane) : 0;
+            ids_nxt = page_id(pbase + rel * C::PAGES + IDS_PER_BATCH + lane);
           }
           if (C::NPW > 1 && it % C::NPW != pw) continue;
           const int slot = it % NST;

@@ -1,5 +1,6 @@
 // Host side of libpdattn: argument checks, the host partitioner call, TMA tensor maps, launches.
-// No allocation, no synchronisation (except pdattn_check), no state beyond thread-locals.
+// No allocation, no synchronisation (except pdattn_check).  State: the process-wide pdattn_set_* settings, and per
+// thread the pdattn_bind binding, the profiling events, the tensor-map cache and the last error text.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -21,29 +22,38 @@ using namespace pdattn;
 thread_local char g_cuda_err[256] = "";
 thread_local int g_last_launches = 0;
 thread_local cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
-thread_local bool g_probe_mode = false;   // set only inside pdattn_gather_probe
-struct GroupedCall {                      // set only inside pdattn_decode_grouped
-  bool active = false;
-  int group_size = 0;
-  const int32_t* prefix_tiles = nullptr;        // device, per group
-  const int32_t* prefix_tiles_host = nullptr;   // host copy
-};
-thread_local GroupedCall g_grouped;
-thread_local std::vector<int32_t> g_start_tiles_host;
+// Process-wide settings (the pdattn_set_* calls); everything that belongs to one call travels in a CallDesc.
 int g_dyn_per_cta = -1;                   // run-time spans per CTA (pdattn_set_dynamic_spans); -1: by batch shape
 constexpr int kAutoDynPerCta = 4;         // ... then this many when the batch has at least kAutoDynUnits units per CTA
 constexpr int kAutoDynUnits = 4;
 int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (chained), 0 barrier, 1 chained
-thread_local bool g_use_chain = true;     // decided per call, read by the launcher
-struct Fp8Call {
-  bool active = false;
-  const float* k_scale = nullptr;
-  const float* v_scale = nullptr;
-};
-thread_local Fp8Call g_fp8;               // set by pdattn_decode_fp8 around the common path
-thread_local int g_query_tokens = 1;      // query tokens per sequence of the call (pdattn_decode_multi)
 int g_host_zero_copy = -1;                // pdattn_set_host_zero_copy: -1 default (when possible), 0 never, 1 as -1
 int g_prefix_engine = -1;                 // pdattn_set_prefix_engine: -1 default (tcgen05), 0 warp MMAs, 1 tcgen05
+thread_local std::vector<int32_t> g_start_tiles_host;   // scratch of the grouped path (no call parameter lives here)
+
+// What one decode call is, beyond the plain arguments: every entry point fills one of these and hands it to
+// decode_common.
+struct CallDesc {
+  int query_tokens = 1;                         // pdattn_decode_multi
+  bool probe = false;                           // pdattn_gather_probe: same walk and loads, no math, no output
+  bool fp8 = false;                             // pdattn_decode_fp8: e4m3 codes, one scale per KV head
+  const float* k_scale = nullptr;
+  const float* v_scale = nullptr;
+  int group_size = 0;                           // pdattn_decode_grouped: > 0, with the shared tiles per group
+  const int32_t* prefix_tiles = nullptr;        //   device copy
+  const int32_t* prefix_tiles_host = nullptr;   //   host copy
+  bool static_scratch = false;                  // pdattn_decode_static_scratch: scratch is the built-in array
+  int32_t* status_out = nullptr;                //   device word that receives the error word after the call
+};
+
+// What the launchers need to pick a kernel instantiation.
+struct DevInfo;
+struct LaunchCtx {
+  int block_size;
+  bool chain, probe, fp8;
+  DevInfo* di;
+  cudaStream_t stream;
+};
 
 struct Binding {
   bool set = false;
@@ -65,16 +75,17 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct WsLayout {
   size_t hdr, spans, rec, prefix, partials, total;
 };
-WsLayout ws_layout(int num_seqs, int G, int head_dim) {
+// max_spans: spans the span table, the records and the partial slots are sized for
+WsLayout ws_layout(int num_seqs, int G, int head_dim, int max_spans = MAX_SPANS) {
   const int NT = G > 8 ? 2 : 1;
   const size_t slot_bytes = static_cast<size_t>(8 * NT) * (head_dim + 2) * 4;
   WsLayout w;
   w.hdr = 0;
   w.spans = 256;
-  w.rec = w.spans + align_up(static_cast<size_t>(MAX_SPANS + 1) * sizeof(SpanStart), 256);
-  w.prefix = w.rec + align_up(static_cast<size_t>(MAX_SPANS) * sizeof(int4), 256);
+  w.rec = w.spans + align_up(static_cast<size_t>(max_spans + 1) * sizeof(SpanStart), 256);
+  w.prefix = w.rec + align_up(static_cast<size_t>(max_spans) * sizeof(int4), 256);
   w.partials = w.prefix + align_up(static_cast<size_t>(num_seqs + 1) * 8, 256);
-  w.total = w.partials + align_up(static_cast<size_t>(MAX_SPANS) * 2 * slot_bytes, 256);
+  w.total = w.partials + align_up(static_cast<size_t>(max_spans) * 2 * slot_bytes, 256);
   return w;
 }
 
@@ -264,8 +275,10 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size
 
 template <int D, int NT, int BS>
 pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
-                     int n_spans_host, DevInfo* di, cudaStream_t stream) {
+                     int n_spans_host, const LaunchCtx& lc) {
   using C = Cfg<D, NT, BS>;
+  DevInfo* di = lc.di;
+  cudaStream_t stream = lc.stream;
   auto kern = decode_kernel<D, NT, BS>;
   bool& done = di->attr_set[D == 128][NT == 2][BS / 32];
   if (!done) {
@@ -273,7 +286,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
     done = true;
   }
-  if (g_probe_mode) {
+  if (lc.probe) {
     auto probe = decode_kernel<D, NT, BS, true>;
     cudaError_t pe = cudaFuncSetAttribute(probe, cudaFuncAttributeMaxDynamicSharedMemorySize, C::DYN_BYTES);
     if (pe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", pe);
@@ -287,7 +300,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   // the kernel may be set up while its predecessor on the stream drains (and waits for it inside)
   const bool dependent = g_prof_start == nullptr;
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
-  if (g_fp8.active) {
+  if (lc.fp8) {
     if constexpr (D == 128) {
       using C8 = Cfg<D, NT, BS, 1>;
       auto k8 = decode_kernel<D, NT, BS, false, true, 1>;
@@ -301,7 +314,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
     } else {
       return PDATTN_UNSUPPORTED;
     }
-  } else if (g_use_chain) {
+  } else if (lc.chain) {
     auto chain = decode_kernel<D, NT, BS, false, true>;
     bool& cdone = di->chain_attr_set[D == 128][NT == 2][BS / 32];
     if (!cdone) {
@@ -372,29 +385,29 @@ pdattn_status launch_prefix_umma_bs(const CUtensorMap& mk, const CUtensorMap& mv
   return PDATTN_OK;
 }
 
-thread_local int g_block_size = 16;   // page size of the call being launched (set by the entry points)
-
 template <int D, int NT>
 pdattn_status launch(const CUtensorMap& mk, const CUtensorMap& mv, const DecodeParams& P, int grid, int combine_grid,
-                     int n_spans_host, DevInfo* di, cudaStream_t stream) {
-  return g_block_size == 64   ? launch_bs<D, NT, 64>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
-         : g_block_size == 32 ? launch_bs<D, NT, 32>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
-                              : launch_bs<D, NT, 16>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+                     int n_spans_host, const LaunchCtx& lc) {
+  return lc.block_size == 64   ? launch_bs<D, NT, 64>(mk, mv, P, grid, combine_grid, n_spans_host, lc)
+         : lc.block_size == 32 ? launch_bs<D, NT, 32>(mk, mv, P, grid, combine_grid, n_spans_host, lc)
+                               : launch_bs<D, NT, 16>(mk, mv, P, grid, combine_grid, n_spans_host, lc);
 }
 template <int D>
-pdattn_status launch_prefix_umma(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
-                                 cudaStream_t stream) {
-  return g_block_size == 64   ? launch_prefix_umma_bs<D, 64>(mk, mv, X, grid, di, stream)
-         : g_block_size == 32 ? launch_prefix_umma_bs<D, 32>(mk, mv, X, grid, di, stream)
-                              : launch_prefix_umma_bs<D, 16>(mk, mv, X, grid, di, stream);
+pdattn_status launch_prefix_umma(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid,
+                                 const LaunchCtx& lc) {
+  return lc.block_size == 64   ? launch_prefix_umma_bs<D, 64>(mk, mv, X, grid, lc.di, lc.stream)
+         : lc.block_size == 32 ? launch_prefix_umma_bs<D, 32>(mk, mv, X, grid, lc.di, lc.stream)
+                               : launch_prefix_umma_bs<D, 16>(mk, mv, X, grid, lc.di, lc.stream);
 }
 template <int D>
-pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
-                            cudaStream_t stream) {
-  return g_block_size == 64   ? launch_prefix_bs<D, 64>(mk, mv, X, grid, di, stream)
-         : g_block_size == 32 ? launch_prefix_bs<D, 32>(mk, mv, X, grid, di, stream)
-                              : launch_prefix_bs<D, 16>(mk, mv, X, grid, di, stream);
+pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid,
+                            const LaunchCtx& lc) {
+  return lc.block_size == 64   ? launch_prefix_bs<D, 64>(mk, mv, X, grid, lc.di, lc.stream)
+         : lc.block_size == 32 ? launch_prefix_bs<D, 32>(mk, mv, X, grid, lc.di, lc.stream)
+                               : launch_prefix_bs<D, 16>(mk, mv, X, grid, lc.di, lc.stream);
 }
+
+pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_stream_t stream_);
 
 }  // namespace
 
@@ -498,201 +511,8 @@ pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, i
   return PDATTN_OK;
 }
 
-pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream_) {
-  g_last_launches = 0;
-  if (!a) return PDATTN_INVALID_ARG;
-  pdattn_status s = check_shape(a->num_seqs, a->num_q_heads, a->num_kv_heads, a->head_dim, a->block_size);
-  if (s != PDATTN_OK) return s;
-  if (a->num_seqs == 0) return PDATTN_OK;
-  g_block_size = a->block_size;
-  if (!a->q || !a->k_cache || !a->v_cache || !a->out || !a->block_table || !a->context_lens || !a->workspace)
-    return PDATTN_INVALID_ARG;
-  if (a->max_blocks_per_seq <= 0 || a->num_blocks <= 0) return PDATTN_INVALID_ARG;
-  if (a->kv_block_stride <= 0 || a->kv_head_stride <= 0 || a->kv_token_stride < a->head_dim) return PDATTN_INVALID_ARG;
-  if ((a->kv_block_stride | a->kv_head_stride | a->kv_token_stride) % 8 != 0) return PDATTN_UNSUPPORTED;
-  auto mis = [](const void* p, size_t al) { return (reinterpret_cast<uintptr_t>(p) & (al - 1)) != 0; };
-  if (mis(a->q, 16) || mis(a->k_cache, 16) || mis(a->v_cache, 16) || mis(a->out, 16) || mis(a->workspace, 256))
-    return PDATTN_MISALIGNED;
-  const int G = a->num_q_heads / a->num_kv_heads;
-  const int T = g_query_tokens;
-  const bool grouped = g_grouped.active;
-  if (T < 1) return PDATTN_INVALID_ARG;
-  if (G * T > 16 || (T > 1 && grouped)) return PDATTN_UNSUPPORTED;
-  const bool fp8 = g_fp8.active;
-  if (fp8 && (a->head_dim != 128 || grouped || g_probe_mode)) return PDATTN_UNSUPPORTED;
-  const WsLayout wl = ws_layout(a->num_seqs, G * T, a->head_dim);
-  // grouped calls keep two more arrays behind the ordinary layout
-  const size_t off_start = wl.total;
-  const size_t off_pfx = off_start + align_up(static_cast<size_t>(a->num_seqs) * 4, 256);
-  const size_t pfx_bytes = static_cast<size_t>(a->num_seqs) * a->num_kv_heads * (G > 8 ? 16 : 8) * (a->head_dim + 2) * 4;
-  const size_t need = grouped ? off_pfx + align_up(pfx_bytes, 256) : wl.total;
-  if (a->workspace_bytes < need) return PDATTN_WORKSPACE_TOO_SMALL;
-  const int32_t* start_tiles_host = nullptr;
-  int n_groups = 0;
-  if (grouped) {
-    const int Gs = g_grouped.group_size;
-    // rows the kernel for the shared tiles takes per unit: 64 on tensor memory, 48 with warp MMAs
-    const int max_rows = g_prefix_engine != 0 ? UMMA_MAX_QUERY_ROWS : MAX_PREFIX_ROWS;
-    if (!a->context_lens_host || Gs <= 0 || a->num_seqs % Gs != 0 || G > 8 || Gs * G > max_rows)
-      return Gs > 0 && (G > 8 || Gs * G > max_rows) ? PDATTN_UNSUPPORTED : PDATTN_INVALID_ARG;
-    n_groups = a->num_seqs / Gs;
-    g_start_tiles_host.resize(a->num_seqs);
-    for (int sq = 0; sq < a->num_seqs; ++sq) {
-      const int pt = g_grouped.prefix_tiles_host[sq / Gs];
-      // every member must own at least one token past the shared tiles
-      if (pt < 0 || static_cast<int64_t>(pt) * kTileTokens >= a->context_lens_host[sq]) return PDATTN_INVALID_ARG;
-      if (static_cast<int64_t>(pt) * kTileTokens / a->block_size > a->max_blocks_per_seq) return PDATTN_INVALID_ARG;
-      g_start_tiles_host[sq] = pt;
-    }
-    start_tiles_host = g_start_tiles_host.data();
-  }
-
-  int dev = 0;
-  DevInfo* di = nullptr;
-  s = device_info(&dev, &di);
-  if (s != PDATTN_OK) return s;
-  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
-  uint8_t* ws = static_cast<uint8_t*>(a->workspace);
-
-  static_assert(sizeof(DecodeParams) + 2 * sizeof(CUtensorMap) <= 32000, "kernel parameters");
-  DecodeParams P;
-  P.q = static_cast<const __nv_bfloat16*>(a->q);
-  P.out = static_cast<__nv_bfloat16*>(a->out);
-  P.block_table = a->block_table;
-  P.context_lens = a->context_lens;
-  P.start_tiles = nullptr;
-  P.pfx_partials = nullptr;
-  P.hdr = reinterpret_cast<WsHeader*>(ws + wl.hdr);
-  P.spans_ws = reinterpret_cast<const SpanStart*>(ws + wl.spans);
-  P.rec = reinterpret_cast<int4*>(ws + wl.rec);
-  P.partials = reinterpret_cast<float*>(ws + wl.partials);
-  P.S = a->num_seqs;
-  P.Hq = a->num_q_heads;
-  P.Hkv = a->num_kv_heads;
-  P.G = G;
-  P.T = T;
-  P.MB = a->max_blocks_per_seq;
-  P.NB = a->num_blocks;
-  P.scale_log2 = a->scale * 1.4426950408889634f;
-  P.use_ws_plan = 0;
-  P.box5d = 0;
-  P.k_scale = fp8 ? g_fp8.k_scale : nullptr;
-  P.v_scale = fp8 ? g_fp8.v_scale : nullptr;
-
-  int n_ctas = di->sm_count;
-  if (n_ctas > MAX_SPANS / (1 + kMaxDynPerCta)) n_ctas = MAX_SPANS / (1 + kMaxDynPerCta);
-  // Run-time spans even out the CTAs' finishing times when there are many units; with few long sequences
-  // they only lengthen the chains the combine kernel walks.  The choice depends on the batch shape alone.
-  const int dyn_per_cta = g_dyn_per_cta >= 0 ? g_dyn_per_cta
-                          : (static_cast<int64_t>(a->num_seqs) * a->num_kv_heads >= static_cast<int64_t>(kAutoDynUnits) * n_ctas
-                                 ? kAutoDynPerCta
-                                 : 0);
-  int grid = n_ctas, combine_grid = 0, n_spans_host = -1;
-  if (a->context_lens_host) {
-    if (!plan_spans(a->context_lens_host, start_tiles_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta,
-                    MAX_PARAM_SPANS, P.spans, &P.plan))
-      return PDATTN_INVALID_ARG;
-    n_spans_host = P.plan.n_static + P.plan.n_dyn;
-    combine_grid = n_spans_host;
-  } else {
-    P.use_ws_plan = 1;
-    memset(&P.plan, 0, sizeof P.plan);
-    const int n_dyn_max = n_ctas * dyn_per_cta;
-    cudaError_t e = launch_dependent(plan_kernel, 1, 1024, 0, stream, true, a->context_lens,
-                                     static_cast<const int32_t*>(nullptr), a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
-                                     reinterpret_cast<int32_t*>(ws + wl.prefix),
-                                     reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr);
-    if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
-    g_last_launches += 1;
-    combine_grid = n_ctas + n_dyn_max;
-  }
-
-  // One TMA op per page-head (rank-5 view) when head_dim is 128; the rank-4 view otherwise, or if
-  // the driver refuses the rank-5 encoding.
-  static const bool force4d = getenv("PDATTN_BOX4D") != nullptr;
-  CUtensorMap mk, mv;
-  int rank = (a->head_dim == 128 && !force4d) ? 5 : 4;
-  if (fp8) rank = kMapK8;
-  s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-               a->kv_head_stride, a->kv_token_stride, rank, &mk);
-  if (s != PDATTN_OK && rank == 5) {
-    rank = 4;
-    s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-                 a->kv_head_stride, a->kv_token_stride, rank, &mk);
-  }
-  if (s != PDATTN_OK) return s;
-  s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-               a->kv_head_stride, a->kv_token_stride, fp8 ? kMapV8 : rank, &mv);
-  if (s != PDATTN_OK) return s;
-  P.box5d = rank == 5;
-  g_use_chain = g_merge_mode != 0;
-
-  if (grouped) {
-    // shared prompt tiles first: one pass per (group, kv head) for the query rows of all samples
-    PrefixParams X;
-    X.q = P.q;
-    X.block_table = a->block_table;
-    X.prefix_tiles = g_grouped.prefix_tiles;
-    X.start_tiles = reinterpret_cast<int32_t*>(ws + off_start);
-    X.pfx_partials = reinterpret_cast<float*>(ws + off_pfx);
-    X.err = &P.hdr->err;
-    X.S = a->num_seqs;
-    X.Hq = a->num_q_heads;
-    X.Hkv = a->num_kv_heads;
-    X.G = G;
-    X.Gs = g_grouped.group_size;
-    X.MB = a->max_blocks_per_seq;
-    X.NB = a->num_blocks;
-    X.scale_log2 = P.scale_log2;
-    X.box5d = P.box5d;
-    // whole units, contiguous ranges of equal tile count (to within one unit)
-    const int n_units = n_groups * a->num_kv_heads;
-    int64_t total = 0;
-    for (int gi = 0; gi < n_groups; ++gi) total += static_cast<int64_t>(g_grouped.prefix_tiles_host[gi]) * a->num_kv_heads;
-    int pgrid = n_ctas < 160 ? n_ctas : 160;
-    if (pgrid > n_units) pgrid = n_units;
-    int u = 0;
-    int64_t done = 0;
-    for (int c = 0; c < pgrid; ++c) {
-      const int64_t target = total * (c + 1) / pgrid;
-      const int u0 = u;
-      while (u < n_units && (done < target || c == pgrid - 1)) {
-        done += g_grouped.prefix_tiles_host[u / a->num_kv_heads];
-        ++u;
-      }
-      X.ranges[c] = make_int2(u0, u);
-    }
-    if (g_prefix_engine != 0) {
-      // tensor-memory kernel: its tiles are laid out per 64-column block, so it takes the rank-4 view
-      CUtensorMap pk = mk, pv = mv;
-      if (rank != 4) {
-        s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-                     a->kv_head_stride, a->kv_token_stride, 4, &pk);
-        if (s != PDATTN_OK) return s;
-        s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-                     a->kv_head_stride, a->kv_token_stride, 4, &pv);
-        if (s != PDATTN_OK) return s;
-      }
-      s = a->head_dim == 128 ? launch_prefix_umma<128>(pk, pv, X, pgrid, di, stream)
-                             : launch_prefix_umma<64>(pk, pv, X, pgrid, di, stream);
-    } else {
-      s = a->head_dim == 128 ? launch_prefix<128>(mk, mv, X, pgrid, di, stream) : launch_prefix<64>(mk, mv, X, pgrid, di, stream);
-    }
-    if (s != PDATTN_OK) return s;
-    g_last_launches += 1;
-    P.start_tiles = X.start_tiles;
-    P.pfx_partials = X.pfx_partials;
-  }
-
-  const bool nt2 = G * T > 8;
-  if (a->head_dim == 128)
-    s = nt2 ? launch<128, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
-            : launch<128, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
-  else
-    s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
-            : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
-  if (s == PDATTN_OK) g_last_launches += 2;
-  return s;
+pdattn_status pdattn_decode_ex(const pdattn_args* a, pdattn_stream_t stream) {
+  return decode_common(a, CallDesc{}, stream);
 }
 
 pdattn_status pdattn_multi_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim, int block_size,
@@ -708,35 +528,30 @@ pdattn_status pdattn_multi_workspace_size(int num_seqs, int num_q_heads, int num
 }
 
 pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens, pdattn_stream_t stream) {
-  if (!args) return PDATTN_INVALID_ARG;
-  g_query_tokens = num_query_tokens;
-  const pdattn_status s = pdattn_decode_ex(args, stream);
-  g_query_tokens = 1;
-  return s;
+  CallDesc cd;
+  cd.query_tokens = num_query_tokens;
+  return decode_common(args, cd, stream);
 }
 
-pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, const float* v_scale,
-                                pdattn_stream_t stream) {
+pdattn_status pdattn_decode_fp8_multi(const pdattn_args* args, int num_query_tokens, const float* k_scale,
+                                      const float* v_scale, pdattn_stream_t stream) {
   if (!args || !k_scale || !v_scale) return PDATTN_INVALID_ARG;
   pdattn_args a = *args;
   // dense pools of one-byte codes; the stride fields are not used by this variant
   a.kv_token_stride = a.head_dim;
   a.kv_head_stride = static_cast<int64_t>(a.block_size) * a.head_dim;
   a.kv_block_stride = static_cast<int64_t>(a.num_kv_heads) * a.block_size * a.head_dim;
-  g_fp8.active = true;
-  g_fp8.k_scale = k_scale;
-  g_fp8.v_scale = v_scale;
-  const pdattn_status s = pdattn_decode_ex(&a, stream);
-  g_fp8 = Fp8Call{};
-  return s;
+  CallDesc cd;
+  cd.query_tokens = num_query_tokens;
+  cd.fp8 = true;
+  cd.k_scale = k_scale;
+  cd.v_scale = v_scale;
+  return decode_common(&a, cd, stream);
 }
 
-pdattn_status pdattn_decode_fp8_multi(const pdattn_args* args, int num_query_tokens, const float* k_scale,
-                                      const float* v_scale, pdattn_stream_t stream) {
-  g_query_tokens = num_query_tokens;
-  const pdattn_status s = pdattn_decode_fp8(args, k_scale, v_scale, stream);
-  g_query_tokens = 1;
-  return s;
+pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, const float* v_scale,
+                                pdattn_stream_t stream) {
+  return pdattn_decode_fp8_multi(args, 1, k_scale, v_scale, stream);
 }
 
 pdattn_status pdattn_grouped_workspace_size(int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
@@ -754,13 +569,12 @@ pdattn_status pdattn_grouped_workspace_size(int num_seqs, int num_q_heads, int n
 pdattn_status pdattn_decode_grouped(const pdattn_args* args, int group_size, const int32_t* prefix_tiles,
                                     const int32_t* prefix_tiles_host, pdattn_stream_t stream) {
   if (!args || !prefix_tiles || !prefix_tiles_host) return PDATTN_INVALID_ARG;
-  g_grouped.active = true;
-  g_grouped.group_size = group_size;
-  g_grouped.prefix_tiles = prefix_tiles;
-  g_grouped.prefix_tiles_host = prefix_tiles_host;
-  const pdattn_status s = pdattn_decode_ex(args, stream);
-  g_grouped = GroupedCall();
-  return s;
+  if (group_size <= 0) return PDATTN_INVALID_ARG;
+  CallDesc cd;
+  cd.group_size = group_size;
+  cd.prefix_tiles = prefix_tiles;
+  cd.prefix_tiles_host = prefix_tiles_host;
+  return decode_common(args, cd, stream);
 }
 
 pdattn_status pdattn_bind(int max_blocks_per_seq, int num_blocks, void* workspace, size_t workspace_bytes,
@@ -951,92 +765,161 @@ pdattn_status static_scratch_address(int dev, uint8_t** out) {
 }
 }  // namespace
 
-extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int32_t* status_out,
-                                                      pdattn_stream_t stream_) {
+// ---- the one decode path -----------------------------------------------------------------------
+namespace {
+
+pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_stream_t stream_) {
   g_last_launches = 0;
   if (!a) return PDATTN_INVALID_ARG;
   pdattn_status s = check_shape(a->num_seqs, a->num_q_heads, a->num_kv_heads, a->head_dim, a->block_size);
   if (s != PDATTN_OK) return s;
   if (a->num_seqs == 0) return PDATTN_OK;
-  g_block_size = a->block_size;
   if (!a->q || !a->k_cache || !a->v_cache || !a->out || !a->block_table || !a->context_lens) return PDATTN_INVALID_ARG;
+  if (!cd.static_scratch && !a->workspace) return PDATTN_INVALID_ARG;
   if (a->max_blocks_per_seq <= 0 || a->num_blocks <= 0) return PDATTN_INVALID_ARG;
   if (a->kv_block_stride <= 0 || a->kv_head_stride <= 0 || a->kv_token_stride < a->head_dim) return PDATTN_INVALID_ARG;
   if ((a->kv_block_stride | a->kv_head_stride | a->kv_token_stride) % 8 != 0) return PDATTN_UNSUPPORTED;
   auto mis = [](const void* p, size_t al) { return (reinterpret_cast<uintptr_t>(p) & (al - 1)) != 0; };
   if (mis(a->q, 16) || mis(a->k_cache, 16) || mis(a->v_cache, 16) || mis(a->out, 16)) return PDATTN_MISALIGNED;
+  if (!cd.static_scratch && mis(a->workspace, 256)) return PDATTN_MISALIGNED;
+  const int G = a->num_q_heads / a->num_kv_heads;
+  const int T = cd.query_tokens;
+  const bool grouped = cd.group_size > 0;
+  const bool fp8 = cd.fp8;
+  if (T < 1) return PDATTN_INVALID_ARG;
+  if (G * T > 16 || (T > 1 && grouped)) return PDATTN_UNSUPPORTED;
+  if (fp8 && (a->head_dim != 128 || grouped || cd.probe)) return PDATTN_UNSUPPORTED;
+  if (fp8 && (!cd.k_scale || !cd.v_scale)) return PDATTN_INVALID_ARG;
+  if (cd.static_scratch && (grouped || fp8 || T != 1 || cd.probe)) return PDATTN_UNSUPPORTED;
+  // a context longer than its block_table row can describe is refused here when the host knows the lengths;
+  // without a host copy the kernel treats the tokens past the row as a bad page
+  if (a->context_lens_host) {
+    const int64_t row_tokens = static_cast<int64_t>(a->max_blocks_per_seq) * a->block_size;
+    for (int sq = 0; sq < a->num_seqs; ++sq)
+      if (a->context_lens_host[sq] > row_tokens) return PDATTN_INVALID_ARG;
+  }
+
+  // ---- scratch: the caller's workspace (checked before any CUDA call), or the array built into the library
+  // (static spans only, sized by the CTA count).  Grouped calls keep two more arrays behind the ordinary layout.
+  auto scratch_need = [&](const WsLayout& w, size_t* off_start, size_t* off_pfx) {
+    const size_t pfx_bytes = static_cast<size_t>(a->num_seqs) * a->num_kv_heads * (G > 8 ? 16 : 8) * (a->head_dim + 2) * 4;
+    *off_start = w.total;
+    *off_pfx = *off_start + align_up(static_cast<size_t>(a->num_seqs) * 4, 256);
+    return grouped ? *off_pfx + align_up(pfx_bytes, 256) : w.total;
+  };
+  WsLayout wl = ws_layout(a->num_seqs, G * T, a->head_dim, MAX_SPANS);
+  size_t off_start = 0, off_pfx = 0;
+  size_t need = scratch_need(wl, &off_start, &off_pfx);
+  if (!cd.static_scratch && a->workspace_bytes < need) return PDATTN_WORKSPACE_TOO_SMALL;
 
   int dev = 0;
   DevInfo* di = nullptr;
   s = device_info(&dev, &di);
   if (s != PDATTN_OK) return s;
-  int n_ctas = di->sm_count;
-  if (n_ctas > 256) n_ctas = 256;
-
-  // layout inside the static array: header | spans | records | prefix sums | partial slots
-  const int G = a->num_q_heads / a->num_kv_heads;
-  const size_t slot_bytes = static_cast<size_t>(G > 8 ? 16 : 8) * (a->head_dim + 2) * 4;
-  const size_t off_spans = 256;
-  const size_t off_rec = off_spans + align_up(static_cast<size_t>(n_ctas + 1) * sizeof(SpanStart), 256);
-  const size_t off_prefix = off_rec + align_up(static_cast<size_t>(n_ctas) * sizeof(int4), 256);
-  const size_t off_part = off_prefix + align_up(static_cast<size_t>(a->num_seqs + 1) * 8, 256);
-  const size_t need = off_part + align_up(static_cast<size_t>(n_ctas) * 2 * slot_bytes, 256);
-  if (a->num_seqs > PDATTN_STATIC_SCRATCH_MAX_SEQS || need > PDATTN_STATIC_SCRATCH_BYTES) {
-    snprintf(g_cuda_err, sizeof g_cuda_err,
-             "pdattn_decode_static_scratch: %d sequences need %zu bytes of scratch; the built-in array holds %u "
-             "bytes and at most %d sequences",
-             a->num_seqs, need, PDATTN_STATIC_SCRATCH_BYTES, PDATTN_STATIC_SCRATCH_MAX_SEQS);
-    return PDATTN_WORKSPACE_TOO_SMALL;
-  }
-  uint8_t* ws = nullptr;
-  s = static_scratch_address(dev, &ws);
-  if (s != PDATTN_OK) return s;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  int n_ctas = di->sm_count;
+  if (n_ctas > MAX_SPANS / (1 + kMaxDynPerCta)) n_ctas = MAX_SPANS / (1 + kMaxDynPerCta);
 
-  // The array still holds whatever the previous call left: the error word and the span counter
-  // must start at zero; everything else is written before it is read.
-  cudaError_t e = cudaMemsetAsync(ws, 0, 256, stream);
-  if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync(static scratch header)", e);
+  uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+  if (cd.static_scratch) {
+    wl = ws_layout(a->num_seqs, G * T, a->head_dim, n_ctas);
+    need = scratch_need(wl, &off_start, &off_pfx);
+    if (a->num_seqs > PDATTN_STATIC_SCRATCH_MAX_SEQS || need > PDATTN_STATIC_SCRATCH_BYTES) {
+      snprintf(g_cuda_err, sizeof g_cuda_err,
+               "pdattn_decode_static_scratch: %d sequences need %zu bytes of scratch; the built-in array holds %u "
+               "bytes and at most %d sequences",
+               a->num_seqs, need, PDATTN_STATIC_SCRATCH_BYTES, PDATTN_STATIC_SCRATCH_MAX_SEQS);
+      return PDATTN_WORKSPACE_TOO_SMALL;
+    }
+    s = static_scratch_address(dev, &ws);
+    if (s != PDATTN_OK) return s;
+    // The array still holds whatever the previous call left: the error word and the span counter
+    // must start at zero; everything else is written before it is read.
+    cudaError_t e = cudaMemsetAsync(ws, 0, 256, stream);
+    if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync(static scratch header)", e);
+  }
 
-  DecodeParams P;
+  const int32_t* start_tiles_host = nullptr;
+  int n_groups = 0;
+  if (grouped) {
+    const int Gs = cd.group_size;
+    // rows the kernel for the shared tiles takes per unit: 64 on tensor memory, 48 with warp MMAs
+    const int max_rows = g_prefix_engine != 0 ? UMMA_MAX_QUERY_ROWS : MAX_PREFIX_ROWS;
+    if (G > 8 || Gs * G > max_rows) return PDATTN_UNSUPPORTED;
+    if (!a->context_lens_host || a->num_seqs % Gs != 0) return PDATTN_INVALID_ARG;
+    n_groups = a->num_seqs / Gs;
+    g_start_tiles_host.resize(a->num_seqs);
+    for (int sq = 0; sq < a->num_seqs; ++sq) {
+      const int pt = cd.prefix_tiles_host[sq / Gs];
+      // every member must own at least one token past the shared tiles
+      if (pt < 0 || static_cast<int64_t>(pt) * kTileTokens >= a->context_lens_host[sq]) return PDATTN_INVALID_ARG;
+      if (static_cast<int64_t>(pt) * kTileTokens / a->block_size > a->max_blocks_per_seq) return PDATTN_INVALID_ARG;
+      g_start_tiles_host[sq] = pt;
+    }
+    start_tiles_host = g_start_tiles_host.data();
+  }
+
+  static_assert(sizeof(DecodeParams) + 2 * sizeof(CUtensorMap) <= 32000, "kernel parameters");
+  DecodeParams P{};
   P.q = static_cast<const __nv_bfloat16*>(a->q);
   P.out = static_cast<__nv_bfloat16*>(a->out);
   P.block_table = a->block_table;
   P.context_lens = a->context_lens;
   P.start_tiles = nullptr;
   P.pfx_partials = nullptr;
-  P.hdr = reinterpret_cast<WsHeader*>(ws);
-  P.spans_ws = reinterpret_cast<const SpanStart*>(ws + off_spans);
-  P.rec = reinterpret_cast<int4*>(ws + off_rec);
-  P.partials = reinterpret_cast<float*>(ws + off_part);
+  P.hdr = reinterpret_cast<WsHeader*>(ws + wl.hdr);
+  P.spans_ws = reinterpret_cast<const SpanStart*>(ws + wl.spans);
+  P.rec = reinterpret_cast<int4*>(ws + wl.rec);
+  P.partials = reinterpret_cast<float*>(ws + wl.partials);
   P.S = a->num_seqs;
   P.Hq = a->num_q_heads;
   P.Hkv = a->num_kv_heads;
   P.G = G;
-  P.T = 1;
+  P.T = T;
   P.MB = a->max_blocks_per_seq;
   P.NB = a->num_blocks;
   P.scale_log2 = a->scale * 1.4426950408889634f;
   P.use_ws_plan = 0;
   P.box5d = 0;
-  int grid = n_ctas, combine_grid = n_ctas, n_spans_host = -1;
-  g_use_chain = g_merge_mode != 0;
+  P.k_scale = fp8 ? cd.k_scale : nullptr;
+  P.v_scale = fp8 ? cd.v_scale : nullptr;
+
+  // Run-time spans even out the CTAs' finishing times when there are many units; with few long sequences
+  // they only lengthen the chains the combine kernel walks.  The choice depends on the batch shape alone.
+  const int dyn_per_cta =
+      cd.static_scratch ? 0
+      : g_dyn_per_cta >= 0
+          ? g_dyn_per_cta
+          : (static_cast<int64_t>(a->num_seqs) * a->num_kv_heads >= static_cast<int64_t>(kAutoDynUnits) * n_ctas
+                 ? kAutoDynPerCta
+                 : 0);
+  int grid = n_ctas, combine_grid = 0, n_spans_host = -1;
   if (a->context_lens_host) {
-    if (!plan_spans(a->context_lens_host, nullptr, a->num_seqs, a->num_kv_heads, n_ctas, 0, n_ctas, P.spans, &P.plan))
+    const int max_param_spans = cd.static_scratch ? n_ctas : MAX_PARAM_SPANS;
+    if (!plan_spans(a->context_lens_host, start_tiles_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta,
+                    max_param_spans, P.spans, &P.plan))
       return PDATTN_INVALID_ARG;
-    n_spans_host = n_ctas;
-    combine_grid = n_ctas;
+    n_spans_host = P.plan.n_static + P.plan.n_dyn;
+    combine_grid = n_spans_host;
   } else {
     P.use_ws_plan = 1;
     memset(&P.plan, 0, sizeof P.plan);
-    e = launch_dependent(plan_kernel, 1, 1024, 0, stream, true, a->context_lens, static_cast<const int32_t*>(nullptr),
-                         a->num_seqs, a->num_kv_heads, n_ctas, 0, reinterpret_cast<int32_t*>(ws + off_prefix),
-                         reinterpret_cast<SpanStart*>(ws + off_spans), P.hdr);
+    const int n_dyn_max = n_ctas * dyn_per_cta;
+    cudaError_t e = launch_dependent(plan_kernel, 1, 1024, 0, stream, true, a->context_lens,
+                                     static_cast<const int32_t*>(nullptr), a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
+                                     reinterpret_cast<int32_t*>(ws + wl.prefix),
+                                     reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr);
     if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
     g_last_launches += 1;
+    combine_grid = n_ctas + n_dyn_max;
   }
+
+  // One TMA op per page-head (rank-5 view) when head_dim is 128; the rank-4 view otherwise, or if
+  // the driver refuses the rank-5 encoding.
+  static const bool force4d = getenv("PDATTN_BOX4D") != nullptr;
   CUtensorMap mk, mv;
-  int rank = a->head_dim == 128 ? 5 : 4;
+  int rank = (a->head_dim == 128 && !force4d) ? 5 : 4;
+  if (fp8) rank = kMapK8;
   s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
                a->kv_head_stride, a->kv_token_stride, rank, &mk);
   if (s != PDATTN_OK && rank == 5) {
@@ -1046,32 +929,100 @@ extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int3
   }
   if (s != PDATTN_OK) return s;
   s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
-               a->kv_head_stride, a->kv_token_stride, rank, &mv);
+               a->kv_head_stride, a->kv_token_stride, fp8 ? kMapV8 : rank, &mv);
   if (s != PDATTN_OK) return s;
   P.box5d = rank == 5;
-  const bool nt2 = G > 8;
+  const LaunchCtx lc{a->block_size, g_merge_mode != 0, cd.probe, fp8, di, stream};
+
+  if (grouped) {
+    // shared prompt tiles first: one pass per (group, kv head) for the query rows of all samples
+    PrefixParams X;
+    X.q = P.q;
+    X.block_table = a->block_table;
+    X.prefix_tiles = cd.prefix_tiles;
+    X.start_tiles = reinterpret_cast<int32_t*>(ws + off_start);
+    X.pfx_partials = reinterpret_cast<float*>(ws + off_pfx);
+    X.err = &P.hdr->err;
+    X.S = a->num_seqs;
+    X.Hq = a->num_q_heads;
+    X.Hkv = a->num_kv_heads;
+    X.G = G;
+    X.Gs = cd.group_size;
+    X.MB = a->max_blocks_per_seq;
+    X.NB = a->num_blocks;
+    X.scale_log2 = P.scale_log2;
+    X.box5d = P.box5d;
+    // whole units, contiguous ranges of equal tile count (to within one unit)
+    const int n_units = n_groups * a->num_kv_heads;
+    int64_t total = 0;
+    for (int gi = 0; gi < n_groups; ++gi) total += static_cast<int64_t>(cd.prefix_tiles_host[gi]) * a->num_kv_heads;
+    int pgrid = n_ctas < 160 ? n_ctas : 160;
+    if (pgrid > n_units) pgrid = n_units;
+    int u = 0;
+    int64_t done = 0;
+    for (int c = 0; c < pgrid; ++c) {
+      const int64_t target = total * (c + 1) / pgrid;
+      const int u0 = u;
+      while (u < n_units && (done < target || c == pgrid - 1)) {
+        done += cd.prefix_tiles_host[u / a->num_kv_heads];
+        ++u;
+      }
+      X.ranges[c] = make_int2(u0, u);
+    }
+    if (g_prefix_engine != 0) {
+      // tensor-memory kernel: its tiles are laid out per 64-column block, so it takes the rank-4 view
+      CUtensorMap pk = mk, pv = mv;
+      if (rank != 4) {
+        s = make_map(a->k_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+                     a->kv_head_stride, a->kv_token_stride, 4, &pk);
+        if (s != PDATTN_OK) return s;
+        s = make_map(a->v_cache, a->head_dim, a->block_size, a->num_kv_heads, a->num_blocks, a->kv_block_stride,
+                     a->kv_head_stride, a->kv_token_stride, 4, &pv);
+        if (s != PDATTN_OK) return s;
+      }
+      s = a->head_dim == 128 ? launch_prefix_umma<128>(pk, pv, X, pgrid, lc) : launch_prefix_umma<64>(pk, pv, X, pgrid, lc);
+    } else {
+      s = a->head_dim == 128 ? launch_prefix<128>(mk, mv, X, pgrid, lc) : launch_prefix<64>(mk, mv, X, pgrid, lc);
+    }
+    if (s != PDATTN_OK) return s;
+    g_last_launches += 1;
+    P.start_tiles = X.start_tiles;
+    P.pfx_partials = X.pfx_partials;
+  }
+
+  const bool nt2 = G * T > 8;
   if (a->head_dim == 128)
-    s = nt2 ? launch<128, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
-            : launch<128, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+    s = nt2 ? launch<128, 2>(mk, mv, P, grid, combine_grid, n_spans_host, lc)
+            : launch<128, 1>(mk, mv, P, grid, combine_grid, n_spans_host, lc);
   else
-    s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream)
-            : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, di, stream);
+    s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, lc)
+            : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, lc);
   if (s != PDATTN_OK) return s;
-  g_last_launches += 2;
-  if (status_out) {
-    e = cudaMemcpyAsync(status_out, ws, 4, cudaMemcpyDeviceToDevice, stream);
+  if (!cd.probe) g_last_launches += 2;
+  if (cd.status_out) {
+    cudaError_t e = cudaMemcpyAsync(cd.status_out, ws, 4, cudaMemcpyDeviceToDevice, stream);
     if (e != cudaSuccess) return cuda_fail("cudaMemcpyAsync(status_out)", e);
   }
   return PDATTN_OK;
 }
 
+}  // namespace
+
+extern "C" pdattn_status pdattn_decode_static_scratch(const pdattn_args* a, int32_t* status_out,
+                                                      pdattn_stream_t stream) {
+  CallDesc cd;
+  cd.static_scratch = true;
+  cd.status_out = status_out;
+  return decode_common(a, cd, stream);
+}
+
 extern "C" {
 
 pdattn_status pdattn_gather_probe(const pdattn_args* args, pdattn_stream_t stream) {
-  g_probe_mode = true;
-  pdattn_status s = pdattn_decode_ex(args, stream);
-  g_probe_mode = false;
-  g_last_launches = 0;
+  CallDesc cd;
+  cd.probe = true;
+  const pdattn_status s = decode_common(args, cd, stream);
+  g_last_launches = 0;   // a probe is not a decode step
   return s;
 }
 

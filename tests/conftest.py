@@ -71,3 +71,19 @@ def merge_mode(request):
         yield name
     finally:
         pdattn.set_merge_mode(-1)
+
+
+# The fp64 oracle's output for a benchmark configuration at full size, every (sequence, head) row.  The
+# configurations are seeded, so the reference is a function of the configuration number alone and is computed
+# once per session (a few seconds of all host cores each); several GPU test modules compare against it.
+_FULL_REFERENCE = {}
+
+
+@pytest.fixture(scope="session")
+def full_reference():
+    def get(cfg, w_gpu):
+        if cfg not in _FULL_REFERENCE:
+            from oracle import pdattn_oracle
+            _FULL_REFERENCE[cfg] = pdattn_oracle.decode_workload(w_gpu.to("cpu"))
+        return _FULL_REFERENCE[cfg]
+    return get

@@ -116,6 +116,14 @@ def test_decode_rejects_bad_arguments_before_any_cuda_call():
     assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.UNSUPPORTED
     a.head_dim = 80
     assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.UNSUPPORTED
+    # a context longer than its block_table row can describe (4 pages of 16 tokens): refused from the host copy of
+    # the lengths, in every entry point that takes one, before anything is launched
+    a.head_dim, a.kv_token_stride = 64, 64
+    lens = (ctypes.c_int32 * 2)(64, 65)
+    a.context_lens_host = ctypes.cast(lens, ctypes.c_void_p).value
+    assert L.pdattn_decode_ex(ctypes.byref(a), None) == pdattn.INVALID_ARG
+    assert L.pdattn_decode_multi(ctypes.byref(a), 2, None) == pdattn.INVALID_ARG
+    assert L.pdattn_decode_static_scratch(ctypes.byref(a), None, None) == pdattn.INVALID_ARG
 
 
 def test_short_form_needs_a_binding():

@@ -1,7 +1,7 @@
 """Accuracy figures of the decode step per benchmark configuration, beyond the pass/fail gate.
 
-For each configuration at full size (config 1 and 2: every output; 3 to 5: a sample of (sequence, head)
-rows that includes the longest and the shortest sequence) this reports and bounds
+For each configuration at full size, every output element (configuration 3 also through the grouped entry
+point), this reports and bounds
 
   - the gate |gpu - ref| <= max(2e-3, 1e-2 |ref|): failures, max abs error, max relative error over |ref| >= 0.2;
   - a tight metric that scales with the row: |gpu - ref| <= 2^-7 |ref| + 2^-8 rms(ref row).  The gate is
@@ -53,33 +53,9 @@ def figures(out_rows: torch.Tensor, ref: np.ndarray):
     }
 
 
-def rows_for(cfg, w):
-    if cfg <= 2:
-        return None
-    rng = np.random.default_rng(100 + cfg)
-    L = w.context_lens_host
-    seqs = set(rng.integers(0, len(L), size=10 if cfg != 5 else 4).tolist())
-    seqs.update([int(np.argmax(L)), int(np.argmin(L))])
-    return np.array([(s, int(h)) for s in sorted(seqs) for h in rng.choice(w.num_q_heads, size=4, replace=False)],
-                    dtype=np.int32)
-
-
-@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
-def test_accuracy_figures_per_config(cfg):
-    w = W.make_config(cfg, device=DEV)
-    ws = pdattn.alloc_workspace(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size)
-    out = pdattn.decode_workload(w, workspace=ws)
-    assert pdattn.check(ws) == pdattn.OK
-    pairs = rows_for(cfg, w)
-    wc = w.to("cpu")
-    if pairs is None:
-        ref = orc.decode_workload(wc).reshape(-1, w.head_dim)
-        got = out.reshape(-1, w.head_dim)
-    else:
-        ref = orc.decode_workload(wc, pairs=pairs).reshape(-1, w.head_dim)
-        got = out[torch.as_tensor(pairs[:, 0], device=DEV), torch.as_tensor(pairs[:, 1], device=DEV)]
-    f = figures(got, ref)
-    print(f"\nconfig {cfg}: {f['n']} elements, gate failures {f['gate_failures']}, max abs err {f['max_abs']:.3e}, "
+def report(what, out, ref, d):
+    f = figures(out.reshape(-1, d), ref.reshape(-1, d))
+    print(f"\n{what}: {f['n']} elements, gate failures {f['gate_failures']}, max abs err {f['max_abs']:.3e}, "
           f"max rel err (|ref| >= 0.2) {f['max_rel_big']:.3e}, tight-metric failures {f['tight_failures']}, "
           f"bf16 steps from the rounded oracle 0/1/2/3+: {f['ulp_hist']}, smallest row rms {f['rms_min']:.3e}")
     assert f["finite"] and f["gate_failures"] == 0
@@ -88,5 +64,23 @@ def test_accuracy_figures_per_config(cfg):
     assert f["max_rel_big"] <= 2.0 ** -7
     h = f["ulp_hist"]
     assert h[0] + h[1] >= 0.98 * f["n"]          # at most one bf16 step away nearly everywhere
-    del w, wc
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_accuracy_figures_per_config(cfg, full_reference):
+    w = W.make_config(cfg, device=DEV)
+    ws = pdattn.alloc_workspace(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size)
+    out = pdattn.decode_workload(w, workspace=ws)
+    assert pdattn.check(ws) == pdattn.OK
+    ref = full_reference(cfg, w)
+    report(f"config {cfg}", out, ref, w.head_dim)
+    if cfg == 3:
+        gws = pdattn.alloc_grouped_workspace(w.num_seqs, w.num_q_heads, w.num_kv_heads, w.head_dim)
+        pth = np.full(w.num_seqs // 8, 16, dtype=np.int32)
+        og = torch.empty_like(w.q)
+        pdattn.decode_grouped(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, og, gws,
+                              w.context_lens_host, 8, torch.from_numpy(pth).to(DEV), pth)
+        assert pdattn.check(gws) == pdattn.OK
+        report("config 3, grouped", og, ref, w.head_dim)
+    del w
     torch.cuda.empty_cache()

@@ -126,24 +126,22 @@ def sample_pairs(w, n, seed):
 
 
 @pytest.mark.parametrize("cfg", [2, 3, 4, 5])
-def test_full_size_configs_on_sampled_outputs(cfg):
-    """The benchmark's configurations at full size in the benchmark's launch configuration; the oracle
-    computes a sample of (sequence, head) outputs one by one (longest and shortest sequences included),
-    and the bitwise properties below hold at any size."""
+def test_full_size_configs_every_output(cfg, full_reference):
+    """The benchmark's configurations at full size in the benchmark's launch configuration: every output
+    element against the oracle (all (sequence, head) rows, computed once per session), and the bitwise
+    properties that hold at any size."""
     w = W.make_config(cfg, device=DEV)
-    pairs = sample_pairs(w, 6 if cfg != 5 else 4, seed=cfg)
-    out = check_against_oracle(w, f"config {cfg} full", pairs=pairs)
+    out, st = run(w)
+    assert st == pdattn.OK
+    ref = full_reference(cfg, w)
+    assert ref.shape == tuple(out.shape)
+    assert_parity(out, ref, f"config {cfg} full, all {ref.size} outputs")
     out2, st = run(w)
     assert st == pdattn.OK and torch.equal(out, out2)                      # run to run
     out3, _ = run(w, use_host_lens=False)
     assert torch.equal(out, out3)                                          # host plan == device plan
     del w
     torch.cuda.empty_cache()
-
-
-def test_full_config2_every_output():
-    w = W.make_config(2, device=DEV)
-    check_against_oracle(w, "config 2 full, all outputs")
 
 
 # ---------------------------------------------------------------------------- exact pins
@@ -362,6 +360,26 @@ def test_out_of_range_page_ids_are_masked_and_reported():
     bt2[1, 3:] = 1 << 30
     out2, st = run(dataclasses.replace(w, block_table=bt2), ws=ws)
     assert st == pdattn.OK and torch.equal(out, out2)
+
+
+def test_a_context_longer_than_its_table_row_is_masked_and_reported_without_reading_past_the_row():
+    """Device-side plan (no host copy of the lengths to refuse the call with): the last sequence claims 200 tokens
+    while its block_table row describes 128.  The entries past the row's end would lie past the end of the table's
+    allocation; they are not read, those tokens count as a bad page, and the result is the attention over the 128
+    tokens the row does describe.  With the host copy the call is refused instead."""
+    import dataclasses
+    w = W.make_custom([100, 128], Hq=8, Hkv=2, d=128, seed=21, device=DEV, num_blocks=64, poison=False)
+    assert w.max_blocks_per_seq == 8
+    lens = torch.tensor([100, 200], dtype=torch.int32, device=DEV)
+    wl = dataclasses.replace(w, context_lens=lens, context_lens_host=np.array([100, 200], dtype=np.int32))
+    ws = pdattn.alloc_workspace(2, 8, 2, 128)
+    out, st = run(wl, use_host_lens=False, ws=ws)
+    assert st == pdattn.BAD_PAGE_INDEX
+    assert_parity(out, orc.decode_workload(w.to("cpu")), "tokens past the row masked")
+    out2 = torch.empty_like(w.q)
+    st = pdattn.decode_ex(wl.q, wl.k_cache, wl.v_cache, wl.block_table, wl.context_lens, wl.scale, out2, ws,
+                          context_lens_host=wl.context_lens_host, check=False)
+    assert st == pdattn.INVALID_ARG
 
 
 def test_token_major_cache_layout_through_strides():
