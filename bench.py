@@ -61,6 +61,8 @@ def parse():
                          "early in its rollout under both prefix kernels (secondary results, N = 1)")
     ap.add_argument("--grouped", action="store_true",
                     help="config 3 only: time pdattn_decode_grouped (shared prompt pages read once per group)")
+    ap.add_argument("--no-all-configs", action="store_true",
+                    help="skip secondary.configs (the other four workloads; taken by the default run at N = 1)")
     ap.add_argument("--num-seqs", type=int, default=None,
                     help="shrink the batch (profiling captures only; not the metric's workload)")
     return ap.parse_args()
@@ -76,13 +78,25 @@ def measured_peak():
 
 
 def profiled_traffic(cfg):
-    """dram bytes per decode_kernel launch from the committed ncu summary, or None."""
+    """DRAM bytes per decode_kernel launch from the committed ncu summary, with where it comes from.  The summary
+    records the fingerprint of the kernel sources it was captured on; when the sources have changed since, the
+    figure is withheld (None) rather than passed off as a measurement of the current kernel."""
+    from paper_2607_09207_b200 import build as pd_build
     p = os.path.join(ROOT, "profiles", f"decode_kernel_cfg{cfg}_ncu.md")
     try:
-        m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)", open(p).read())
-        return float(m.group(1)) if m else None
-    except Exception:
-        return None
+        text = open(p).read()
+        m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)", text)
+        f = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
+        if not m:
+            return None, f"no traffic figure in profiles/{os.path.basename(p)}"
+        now = pd_build.source_fingerprint()
+        if not f or f.group(1) != now:
+            return None, (f"withheld: profiles/{os.path.basename(p)} was captured on kernel sources "
+                          f"{f.group(1)[:12] if f else 'unknown'}, this build is {now[:12]}")
+        return float(m.group(1)), (f"ncu dram__bytes_read.sum + dram__bytes_write.sum, profiles/{os.path.basename(p)}, "
+                                   f"kernel sources {now[:12]} (same as this build)")
+    except Exception as e:
+        return None, f"unavailable: {e}"
 
 
 class ClockSampler:
@@ -187,6 +201,123 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def batch_stats(step, stream, n_batches=10, calls=20, warm=5):
+    """Procedure of the metric: `warm` untimed calls, then n_batches batches of `calls` back-to-back calls with
+    one CUDA-event pair per batch (time / calls includes launch gaps and the hand-off between the step's kernels
+    as an engine would see them); median and best batch."""
+    i = 0
+    for _ in range(warm):
+        step(i)
+        i += 1
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(n_batches):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(calls):
+            step(i)
+            i += 1
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms.append(a.elapsed_time(b) / calls)
+    return {"batches": n_batches, "calls_per_batch": calls, "median_ms": float(np.median(ms)), "best_ms": float(min(ms))}
+
+
+def kernel_events_ms(pdattn, step, stream, n=40):
+    """Mean duration of the split-KV kernel alone: CUDA events the library records around it on its stream."""
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for a, b in evs:                      # force creation of the underlying CUDA events
+        a.record(stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    L = pdattn.lib()
+    for i, (a, b) in enumerate(evs):
+        L.pdattn_profile_events(a.cuda_event, b.cuda_event)
+        step(i)
+    L.pdattn_profile_events(None, None)
+    torch.cuda.synchronize()
+    return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+
+
+def oracle_full(wc, threads):
+    """One oracle pass over every sequence of the host copy of a workload with `threads` threads: seconds."""
+    from oracle import pdattn_oracle as orc
+    t0 = time.perf_counter()
+    orc.decode(wc.q, wc.k_cache, wc.v_cache, wc.block_table, wc.context_lens, wc.scale, num_threads=threads)
+    return time.perf_counter() - t0
+
+
+def other_configs(pdattn, W, dev, stream, local, peak, with_oracle):
+    """The metric's other workloads (configurations 1, 3, 3 through the grouped entry point, 4 and 5), each at full
+    size: step time as median and best of 10 batches of 20 calls, the split-KV kernel's own time, unique KV bytes,
+    TB/s and fraction of the measured copy bandwidth, the SM clock and throttle reasons seen during that region,
+    and the oracle timed once on the host cores.  Configuration 1 (96 KB, cache resident) reports latency only."""
+    from oracle import pdattn_oracle as orc
+    res = {}
+    for cfg in (1, 3, 4, 5):
+        w = W.make_config(cfg, device=dev)
+        S = w.num_seqs
+        uniq = w.unique_kv_bytes()
+        copies = [w]
+        if cfg != 1 and uniq < (24 << 30):
+            copies.append(_physical_copy(w, seed=177 + cfg))
+        outs = [torch.empty_like(c.q) for c in copies]
+        ws = pdattn.alloc_grouped_workspace(S, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_size, device=dev)
+        variants = [("", False)] + ([("_grouped", True)] if cfg == 3 else [])
+        for suffix, grouped in variants:
+            if grouped:
+                pth = np.full(S // 8, 1024 // 64, dtype=np.int32)
+                ptd = torch.from_numpy(pth).to(dev)
+
+            def step(i):
+                c, o = copies[i % len(copies)], outs[i % len(copies)]
+                if grouped:
+                    pdattn.decode_grouped(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale, o, ws,
+                                          c.context_lens_host, 8, ptd, pth, stream=stream)
+                else:
+                    pdattn.decode_ex(c.q, c.k_cache, c.v_cache, c.block_table, c.context_lens, c.scale, o, ws,
+                                     context_lens_host=c.context_lens_host, stream=stream)
+
+            sampler = ClockSampler(local)
+            sampler.start()
+            bt = batch_stats(step, stream)
+            k_ms = None if grouped else kernel_events_ms(pdattn, step, stream)
+            sampler.stop()
+            assert pdattn.check(ws) == pdattn.OK
+            row = {"workload": CFG_DESC[cfg] + (" [grouped entry point: shared prompt tiles read once per group]"
+                                                if grouped else ""),
+                   "num_seqs": S, "step_ms": bt, "clocks": sampler.summary()}
+            if cfg == 1:
+                row["latency_us"] = {"median": bt["median_ms"] * 1e3, "best": bt["best_ms"] * 1e3}
+                row["note"] = "96 KB of KV, cache resident: latency only"
+            else:
+                ms = bt["median_ms"]
+                row.update({"seq_steps_per_s": S / (ms * 1e-3), "unique_kv_bytes": uniq,
+                            "logical_kv_bytes": w.logical_kv_bytes(),
+                            "hbm_tbs_step": uniq / (ms * 1e-3) / 1e12, "frac_of_measured_peak_step": uniq / (ms * 1e-3) / 1e9 / peak,
+                            "pct_of_8tbs_nominal_step": uniq / (ms * 1e-3) / 8e12 * 100.0,
+                            "l2": f"steps rotate over {len(copies)} physically distinct copies of pools/tables"})
+                if k_ms is not None:
+                    row.update({"kernel_ms": k_ms, "kernel_tbs": uniq / (k_ms * 1e-3) / 1e12,
+                                "kernel_frac_of_measured_peak": uniq / (k_ms * 1e-3) / 1e9 / peak})
+            res[f"cfg{cfg}{suffix}"] = row
+        if with_oracle:
+            del copies[1:], outs[1:]
+            wc = w.to("cpu")
+            cores = orc.host_cores()
+            t_all = oracle_full(wc, cores)
+            res[f"cfg{cfg}"]["oracle"] = {"seq_steps_per_s": S / t_all, "seconds_per_pass": t_all, "cores": cores,
+                                          "sample": f"one pass over all {S} sequences"}
+            if cfg == 1:
+                t_one = oracle_full(wc, 1)
+                res["cfg1"]["oracle_single_thread"] = {"seq_steps_per_s": S / t_one, "seconds_per_pass": t_one, "cores": 1,
+                                                       "sample": f"one pass over all {S} sequences"}
+            del wc
+        del w, copies, outs, ws
+        torch.cuda.empty_cache()
+    return res
+
+
 def main():
     args = parse()
     if args.impl == "reference":
@@ -285,26 +416,17 @@ def main():
         ms_total = float(t.item())
     ms_step = ms_total / K
     value = world * S / (ms_step * 1e-3)
+    # the same step as 10 batches of 20 calls, one event pair per batch: median and best batch (this rank)
+    batch_timing = batch_stats(step, stream)
 
     # ---- region B: the split-KV kernel's own duration, CUDA events recorded around it by the library
-    nb = min(K, 200)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nb)]
-    for a, b in evs:                      # force creation of the underlying CUDA events
-        a.record(stream)
-        b.record(stream)
-    torch.cuda.synchronize()
-    L = pdattn.lib()
-    for i, (a, b) in enumerate(evs):
-        L.pdattn_profile_events(a.cuda_event, b.cuda_event)
-        step(i)
-    L.pdattn_profile_events(None, None)
-    torch.cuda.synchronize()
-    k1_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    k1_ms = kernel_events_ms(pdattn, step, stream, n=min(K, 200))
     kernel_name = "decode_kernel"
     if grouped:      # the prefix kernel does part of the reading: account the whole step
         k1_ms, kernel_name = ms_step, "prefix_kernel + decode_kernel + combine_kernel (whole step)"
     peak, peak_src = measured_peak()
     achieved = uniq / (k1_ms * 1e-3) / 1e9
+    traffic, traffic_src = (None, "not captured for the fp8 step") if fp8 is not None else profiled_traffic(args.cfg)
 
     # ---- region C: end to end from pinned host buffers through pdattn_decode_host
     c0 = copies[0]
@@ -414,6 +536,8 @@ def main():
 
         if args.short_batches:
             extras["short_context_batches"] = short_batches(pdattn, W, dev, timed)
+        if args.cfg == 2 and args.num_seqs is None and not args.no_all_configs:
+            extras["configs"] = other_configs(pdattn, W, dev, stream, local, peak, with_oracle=not args.no_cpu_baseline)
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only)
     cpu_baseline = None
@@ -428,11 +552,21 @@ def main():
             passes += 1
         cpu_baseline = {"value": n * passes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"{passes} oracle passes over the first {n} of {S} sequences ({dt:.2f} s in all)"}
+        if args.cfg <= 2:
+            # single-threaded as well, on a sample sized for about 5 s
+            n1 = int(max(1, min(S, 5.0 / max(t_probe / min(S, 8) * cores, 1e-9))))
+            from oracle import pdattn_oracle as orc
+            t0 = time.perf_counter()
+            orc.decode(wc.q[:n1], wc.k_cache, wc.v_cache, wc.block_table[:n1], wc.context_lens[:n1], wc.scale, num_threads=1)
+            t1 = time.perf_counter() - t0
+            cpu_baseline["single_thread"] = {"value": n1 / t1, "unit": UNIT, "cores": 1,
+                                             "sample": f"one oracle pass over the first {n1} of {S} sequences ({t1:.2f} s)"}
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_step, "step_ms_batches": batch_timing,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if fp8 is None else "e4m3 cache, fp16 products, fp32 accumulate", "data": "synthetic",
             "config": {"workload": CFG_DESC[args.cfg] + (f" [REDUCED to {S} seqs]" if args.num_seqs else "")
                        + (" [grouped: shared prompt tiles read once per group]" if grouped else "")
@@ -449,7 +583,7 @@ def main():
                                                / (uniq / (ms_step * 1e-3)),
             "pct_of_8tbs_nominal_step": uniq / (ms_step * 1e-3) / 8e12 * 100.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": None if fp8 is not None else profiled_traffic(args.cfg),
+                         "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_src,
                          "kernel": kernel_name, "kernel_ms": k1_ms, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": uniq,
                          "pct_of_8tbs_nominal": achieved / 8000.0 * 100.0},
@@ -568,12 +702,19 @@ def _physical_copy(w, seed):
 
 
 def _reseeded(W, cfg, rank, dev, lens, rng):
-    """Another batch of the same configuration for rank > 0: lengths shuffled, values reseeded."""
+    """Another batch of the same configuration for rank > 0: lengths shuffled, values reseeded; what makes the
+    configuration what it is stays (config 3: the 8 rows of a group share their 64 prompt pages; config 4: per-head
+    scales on K and V)."""
     lens = rng.permutation(lens)
     shapes = {2: (28, 4), 3: (40, 8), 4: (64, 8), 5: (28, 4), 1: (4, 1)}
     Hq, Hkv = shapes[cfg]
     d = 64 if cfg == 1 else 128
-    return W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, seed=1000 * cfg + rank, device=dev)
+    kw = {}
+    if cfg == 3:
+        kw.update(shared_prefix_pages=1024 // 16, group=8)
+    if cfg == 4:
+        kw.update(head_scales=True)
+    return W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, seed=1000 * cfg + rank, device=dev, **kw)
 
 
 if __name__ == "__main__":

@@ -21,6 +21,19 @@ def _nvcc() -> str:
     return "nvcc"
 
 
+def source_fingerprint() -> str:
+    """sha256 over the kernel and host sources the library is built from (in a fixed order): names a build
+    without needing the version control history, e.g. to tie a profile summary to the kernels it measured."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted(SOURCES + HEADERS):
+        path = os.path.join(CSRC, f)
+        h.update(os.path.basename(f).encode())
+        with open(path, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
 def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
