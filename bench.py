@@ -457,7 +457,10 @@ def main():
         e2e_s = float(t.item())
     sampler.stop()
     e2e_value = world * S * ke / e2e_s
-    h2d = qh.numel() * 2 + bth.numel() * 4 + lh.numel() * 4
+    # bytes that cross the bus per step: q rows, the lengths, and the used part of every block_table row (fetched in
+    # 16-byte units by the library's gather kernel when the table is pinned and mapped, as here)
+    used_pages = (c0.context_lens_host.astype(np.int64) + c0.block_size - 1) // c0.block_size
+    h2d = qh.numel() * 2 + int((((used_pages * 4) + 15) // 16 * 16).sum()) + lh.numel() * 4
     d2h = oh.numel() * 2
     assert pdattn.check(ws) == pdattn.OK
 
@@ -590,9 +593,10 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": ke, "note": ("bf16 step (pdattn_decode_host has no fp8 form); " if fp8 is not None else "")
                                          + "q/block_table/context_lens in pinned host memory, out in pinned host memory "
-                                         "and the stream synchronised every step: block_table and context_lens are "
-                                         "copied, q rows are fetched and out rows written over the bus by the kernels "
-                                         "themselves (same bytes, off the critical path); KV pools are resident state"},
+                                         "and the stream synchronised every step: the lengths and the used part of each "
+                                         "block_table row are fetched by a gather kernel (bulk copies over the bus), q rows "
+                                         "are fetched and out rows written over the bus by the decode kernels themselves; "
+                                         "KV pools are resident state"},
             "gpu_launches": launches_per_step * K,
             "clocks": sampler.summary(),
             "cpu_baseline": cpu_baseline,

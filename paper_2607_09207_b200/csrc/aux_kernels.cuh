@@ -43,6 +43,74 @@ append_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __re
   if (threadIdx.x == 0) context_lens[s] = L + 1;
 }
 
+// ------------------------------------------------------------------------------------------
+// Host-resident step inputs: block s copies the used part of row s of a block table that lives in pinned,
+// mapped host memory (ceil(L_s / bs) entries, the only ones a decode step reads) and the length itself into
+// their device staging copies.  All loads are independent, so the whole batch costs about one round trip over
+// the bus plus the bytes actually used, and the launch replaces two host-to-device copies of the full arrays.
+// ------------------------------------------------------------------------------------------
+constexpr int kGatherRows = 8;     // sequences per block of host_table_gather_kernel (one warp each)
+
+// The fetches go through the bulk-copy engine (plain loads from host memory reach a small fraction of the
+// bus rate): per block one bulk copy brings the kGatherRows lengths, then warp w brings the used part of its
+// row into shared memory and sends it on to the device copy.  Needs MB % 4 == 0 (16-byte aligned rows) and
+// num_seqs-padded length arrays are not assumed: the last block copies only the lengths that exist.
+__global__ void __launch_bounds__(32 * kGatherRows)
+host_table_gather_kernel(const int32_t* __restrict__ table_host, const int32_t* __restrict__ lens_host,
+                         int32_t* __restrict__ table_dev, int32_t* __restrict__ lens_dev, int S, int MB, int bs,
+                         int32_t* err) {
+  extern __shared__ __align__(128) uint8_t gsm[];
+  __shared__ __align__(16) int32_t lens_s[kGatherRows];
+  __shared__ uint64_t bar_len, bar_row[kGatherRows];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int s0 = blockIdx.x * kGatherRows;
+  const int nseq = min(kGatherRows, S - s0);
+  const int row_bytes = MB * 4;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar_len), 1);
+    for (int i = 0; i < kGatherRows; ++i) mbar_init(smem_u32(&bar_row[i]), 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the staging copies may still be read by the step before
+  const bool whole = nseq == kGatherRows;              // 32 bytes from a 32-byte aligned offset: one bulk copy
+  if (threadIdx.x == 0) {
+    if (whole) {
+      mbar_arrive_expect_tx(smem_u32(&bar_len), kGatherRows * 4);
+      bulk_load(smem_u32(lens_s), lens_host + s0, kGatherRows * 4, smem_u32(&bar_len));
+    } else {
+      for (int i = 0; i < nseq; ++i) lens_s[i] = *reinterpret_cast<const volatile int32_t*>(lens_host + s0 + i);
+      mbar_arrive(smem_u32(&bar_len));
+    }
+  }
+  bool ok = mbar_wait(smem_u32(&bar_len), 0);
+  if (ok && warp < nseq) {
+    const int s = s0 + warp;
+    const int L = lens_s[warp];
+    int n = L > 0 ? (L + bs - 1) / bs : 0;
+    if (n > MB) n = MB;
+    const uint32_t bytes = static_cast<uint32_t>((n * 4 + 15) & ~15);   // within the row: MB is a multiple of 4
+    const uint32_t dst_s = smem_u32(gsm) + warp * row_bytes;
+    if (bytes > 0) {
+      if (lane == 0) {
+        mbar_arrive_expect_tx(smem_u32(&bar_row[warp]), bytes);
+        bulk_load(dst_s, table_host + static_cast<int64_t>(s) * MB, bytes, smem_u32(&bar_row[warp]));
+      }
+      ok = mbar_wait(smem_u32(&bar_row[warp]), 0);
+      if (ok && lane == 0) {
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(
+                         reinterpret_cast<uint64_t>(table_dev + static_cast<int64_t>(s) * MB)),
+                     "r"(dst_s), "r"(bytes)
+                     : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+      }
+    }
+    if (lane == 0) lens_dev[s] = L;
+  }
+  if (!ok && lane == 0 && err) atomicOr(err, ERR_TIMEOUT);
+}
+
 // Read-only streaming ceiling: every thread block sums a contiguous slice with 16-byte loads.
 __global__ void __launch_bounds__(512)
 stream_read_kernel(const uint4* __restrict__ src, size_t n_vec, uint32_t* __restrict__ sink) {

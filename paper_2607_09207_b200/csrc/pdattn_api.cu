@@ -683,10 +683,33 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
   cudaError_t e;
   if (!in_place && (e = cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
     return cuda_fail("cudaMemcpyAsync(q)", e);
-  if ((e = cudaMemcpyAsync(bt_dev, block_table_host, t_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
-    return cuda_fail("cudaMemcpyAsync(block_table)", e);
-  if ((e = cudaMemcpyAsync(len_dev, context_lens_host, l_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
-    return cuda_fail("cudaMemcpyAsync(context_lens)", e);
+  // block_table and context_lens: when both are pinned and mapped, one small kernel fetches the lengths and the
+  // used part of every table row over the bus (about a third of the table for a long-tailed batch); otherwise
+  // two copies of the whole arrays
+  const void* btm = g_host_zero_copy != 0 ? mapped_host_pointer(block_table_host) : nullptr;
+  const void* lm = g_host_zero_copy != 0 ? mapped_host_pointer(context_lens_host) : nullptr;
+  const size_t gather_smem = static_cast<size_t>(kGatherRows) * max_blocks_per_seq * 4;
+  if (btm && lm && !(reinterpret_cast<uintptr_t>(btm) & 15) && !(reinterpret_cast<uintptr_t>(lm) & 31) &&
+      max_blocks_per_seq % 4 == 0 && gather_smem <= 200 * 1024) {
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev >= 0 && dev < kMaxDevices && !attr_set[dev]) {
+      e = cudaFuncSetAttribute(host_table_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
+      attr_set[dev] = true;
+    }
+    e = launch_dependent(host_table_gather_kernel, (num_seqs + kGatherRows - 1) / kGatherRows, 32 * kGatherRows,
+                         gather_smem, stream, true, static_cast<const int32_t*>(btm), static_cast<const int32_t*>(lm),
+                         static_cast<int32_t*>(bt_dev), static_cast<int32_t*>(len_dev), num_seqs, max_blocks_per_seq,
+                         block_size, static_cast<int32_t*>(workspace));
+    if (e != cudaSuccess) return cuda_fail("host_table_gather_kernel launch", e);
+  } else {
+    if ((e = cudaMemcpyAsync(bt_dev, block_table_host, t_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+      return cuda_fail("cudaMemcpyAsync(block_table)", e);
+    if ((e = cudaMemcpyAsync(len_dev, context_lens_host, l_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+      return cuda_fail("cudaMemcpyAsync(context_lens)", e);
+  }
   pdattn_args a;
   memset(&a, 0, sizeof a);
   a.q = q_dev;
