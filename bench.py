@@ -438,8 +438,10 @@ def main():
 
     oh_bits = oh.view(torch.int16).numpy()        # the host buffer itself, for the per-step read
 
+    host_step = pdattn.HostStep(qh, bth, lh, oh, c0.k_cache, c0.v_cache, c0.scale, staging, ws, stream=stream)
+
     def e2e_step():
-        pdattn.decode_host(qh, bth, lh, oh, c0.k_cache, c0.v_cache, c0.scale, staging, ws, stream=stream)
+        host_step()                       # pdattn_decode_host on the same pinned buffers every step
         stream.synchronize()              # the caller reads `out` on the host every step
         return int(oh_bits[0, 0, 0])
 

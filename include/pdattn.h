@@ -65,8 +65,9 @@ pdattn_status pdattn_workspace_size(int num_seqs, int num_q_heads, int num_kv_he
                                     size_t* device_bytes, size_t* pinned_host_bytes);
 
 /*
- * Clear the workspace's error word.  Call once after allocating a workspace (and at will later);
- * enqueued on `stream`.  workspace: DEVICE.
+ * Clear the words of the workspace that must be zero before its first use (error word, span counter, the
+ * ticket words of the in-kernel merge: the first 8448 bytes).  Call once after allocating a workspace, and at
+ * will later while no call that uses the workspace is in flight; enqueued on `stream`.  workspace: DEVICE.
  */
 pdattn_status pdattn_workspace_init(void* workspace, size_t workspace_bytes, pdattn_stream_t stream);
 
@@ -281,14 +282,20 @@ pdattn_status pdattn_plan_host(const int32_t* context_lens_host, int num_seqs, i
 pdattn_status pdattn_set_dynamic_spans(int per_cta);
 
 /*
- * Process-wide choice of how the consumer warps of a CTA merge their online-softmax states at
- * the end of a piece (a sequence's run of tiles inside one span).  1: the state is handed down a
- * chain of warps through shared memory and no warp waits for the others, so several short pieces
- * are in work at once.  0: all warps meet at a barrier and sum their states together; on long
- * pieces (tens of tiles) this costs the same, on batches of short contexts one barrier round per
- * piece.  -1 (default): 1, with static and with run-time spans alike.  Either way the order of every
- * sum is fixed by tile indices, so a setting's results are bit-identical from run to run and under any
- * renumbering of the physical pages.
+ * Process-wide choice of how partial online-softmax states (m, l, acc) are merged (the split-combine of the
+ * split-KV method; no paper counterpart beyond the decoding step of Section 2.3).  Two places merge:
+ *   - inside a CTA, at the end of a piece (a sequence's run of tiles inside one span), the states of its
+ *     consumer warps: "chained" hands the state down a chain of warps through shared memory and no warp waits
+ *     for the others, so several short pieces are in work at once; "barrier" makes all warps meet and sum
+ *     together (same cost on long pieces, one barrier round per piece on batches of short contexts);
+ *   - across CTAs, the partials of a sequence that span boundaries cut: either inside the decode kernel, by
+ *     whichever CTA writes the unit's last partial (found with one atomic ticket per unit; no CTA waits for
+ *     another; units cut into more than 16 consecutive spans are left to the combine kernel), or by the separate
+ *     combine kernel launched behind it.
+ * mode 1: chained + merge of cut units inside the decode kernel (one launch per step when every chain is short
+ * enough and context_lens_host is given); mode 2: chained + combine kernel; mode 0: barrier + combine kernel;
+ * -1 (default): 1.  In every mode the order of every sum is fixed by tile and span indices, so a setting's
+ * results are bit-identical from run to run and under any renumbering of the physical pages.
  */
 pdattn_status pdattn_set_merge_mode(int mode);
 
@@ -365,7 +372,8 @@ pdattn_status pdattn_stream_read_probe(const void* src, size_t bytes, void* sink
  */
 pdattn_status pdattn_wait_limit_probe(void* workspace, int limit_us, pdattn_stream_t stream);
 
-/* Number of kernels the last pdattn_decode_ex on this thread launched (2 or 3). */
+/* Number of kernels the last decode call on this thread launched (1 to 4: planner, shared-prefix kernel,
+ * split-KV kernel, combine kernel, each only when it is needed). */
 int pdattn_last_launch_count(void);
 
 /* Fixed English text for a status code (no paper counterpart); never NULL, never freed. */

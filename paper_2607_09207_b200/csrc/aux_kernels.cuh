@@ -179,20 +179,20 @@ append_fp8_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* 
 // Split-combine: block i merges the unit that started in span i and ran past its end.  The
 // pieces live in the following spans (slot 0 of each follower), merged in ascending token order:
 //   M = max m_c;  Lsum = sum l_c 2^(m_c - M);  out = bf16( sum acc_c 2^(m_c - M) / Lsum ).
-// Block 0 also rearms the run-time span counter for the next call.
+// With inkernel_max > 0 the decode kernel has already merged every unit whose followers lie within
+// inkernel_max spans of its first one; this kernel then only takes the longer chains.
 // ------------------------------------------------------------------------------------------
 template <int D, int NT>
 __global__ void __launch_bounds__(256)
 combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, const float* __restrict__ partials,
                __nv_bfloat16* __restrict__ out, int Hq, int Hkv, int G, const int32_t* __restrict__ start_tiles,
-               const float* __restrict__ pfx_partials, int T) {
+               const float* __restrict__ pfx_partials, int T, int inkernel_max) {
   constexpr int HP = 8 * NT;
   constexpr int SLOT_FLOATS = HP * (D + 2);
   const int c = blockIdx.x;
   // launched as a programmatic dependent of the decode kernel: nothing of that kernel may be read
   // before this returns (it waits for the kernel's completion and memory flush)
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (c == 0 && threadIdx.x == 0) hdr->counter = 0;
   const int n_spans = n_spans_host >= 0 ? n_spans_host : hdr->plan.n_static + hdr->plan.n_dyn;
   if (c >= n_spans) return;
   const int4 r = rec[c];
@@ -201,9 +201,12 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
   // followers: later spans whose first piece continues `unit` (spans without tiles may sit between).
   // The block looks at blockDim.x span records at a time instead of walking them one dependent load after
   // the other: a long sequence can be cut by hundreds of spans.
-  __shared__ int n_follow, first_break;
+  __shared__ int n_follow, first_break, run_len;
   __shared__ int follow[MAX_SPANS];
-  if (threadIdx.x == 0) n_follow = 0;
+  if (threadIdx.x == 0) {
+    n_follow = 0;
+    run_len = n_spans - (c + 1);
+  }
   for (int base = c + 1; base < n_spans; base += blockDim.x) {
     if (threadIdx.x == 0) first_break = blockDim.x;
     __syncthreads();
@@ -231,11 +234,14 @@ combine_kernel(WsHeader* hdr, int n_spans_host, const int4* __restrict__ rec, co
       int tot = 0;
       for (int w = 0; w < static_cast<int>(blockDim.x) / 32; ++w) tot += warp_count[w];
       n_follow += tot;
+      if (fb < static_cast<int>(blockDim.x)) run_len = base - (c + 1) + fb;
     }
     __syncthreads();
     if (fb < static_cast<int>(blockDim.x)) break;
   }
   __syncthreads();
+  // a short chain has been merged inside the decode kernel by the CTA that wrote its last partial
+  if (inkernel_max > 0 && run_len <= inkernel_max) return;
   const int np = n_follow + 1;
   const int s = unit / Hkv, g = unit - s * Hkv;
   // piece -1: the partial of the unit's leading tiles when those were handled elsewhere (shared prefix)
@@ -351,7 +357,7 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
     sp.unit = S * Hkv;
     sp.tile = 0;
     sp.flat = pp.total;
-    sp.pad = 0;
+    sp.merge = 0;
     const int x = static_cast<int>(span_cost_start(pp, c));
     if (c < n_spans && x < total_cost) {
       int lo = 0, hi = S;   // find s with pcost[s] <= x < pcost[s+1]
@@ -368,6 +374,9 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
     }
     spans[c] = sp;
   }
+  // how the cut units are put together again: one word per span, from the finished table
+  __syncthreads();
+  for (int c = tid; c < n_spans; c += 1024) spans[c].merge = span_merge_info(spans, n_spans, c);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -30,6 +30,7 @@ constexpr int MAX_SPANS = 2048;                  // spans per call (static + run
 constexpr int MAX_PARAM_SPANS = 768;             // spans that can travel in kernel parameters
 constexpr int SPAN_QUEUE = 32;                   // in-CTA queue of run-time span ids
 constexpr int MAX_STAGES = 14;
+constexpr int MERGE_QUEUE = 8;                  // entries of the in-CTA queue of merge jobs
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2 };
@@ -37,11 +38,18 @@ enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2 };
 // Workspace header (first 256 bytes of the workspace)
 struct WsHeader {
   int32_t err;        // sticky error bits
-  int32_t counter;    // next run-time span; zero between calls (combine_kernel resets it)
+  int32_t counter;    // next run-time span; zero between calls (the last CTA out resets it)
   PlanParams plan;    // written by plan_kernel
-  int32_t pad[54];
+  int32_t done;       // CTAs of the running decode kernel whose span draws are over; zero between calls
+  int32_t pad[53];
 };
 static_assert(sizeof(WsHeader) == 256, "header size");
+// Behind the header: one ticket word per span, zero between calls.  Word c counts the partials written so far
+// for the unit that starts in span c and runs past its end; the CTA that brings the count to the unit's number
+// of pieces merges them and writes the output (no CTA ever waits for another).
+constexpr int WS_TICKETS_OFFSET = 256;
+constexpr int WS_TICKETS_BYTES = MAX_SPANS * 4;
+constexpr int WS_CLEARED_BYTES = WS_TICKETS_OFFSET + WS_TICKETS_BYTES;   // what must be zero before the first call
 
 struct DecodeParams {
   const __nv_bfloat16* q;
@@ -62,6 +70,9 @@ struct DecodeParams {
   PlanParams plan;          // host plan (ignored when use_ws_plan)
   int use_ws_plan;
   int box5d;                // 1: the tensor maps are 5-D and one TMA op brings a whole page-head
+  int32_t* tickets;         // [MAX_SPANS] ticket words (see WS_TICKETS_OFFSET)
+  int inkernel_max;         // > 0: a cut unit whose followers all lie within this many spans after its first one is
+                            // merged by the CTA that writes its last partial; 0: every cut unit is left to combine_kernel
   SpanStart spans[MAX_PARAM_SPANS + 1];
 };
 
@@ -237,7 +248,7 @@ struct Cfg {
   // tile is kept back and the warps exchange their accumulators through it.
   static constexpr int ACC_STRIDE = D + 4;             // floats; keeps the parked stores conflict-free
   static constexpr int SMEM_MAX = 232448;              // 227 KB
-  static constexpr int CTRL_BYTES = 1024;
+  static constexpr int CTRL_BYTES = 1280;
   static constexpr int NCW = PDATTN_NCW;                               // consumer warps
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
   static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged by producer 0
@@ -246,7 +257,12 @@ struct Cfg {
   static constexpr int NSTAGES = (NSTAGES_FIT > MAX_STAGES ? MAX_STAGES : NSTAGES_FIT) / NCW * NCW;
   static constexpr int NCT = NCW * 32;                                 // consumer threads
   static constexpr int NPW = (NT == 2 && PDATTN_NPW > 2) ? 2 : PDATTN_NPW;   // producer warps (8 warps in all for 16-row tiles: 255 registers)
-  static constexpr int NTHREADS = NCT + 32 * NPW;
+  // One more warp (8-row tiles only: with 16-row tiles the consumers need every register a smaller block leaves
+  // them) does the final merge of cut units: consumers post jobs to it through shared memory and never wait
+  // on global memory for a merge themselves.
+  static constexpr bool MERGE_WARP = NT == 1;
+  static constexpr int NTHREADS_BASE = NCT + 32 * NPW;                      // consumers and producers
+  static constexpr int NTHREADS = NTHREADS_BASE + (MERGE_WARP ? 32 : 0);    // decode_kernel's block
   static constexpr int DYN_BYTES = 1024 + NSTAGES * STAGE_BYTES + QSLOTS * Q_BYTES + ML_BYTES + CTRL_BYTES;
   static constexpr int SLOT_FLOATS = HP * (D + 2);     // one partial: m[HP], l[HP], acc[HP][D]
   // Chained merge (decode_kernel with CHAIN): a warp's running (m, l, acc) of a piece in MMA fragment
@@ -276,8 +292,14 @@ struct Ctrl {                 // lives in the CTRL_BYTES area
   uint64_t q_empty[4];        // ... and every consumer warp has copied them to registers
   int32_t qseq[4];            // CHAIN: piece whose rows the producer last armed the query slot for
   int32_t turn[8];            // CHAIN: hand-off slot e is waiting for class (turn % 8) of merge number (turn / 8)
+  // queue of merge jobs from the consumer warps to the merge warp (CHAIN with Cfg::MERGE_WARP)
+  int32_t mq_head;            // jobs claimed so far (shared-memory atomic)
+  int32_t mq_tail;            // jobs the merge warp has taken over
+  int32_t mq_done;            // consumer warps that will post no more jobs
+  int32_t mq_tag[MERGE_QUEUE];   // job k has been written to entry k % MERGE_QUEUE when its tag is k + 1
+  int4 mq_job[MERGE_QUEUE];   // (first span c, hold mask, ticket increment, unit | has-prefix flag << 30)
 };
-static_assert(sizeof(Ctrl) <= 1024, "control block");
+static_assert(sizeof(Ctrl) <= 1280, "control block");
 
 // ------------------------------------------------------------------------------------------
 // The walk over a span: pieces = (unit, tile range) in order.  Every warp runs the same walk.

@@ -14,6 +14,188 @@
 namespace pdattn {
 
 // ------------------------------------------------------------------------------------------
+// Final merge of a cut unit inside the decode kernel.  The span table's merge words tell every warp that writes
+// a partial (m, l, acc) of a cut unit which span c the unit starts in and which of the spans after it hold a
+// piece.  The warp posts a job to its CTA's merge warp, which publishes the partial device-wide by taking a
+// ticket on word c; the merge warp that draws a unit's last ticket -- whichever CTA it belongs to, no one
+// waits -- merges all the pieces in ascending token order (the shared-prefix partial first when there is one)
+// and writes the output rows.  The order of the sum is fixed by the span table, so the bits do not depend on
+// who merges.  merge_cut_unit takes plain values only: a reference to the kernel parameters inside a function
+// that is not inlined would turn every access into a generic load.
+// ------------------------------------------------------------------------------------------
+struct MergeJob {
+  const float* partials;      // [span][2][SLOT_FLOATS]
+  const float* pfx;           // this unit's shared-prefix partial, or null
+  __nv_bfloat16* out;
+  int c, hold_mask, n_parts;
+  int s, g, G, T, Hq;
+};
+template <int D, int NT>
+__device__ __noinline__ void merge_cut_unit(const MergeJob J, int own_slot, int lane) {
+  constexpr int HP = 8 * NT;
+  constexpr int SLOT_FLOATS = HP * (D + 2);
+  const float NEG_INF = __int_as_float(0xff800000);
+  // piece p: -1 the partial of the unit's leading tiles (shared prefix, written by an earlier kernel), 0 the one
+  // of span c, p >= 1 the p-th follower that holds tiles; lane p keeps the address of piece p
+  const int p0 = J.pfx ? -1 : 0;
+  const float* mine = nullptr;
+  if (lane == 0) mine = J.partials + (static_cast<int64_t>(J.c) * 2 + own_slot) * SLOT_FLOATS;
+  else if (lane < J.n_parts) mine = J.partials + static_cast<int64_t>(J.c + 1 + __fns(J.hold_mask, 0, lane)) * 2 * SLOT_FLOATS;
+  auto piece = [&](int p) -> const float* {
+    const unsigned long long a = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(mine), p < 0 ? 0 : p);
+    return p < 0 ? J.pfx : reinterpret_cast<const float*>(a);
+  };
+  // Pieces are taken two at a time and every load of a pair is issued before anything is computed:
+  // one round trip to the L2 per pair, however loaded the memory system is.  Pairs are folded into the
+  // running (M, Ls, a) like tiles into an online softmax; the order is fixed by the span table.
+  const int R = J.G * J.T;
+  constexpr int ITEMS = HP * (D / 4);
+  constexpr int IPL = ITEMS / 32;                   // items per lane: item = (row h, four consecutive dims dq)
+  constexpr int CH = 2;
+  static_assert(ITEMS % 32 == 0 && HP <= 32, "merge layout");
+  int h[IPL], dq[IPL];
+  float M[IPL], Ls[IPL];
+  float4 a[IPL];
+#pragma unroll
+  for (int j = 0; j < IPL; ++j) {
+    const int idx = j * 32 + lane;
+    h[j] = idx / (D / 4);
+    dq[j] = idx % (D / 4);
+    M[j] = NEG_INF;
+    Ls[j] = 0.f;
+    a[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll 1
+  for (int pb = p0; pb < J.n_parts; pb += CH) {
+    float pm[CH], pl[CH];                           // lane t < HP: m and l of row t of each piece of the group
+    float4 v[CH][IPL];
+    bool valid[CH];
+#pragma unroll
+    for (int q = 0; q < CH; ++q) {
+      valid[q] = pb + q < J.n_parts;
+      const float* part = piece(valid[q] ? pb + q : pb);
+      pm[q] = __ldcg(part + (lane % HP));
+      pl[q] = __ldcg(part + HP + (lane % HP));
+#pragma unroll
+      for (int j = 0; j < IPL; ++j) v[q][j] = __ldcg(reinterpret_cast<const float4*>(part + 2 * HP + h[j] * D + dq[j] * 4));
+    }
+#pragma unroll
+    for (int j = 0; j < IPL; ++j) {
+      float mq[CH], lq[CH];
+      float Mn = M[j];
+#pragma unroll
+      for (int q = 0; q < CH; ++q) {
+        mq[q] = __shfl_sync(0xffffffffu, pm[q], h[j]);
+        lq[q] = __shfl_sync(0xffffffffu, pl[q], h[j]);
+        if (valid[q]) Mn = fmaxf(Mn, mq[q]);
+      }
+      const float Mu = (Mn == NEG_INF) ? 0.f : Mn;
+      const float fo = fast_exp2(M[j] - Mu);        // 0 for the first group (M = -inf)
+      M[j] = Mn;
+      Ls[j] *= fo;
+      a[j].x *= fo;
+      a[j].y *= fo;
+      a[j].z *= fo;
+      a[j].w *= fo;
+#pragma unroll
+      for (int q = 0; q < CH; ++q) {
+        if (valid[q]) {
+          const float f = fast_exp2(mq[q] - Mu);
+          Ls[j] += lq[q] * f;
+          a[j].x += v[q][j].x * f;
+          a[j].y += v[q][j].y * f;
+          a[j].z += v[q][j].z * f;
+          a[j].w += v[q][j].w * f;
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < IPL; ++j) {
+    if (h[j] < R) {   // row h = query token * G + head
+      const float inv = Ls[j] > 0.f ? 1.f / Ls[j] : 0.f;
+      uint2 o;
+      o.x = pack_bf16x2(a[j].x * inv, a[j].y * inv);
+      o.y = pack_bf16x2(a[j].z * inv, a[j].w * inv);
+      const int qtok = h[j] / J.G;
+      *reinterpret_cast<uint2*>(J.out + ((static_cast<int64_t>(J.s) * J.T + qtok) * J.Hq + J.g * J.G + (h[j] - qtok * J.G)) * D +
+                                dq[j] * 4) = o;
+    }
+  }
+}
+
+// The merge warp of a CTA: takes the jobs the consumer warps post (one per partial written for a unit that the
+// decode kernel merges itself), in order, and runs merge_cut_unit for each.  It is the only warp of the kernel
+// that waits on global memory for a merge, and nothing waits for it: while the ring is full a dependent access
+// to global memory takes several microseconds (it queues behind the CTA's own bulk copies), which a consumer
+// warp cannot afford -- its ring slot would stay occupied.  Ends when every consumer warp has said it is done
+// and the queue is empty.  Every wait is bounded.
+template <int D, int NT>
+__device__ __forceinline__ void merge_warp_loop(const DecodeParams& P, Ctrl* ctrl, int ncw, int lane) {
+  constexpr int SLOT_FLOATS = 8 * NT * (D + 2);
+  constexpr int BATCH = 4;          // jobs whose tickets are drawn together (one lane each)
+  const unsigned long long t_start = globaltimer_ns();
+  for (int next = 0;;) {
+    bool have = false;
+    for (;;) {
+      if (ld_acquire_shared(&ctrl->mq_tag[next % MERGE_QUEUE]) == next + 1) {
+        have = true;
+        break;
+      }
+      if (ld_acquire_shared(&ctrl->mq_done) == ncw && ld_acquire_shared(&ctrl->mq_head) == next) break;
+      if (*reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) break;
+      if (globaltimer_ns() - t_start > 4 * kWaitLimitNs) {   // the whole kernel is bounded well below this
+        if (lane == 0) atomicOr(&P.hdr->err, ERR_TIMEOUT);
+        break;
+      }
+      __nanosleep(64);
+    }
+    if (!have) return;
+    // every job that is already there, up to BATCH: their round trips to global memory overlap
+    int nj = 1;
+    while (nj < BATCH && ld_acquire_shared(&ctrl->mq_tag[(next + nj) % MERGE_QUEUE]) == next + nj + 1) ++nj;
+    int4 j = make_int4(0, 0, 0, 0);
+    if (lane < nj) j = ctrl->mq_job[(next + lane) % MERGE_QUEUE];
+    __syncwarp();
+    if (lane == 0) st_release_shared(&ctrl->mq_tail, next + nj);   // the entries may be reused
+    next += nj;
+    // ---- tickets: the partials the consumer warps wrote (made visible to this warp by the queue's release /
+    // acquire) are published device-wide before them, the other CTAs' partials are read after them
+    int tot = 0;
+    if (lane < nj) {
+      // release: what this thread has observed so far (the posted partials) is visible device-wide before the
+      // ticket; acquire: what the earlier ticket holders published is visible to the loads that follow (the
+      // other lanes' loads are ordered behind this one by the warp-wide ballot below)
+      asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(tot) : "l"(P.tickets + j.x), "r"(j.z) : "memory");
+      tot += j.z;
+    }
+    const bool last = lane < nj && (tot & 0xffff) == 1 + __popc(j.y);
+    if (last) P.tickets[j.x] = 0;                   // everyone has drawn: rearm for the next call
+    uint32_t todo = __ballot_sync(0xffffffffu, last);
+    while (todo) {
+      const int i = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const int c = __shfl_sync(0xffffffffu, j.x, i), mask = __shfl_sync(0xffffffffu, j.y, i);
+      const int uw = __shfl_sync(0xffffffffu, j.w, i), own = __shfl_sync(0xffffffffu, tot, i) >> 16;
+      const int unit = uw & 0x3fffffff;
+      MergeJob J;
+      J.partials = P.partials;
+      J.pfx = (uw >> 30) ? P.pfx_partials + static_cast<int64_t>(unit) * SLOT_FLOATS : nullptr;
+      J.out = P.out;
+      J.c = c;
+      J.hold_mask = mask;
+      J.n_parts = 1 + __popc(mask);
+      J.s = unit / P.Hkv;
+      J.g = unit - J.s * P.Hkv;
+      J.G = P.G;
+      J.T = P.T;
+      J.Hq = P.Hq;
+      merge_cut_unit<D, NT>(J, own, lane);   // the piece in span c said which of its two slots it used
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Consumer side of decode_kernel<.., CHAIN = true>: the variant for batches of many short pieces.
 //
 // Tiles are dealt to the consumer warps exactly as in the default variant (tile i of the CTA to warp
@@ -336,12 +518,47 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
             a1[jm * 16 + 8] = acc[nt][jm][3];
           }
         }
+        // the unit's last partial to be written triggers its final merge; this warp only posts the job
+        if (C::MERGE_WARP && P.inkernel_max > 0) {
+          const int back = pc.tb > 0 ? merge_back(sp.merge) : 0;
+          if (back != kMergeTooLong) {
+            const int c = span - back;
+            const int32_t w = back == 0 ? sp.merge : (P.use_ws_plan ? P.spans_ws[c].merge : P.spans[c].merge);
+            const int run = merge_run(w);
+            if (run >= 1 && run <= P.inkernel_max) {
+              __syncwarp();            // every lane's part of the partial is written ...
+              if (lane == 0) {
+                const int k = atomicAdd(&ctrl->mq_head, 1);
+                bool room = k - ld_acquire_shared(&ctrl->mq_tail) < MERGE_QUEUE;
+                if (!room) {
+                  const unsigned long long t0 = globaltimer_ns();
+                  while (!(room = k - ld_acquire_shared(&ctrl->mq_tail) < MERGE_QUEUE))
+                    if (*reinterpret_cast<volatile uint32_t*>(&ctrl->abort) || globaltimer_ns() - t0 > kWaitLimitNs) break;
+                }
+                if (room) {
+                  const bool has_pfx = P.start_tiles != nullptr && pc.t0 > 0;
+                  ctrl->mq_job[k % MERGE_QUEUE] = make_int4(c, merge_hold_mask(w), 1 + (pc.tb == 0 ? (slot_idx << 16) : 0),
+                                                            pc.unit | (has_pfx ? (1 << 30) : 0));
+                  st_release_shared(&ctrl->mq_tag[k % MERGE_QUEUE], k + 1);   // ... before the job becomes visible
+                } else {
+                  atomicOr(&P.hdr->err, ERR_TIMEOUT);
+                  atomicExch(&ctrl->abort, 1u);
+                }
+              }
+            }
+          }
+        }
       }
     }
     if (warp == 0 && lane == 0) P.rec[span] = make_int4(first_unit, first_tb, own_unit, own_slot);
     span = read_span(ctrl, k + 1, aborted);
   }
   if (aborted && lane == 0) atomicOr(&P.hdr->err, ERR_TIMEOUT);
+  __syncwarp();
+  if (C::MERGE_WARP && lane == 0) {
+    __threadfence_block();
+    atomicAdd(&ctrl->mq_done, 1);     // this warp posts no more merge jobs
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -390,6 +607,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       ctrl->qseq[i] = -1;
     }
     for (int i = 0; i < 8; ++i) ctrl->turn[i] = i * 8;   // slot i first serves merge number i, class 0
+    ctrl->mq_head = ctrl->mq_tail = ctrl->mq_done = 0;
+    for (int i = 0; i < MERGE_QUEUE; ++i) ctrl->mq_tag[i] = 0;
     fence_mbar_init();
   }
   __syncthreads();
@@ -406,6 +625,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
   // split stage halves: only where the consumers use them (chained merge over the bf16 cache)
   constexpr bool SPLIT = CHAIN && EB == 2 && !PROBE;
+  if (C::MERGE_WARP && warp == NCW + C::NPW) {
+    // ================= merge warp =================
+    if constexpr (CHAIN && !PROBE && NT == 1) {
+      if (P.inkernel_max > 0) merge_warp_loop<D, NT>(P, ctrl, NCW, lane);
+    }
+    return;
+  }
   if (warp >= NCW) {
     // ================= producer warp(s) =================
     const int pw = warp - NCW;
@@ -566,6 +792,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       if (aborted) {
         atomicOr(&P.hdr->err, ERR_TIMEOUT);
         atomicExch(&ctrl->abort, 1u);
+      }
+      // this CTA draws no more run-time spans; the last CTA to say so rearms the counter for the next call
+      if (pw == 0 && atomicAdd(&P.hdr->done, 1) == static_cast<int>(gridDim.x) - 1) {
+        P.hdr->done = 0;
+        P.hdr->counter = 0;
       }
     }
     return;

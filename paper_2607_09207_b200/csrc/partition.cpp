@@ -35,7 +35,7 @@ bool plan_spans(const int32_t* context_lens, const int32_t* start_tiles, int num
       spans[c].unit = static_cast<int32_t>(static_cast<int64_t>(s) * num_kv_heads + k);
       spans[c].tile = tile;
       spans[c].flat = static_cast<int32_t>(tbase + static_cast<int64_t>(k) * nt + tile);
-      spans[c].pad = 0;
+      spans[c].merge = 0;
       ++c;
     }
     cbase += sc;
@@ -45,8 +45,9 @@ bool plan_spans(const int32_t* context_lens, const int32_t* start_tiles, int num
     spans[c].unit = num_seqs * num_kv_heads;
     spans[c].tile = 0;
     spans[c].flat = static_cast<int32_t>(total);
-    spans[c].pad = 0;
+    spans[c].merge = 0;
   }
+  for (int k = 0; k < n_spans; ++k) spans[k].merge = span_merge_info(spans, n_spans, k);
   return true;
 }
 

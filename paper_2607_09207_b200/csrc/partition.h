@@ -45,9 +45,52 @@ struct PlanParams {
 
 // One span: where it starts and the index of its first tile in the flattened stream.  Span i
 // holds spans[i + 1].flat - spans[i].flat tiles, so the table has n_static + n_dyn + 1 entries.
+// `merge` describes how the units that span boundaries cut are put together again (see span_merge_info).
 struct SpanStart {
-  int32_t unit, tile, flat, pad;
+  int32_t unit, tile, flat, merge;
 };
+
+// Merge word of span k.  A unit that starts in span c and runs past its end is followed by a run of spans that
+// begin inside it; each of those that holds tiles produces one partial (m, l, acc), as does span c itself.
+//   bits  0..14  as first span of such a unit: bit r set = span c + 1 + r holds tiles (a partial will exist)
+//   bits 16..20  ... the length of that run (0 = no unit runs past this span's end; kMergeTooLong = longer than
+//                kMaxMergeRun: left to the combine kernel)
+//   bits 24..28  as a span that begins inside a unit: how many spans back that unit's first span lies
+//                (0 = this span begins at a unit's tile 0; kMergeTooLong = too far back)
+constexpr int kMaxMergeRun = 15;
+constexpr int kMergeTooLong = 31;
+PDATTN_HD inline int merge_hold_mask(int32_t w) { return w & 0x7fff; }
+PDATTN_HD inline int merge_run(int32_t w) { return (w >> 16) & 31; }
+PDATTN_HD inline int merge_back(int32_t w) { return (w >> 24) & 31; }
+// spans: the finished table of n_spans + 1 entries (unit, tile, flat valid)
+PDATTN_HD inline int32_t span_merge_info(const SpanStart* spans, int n_spans, int k) {
+  const int unit_k = spans[k].unit;
+  int32_t w = 0;
+  // backwards: the first span of the unit this span begins inside
+  if (spans[k].tile > 0) {
+    int d = 1;
+    while (d <= kMaxMergeRun && k - d > 0 && spans[k - d].unit == unit_k && spans[k - d].tile > 0) ++d;
+    // span k - d is now the nearest one that does not begin inside the unit, or we gave up
+    const bool found = d <= kMaxMergeRun && !(spans[k - d].unit == unit_k && spans[k - d].tile > 0);
+    w |= (found ? d : kMergeTooLong) << 24;
+  }
+  // forwards: the run of spans that begin inside the unit that holds the last tile of span k, if that unit starts
+  // in span k (a unit that started earlier is described by its own first span)
+  if (k + 1 < n_spans && spans[k + 1].tile > 0 && spans[k + 1].flat > spans[k].flat) {
+    const int u = spans[k + 1].unit;
+    const bool starts_here = spans[k].unit < u || (spans[k].unit == u && spans[k].tile == 0);
+    if (starts_here) {
+      int run = 0, mask = 0;
+      while (k + 1 + run < n_spans && spans[k + 1 + run].unit == u && spans[k + 1 + run].tile > 0) {
+        if (run < kMaxMergeRun && spans[k + 2 + run].flat > spans[k + 1 + run].flat) mask |= 1 << run;
+        ++run;
+        if (run > kMaxMergeRun) break;
+      }
+      w |= mask | ((run > kMaxMergeRun ? kMergeTooLong : run) << 16);
+    }
+  }
+  return w;
+}
 
 PDATTN_HD inline PlanParams make_plan_params(int64_t total_cost, int64_t total_tiles, int n_static, int n_dyn_max) {
   PlanParams p;

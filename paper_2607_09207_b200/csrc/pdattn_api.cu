@@ -26,7 +26,9 @@ thread_local cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 int g_dyn_per_cta = -1;                   // run-time spans per CTA (pdattn_set_dynamic_spans); -1: by batch shape
 constexpr int kAutoDynPerCta = 4;         // ... then this many when the batch has at least kAutoDynUnits units per CTA
 constexpr int kAutoDynUnits = 4;
-int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (chained), 0 barrier, 1 chained
+int g_merge_mode = -1;                    // pdattn_set_merge_mode: -1 default (= 1), 0 barrier + combine kernel, 1 chained + merge
+                                          // of cut units inside the decode kernel, 2 chained + combine kernel
+constexpr int kInKernelMergeSpans = kMaxMergeRun;   // a cut unit followed by at most this many spans is merged inside the decode kernel
 int g_host_zero_copy = -1;                // pdattn_set_host_zero_copy: -1 default (when possible), 0 never, 1 as -1
 int g_prefix_engine = -1;                 // pdattn_set_prefix_engine: -1 default (tcgen05), 0 warp MMAs, 1 tcgen05
 thread_local std::vector<int32_t> g_start_tiles_host;   // scratch of the grouped path (no call parameter lives here)
@@ -81,7 +83,7 @@ WsLayout ws_layout(int num_seqs, int G, int head_dim, int max_spans = MAX_SPANS)
   const size_t slot_bytes = static_cast<size_t>(8 * NT) * (head_dim + 2) * 4;
   WsLayout w;
   w.hdr = 0;
-  w.spans = 256;
+  w.spans = WS_CLEARED_BYTES;   // header, then the ticket words
   w.rec = w.spans + align_up(static_cast<size_t>(max_spans + 1) * sizeof(SpanStart), 256);
   w.prefix = w.rec + align_up(static_cast<size_t>(max_spans) * sizeof(int4), 256);
   w.partials = w.prefix + align_up(static_cast<size_t>(num_seqs + 1) * 8, 256);
@@ -331,6 +333,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   if (g_prof_stop) cudaEventRecord(g_prof_stop, stream);
   // Programmatic dependent launch: the combine grid is set up while the decode kernel drains and
   // waits (griddepcontrol.wait in the kernel) until that kernel has completed and flushed.
+  if (combine_grid <= 0) return PDATTN_OK;   // every cut unit is merged inside the decode kernel
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(combine_grid);
   cfg.blockDim = dim3(256);
@@ -343,7 +346,7 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   cfg.numAttrs = 1;
   e = cudaLaunchKernelEx(&cfg, combine_kernel<D, NT>, P.hdr, n_spans_host, static_cast<const int4*>(P.rec),
                          static_cast<const float*>(P.partials), P.out, P.Hq, P.Hkv, P.G, P.start_tiles,
-                         P.pfx_partials, P.T);
+                         P.pfx_partials, P.T, P.inkernel_max);
   if (e != cudaSuccess) return cuda_fail("combine_kernel launch", e);
   return PDATTN_OK;
 }
@@ -361,7 +364,7 @@ pdattn_status launch_prefix_bs(const CUtensorMap& mk, const CUtensorMap& mv, con
     done = true;
   }
   if (grid <= 0) return PDATTN_OK;
-  kern<<<grid, C::NTHREADS, smem, stream>>>(mk, mv, X);
+  kern<<<grid, C::NTHREADS_BASE, smem, stream>>>(mk, mv, X);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail("prefix_kernel launch", e);
   return PDATTN_OK;
@@ -425,8 +428,9 @@ pdattn_status pdattn_workspace_size(int num_seqs, int num_q_heads, int num_kv_he
 }
 
 pdattn_status pdattn_workspace_init(void* workspace, size_t workspace_bytes, pdattn_stream_t stream) {
-  if (!workspace || workspace_bytes < 256) return PDATTN_INVALID_ARG;
-  cudaError_t e = cudaMemsetAsync(workspace, 0, 256, reinterpret_cast<cudaStream_t>(stream));
+  if (!workspace || workspace_bytes < static_cast<size_t>(WS_CLEARED_BYTES)) return PDATTN_INVALID_ARG;
+  // the header (error word, span counter) and the ticket words of the in-kernel merge start at zero
+  cudaError_t e = cudaMemsetAsync(workspace, 0, WS_CLEARED_BYTES, reinterpret_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
   return PDATTN_OK;
 }
@@ -491,7 +495,7 @@ pdattn_status pdattn_set_prefix_engine(int engine) {
 }
 
 pdattn_status pdattn_set_merge_mode(int mode) {
-  if (mode < -1 || mode > 1) return PDATTN_INVALID_ARG;
+  if (mode < -1 || mode > 2) return PDATTN_INVALID_ARG;
   g_merge_mode = mode;
   return PDATTN_OK;
 }
@@ -748,7 +752,8 @@ pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream_) {
   e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
   if (word == 0) return PDATTN_OK;
-  e = cudaMemsetAsync(workspace, 0, 4, stream);
+  // a failed call may have left ticket words and counters half-way: put all of them back to zero
+  e = cudaMemsetAsync(workspace, 0, WS_CLEARED_BYTES, stream);
   if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
   e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
@@ -856,9 +861,9 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
     }
     s = static_scratch_address(dev, &ws);
     if (s != PDATTN_OK) return s;
-    // The array still holds whatever the previous call left: the error word and the span counter
-    // must start at zero; everything else is written before it is read.
-    cudaError_t e = cudaMemsetAsync(ws, 0, 256, stream);
+    // The array still holds whatever the previous call left: the error word, the span counter and the
+    // ticket words must start at zero; everything else is written before it is read.
+    cudaError_t e = cudaMemsetAsync(ws, 0, WS_CLEARED_BYTES, stream);
     if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync(static scratch header)", e);
   }
 
@@ -906,6 +911,11 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
   P.box5d = 0;
   P.k_scale = fp8 ? cd.k_scale : nullptr;
   P.v_scale = fp8 ? cd.v_scale : nullptr;
+  P.tickets = reinterpret_cast<int32_t*>(ws + WS_TICKETS_OFFSET);
+  // the final merge of cut units: inside the decode kernel with the chained merge (modes -1 and 1) and 8-row
+  // tiles, in combine_kernel alone with the barrier merge (0), with 16-row tiles or when asked for (2)
+  const bool chain = g_merge_mode != 0;
+  P.inkernel_max = (chain && g_merge_mode != 2 && !cd.probe && G * T <= 8) ? kInKernelMergeSpans : 0;
 
   // Run-time spans even out the CTAs' finishing times when there are many units; with few long sequences
   // they only lengthen the chains the combine kernel walks.  The choice depends on the batch shape alone.
@@ -924,6 +934,13 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
       return PDATTN_INVALID_ARG;
     n_spans_host = P.plan.n_static + P.plan.n_dyn;
     combine_grid = n_spans_host;
+    if (P.inkernel_max > 0) {
+      // if every cut unit is short enough for the decode kernel's own merge, combine_kernel has nothing to do
+      // and is not launched
+      bool all_short = true;
+      for (int k = 0; k < n_spans_host && all_short; ++k) all_short = merge_run(P.spans[k].merge) <= P.inkernel_max;
+      if (all_short) combine_grid = 0;
+    }
   } else {
     P.use_ws_plan = 1;
     memset(&P.plan, 0, sizeof P.plan);
@@ -955,7 +972,7 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
                a->kv_head_stride, a->kv_token_stride, fp8 ? kMapV8 : rank, &mv);
   if (s != PDATTN_OK) return s;
   P.box5d = rank == 5;
-  const LaunchCtx lc{a->block_size, g_merge_mode != 0, cd.probe, fp8, di, stream};
+  const LaunchCtx lc{a->block_size, chain, cd.probe, fp8, di, stream};
 
   if (grouped) {
     // shared prompt tiles first: one pass per (group, kv head) for the query rows of all samples
@@ -1021,7 +1038,7 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
     s = nt2 ? launch<64, 2>(mk, mv, P, grid, combine_grid, n_spans_host, lc)
             : launch<64, 1>(mk, mv, P, grid, combine_grid, n_spans_host, lc);
   if (s != PDATTN_OK) return s;
-  if (!cd.probe) g_last_launches += 2;
+  if (!cd.probe) g_last_launches += combine_grid > 0 ? 2 : 1;
   if (cd.status_out) {
     cudaError_t e = cudaMemcpyAsync(cd.status_out, ws, 4, cudaMemcpyDeviceToDevice, stream);
     if (e != cudaSuccess) return cuda_fail("cudaMemcpyAsync(status_out)", e);

@@ -30,7 +30,7 @@ struct PrefixParams {
 };
 
 template <int D, int BS>
-__global__ void __launch_bounds__(Cfg<D, 1, BS>::NTHREADS, 1)
+__global__ void __launch_bounds__(Cfg<D, 1, BS>::NTHREADS_BASE, 1)
 prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
               const __grid_constant__ PrefixParams P) {
   using C = Cfg<D, 1, BS>;

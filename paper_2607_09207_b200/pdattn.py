@@ -390,6 +390,32 @@ def decode_host(q_host, block_table_host, context_lens_host, out_host, k_cache, 
     return st
 
 
+class HostStep:
+    """pdattn_decode_host for a decode loop that reuses its buffers: the engine rewrites q_host, block_table_host
+    and context_lens_host in place every step and reads out_host after synchronising the stream.  The arguments
+    are marshalled once, so a step is a single foreign call (argument marshalling only; same entry point, same
+    results as decode_host)."""
+
+    def __init__(self, q_host, block_table_host, context_lens_host, out_host, k_cache, v_cache, scale, staging,
+                 workspace, stream=None):
+        S, Hq, d = q_host.shape
+        NB, Hkv, bs, _ = k_cache.shape
+        self._keep = (q_host, block_table_host, context_lens_host, out_host, k_cache, v_cache, staging, workspace)
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        self._args = (vp(q_host.data_ptr()), vp(block_table_host.data_ptr()), vp(context_lens_host.data_ptr()),
+                      vp(out_host.data_ptr()), vp(k_cache.data_ptr()), vp(v_cache.data_ptr()), ci(S), ci(Hq), ci(Hkv),
+                      ci(d), ci(bs), ci(block_table_host.shape[1]), ci(NB), ctypes.c_float(float(scale)),
+                      vp(staging.data_ptr()), ctypes.c_size_t(staging.numel()), vp(workspace.data_ptr()),
+                      ctypes.c_size_t(workspace.numel()), vp(_stream_ptr(stream)))
+        self._fn = lib().pdattn_decode_host
+
+    def __call__(self, check: bool = True) -> int:
+        st = self._fn(*self._args)
+        if check and st != OK:
+            raise PdattnError(st, "pdattn_decode_host")
+        return st
+
+
 def set_dynamic_spans(per_cta: int):
     st = lib().pdattn_set_dynamic_spans(per_cta)
     if st != OK:
@@ -397,7 +423,8 @@ def set_dynamic_spans(per_cta: int):
 
 
 def set_merge_mode(mode: int):
-    """-1: by piece length (default); 0: barrier merge; 1: chained merge."""
+    """-1: default (= 1); 0: barrier merge + combine kernel; 1: chained merge + final merge of cut units inside the
+    decode kernel; 2: chained merge + combine kernel."""
     st = lib().pdattn_set_merge_mode(mode)
     if st != OK:
         raise PdattnError(st, "pdattn_set_merge_mode")

@@ -26,10 +26,11 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
-# The GPU parity modules run once per merge mode of the decode kernel's consumer warps: the barrier
-# merge and the chained merge must each pass every case, whatever the library would pick by itself.
+# The GPU parity modules run once per merge mode: the barrier merge with the combine kernel, the chained merge
+# with the final merge of cut units inside the decode kernel (the default), and the chained merge with the
+# combine kernel must each pass every case, whatever the library would pick by itself.
 MERGE_MODE_MODULES = ("test_gpu_parity", "test_gpu_grouped", "test_gpu_decode_loop", "test_gpu_multi_token")
-MERGE_MODES = {"barrier": 0, "chain": 1}
+MERGE_MODES = {"barrier": 0, "chain": 1, "chain_combine": 2}
 
 
 # ... and the grouped-decode module once per kernel for the shared prompt tiles.

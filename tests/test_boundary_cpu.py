@@ -66,9 +66,9 @@ def test_status_strings():
 
 def test_tuning_setters_check_their_ranges():
     L = pdattn.lib()
-    for mode in (-1, 0, 1):
+    for mode in (-1, 0, 1, 2):
         assert L.pdattn_set_merge_mode(mode) == pdattn.OK
-    for mode in (-2, 2, 100):
+    for mode in (-2, 3, 100):
         assert L.pdattn_set_merge_mode(mode) == pdattn.INVALID_ARG
     L.pdattn_set_merge_mode(-1)
     assert L.pdattn_set_dynamic_spans(-2) == pdattn.INVALID_ARG

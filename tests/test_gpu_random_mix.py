@@ -41,7 +41,7 @@ def test_random_mix_of_everything(seed):
             hi = {"short": 130, "mid": 1200, "long": 9000, "mixed": 3000}[kind]
             lens = rng.integers(0, hi, size=S)
             if kind == "mixed": lens[rng.integers(S)] = int(rng.integers(20000, 60000))
-            mode = int(rng.choice([-1, 0, 1])); dyn = int(rng.choice([-1, 0, 3, 8])); host = bool(rng.integers(2))
+            mode = int(rng.choice([-1, 0, 1, 2])); dyn = int(rng.choice([-1, 0, 3, 8])); host = bool(rng.integers(2))
             pdattn.set_merge_mode(mode); pdattn.set_dynamic_spans(dyn)
             variant = rng.choice(["plain", "multi", "fp8", "grouped", "fp8multi"])
             G = Hq // Hkv
