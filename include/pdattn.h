@@ -294,7 +294,9 @@ pdattn_status pdattn_set_dynamic_spans(int per_cta);
  *     combine kernel launched behind it.
  * mode 1: chained + merge of cut units inside the decode kernel (one launch per step when every chain is short
  * enough and context_lens_host is given); mode 2: chained + combine kernel; mode 0: barrier + combine kernel;
- * -1 (default): 1.  In every mode the order of every sum is fixed by tile and span indices, so a setting's
+ * -1 (default): 1 when context_lens_host is given and the batch averages at least 8 tiles (512 tokens) per
+ * sequence and KV head, else 2 (on batches of short ragged sequences the in-kernel merge costs more than the
+ * launch it saves).  In every mode the order of every sum is fixed by tile and span indices, so a setting's
  * results are bit-identical from run to run and under any renumbering of the physical pages.
  */
 pdattn_status pdattn_set_merge_mode(int mode);

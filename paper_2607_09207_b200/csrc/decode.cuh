@@ -676,7 +676,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const int pbase = (pc.t0 + pc.tb) * C::PAGES;
         // A context length beyond what the table row can describe: the entries past the row's end are not
         // read (they belong to the next row, or lie past the allocation); their tokens count as a bad page.
-        auto page_id = [&](int idx) { return idx < npages ? (idx < P.MB ? __ldg(row + idx) : -1) : 0; };
+        const int nread = min(npages, P.MB);
+        auto page_id = [&](int idx) {
+          int id = idx < npages ? -1 : 0;
+          if (idx < nread) id = __ldg(row + idx);
+          return id;
+        };
         int ids_cur = page_id(pbase + lane);
         int ids_nxt = page_id(pbase + IDS_PER_BATCH + lane);
         for (int t = pc.tb; t < pc.te; ++t, ++it) {

@@ -423,7 +423,7 @@ def set_dynamic_spans(per_cta: int):
 
 
 def set_merge_mode(mode: int):
-    """-1: default (= 1); 0: barrier merge + combine kernel; 1: chained merge + final merge of cut units inside the
+    """-1: default (1 for batches of long sequences with host lengths, else 2); 0: barrier merge + combine kernel; 1: chained merge + final merge of cut units inside the
     decode kernel; 2: chained merge + combine kernel."""
     st = lib().pdattn_set_merge_mode(mode)
     if st != OK:

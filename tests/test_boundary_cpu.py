@@ -186,6 +186,53 @@ def test_partitioner_covers_every_tile_exactly_once(case, n_ctas, dyn):
     assert plan.n_dynamic <= 8 * n_ctas
 
 
+@pytest.mark.parametrize("case", ["cfg1", "cfg2", "cfg5", "zeros", "short", "one", "long"])
+@pytest.mark.parametrize("n_ctas", [7, 148])
+@pytest.mark.parametrize("dyn", [0, 8])
+def test_merge_words_describe_every_cut_unit(case, n_ctas, dyn):
+    """The fourth word of a span says how the units that span boundaries cut are put together again.  Rebuilt here
+    from the coverage alone: for a unit that starts in span c and has tiles in later spans, word c holds the number
+    of spans up to the last one that begins inside the unit and one bit per such span that holds tiles; every span
+    that begins inside a unit says how far back the unit's first span lies.  Chains longer than 15 spans say so."""
+    lens, Hkv = {
+        "cfg1": (W.config_lengths(1), 1), "cfg2": (W.config_lengths(2), 4), "cfg5": (W.config_lengths(5), 4),
+        "zeros": (np.array([0, 5, 0, 0, 300, 0]), 2), "short": (np.arange(1, 40), 3), "one": (np.array([1]), 8),
+        "long": (np.array([40000, 3, 70000]), 1),
+    }[case]
+    spans, plan = pdattn.plan_host(lens, Hkv, n_ctas, dynamic_per_cta=dyn)
+    cover, _ = walk_spans(lens, Hkv, n_ctas, dyn)
+    n = len(cover)
+    word = [int(spans[k, 3]) for k in range(n)]
+    first_span, holders = {}, {}
+    for k, mine in enumerate(cover):
+        for u in sorted({u for u, _ in mine}):
+            first_span.setdefault(u, k)
+            holders.setdefault(u, []).append(k)
+    seen_owner = set()
+    for u, ks in holders.items():
+        if len(ks) == 1:
+            continue                                         # not cut
+        c = first_span[u]
+        seen_owner.add(c)
+        inside = [k for k in range(c + 1, n) if int(spans[k, 0]) == u and int(spans[k, 1]) > 0]
+        assert inside and inside == list(range(c + 1, c + 1 + len(inside)))       # a run right behind span c
+        assert set(ks[1:]) <= set(inside)
+        run = (word[c] >> 16) & 31
+        if len(inside) > 15:
+            assert run == 31
+        else:
+            assert run == len(inside)
+            assert (word[c] & 0x7fff) == sum(1 << (k - c - 1) for k in ks[1:])
+        for k in inside:
+            back = (word[k] >> 24) & 31
+            assert back == (k - c if k - c <= 15 else 31)
+    for k in range(n):
+        if k not in seen_owner:
+            assert (word[k] >> 16) & 31 == 0                 # no unit runs past this span's end
+        if int(spans[k, 1]) == 0:
+            assert (word[k] >> 24) & 31 == 0                 # begins at a unit's first tile
+
+
 def test_partitioner_balances_cost_not_tiles():
     """Config 2: CTAs inside long sequences get more tiles than CTAs that walk many short ones, and the
     cost (tiles + 2 per unit touched) is even to within one unit's start-up plus the cut unit."""
