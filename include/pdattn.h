@@ -167,8 +167,7 @@ pdattn_status pdattn_decode_multi(const pdattn_args* args, int num_query_tokens,
  * including the treatment of bad page ids and of slots past the end (any code, NaN codes too).
  * The codes are widened exactly; q is rounded to fp16 for the products (values below 2^-14 lose bits) and
  * the softmax weights to fp16 (11 bits), accumulation in fp32; out is bf16.
- *   Requirements: head_dim 128 (else PDATTN_UNSUPPORTED; every page size of pdattn_decode_ex); not combined with
- *   pdattn_decode_grouped.  Workspace as for pdattn_decode_ex.
+ *   Requirements: head_dim 128 or 64, every page size of pdattn_decode_ex.  Workspace as for pdattn_decode_ex.
  */
 pdattn_status pdattn_decode_fp8(const pdattn_args* args, const float* k_scale, const float* v_scale,
                                 pdattn_stream_t stream);
@@ -178,11 +177,21 @@ pdattn_status pdattn_decode_fp8_multi(const pdattn_args* args, int num_query_tok
                                       const float* v_scale, pdattn_stream_t stream);
 
 /*
+ * pdattn_decode_grouped over the fp8 cache of pdattn_decode_fp8 (GRPO prompt groups, Section 2.1, with the one-byte
+ * cache elements of Appendix A.1.2's b_dtype): same group rules, same workspace size, same layouts as
+ * pdattn_decode_fp8.  The shared tiles are scored with warp-level MMAs on the widened codes, eight query rows per
+ * warp, so group_size * G <= 48 (else PDATTN_UNSUPPORTED; pass a larger group as several smaller ones).
+ */
+pdattn_status pdattn_decode_grouped_fp8(const pdattn_args* args, int group_size, const int32_t* prefix_tiles,
+                                        const int32_t* prefix_tiles_host, const float* k_scale, const float* v_scale,
+                                        pdattn_stream_t stream);
+
+/*
  * KV append into the fp8 cache of pdattn_decode_fp8 (same layouts): the rows k_new[s], v_new[s] (DEVICE
  * bf16 [num_seqs, num_kv_heads, head_dim]) are divided by their KV head's scale, rounded to e4m3 (nearest
  * even; magnitudes beyond the largest finite code 448 saturate to it) and written at position
  * context_lens[s], which then becomes context_lens[s] + 1.  Page rules and error reporting as in
- * pdattn_append_kv.  head_dim 128.
+ * pdattn_append_kv.  head_dim 128 or 64.
  */
 pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                                    const float* k_scale, const float* v_scale, const int32_t* block_table,
@@ -251,6 +260,19 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
                                  void* workspace, size_t workspace_bytes, pdattn_stream_t stream);
 
 /*
+ * pdattn_decode_host over the fp8 cache of pdattn_decode_fp8: k_cache / v_cache are the DEVICE code pools in that
+ * entry point's layouts, k_scale / v_scale DEVICE fp32 [num_kv_heads]; everything else as pdattn_decode_host
+ * (the per-step inputs q, block_table, context_lens and the result `out` live in HOST memory; same staging size).
+ */
+pdattn_status pdattn_decode_host_fp8(const void* q_host, const int32_t* block_table_host,
+                                     const int32_t* context_lens_host, void* out_host,
+                                     const void* k_cache, const void* v_cache, const float* k_scale,
+                                     const float* v_scale, int num_seqs, int num_q_heads, int num_kv_heads,
+                                     int head_dim, int block_size, int max_blocks_per_seq, int num_blocks, float scale,
+                                     void* staging, size_t staging_bytes,
+                                     void* workspace, size_t workspace_bytes, pdattn_stream_t stream);
+
+/*
  * The host partitioner on its own (no GPU needed).  It flattens the batch into a stream of
  * 64-token tiles, unit-major (unit = s * num_kv_heads + kv_head; unit u has ceil(L_s / 64)
  * tiles), and cuts it into contiguous spans so that long-tail sequences are spread over all SMs
@@ -259,9 +281,13 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
  * tiles than one inside a long sequence.  n_static spans, one per CTA, cover the stream; with
  * dynamic_per_cta > 0 they cover only its first three quarters (by cost) and up to n_ctas *
  * dynamic_per_cta short spans cover the rest, taken at run time by whichever CTA is free.
- * spans: HOST int32 [4 * (max_spans + 1)], one (unit, tile, flat, 0) entry per span plus an end
+ * spans: HOST int32 [4 * (max_spans + 1)], one (unit, tile, flat, merge) entry per span plus an end
  * marker: span i starts at tile `tile` of unit `unit`, which is tile number `flat` of the stream,
  * and holds flat[i + 1] - flat[i] tiles (possibly none).  n_static + n_dynamic <= max_spans.
+ * `merge` says how a unit that span boundaries cut is put together again: bits 16-20 the number of spans
+ * right behind span i that begin inside the unit that starts in span i and runs past its end (0 = none,
+ * 31 = more than 15), bits 0-14 which of those hold tiles (each writes one partial), bits 24-28, for a span
+ * that begins inside a unit, how many spans back that unit's first span lies (31 = more than 15).
  * The plan depends on the context lengths only, never on page ids.
  */
 typedef struct {

@@ -231,7 +231,7 @@ __device__ __forceinline__ void bar_consumers() {   // named barrier 1: the NCT 
 template <int D, int NT, int BS, int EB = 2>   // EB: bytes per cache element (2 = bf16, 1 = fp8 codes)
 struct Cfg {
   static constexpr int PAGES = TILE / BS;              // pages per tile
-  static constexpr int HALVES = D * EB / 128;          // 128-byte column blocks per row
+  static constexpr int HALVES = D * EB / 128 > 0 ? D * EB / 128 : 1;   // copies per page-head with the rank-4 view
   static constexpr int HALF_BYTES = BS * 128;          // one TMA box: BS rows x 128 bytes
   static constexpr int PAGE_BYTES = BS * D * EB;
   static constexpr int KV_BYTES = TILE * D * EB;

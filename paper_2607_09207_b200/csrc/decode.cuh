@@ -213,7 +213,6 @@ template <int D, int NT, int BS, int EB>
 __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanParams& pp, Ctrl* ctrl, uint32_t ring,
                                               uint32_t qbuf, uint8_t* handoff, int warp, int lane) {
   using C = Cfg<D, NT, BS, EB>;
-  static_assert(EB == 2 || (EB == 1 && D == 128), "the fp8 cache path is built for head_dim 128");
   constexpr int NST = C::NSTAGES;
   constexpr int NCW = C::NCW;
   constexpr int E = C::HANDOFFS;
@@ -367,9 +366,9 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
           continue;
         } else {
           if (n_left - (P.T - 1) >= TILE) {
-            compute_tile_f8<NT, BS, false>(sK, sV, qf, acc, m, l, sl2, TILE, badmask, lane, lag);
+            compute_tile_f8<D, NT, BS, false>(sK, sV, qf, acc, m, l, sl2, TILE, badmask, lane, lag);
           } else {
-            compute_tile_f8<NT, BS, true>(sK, sV, qf, acc, m, l, sl2, n_left, badmask, lane, lag);
+            compute_tile_f8<D, NT, BS, true>(sK, sV, qf, acc, m, l, sl2, n_left, badmask, lane, lag);
           }
         }
         __syncwarp();

@@ -108,7 +108,8 @@ struct DevInfo {
   bool attr_set[2][2][3] = {};      // [D==128][NT==2][page size / 32]
   bool probe_attr_set[2][2][3] = {};
   bool chain_attr_set[2][2][3] = {};
-  bool fp8_attr_set[2][3] = {};     // [NT==2][page size / 32]
+  bool fp8_attr_set[2][2][3] = {};  // [D==128][NT==2][page size / 32]
+  bool prefix_fp8_attr_set[2][3] = {};
   bool prefix_attr_set[2][3] = {};  // [D==128][page size / 32]
   bool prefix_umma_attr_set[2][3] = {};
 };
@@ -208,9 +209,10 @@ pdattn_status make_map(const void* ptr, int d, int bs, int hkv, int nb, int64_t 
                              static_cast<cuuint64_t>(hkv) * bs * d};
     cuuint32_t box[4] = {static_cast<cuuint32_t>(d), static_cast<cuuint32_t>(bs), 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
+    // rows of d bytes: 128-byte swizzle at head_dim 128, 64-byte swizzle at head_dim 64
     r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, d == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else if (rank == kMapV8) {
     // fp8 V pool [pages, kv heads, d, slots] (transposed inside a page): a page-head is d * block_size
     // contiguous bytes and lands in shared memory in the same order, so it is described as rows of 256
@@ -304,19 +306,15 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   const bool dependent = g_prof_start == nullptr;
   if (g_prof_start) cudaEventRecord(g_prof_start, stream);
   if (lc.fp8) {
-    if constexpr (D == 128) {
-      using C8 = Cfg<D, NT, BS, 1>;
-      auto k8 = decode_kernel<D, NT, BS, false, true, 1>;
-      bool& fdone = di->fp8_attr_set[NT == 2][BS / 32];
-      if (!fdone) {
-        cudaError_t fe = cudaFuncSetAttribute(k8, cudaFuncAttributeMaxDynamicSharedMemorySize, C8::CHAIN_DYN_BYTES);
-        if (fe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", fe);
-        fdone = true;
-      }
-      launch_dependent(k8, grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream, dependent, mk, mv, P);
-    } else {
-      return PDATTN_UNSUPPORTED;
+    using C8 = Cfg<D, NT, BS, 1>;
+    auto k8 = decode_kernel<D, NT, BS, false, true, 1>;
+    bool& fdone = di->fp8_attr_set[D == 128][NT == 2][BS / 32];
+    if (!fdone) {
+      cudaError_t fe = cudaFuncSetAttribute(k8, cudaFuncAttributeMaxDynamicSharedMemorySize, C8::CHAIN_DYN_BYTES);
+      if (fe != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", fe);
+      fdone = true;
     }
+    launch_dependent(k8, grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream, dependent, mk, mv, P);
   } else if (lc.chain) {
     auto chain = decode_kernel<D, NT, BS, false, true>;
     bool& cdone = di->chain_attr_set[D == 128][NT == 2][BS / 32];
@@ -352,13 +350,13 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
   return PDATTN_OK;
 }
 
-template <int D, int BS>
+template <int D, int BS, int EB>
 pdattn_status launch_prefix_bs(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid, DevInfo* di,
                             cudaStream_t stream) {
-  using C = Cfg<D, 1, BS>;
+  using C = Cfg<D, 1, BS, EB>;
   const int smem = 1024 + C::NSTAGES * C::STAGE_BYTES + C::CTRL_BYTES;
-  auto kern = prefix_kernel<D, BS>;
-  bool& done = di->prefix_attr_set[D == 128][BS / 32];
+  auto kern = prefix_kernel<D, BS, EB>;
+  bool& done = EB == 1 ? di->prefix_fp8_attr_set[D == 128][BS / 32] : di->prefix_attr_set[D == 128][BS / 32];
   if (!done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
@@ -406,9 +404,13 @@ pdattn_status launch_prefix_umma(const CUtensorMap& mk, const CUtensorMap& mv, c
 template <int D>
 pdattn_status launch_prefix(const CUtensorMap& mk, const CUtensorMap& mv, const PrefixParams& X, int grid,
                             const LaunchCtx& lc) {
-  return lc.block_size == 64   ? launch_prefix_bs<D, 64>(mk, mv, X, grid, lc.di, lc.stream)
-         : lc.block_size == 32 ? launch_prefix_bs<D, 32>(mk, mv, X, grid, lc.di, lc.stream)
-                               : launch_prefix_bs<D, 16>(mk, mv, X, grid, lc.di, lc.stream);
+  if (lc.fp8)
+    return lc.block_size == 64   ? launch_prefix_bs<D, 64, 1>(mk, mv, X, grid, lc.di, lc.stream)
+           : lc.block_size == 32 ? launch_prefix_bs<D, 32, 1>(mk, mv, X, grid, lc.di, lc.stream)
+                                 : launch_prefix_bs<D, 16, 1>(mk, mv, X, grid, lc.di, lc.stream);
+  return lc.block_size == 64   ? launch_prefix_bs<D, 64, 2>(mk, mv, X, grid, lc.di, lc.stream)
+         : lc.block_size == 32 ? launch_prefix_bs<D, 32, 2>(mk, mv, X, grid, lc.di, lc.stream)
+                               : launch_prefix_bs<D, 16, 2>(mk, mv, X, grid, lc.di, lc.stream);
 }
 
 pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_stream_t stream_);
@@ -474,7 +476,8 @@ pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k
                                    pdattn_stream_t stream) {
   if (num_seqs < 0 || num_kv_heads <= 0 || num_kv_heads > 16 || max_blocks_per_seq <= 0 || num_blocks <= 0)
     return PDATTN_INVALID_ARG;
-  if (head_dim != 128 || (block_size != 16 && block_size != 32 && block_size != 64)) return PDATTN_UNSUPPORTED;
+  if ((head_dim != 128 && head_dim != 64) || (block_size != 16 && block_size != 32 && block_size != 64))
+    return PDATTN_UNSUPPORTED;
   if (num_seqs == 0) return PDATTN_OK;
   if (!k_new || !v_new || !k_cache || !v_cache || !k_scale || !v_scale || !block_table || !context_lens)
     return PDATTN_INVALID_ARG;
@@ -650,12 +653,12 @@ static void* mapped_host_pointer(const void* p) {
   return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
 }
 
-pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_host,
-                                 const int32_t* context_lens_host, void* out_host, const void* k_cache,
-                                 const void* v_cache, int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
-                                 int block_size, int max_blocks_per_seq, int num_blocks, float scale, void* staging,
-                                 size_t staging_bytes, void* workspace, size_t workspace_bytes,
-                                 pdattn_stream_t stream_) {
+static pdattn_status decode_host_common(const void* q_host, const int32_t* block_table_host,
+                                        const int32_t* context_lens_host, void* out_host, const void* k_cache,
+                                        const void* v_cache, int num_seqs, int num_q_heads, int num_kv_heads,
+                                        int head_dim, int block_size, int max_blocks_per_seq, int num_blocks, float scale,
+                                        void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                        const CallDesc& cd, pdattn_stream_t stream_) {
   if (num_seqs == 0) return PDATTN_OK;
   if (!q_host || !block_table_host || !context_lens_host || !out_host || !staging) return PDATTN_INVALID_ARG;
   size_t need = 0;
@@ -737,11 +740,58 @@ pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_
   a.scale = scale;
   a.workspace = workspace;
   a.workspace_bytes = workspace_bytes;
-  s = pdattn_decode_ex(&a, stream_);
+  s = decode_common(&a, cd, stream_);
   if (s != PDATTN_OK) return s;
   if (!in_place && (e = cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
     return cuda_fail("cudaMemcpyAsync(out)", e);
   return PDATTN_OK;
+}
+
+pdattn_status pdattn_decode_host(const void* q_host, const int32_t* block_table_host,
+                                 const int32_t* context_lens_host, void* out_host, const void* k_cache,
+                                 const void* v_cache, int num_seqs, int num_q_heads, int num_kv_heads, int head_dim,
+                                 int block_size, int max_blocks_per_seq, int num_blocks, float scale, void* staging,
+                                 size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                 pdattn_stream_t stream) {
+  return decode_host_common(q_host, block_table_host, context_lens_host, out_host, k_cache, v_cache, num_seqs,
+                            num_q_heads, num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks, scale,
+                            staging, staging_bytes, workspace, workspace_bytes, CallDesc{}, stream);
+}
+
+pdattn_status pdattn_decode_host_fp8(const void* q_host, const int32_t* block_table_host,
+                                     const int32_t* context_lens_host, void* out_host, const void* k_cache,
+                                     const void* v_cache, const float* k_scale, const float* v_scale, int num_seqs,
+                                     int num_q_heads, int num_kv_heads, int head_dim, int block_size,
+                                     int max_blocks_per_seq, int num_blocks, float scale, void* staging,
+                                     size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                     pdattn_stream_t stream) {
+  if (!k_scale || !v_scale) return PDATTN_INVALID_ARG;
+  CallDesc cd;
+  cd.fp8 = true;
+  cd.k_scale = k_scale;
+  cd.v_scale = v_scale;
+  return decode_host_common(q_host, block_table_host, context_lens_host, out_host, k_cache, v_cache, num_seqs,
+                            num_q_heads, num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks, scale,
+                            staging, staging_bytes, workspace, workspace_bytes, cd, stream);
+}
+
+pdattn_status pdattn_decode_grouped_fp8(const pdattn_args* args, int group_size, const int32_t* prefix_tiles,
+                                        const int32_t* prefix_tiles_host, const float* k_scale, const float* v_scale,
+                                        pdattn_stream_t stream) {
+  if (!args || !prefix_tiles || !prefix_tiles_host || !k_scale || !v_scale) return PDATTN_INVALID_ARG;
+  if (group_size <= 0) return PDATTN_INVALID_ARG;
+  pdattn_args a = *args;
+  a.kv_token_stride = a.head_dim;
+  a.kv_head_stride = static_cast<int64_t>(a.block_size) * a.head_dim;
+  a.kv_block_stride = static_cast<int64_t>(a.num_kv_heads) * a.block_size * a.head_dim;
+  CallDesc cd;
+  cd.group_size = group_size;
+  cd.prefix_tiles = prefix_tiles;
+  cd.prefix_tiles_host = prefix_tiles_host;
+  cd.fp8 = true;
+  cd.k_scale = k_scale;
+  cd.v_scale = v_scale;
+  return decode_common(&a, cd, stream);
 }
 
 pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream_) {
@@ -817,7 +867,7 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
   const bool fp8 = cd.fp8;
   if (T < 1) return PDATTN_INVALID_ARG;
   if (G * T > 16 || (T > 1 && grouped)) return PDATTN_UNSUPPORTED;
-  if (fp8 && (a->head_dim != 128 || grouped || cd.probe)) return PDATTN_UNSUPPORTED;
+  if (fp8 && cd.probe) return PDATTN_UNSUPPORTED;
   if (fp8 && (!cd.k_scale || !cd.v_scale)) return PDATTN_INVALID_ARG;
   if (cd.static_scratch && (grouped || fp8 || T != 1 || cd.probe)) return PDATTN_UNSUPPORTED;
   // a context longer than its block_table row can describe is refused here when the host knows the lengths;
@@ -870,10 +920,12 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
 
   const int32_t* start_tiles_host = nullptr;
   int n_groups = 0;
+  const bool umma = g_prefix_engine != 0 && !fp8;   // which kernel takes the shared tiles of a grouped call
   if (grouped) {
     const int Gs = cd.group_size;
-    // rows the kernel for the shared tiles takes per unit: 64 on tensor memory, 48 with warp MMAs
-    const int max_rows = g_prefix_engine != 0 ? UMMA_MAX_QUERY_ROWS : MAX_PREFIX_ROWS;
+    // rows the kernel for the shared tiles takes per unit: 64 on tensor memory, 48 with warp MMAs (the only
+    // kernel for the shared tiles of an fp8 cache)
+    const int max_rows = umma ? UMMA_MAX_QUERY_ROWS : MAX_PREFIX_ROWS;
     if (G > 8 || Gs * G > max_rows) return PDATTN_UNSUPPORTED;
     if (!a->context_lens_host || a->num_seqs % Gs != 0) return PDATTN_INVALID_ARG;
     n_groups = a->num_seqs / Gs;
@@ -1000,6 +1052,8 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
     X.NB = a->num_blocks;
     X.scale_log2 = P.scale_log2;
     X.box5d = P.box5d;
+    X.k_scale = P.k_scale;
+    X.v_scale = P.v_scale;
     // whole units, contiguous ranges of equal tile count (to within one unit)
     const int n_units = n_groups * a->num_kv_heads;
     int64_t total = 0;
@@ -1017,7 +1071,7 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
       }
       X.ranges[c] = make_int2(u0, u);
     }
-    if (g_prefix_engine != 0) {
+    if (umma) {
       // tensor-memory kernel: its tiles are laid out per 64-column block, so it takes the rank-4 view
       CUtensorMap pk = mk, pv = mv;
       if (rank != 4) {

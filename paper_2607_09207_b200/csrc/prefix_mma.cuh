@@ -3,6 +3,7 @@
 
 #include "common.cuh"
 #include "tile_bf16.cuh"
+#include "tile_fp8.cuh"
 
 namespace pdattn {
 
@@ -26,14 +27,17 @@ struct PrefixParams {
   int S, Hq, Hkv, G, Gs, MB, NB;
   float scale_log2;
   int box5d;
+  const float* k_scale;          // fp8 cache only (EB = 1): per KV head, value = scale * e4m3 code
+  const float* v_scale;
   int2 ranges[160];
 };
 
-template <int D, int BS>
-__global__ void __launch_bounds__(Cfg<D, 1, BS>::NTHREADS_BASE, 1)
+// EB: bytes per cache element (2 = bf16 through compute_tile, 1 = e4m3 codes through compute_tile_f8)
+template <int D, int BS, int EB = 2>
+__global__ void __launch_bounds__(Cfg<D, 1, BS, EB>::NTHREADS_BASE, 1)
 prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
               const __grid_constant__ PrefixParams P) {
-  using C = Cfg<D, 1, BS>;
+  using C = Cfg<D, 1, BS, EB>;
   constexpr int NST = C::NSTAGES;
   constexpr int NCW = C::NCW;
   static_assert(NST % C::NPW == 0, "a slot is always refilled by the same producer warp");
@@ -146,10 +150,20 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           reinterpret_cast<const uint32_t*>(P.q + (static_cast<int64_t>(s0 + j) * P.Hq + g * P.G + h) * D);
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
-        qf[0][kk][0] = live ? __ldg(qp + (kk * 16 + qcol) / 2) : 0u;
-        qf[0][kk][1] = live ? __ldg(qp + (kk * 16 + 8 + qcol) / 2) : 0u;
+        if constexpr (EB == 2) {
+          qf[0][kk][0] = live ? __ldg(qp + (kk * 16 + qcol) / 2) : 0u;
+          qf[0][kk][1] = live ? __ldg(qp + (kk * 16 + 8 + qcol) / 2) : 0u;
+        } else {
+          // fp16 fragments in the permuted order of compute_tile_f8: four consecutive elements per lane
+          const uint32_t v0 = live ? __ldg(qp + (kk * 16 + qcol * 2) / 2) : 0u;
+          const uint32_t v1 = live ? __ldg(qp + (kk * 16 + qcol * 2) / 2 + 1) : 0u;
+          qf[0][kk][0] = pack_f16x2(__uint_as_float(v0 << 16), __uint_as_float(v0 & 0xffff0000u));
+          qf[0][kk][1] = pack_f16x2(__uint_as_float(v1 << 16), __uint_as_float(v1 & 0xffff0000u));
+        }
       }
     }
+    // fp8 cache: the K scale of this KV head joins the softmax scale
+    const float sl2 = EB == 1 ? P.scale_log2 * __ldg(P.k_scale + g) : P.scale_log2;
     float acc[1][D / 16][4];
     float m[1][2] = {{NEG_INF, NEG_INF}}, l[1][2] = {{0.f, 0.f}};
 #pragma unroll
@@ -169,7 +183,10 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
       if (has_rows) {
         const uint32_t sK = ring + slot * C::STAGE_BYTES;
-        compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, P.scale_log2, TILE, ctrl->meta[slot], lane, no_lag, [] {}, [] {});
+        if constexpr (EB == 2)
+          compute_tile<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, sl2, TILE, ctrl->meta[slot], lane, no_lag, [] {}, [] {});
+        else
+          compute_tile_f8<D, 1, BS, false>(sK, sK + C::KV_BYTES, qf, acc, m, l, sl2, TILE, ctrl->meta[slot], lane, no_lag);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
@@ -184,6 +201,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         l[0][e] = v;
       }
       const int drow = lane >> 2;
+      const float vs = EB == 1 ? __ldg(P.v_scale + g) : 1.f;   // fp8 cache: the accumulator is linear in V
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const int r = warp * 8 + qcol + e;
@@ -197,8 +215,8 @@ prefix_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           float* a = slotp + 2 * C::HP + h * D;
 #pragma unroll
           for (int jm = 0; jm < D / 16; ++jm) {
-            a[jm * 16 + drow] = acc[0][jm][e];
-            a[jm * 16 + drow + 8] = acc[0][jm][2 + e];
+            a[jm * 16 + drow] = acc[0][jm][e] * vs;
+            a[jm * 16 + drow + 8] = acc[0][jm][2 + e] * vs;
           }
         }
       }

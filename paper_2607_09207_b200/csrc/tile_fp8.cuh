@@ -6,8 +6,10 @@
 namespace pdattn {
 
 // ------------------------------------------------------------------------------------------
-// One 64-token tile on one warp, fp8 cache (e4m3 codes; head_dim 128).
-// K tile: [64 tokens][128 B] (one code per element, 128-byte swizzle); V tile: per page [128 d][BS tokens]
+// One 64-token tile on one warp, fp8 cache (e4m3 codes; head_dim D = 128 or 64).
+// K tile: [64 tokens][D bytes] (one code per element; 128-byte swizzle at D = 128, 64-byte swizzle at D = 64:
+// the 16-byte chunk index is XORed with the row's low three bits, or with bits 1-2 of the row, as the copy
+// engine does it); V tile: per page [D][BS tokens]
 // (V is stored transposed inside a page; with pages of 32 or 64 tokens the 16-byte rows that ldmatrix
 // reads lie 32 or 64 bytes apart and collide two or four ways in the banks).  The codes are widened to fp16 in registers (exact) and both
 // products run as fp16 MMAs; Q arrives as fp16 fragments and P is rounded to fp16 (11 bits, one term).
@@ -20,9 +22,9 @@ namespace pdattn {
 // the score MMA holds token pi(rho) of its 16-token group -- a matter of the row addresses handed to
 // ldmatrix for K.
 // ------------------------------------------------------------------------------------------
-template <int NT, int BS, bool TAIL>
-__device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const uint32_t (&qf)[NT][8][2],
-                                                float (&acc)[NT][8][4], float (&m)[NT][2], float (&l)[NT][2],
+template <int D, int NT, int BS, bool TAIL>
+__device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const uint32_t (&qf)[NT][D / 16][2],
+                                                float (&acc)[NT][D / 16][4], float (&m)[NT][2], float (&l)[NT][2],
                                                 float sl2, int n_left, uint32_t badmask, int lane,
                                                 const int (&lag)[NT][2]) {
   constexpr int GROUPS = TILE / 16;
@@ -44,10 +46,10 @@ __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const 
     for (int nt = 0; nt < NT; ++nt) sc[j][nt][0] = sc[j][nt][1] = sc[j][nt][2] = sc[j][nt][3] = 0.f;
     if (!TAIL || j * 16 < n_valid) {
       const int tok = j * 16 + k_tok;
-      const uint32_t base = sK + tok * 128;
+      const uint32_t base = sK + tok * D;
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int ch = (cc * 2 + k_csel) ^ (tok & 7);
+      for (int cc = 0; cc < D / 32; ++cc) {
+        const int ch = (cc * 2 + k_csel) ^ (D == 128 ? (tok & 7) : ((tok >> 1) & 3));
         uint32_t r[4];
         ldsm_x4(r, base + (ch << 4));
         {
@@ -113,7 +115,7 @@ __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const 
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-      for (int jm = 0; jm < 8; ++jm) {
+      for (int jm = 0; jm < D / 16; ++jm) {
         acc[nt][jm][0] *= alpha[nt][0];
         acc[nt][jm][1] *= alpha[nt][1];
         acc[nt][jm][2] *= alpha[nt][0];
@@ -137,7 +139,7 @@ __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const 
       pb[j][nt][1] = movmatrix_trans(pack_f16x2(p2, p3));
     }
 
-  // ---- O^T += V^T . P^T : [128] x [8*NT heads], 16 tokens of a page per MMA step
+  // ---- O^T += V^T . P^T : [D] x [8*NT heads], 16 tokens of a page per MMA step
 #pragma unroll
   for (int j = 0; j < GROUPS; ++j) {
     if (!TAIL || j * 16 < n_valid) {
@@ -148,9 +150,9 @@ __device__ __forceinline__ void compute_tile_f8(uint32_t sK, uint32_t sV, const 
         keep_mask = keep >= 4 ? 0xffffffffu : (keep <= 0 ? 0u : ((1u << (8 * keep)) - 1u));
       }
 #pragma unroll
-      for (int jp = 0; jp < 4; ++jp) {
+      for (int jp = 0; jp < D / 32; ++jp) {
         uint32_t r[4];
-        ldsm_x4(r, sV + ((j * 16) / BS) * (128 * BS) + (jp * 32 + v_drow) * BS + (j * 16) % BS);
+        ldsm_x4(r, sV + ((j * 16) / BS) * (D * BS) + (jp * 32 + v_drow) * BS + (j * 16) % BS);
         if (TAIL) {
           r[0] &= keep_mask;
           r[1] &= keep_mask;

@@ -28,6 +28,7 @@ DEVICE_TIMEOUT = -8
 
 EXPORTS = [
     "pdattn_workspace_size", "pdattn_workspace_init", "pdattn_decode_ex", "pdattn_bind", "pdattn_decode",
+    "pdattn_decode_host_fp8", "pdattn_decode_grouped_fp8",
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_wait_limit_probe", "pdattn_set_dynamic_spans",
@@ -95,6 +96,9 @@ def lib():
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
         L.pdattn_grouped_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_grouped.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp]
+        L.pdattn_decode_grouped_fp8.argtypes = [ctypes.POINTER(Args), i32, vp, vp, vp, vp, vp]
+        L.pdattn_decode_host_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32,
+                                             vp, sz, vp, sz, vp]
         L.pdattn_multi_workspace_size.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.pdattn_decode_multi.argtypes = [ctypes.POINTER(Args), i32, vp]
         L.pdattn_decode_fp8.argtypes = [ctypes.POINTER(Args), vp, vp, vp]
@@ -310,6 +314,49 @@ def decode_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, ou
         st = lib().pdattn_decode_fp8(ctypes.byref(a), k_scale.data_ptr(), v_scale.data_ptr(), _stream_ptr(stream))
     if check and st != OK:
         raise PdattnError(st, "pdattn_decode_fp8")
+    return st
+
+
+def decode_grouped_fp8(q, k8, v8, k_scale, v_scale, block_table, context_lens, scale, out, workspace,
+                       context_lens_host, group_size, prefix_tiles, prefix_tiles_host, stream=None,
+                       check: bool = True) -> int:
+    """pdattn_decode_grouped_fp8: decode_grouped over the e4m3 code pools of decode_fp8."""
+    S, Hq, d = q.shape
+    NB, Hkv, bs, _ = k8.shape
+    assert k8.dtype == torch.uint8 and v8.dtype == torch.uint8 and tuple(v8.shape) == (NB, Hkv, d, bs)
+    assert k8.is_contiguous() and v8.is_contiguous()
+    a = Args()
+    a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k8.data_ptr(), v8.data_ptr(), out.data_ptr()
+    a.block_table, a.context_lens = block_table.data_ptr(), context_lens.data_ptr()
+    lens = np.ascontiguousarray(context_lens_host, dtype=np.int32)
+    a.context_lens_host = lens.ctypes.data
+    a.num_seqs, a.num_q_heads, a.num_kv_heads, a.head_dim, a.block_size = S, Hq, Hkv, d, bs
+    a.max_blocks_per_seq = block_table.shape[1]
+    a.num_blocks = NB
+    a.kv_block_stride, a.kv_head_stride, a.kv_token_stride = Hkv * bs * d, bs * d, d
+    a.scale = float(scale)
+    a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    pth = np.ascontiguousarray(prefix_tiles_host, dtype=np.int32)
+    st = lib().pdattn_decode_grouped_fp8(ctypes.byref(a), int(group_size), prefix_tiles.data_ptr(), pth.ctypes.data,
+                                         k_scale.data_ptr(), v_scale.data_ptr(), _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_grouped_fp8")
+    return st
+
+
+def decode_host_fp8(q_host, block_table_host, context_lens_host, out_host, k8, v8, k_scale, v_scale, scale, staging,
+                    workspace, stream=None, check: bool = True) -> int:
+    """pdattn_decode_host_fp8: q / block_table / context_lens / out are HOST tensors (pinned), code pools and scales
+    on the device."""
+    S, Hq, d = q_host.shape
+    NB, Hkv, bs, _ = k8.shape
+    st = lib().pdattn_decode_host_fp8(q_host.data_ptr(), block_table_host.data_ptr(), context_lens_host.data_ptr(),
+                                      out_host.data_ptr(), k8.data_ptr(), v8.data_ptr(), k_scale.data_ptr(),
+                                      v_scale.data_ptr(), S, Hq, Hkv, d, bs, block_table_host.shape[1], NB, float(scale),
+                                      staging.data_ptr(), staging.numel(), workspace.data_ptr(), workspace.numel(),
+                                      _stream_ptr(stream))
+    if check and st != OK:
+        raise PdattnError(st, "pdattn_decode_host_fp8")
     return st
 
 

@@ -124,14 +124,104 @@ def test_out_of_range_page_ids_are_masked_and_reported():
 
 
 def test_rejects_what_it_cannot_do():
-    w = W.make_custom([100], Hq=4, Hkv=2, d=64, seed=45, device=DEV)
-    ks, vs = scales(2, 5)
-    k8, v8 = W.fp8_caches(w, ks, vs)
-    ws = pdattn.alloc_workspace(1, 4, 2, 64)
-    out = torch.empty_like(w.q)
-    args = (w.block_table, w.context_lens, w.scale, out, ws)
-    assert pdattn.decode_fp8(w.q, k8, v8, ks, vs, *args, check=False) == pdattn.UNSUPPORTED       # head_dim 64
     assert pdattn.lib().pdattn_decode_fp8(None, None, None, None) == pdattn.INVALID_ARG
+    # a grouped call over the fp8 cache scores the shared tiles with warp-level MMAs: at most 48 query rows a group
+    w = W.make_custom([200] * 8, Hq=28, Hkv=4, d=128, seed=45, device=DEV)
+    ks, vs = scales(4, 5)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    ws = pdattn.alloc_grouped_workspace(8, 28, 4, 128)
+    pt = torch.tensor([1], dtype=torch.int32, device=DEV)
+    st = pdattn.decode_grouped_fp8(w.q, k8, v8, ks, vs, w.block_table, w.context_lens, w.scale, torch.empty_like(w.q),
+                                   ws, w.context_lens_host, 8, pt, [1], check=False)
+    assert st == pdattn.UNSUPPORTED                  # 8 * 7 = 56 rows
+
+
+@pytest.mark.parametrize("host_lens", [True, False])
+@pytest.mark.parametrize("Hq,Hkv,bs", [(4, 1, 16), (16, 2, 16), (32, 2, 32), (12, 4, 64)])
+def test_head_dim_64(Hq, Hkv, bs, host_lens):
+    """K rows of 64 bytes land under the copy engine's 64-byte swizzle; 8- and 16-row tiles; every page size."""
+    lens = [1, 2, 3, 15, 16, 17, 31, 33, 47, 49, 63, 64, 65, 127, 129, 191, 193, 255, 257, 1000, 0, 4097, 577]
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=64, bs=bs, seed=460 + Hq, device=DEV)
+    ks, vs = scales(Hkv, Hq + 1)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    out, st = run_fp8(w, k8, v8, ks, vs, host_lens)
+    assert st == pdattn.OK
+    assert_parity(out, reference(w, k8, v8, ks, vs), f"fp8 d=64 Hq={Hq} Hkv={Hkv} bs={bs}")
+    again, _ = run_fp8(w, k8, v8, ks, vs, host_lens)
+    assert torch.equal(out, again)
+
+
+def test_head_dim_64_append_then_decode():
+    lens = [0, 1, 15, 16, 17, 63, 64, 300]
+    w = W.make_custom(lens, Hq=8, Hkv=2, d=64, seed=47, device=DEV, headroom_tokens=40)
+    ks, vs = scales(2, 6)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    ck8, cv8 = k8.cpu().clone(), v8.cpu().clone()
+    ws = pdattn.alloc_workspace(len(lens), 8, 2, 64)
+    dlens, clens = w.context_lens.clone(), w.context_lens.cpu().clone()
+    for step in range(20):
+        k_new = W.normal_bf16(len(lens) * 2 * 64, 600 + step, 3, device=DEV).view(len(lens), 2, 64)
+        v_new = W.normal_bf16(len(lens) * 2 * 64, 600 + step, 4, device=DEV).view(len(lens), 2, 64)
+        pdattn.append_kv_fp8(k_new, v_new, k8, v8, ks, vs, w.block_table, dlens, ws)
+        assert orc.append_kv_fp8(ck8, cv8, ks.cpu(), vs.cpu(), w.block_table.cpu(), clens, k_new.cpu(), v_new.cpu()) == 0
+    assert pdattn.check(ws) == pdattn.OK
+    assert torch.equal(dlens.cpu(), clens) and torch.equal(k8.cpu(), ck8) and torch.equal(v8.cpu(), cv8)
+    wl = dataclasses.replace(w, context_lens=dlens, context_lens_host=clens.numpy().astype(np.int32))
+    out, st = run_fp8(wl, k8, v8, ks, vs, ws=ws)
+    assert st == pdattn.OK
+    assert_parity(out, orc.decode_fp8(w.q.cpu(), ck8, cv8, ks.cpu(), vs.cpu(), w.block_table.cpu(), clens, w.scale),
+                  "fp8 d=64 decode after appends")
+
+
+@pytest.mark.parametrize("Hq,Hkv,group,d,bs", [(40, 8, 8, 128, 16), (28, 4, 4, 128, 16), (8, 2, 8, 64, 16), (16, 4, 6, 128, 32)])
+def test_grouped_over_the_fp8_cache(Hq, Hkv, group, d, bs):
+    """GRPO groups on an fp8 cache: groups that share 0, 1, 5 and 16 tiles; the shared tiles are read once per
+    group (warp-MMA prefix kernel on the widened codes) and merged with every member's own tiles."""
+    rng = np.random.default_rng(Hq * 10 + group)
+    shared_tokens = [0, 70, 330, 1024]
+    lens, tiles = [], []
+    for stok in shared_tokens:
+        tiles.append(stok // 64)
+        for j in range(group):
+            lens.append(stok + (1 if j == 0 else int(rng.integers(1, 700))))
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, bs=bs, seed=70 + group, device=DEV, poison=False)
+    bt = w.block_table.clone()
+    for gi, stok in enumerate(shared_tokens):
+        pages = stok // bs
+        for j in range(1, group):
+            bt[gi * group + j, :pages] = bt[gi * group, :pages]
+    w = dataclasses.replace(w, block_table=bt)
+    W.poison_unused(w)
+    ks, vs = scales(Hkv, group)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    ws = pdattn.alloc_grouped_workspace(w.num_seqs, Hq, Hkv, d, bs)
+    pt = torch.tensor(tiles, dtype=torch.int32, device=DEV)
+    out = torch.full_like(w.q, float("nan"))
+    pdattn.decode_grouped_fp8(w.q, k8, v8, ks, vs, w.block_table, w.context_lens, w.scale, out, ws,
+                              w.context_lens_host, group, pt, tiles)
+    assert pdattn.check(ws) == pdattn.OK
+    assert_parity(out, reference(w, k8, v8, ks, vs), f"fp8 grouped Hq={Hq} Hkv={Hkv} group={group} d={d} bs={bs}")
+    again = torch.full_like(w.q, float("nan"))
+    pdattn.decode_grouped_fp8(w.q, k8, v8, ks, vs, w.block_table, w.context_lens, w.scale, again, ws,
+                              w.context_lens_host, group, pt, tiles)
+    assert pdattn.check(ws) == pdattn.OK and torch.equal(out, again)
+
+
+def test_host_buffer_form_over_the_fp8_cache():
+    """pdattn_decode_host_fp8: the step's q / block_table / context_lens in pinned host memory, out read back."""
+    w = W.make_config(2, device=DEV, num_seqs=12, len_div=4)
+    ks, vs = scales(4, 9)
+    k8, v8 = W.fp8_caches(w, ks, vs)
+    ref, st = run_fp8(w, k8, v8, ks, vs)
+    assert st == pdattn.OK
+    ws = pdattn.alloc_workspace(w.num_seqs, 28, 4, 128)
+    qh, bth, lh = w.q.cpu().pin_memory(), w.block_table.cpu().pin_memory(), w.context_lens.cpu().pin_memory()
+    oh = torch.full_like(qh, float("nan")).pin_memory()
+    staging = torch.empty(pdattn.host_staging_size(w.num_seqs, 28, 128, w.max_blocks_per_seq), dtype=torch.uint8, device=DEV)
+    pdattn.decode_host_fp8(qh, bth, lh, oh, k8, v8, ks, vs, w.scale, staging, ws)
+    torch.cuda.synchronize()
+    assert pdattn.check(ws) == pdattn.OK and torch.equal(ref.cpu(), oh)
+    assert_parity(oh, reference(w, k8, v8, ks, vs), "fp8 host-buffer form")
 
 
 @pytest.mark.parametrize("bs", [16, 32])

@@ -55,7 +55,6 @@ def test_random_mix_of_everything(seed):
                     st = pdattn.check(ws); msg = parity(out, orc.decode_workload(wc))
                 elif variant in ("multi", "fp8multi"):
                     T = int(rng.integers(1, max(2, 16 // G + 1)))
-                    if variant == "fp8multi" and d != 128: continue
                     q = W.normal_bf16(S * T * Hq * d, 5, 7, device=DEV).view(S, T, Hq, d)
                     ws = pdattn.alloc_multi_workspace(S, Hq, Hkv, d, bs, T)
                     out = torch.full_like(q, float("nan"))
@@ -69,7 +68,6 @@ def test_random_mix_of_everything(seed):
                         ref = orc.decode_fp8_multi(q.cpu(), k8.cpu(), v8.cpu(), ks.cpu(), vs.cpu(), wc.block_table, wc.context_lens, wc.scale)
                     st = pdattn.check(ws); msg = parity(out, ref); desc += f" T={T}"
                 elif variant == "fp8":
-                    if d != 128: continue
                     ks = torch.tensor(rng.uniform(0.5, 2, Hkv), dtype=torch.float32, device=DEV); vs = torch.tensor(rng.uniform(0.5, 2, Hkv), dtype=torch.float32, device=DEV)
                     k8, v8 = W.fp8_caches(w, ks, vs)
                     ws = pdattn.alloc_workspace(S, Hq, Hkv, d, bs); out = torch.full_like(w.q, float("nan"))
@@ -88,10 +86,19 @@ def test_random_mix_of_everything(seed):
                         for j in range(1, gs): bt[i * gs + j, :pg] = bt[i * gs, :pg]
                     w = dataclasses.replace(w, block_table=bt); W.poison_unused(w)
                     eng = int(rng.choice([0, 1])) if gs * G <= 48 else 1
+                    f8 = bool(rng.integers(2)) and gs * G <= 48     # the same groups over an e4m3 copy of the pools
                     pdattn.set_prefix_engine(eng)
                     ws = pdattn.alloc_grouped_workspace(S, Hq, Hkv, d, bs); out = torch.full_like(w.q, float("nan"))
-                    pdattn.decode_grouped(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws, w.context_lens_host, gs, torch.tensor(pt, dtype=torch.int32, device=DEV), pt.astype(np.int32))
-                    st = pdattn.check(ws); msg = parity(out, orc.decode_workload(w.to("cpu"))); desc += f" gs={gs} pt={pt.tolist()} eng={eng}"
+                    ptd = torch.tensor(pt, dtype=torch.int32, device=DEV)
+                    if f8:
+                        ks = torch.tensor(rng.uniform(0.5, 2, Hkv), dtype=torch.float32, device=DEV); vs = torch.tensor(rng.uniform(0.5, 2, Hkv), dtype=torch.float32, device=DEV)
+                        k8, v8 = W.fp8_caches(w, ks, vs)
+                        pdattn.decode_grouped_fp8(w.q, k8, v8, ks, vs, w.block_table, w.context_lens, w.scale, out, ws, w.context_lens_host, gs, ptd, pt.astype(np.int32))
+                        ref = orc.decode_fp8(w.q.cpu(), k8.cpu(), v8.cpu(), ks.cpu(), vs.cpu(), w.block_table.cpu(), w.context_lens.cpu(), w.scale)
+                    else:
+                        pdattn.decode_grouped(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws, w.context_lens_host, gs, ptd, pt.astype(np.int32))
+                        ref = orc.decode_workload(w.to("cpu"))
+                    st = pdattn.check(ws); msg = parity(out, ref); desc += f" gs={gs} pt={pt.tolist()} eng={eng} fp8={f8}"
                     pdattn.set_prefix_engine(-1)
                 n += 1
                 if st != pdattn.OK or msg:
