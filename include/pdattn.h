@@ -339,8 +339,10 @@ pdattn_status pdattn_set_prefix_engine(int engine);
 /*
  * Error report of the decode steps enqueued so far (no paper counterpart; the rollout loop of Section 2.3
  * would call it once per step or less).  Synchronises `stream`, reads and clears the workspace's sticky
- * error word (hence a non-const pointer).  Returns PDATTN_OK, PDATTN_BAD_PAGE_INDEX or
- * PDATTN_DEVICE_TIMEOUT.  workspace: DEVICE.
+ * error word (hence a non-const pointer).  Returns PDATTN_OK, PDATTN_BAD_PAGE_INDEX, PDATTN_DEVICE_TIMEOUT, or
+ * PDATTN_UNSUPPORTED when the device-side planner refused a batch of more than 2^30 tiles (with
+ * context_lens_host the call itself returns PDATTN_INVALID_ARG for such a batch); that call computed nothing.
+ * workspace: DEVICE.
  */
 pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream);
 

@@ -321,11 +321,37 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
   // launched as a programmatic dependent of whatever precedes it on the stream (the KV append in a decode
   // loop): nothing may be read or written before that kernel has completed and flushed
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  __shared__ unsigned long long wide_cost;
   if (tid == 0) {
     carry_c = carry_t = 0;
     pcost[0] = ptile[0] = 0;
+    wide_cost = 0ull;
   }
   __syncthreads();
+  // The running sums below are 32-bit, like the host planner's tables; the host refuses a batch whose tile count
+  // does not fit, and so does this kernel: total cost first, in 64 bits.
+  {
+    unsigned long long mine = 0ull;
+    for (int s = tid; s < S; s += 1024)
+      mine += static_cast<unsigned long long>(seq_cost(seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0), Hkv));
+    if (mine) atomicAdd(&wide_cost, mine);
+  }
+  __syncthreads();
+  if (wide_cost > static_cast<unsigned long long>(INT32_MAX / 2)) {
+    // too large: an empty plan (nothing is computed) and an error bit for pdattn_check
+    const PlanParams none = make_plan_params(0, 0, n_static, 0);
+    if (tid == 0) {
+      hdr->plan = none;
+      atomicOr(&hdr->err, ERR_TOO_LARGE);
+    }
+    for (int c = tid; c <= n_static; c += 1024) {
+      SpanStart sp;
+      sp.unit = S * Hkv;
+      sp.tile = sp.flat = sp.merge = 0;
+      spans[c] = sp;
+    }
+    return;
+  }
   for (int base = 0; base < S; base += 1024) {
     const int s = base + tid;
     int nt = 0;

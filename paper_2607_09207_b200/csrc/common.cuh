@@ -33,7 +33,7 @@ constexpr int MAX_STAGES = 14;
 constexpr int MERGE_QUEUE = 8;                  // entries of the in-CTA queue of merge jobs
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2 };
+enum : int { ERR_BAD_PAGE = 1, ERR_TIMEOUT = 2, ERR_TOO_LARGE = 4 };
 
 // Workspace header (first 256 bytes of the workspace)
 struct WsHeader {

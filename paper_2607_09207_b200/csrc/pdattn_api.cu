@@ -809,6 +809,7 @@ pdattn_status pdattn_check(void* workspace, pdattn_stream_t stream_) {
   e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
   if (word & ERR_TIMEOUT) return PDATTN_DEVICE_TIMEOUT;
+  if (word & ERR_TOO_LARGE) return PDATTN_UNSUPPORTED;   // the device-side planner refused the batch (tile count)
   return PDATTN_BAD_PAGE_INDEX;
 }
 

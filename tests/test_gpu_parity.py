@@ -382,6 +382,27 @@ def test_a_context_longer_than_its_table_row_is_masked_and_reported_without_read
     assert st == pdattn.INVALID_ARG
 
 
+def test_device_planner_refuses_a_batch_whose_tile_count_overflows():
+    """Without a host copy of the lengths the planning kernel sums tile counts itself; a batch beyond 2^30 tiles gets
+    an empty plan (nothing is read or computed) and pdattn_check says so.  With the host copy the call is refused."""
+    S = 64
+    w = W.make_custom([16] * S, Hq=8, Hkv=8, d=128, seed=22, device=DEV, num_blocks=64, poison=False)
+    huge = torch.full((S,), 1 << 30, dtype=torch.int32, device=DEV)
+    ws = pdattn.alloc_workspace(S, 8, 8, 128)
+    out = torch.full_like(w.q, 7.0)
+    st = pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, huge, w.scale, out, ws, context_lens_host=None,
+                          check=False)
+    assert st == pdattn.OK
+    assert pdattn.check(ws) == pdattn.UNSUPPORTED
+    assert torch.all(out == 7.0)                       # nothing was written
+    st = pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, huge, w.scale, out, ws,
+                          context_lens_host=np.full(S, 1 << 30, dtype=np.int32), check=False)
+    assert st == pdattn.INVALID_ARG
+    out2, st = run(w, use_host_lens=False, ws=ws)      # the workspace is usable afterwards
+    assert st == pdattn.OK
+    assert_parity(out2, orc.decode_workload(w.to("cpu")), "after a refused batch")
+
+
 def test_token_major_cache_layout_through_strides():
     """[page, slot, head, dim] pools passed through the stride arguments give the same bits."""
     w = W.make_custom([333, 64, 1500], Hq=28, Hkv=4, d=128, seed=19, device=DEV)
