@@ -311,7 +311,8 @@ __device__ __forceinline__ int block_scan_1024(int v, int* warp_sums, int lane, 
 
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict__ start_tiles, int S, int Hkv,
-            int n_static, int n_dyn_max, int32_t* __restrict__ prefix, SpanStart* __restrict__ spans, WsHeader* hdr) {
+            int n_static, int n_dyn_max, int32_t* __restrict__ prefix, SpanStart* __restrict__ spans, WsHeader* hdr,
+            int with_merge_words) {
   __shared__ int warp_sums[32];
   __shared__ int carry_c, carry_t;
   __shared__ PlanParams pp_s;
@@ -328,14 +329,30 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
     wide_cost = 0ull;
   }
   __syncthreads();
-  // The running sums below are 32-bit, like the host planner's tables; the host refuses a batch whose tile count
-  // does not fit, and so does this kernel: total cost first, in 64 bits.
-  {
-    unsigned long long mine = 0ull;
-    for (int s = tid; s < S; s += 1024)
-      mine += static_cast<unsigned long long>(seq_cost(seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0), Hkv));
-    if (mine) atomicAdd(&wide_cost, mine);
+  unsigned long long mine64 = 0ull;   // this thread's share of the total cost, in 64 bits (see the end of the kernel)
+  for (int base = 0; base < S; base += 1024) {
+    const int s = base + tid;
+    int nt = 0;
+    if (s < S) nt = static_cast<int>(seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0));
+    mine64 += static_cast<unsigned long long>(seq_cost(nt, Hkv));
+    const int ic = block_scan_1024(static_cast<int>(seq_cost(nt, Hkv)), warp_sums, lane, wid) + carry_c;
+    const int itl = block_scan_1024(nt * Hkv, warp_sums, lane, wid) + carry_t;
+    if (s < S) {
+      pcost[s + 1] = ic;
+      ptile[s + 1] = itl;
+    }
+    __syncthreads();
+    if (tid == 1023) {
+      carry_c = ic;
+      carry_t = itl;
+    }
+    __syncthreads();
   }
+  // The running sums above are 32-bit, like the host planner's tables; the host refuses a batch whose tile count
+  // does not fit, and so does this kernel: the true total, in 64 bits, decides.
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mine64 += __shfl_xor_sync(0xffffffffu, mine64, o);
+  if (lane == 0 && mine64) atomicAdd(&wide_cost, mine64);
   __syncthreads();
   if (wide_cost > static_cast<unsigned long long>(INT32_MAX / 2)) {
     // too large: an empty plan (nothing is computed) and an error bit for pdattn_check
@@ -351,23 +368,6 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
       spans[c] = sp;
     }
     return;
-  }
-  for (int base = 0; base < S; base += 1024) {
-    const int s = base + tid;
-    int nt = 0;
-    if (s < S) nt = static_cast<int>(seq_tiles(context_lens[s], start_tiles ? start_tiles[s] : 0));
-    const int ic = block_scan_1024(static_cast<int>(seq_cost(nt, Hkv)), warp_sums, lane, wid) + carry_c;
-    const int itl = block_scan_1024(nt * Hkv, warp_sums, lane, wid) + carry_t;
-    if (s < S) {
-      pcost[s + 1] = ic;
-      ptile[s + 1] = itl;
-    }
-    __syncthreads();
-    if (tid == 1023) {
-      carry_c = ic;
-      carry_t = itl;
-    }
-    __syncthreads();
   }
   if (tid == 0) {
     pp_s = make_plan_params(carry_c, carry_t, n_static, n_dyn_max);
@@ -400,7 +400,9 @@ plan_kernel(const int32_t* __restrict__ context_lens, const int32_t* __restrict_
     }
     spans[c] = sp;
   }
-  // how the cut units are put together again: one word per span, from the finished table
+  // how the cut units are put together again: one word per span, from the finished table (only when the decode
+  // kernel that follows merges cut units itself: the scan is a chain of dependent loads per span)
+  if (!with_merge_words) return;
   __syncthreads();
   for (int c = tid; c < n_spans; c += 1024) spans[c].merge = span_merge_info(spans, n_spans, c);
 }

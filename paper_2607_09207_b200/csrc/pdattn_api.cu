@@ -1009,7 +1009,7 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
     cudaError_t e = launch_dependent(plan_kernel, 1, 1024, 0, stream, true, a->context_lens,
                                      static_cast<const int32_t*>(nullptr), a->num_seqs, a->num_kv_heads, n_ctas, n_dyn_max,
                                      reinterpret_cast<int32_t*>(ws + wl.prefix),
-                                     reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr);
+                                     reinterpret_cast<SpanStart*>(ws + wl.spans), P.hdr, P.inkernel_max > 0 ? 1 : 0);
     if (e != cudaSuccess) return cuda_fail("plan_kernel launch", e);
     g_last_launches += 1;
     combine_grid = n_ctas + n_dyn_max;
