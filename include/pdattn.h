@@ -21,8 +21,8 @@
  *     memory, creates no streams, and synchronises only where stated.
  *   - Work is enqueued on `stream`; outputs are valid once the stream reaches that point.
  *   - State.  Per thread: the binding made by pdattn_bind(), the events of pdattn_profile_events(), the
- *     launch count and the text of the last CUDA failure.  Process-wide: the four tuning settings
- *     pdattn_set_dynamic_spans / _merge_mode / _prefix_engine / _host_zero_copy (plain ints; set them
+ *     launch count and the text of the last CUDA failure.  Process-wide: the five tuning settings
+ *     pdattn_set_dynamic_spans / _merge_mode / _short_piece_path / _prefix_engine / _host_zero_copy (plain ints; set them
  *     before the threads that decode start, not concurrently with a call).
  */
 #ifndef PDATTN_H_
@@ -326,6 +326,17 @@ pdattn_status pdattn_set_dynamic_spans(int per_cta);
  * results are bit-identical from run to run and under any renumbering of the physical pages.
  */
 pdattn_status pdattn_set_merge_mode(int mode);
+
+/*
+ * Process-wide choice of the decode kernel's instantiation for batches of very short contexts (early in a rollout
+ * most sequences are a tile or two long: Section 2.3's length skew seen from its short end; no paper counterpart).
+ * In the short-piece instantiation every warp walks the work spans 32 sequences x KV heads at a time (one load of
+ * the lengths, one warp scan, one ballot) instead of piece by piece, and a warp of its own stages the query rows.
+ * It applies to the chained merge over a bf16 cache with at most 8 query rows per KV head and context_lens_host
+ * given; cut sequences are merged by the combine kernel.  -1 (default): used below 1.5 tiles (96 tokens) per
+ * sequence and KV head on average; 0: never; 1: whenever it applies.  Results are the same bits either way.
+ */
+pdattn_status pdattn_set_short_piece_path(int mode);
 
 /*
  * Process-wide choice of the kernel that pdattn_decode_grouped runs over the shared prompt tiles.

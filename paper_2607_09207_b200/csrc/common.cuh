@@ -350,6 +350,69 @@ struct Walker {
 };
 
 // ------------------------------------------------------------------------------------------
+// The same walk, 32 units at a time, for the short-piece instantiation of the chained-merge kernel.  A consumer warp works on
+// the pieces it holds a tile of and has to step over all the others; with the one-piece-at-a-time Walker that step
+// (a dependent load, tile arithmetic, bookkeeping) cost ≈ 700 cycles, and in a batch of one-tile pieces a warp
+// steps over five pieces for every one it works on.  Here lane i looks at unit base + i: one lane-wide load of
+// the lengths (fetched a window ahead), one warp scan of the tile counts, and a ballot tell the warp which of the
+// 32 pieces are its own; only for those are the fields broadcast.
+// ------------------------------------------------------------------------------------------
+struct PieceWindow {
+  // per lane (unit base + lane)
+  int unit, s, L, t0, full;   // full: tiles of the unit that this call covers
+  int tb, take;               // this span's piece of the unit: tiles [tb, tb + take) (take == 0: none)
+  int it0;                    // CTA tile counter at the piece's first tile
+  // uniform
+  int total;                  // tiles of the whole window
+};
+struct WindowWalker {
+  const int32_t* ctx;
+  const int32_t* start_tiles;   // per sequence, may be null (= 0)
+  int Hkv, nunits, lane;
+  int base = 0, rem = 0, first = 0, tb0 = 0;
+  int nL = 0, nT = 0, nS = 0;   // the window at `base`, fetched ahead
+  __device__ __forceinline__ void fetch(int b) {
+    const int u = b + lane;
+    nS = u < nunits ? u / Hkv : 0;
+    nL = u < nunits ? __ldg(ctx + nS) : 0;
+    nT = (start_tiles && u < nunits) ? __ldg(start_tiles + nS) : 0;
+  }
+  __device__ __forceinline__ void begin_span(int unit, int tile, int count) {
+    first = base = unit;
+    tb0 = tile;
+    rem = count;
+    if (rem > 0) fetch(base);
+  }
+  // it: the CTA's tile counter before this window
+  __device__ __forceinline__ bool next(PieceWindow& w, int it) {
+    if (rem <= 0 || base >= nunits) return false;
+    w.unit = base + lane;
+    w.s = nS;
+    w.L = nL;
+    w.t0 = nT;
+    const int all = w.L > 0 ? (w.L + TILE - 1) / TILE : 0;
+    w.full = (w.unit < nunits && all > w.t0) ? all - w.t0 : 0;
+    w.tb = w.unit == first ? tb0 : 0;
+    const int avail = w.full > w.tb ? w.full - w.tb : 0;
+    int incl = avail;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    const int excl = incl - avail;
+    w.take = excl >= rem ? 0 : (rem - excl < avail ? rem - excl : avail);
+    w.it0 = it + excl;
+    const int sum = __shfl_sync(0xffffffffu, incl, 31);
+    w.total = sum < rem ? sum : rem;
+    rem -= w.total;
+    base += 32;
+    if (rem > 0 && base < nunits) fetch(base);   // used a whole window of work later
+    return true;
+  }
+};
+
+// ------------------------------------------------------------------------------------------
 // Span sequencing inside a CTA.  Every warp walks the same sequence of spans: first the CTA's
 // static span, then run-time spans.  Lane 0 of producer warp 0 draws run-time spans from the
 // global counter (one atomic per span, issued a whole span ahead of its use) and publishes the

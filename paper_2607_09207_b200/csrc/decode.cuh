@@ -195,6 +195,61 @@ __device__ __forceinline__ void merge_warp_loop(const DecodeParams& P, Ctrl* ctr
   }
 }
 
+// The tenth warp of the short-piece instantiation (WIN; it never merges cut units itself): it stages the query rows of
+// every piece, which is producer warp 0's job elsewhere.  In such batches a piece is a tile or two, the
+// consumer warps step over pieces in a few hundred cycles (WindowWalker), and the producer that walked the spans piece
+// by piece, staged every piece's rows and issued its third of the tiles set the pace of the CTA.  Walks the same
+// spans in the same order as everybody else, 32 units at a time.
+template <int D, int NT, int BS, int EB>
+__device__ __forceinline__ void stage_queries_loop(const DecodeParams& P, Ctrl* ctrl, uint32_t qbuf, int lane) {
+  using C = Cfg<D, NT, BS, EB>;
+  const int nunits = P.S * P.Hkv;
+  int it = 0, pcnt = 0;
+  bool aborted = false;
+  int span = blockIdx.x;
+  for (int k = 0; span >= 0 && !aborted; ++k) {
+    const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
+    const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
+    WindowWalker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, lane};
+    walk.begin_span(sp.unit, sp.tile, sp_end - sp.flat);
+    PieceWindow W;
+    while (!aborted && walk.next(W, it)) {
+      it += W.total;
+      uint32_t m = __ballot_sync(0xffffffffu, W.take > 0);
+      while (m) {
+        const int wl = __ffs(m) - 1;
+        m &= m - 1;
+        const int unit = __shfl_sync(0xffffffffu, W.unit, wl);
+        const int s = __shfl_sync(0xffffffffu, W.s, wl);
+        const int g = unit - s * P.Hkv;
+        const int qs = pcnt % C::QSLOTS;
+        const uint32_t qphase = (pcnt / C::QSLOTS) & 1;
+        if (!mbar_wait(smem_u32(&ctrl->q_empty[qs]), qphase ^ 1u)) {
+          aborted = true;
+          break;
+        }
+        if (lane == 0) {
+          // the G rows of each of the T query tokens, packed: row = query token * G + head
+          const uint32_t bytes = static_cast<uint32_t>(P.G) * D * 2;
+          const uint32_t qb = smem_u32(&ctrl->q_full[qs]);
+          ctrl->qseq[qs] = pcnt;
+          mbar_arrive_expect_tx(qb, bytes * P.T);
+          for (int qt = 0; qt < P.T; ++qt)
+            bulk_load(qbuf + qs * C::Q_BYTES + qt * bytes,
+                      P.q + ((static_cast<int64_t>(s) * P.T + qt) * P.Hq + g * P.G) * D, bytes, qb);
+        }
+        ++pcnt;
+      }
+    }
+    if (aborted) break;
+    span = read_span(ctrl, k + 1, aborted);
+  }
+  if (aborted && lane == 0) {
+    atomicOr(&P.hdr->err, ERR_TIMEOUT);
+    atomicExch(&ctrl->abort, 1u);
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // Consumer side of decode_kernel<.., CHAIN = true>: the variant for batches of many short pieces.
 //
@@ -209,7 +264,7 @@ __device__ __forceinline__ void merge_warp_loop(const DecodeParams& P, Ctrl* ctr
 // which class of which of those pieces may touch it next.  Warps that hold no tile of a piece skip it
 // (they do not even read its query rows), so up to NCW short pieces are in work at once.
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS, int EB>
+template <int D, int NT, int BS, int EB, bool WIN>
 __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanParams& pp, Ctrl* ctrl, uint32_t ring,
                                               uint32_t qbuf, uint8_t* handoff, int warp, int lane) {
   using C = Cfg<D, NT, BS, EB>;
@@ -246,36 +301,17 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
   for (int k = 0; span >= 0; ++k) {
     const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
     const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
-    Walker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
-    Piece pc;
     int first_unit = -1, first_tb = 0, own_unit = -1, own_slot = 0, piece_idx = 0;
 
-    while (walk.next(pc)) {
+    // ---- one piece that this warp holds a tile of (class `pos` of its n_cls classes)
+    auto piece_body = [&](const Piece& pc, const int it0, const int p, const int mq, const int slot_idx, const int pos) {
       const int n_piece = pc.te - pc.tb;
-      const int it0 = it;
-      it += n_piece;
-      const int p = pcnt++;
       const int n_cls = n_piece < NCW ? n_piece : NCW;
       const bool multi = n_cls > 1;
-      const int mq = mcnt;            // number of this piece among those with more than one class
-      if (multi) ++mcnt;
       const bool complete = (pc.tb == 0 && pc.te == pc.nt);
-      const int slot_idx = piece_idx == 0 ? 0 : 1;
-      if (piece_idx == 0) {
-        first_unit = pc.unit;
-        first_tb = pc.tb;
-      }
-      if (!complete && pc.tb == 0) {
-        own_unit = pc.unit;
-        own_slot = slot_idx;
-      }
-      ++piece_idx;
-      int pos = warp - it0 % NCW;     // this warp's class in the piece
-      if (pos < 0) pos += NCW;
-      if (pos >= n_cls || aborted) continue;
       if (*reinterpret_cast<volatile uint32_t*>(&ctrl->abort)) {
         aborted = true;
-        continue;
+        return;
       }
 
       // ---- packed query rows of this KV head as MMA B fragments, from the staged copy
@@ -284,7 +320,7 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         const int qs = p % C::QSLOTS;
         if (!wait_q<C::QSLOTS>(ctrl, qs, p)) {
           fail();
-          continue;
+          return;
         }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
@@ -374,7 +410,7 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[slot]));
       }
-      if (aborted) continue;
+      if (aborted) return;
       if constexpr (EB == 1) {
         // the V scale of this KV head, once per piece: the accumulator is linear in V
         const float vs = __ldg(P.v_scale + pc.g);
@@ -405,7 +441,7 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
         float4* row4 = reinterpret_cast<float4*>(handoff + e * C::HANDOFF_BYTES) + lane;   // row r: row4[r * 32]
         if (!wait_turn(ctrl, e, mq * 8 + pos)) {
           fail();
-          continue;
+          return;
         }
         if (pos > 0) {
 #pragma unroll
@@ -440,7 +476,7 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
           }
           __syncwarp();
           if (lane == 0) st_release_shared(&ctrl->turn[e], mq * 8 + pos + 1);
-          continue;
+          return;
         }
         __syncwarp();   // the last class has read the slot: it now serves merge number mq + E
         if (lane == 0) st_release_shared(&ctrl->turn[e], (mq + E) * 8);
@@ -548,6 +584,86 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
           }
         }
       }
+    };
+
+    if constexpr (WIN) {
+      // ---- 32 units at a time: which pieces exist, which are this warp's (see WindowWalker)
+      WindowWalker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, lane};
+      walk.begin_span(sp.unit, sp.tile, sp_end - sp.flat);
+      PieceWindow W;
+      while (walk.next(W, it)) {
+        const bool has = W.take > 0;
+        const int w_ncls = W.take < NCW ? W.take : NCW;
+        int w_pos = warp - W.it0 % NCW;
+        if (w_pos < 0) w_pos += NCW;
+        const uint32_t m_has = __ballot_sync(0xffffffffu, has);
+        const uint32_t m_multi = __ballot_sync(0xffffffffu, has && w_ncls > 1);
+        uint32_t m_mine = __ballot_sync(0xffffffffu, has && w_pos < w_ncls);
+        // the span's record: its first piece, and the unit that starts here and runs past the span's end
+        if (piece_idx == 0 && m_has) {
+          const int fl = __ffs(m_has) - 1;
+          first_unit = __shfl_sync(0xffffffffu, W.unit, fl);
+          first_tb = __shfl_sync(0xffffffffu, W.tb, fl);
+        }
+        const uint32_t m_own = __ballot_sync(0xffffffffu, has && W.tb == 0 && W.take < W.full);
+        if (m_own) {
+          const int ol = __ffs(m_own) - 1;
+          own_unit = __shfl_sync(0xffffffffu, W.unit, ol);
+          own_slot = (piece_idx + __popc(m_has & ((1u << ol) - 1u))) == 0 ? 0 : 1;
+        }
+        const int p_w = pcnt, mq_w = mcnt, pi_w = piece_idx;
+        it += W.total;
+        pcnt += __popc(m_has);
+        mcnt += __popc(m_multi);
+        piece_idx += __popc(m_has);
+        while (m_mine) {
+          const int wl = __ffs(m_mine) - 1;
+          m_mine &= m_mine - 1;
+          if (aborted) continue;
+          const uint32_t below = (1u << wl) - 1u;
+          Piece pc;
+          pc.unit = __shfl_sync(0xffffffffu, W.unit, wl);
+          pc.s = __shfl_sync(0xffffffffu, W.s, wl);
+          pc.g = pc.unit - pc.s * P.Hkv;
+          pc.L = __shfl_sync(0xffffffffu, W.L, wl);
+          pc.t0 = __shfl_sync(0xffffffffu, W.t0, wl);
+          pc.nt = __shfl_sync(0xffffffffu, W.full, wl);
+          pc.tb = __shfl_sync(0xffffffffu, W.tb, wl);
+          pc.te = pc.tb + __shfl_sync(0xffffffffu, W.take, wl);
+          const int it0 = __shfl_sync(0xffffffffu, W.it0, wl);
+          int pos = warp - it0 % NCW;     // this warp's class in the piece
+          if (pos < 0) pos += NCW;
+          piece_body(pc, it0, p_w + __popc(m_has & below), mq_w + __popc(m_multi & below),
+                     (pi_w + __popc(m_has & below)) == 0 ? 0 : 1, pos);
+        }
+      }
+    } else {
+      Walker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
+      Piece pc;
+      while (walk.next(pc)) {
+        const int n_piece = pc.te - pc.tb;
+        const int it0 = it;
+        it += n_piece;
+        const int p = pcnt++;
+        const int n_cls = n_piece < NCW ? n_piece : NCW;
+        const int mq = mcnt;            // number of this piece among those with more than one class
+        if (n_cls > 1) ++mcnt;
+        const bool complete = (pc.tb == 0 && pc.te == pc.nt);
+        const int slot_idx = piece_idx == 0 ? 0 : 1;
+        if (piece_idx == 0) {
+          first_unit = pc.unit;
+          first_tb = pc.tb;
+        }
+        if (!complete && pc.tb == 0) {
+          own_unit = pc.unit;
+          own_slot = slot_idx;
+        }
+        ++piece_idx;
+        int pos = warp - it0 % NCW;     // this warp's class in the piece
+        if (pos < 0) pos += NCW;
+        if (pos >= n_cls || aborted) continue;
+        piece_body(pc, it0, p, mq, slot_idx, pos);
+      }
     }
     if (warp == 0 && lane == 0) P.rec[span] = make_int4(first_unit, first_tb, own_unit, own_slot);
     span = read_span(ctrl, k + 1, aborted);
@@ -566,7 +682,9 @@ __device__ __forceinline__ void consume_chain(const DecodeParams& P, const PlanP
 // CHAIN = true replaces the consumers' barrier-and-merge at the end of each piece by the chained
 // hand-off of consume_chain (the producers are the same).
 // ------------------------------------------------------------------------------------------
-template <int D, int NT, int BS, bool PROBE = false, bool CHAIN = false, int EB = 2>
+// WIN: the instantiation for batches of mostly one-tile pieces (chained merge, 8-row tiles, no in-kernel merge):
+// every warp walks the spans 32 units at a time (WindowWalker) and the tenth warp stages the query rows.
+template <int D, int NT, int BS, bool PROBE = false, bool CHAIN = false, int EB = 2, bool WIN = false>
 __global__ void __launch_bounds__(Cfg<D, NT, BS, EB>::NTHREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
               const __grid_constant__ DecodeParams P) {
@@ -627,7 +745,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   if (C::MERGE_WARP && warp == NCW + C::NPW) {
     // ================= merge warp =================
     if constexpr (CHAIN && !PROBE && NT == 1) {
-      if (P.inkernel_max > 0) merge_warp_loop<D, NT>(P, ctrl, NCW, lane);
+      if constexpr (WIN) stage_queries_loop<D, NT, BS, EB>(P, ctrl, qbuf, lane);
+      else if (P.inkernel_max > 0) merge_warp_loop<D, NT>(P, ctrl, NCW, lane);
     }
     return;
   }
@@ -647,29 +766,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
       const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
       const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
-      Walker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
-      Piece pc;
-      while (!aborted && walk.next(pc)) {
-        if (!PROBE && pw == 0) {
-          // stage this piece's packed query rows; the consumers reach the piece several tiles later
-          const int qs = pcnt % C::QSLOTS;
-          const uint32_t qphase = (pcnt / C::QSLOTS) & 1;
-          if (!mbar_wait(smem_u32(&ctrl->q_empty[qs]), qphase ^ 1u)) {
-            aborted = true;
-            break;
-          }
-          if (lane == 0) {
-            // the G rows of each of the T query tokens, packed: row = query token * G + head
-            const uint32_t bytes = static_cast<uint32_t>(P.G) * D * 2;
-            const uint32_t qb = smem_u32(&ctrl->q_full[qs]);
-            if (CHAIN) ctrl->qseq[qs] = pcnt;
-            mbar_arrive_expect_tx(qb, bytes * P.T);
-            for (int qt = 0; qt < P.T; ++qt)
-              bulk_load(qbuf + qs * C::Q_BYTES + qt * bytes,
-                        P.q + ((static_cast<int64_t>(pc.s) * P.T + qt) * P.Hq + pc.g * P.G) * D, bytes, qb);
-          }
-        }
-        ++pcnt;
+      // ---- the tiles of one piece that this warp issues (`it`: the CTA's tile counter at the piece's first tile)
+      auto issue_piece = [&](const Piece& pc) -> bool {
         const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
         const int npages = (pc.L + BS - 1) / BS;
         const int pbase = (pc.t0 + pc.tb) * C::PAGES;
@@ -706,13 +804,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                   break;
                 }
               }
-              if (aborted) break;
+              if (aborted) return false;
             }
           }
-          if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) {
-            aborted = true;
-            break;
-          }
+          if (!mbar_wait(smem_u32(&ctrl->empty[slot]), phase ^ 1u)) return false;
           const int np = min(C::PAGES, npages - (pc.t0 + t) * C::PAGES);
           const int j = lane % C::PAGES;
           int id = __shfl_sync(0xffffffffu, ids_cur, kb * C::PAGES + j);
@@ -737,10 +832,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 for (int h = 0; h < C::HALVES; ++h) tma_load_4d(dst + h * C::HALF_BYTES, &tmK, h * 64, 0, pc.g, id, bar_k);
               }
             }
-            if (!mbar_wait(smem_u32(&ctrl->empty_v[slot]), phase ^ 1u)) {
-              aborted = true;
-              break;
-            }
+            if (!mbar_wait(smem_u32(&ctrl->empty_v[slot]), phase ^ 1u)) return false;
             const uint32_t bar_v = smem_u32(&ctrl->full_v[slot]);
             if (lane == 0) mbar_arrive_expect_tx(bar_v, static_cast<uint32_t>(np) * C::PAGE_BYTES);
             __syncwarp();
@@ -777,6 +869,61 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) st_release_shared(&ctrl->prod_last[pw], it);
           }
+        }
+        return true;
+      };
+      if constexpr (WIN) {
+        // 32 units at a time (see WindowWalker); the query rows are staged by the tenth warp
+        WindowWalker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, lane};
+        walk.begin_span(sp.unit, sp.tile, sp_end - sp.flat);
+        PieceWindow W;
+        while (!aborted && walk.next(W, it)) {
+          const int it_end = it + W.total;
+          int first = pw - W.it0 % C::NPW;          // the first tile of the lane's piece that is this warp's
+          if (first < 0) first += C::NPW;
+          uint32_t m_mine = __ballot_sync(0xffffffffu, W.take > 0 && first < W.take);
+          while (m_mine && !aborted) {
+            const int wl = __ffs(m_mine) - 1;
+            m_mine &= m_mine - 1;
+            Piece pc;
+            pc.unit = __shfl_sync(0xffffffffu, W.unit, wl);
+            pc.s = __shfl_sync(0xffffffffu, W.s, wl);
+            pc.g = pc.unit - pc.s * P.Hkv;
+            pc.L = __shfl_sync(0xffffffffu, W.L, wl);
+            pc.t0 = __shfl_sync(0xffffffffu, W.t0, wl);
+            pc.nt = __shfl_sync(0xffffffffu, W.full, wl);
+            pc.tb = __shfl_sync(0xffffffffu, W.tb, wl);
+            pc.te = pc.tb + __shfl_sync(0xffffffffu, W.take, wl);
+            it = __shfl_sync(0xffffffffu, W.it0, wl);
+            if (!issue_piece(pc)) aborted = true;
+          }
+          it = it_end;
+        }
+      } else {
+        Walker walk{P.context_lens, P.start_tiles, P.Hkv, nunits, sp.unit, sp.tile, sp_end - sp.flat};
+        Piece pc;
+        while (!aborted && walk.next(pc)) {
+          if (!PROBE && pw == 0) {
+            // stage this piece's packed query rows; the consumers reach the piece several tiles later
+            const int qs = pcnt % C::QSLOTS;
+            const uint32_t qphase = (pcnt / C::QSLOTS) & 1;
+            if (!mbar_wait(smem_u32(&ctrl->q_empty[qs]), qphase ^ 1u)) {
+              aborted = true;
+              break;
+            }
+            if (lane == 0) {
+              // the G rows of each of the T query tokens, packed: row = query token * G + head
+              const uint32_t bytes = static_cast<uint32_t>(P.G) * D * 2;
+              const uint32_t qb = smem_u32(&ctrl->q_full[qs]);
+              if (CHAIN) ctrl->qseq[qs] = pcnt;
+              mbar_arrive_expect_tx(qb, bytes * P.T);
+              for (int qt = 0; qt < P.T; ++qt)
+                bulk_load(qbuf + qs * C::Q_BYTES + qt * bytes,
+                          P.q + ((static_cast<int64_t>(pc.s) * P.T + qt) * P.Hq + pc.g * P.G) * D, bytes, qb);
+            }
+          }
+          ++pcnt;
+          if (!issue_piece(pc)) aborted = true;
         }
       }
       if (aborted) break;
@@ -821,7 +968,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const int qcol = (lane & 3) * 2;
 
   if constexpr (CHAIN) {
-    consume_chain<D, NT, BS, EB>(P, pp, ctrl, ring, qbuf,
+    consume_chain<D, NT, BS, EB, WIN>(P, pp, ctrl, ring, qbuf,
                              smem + NST * C::STAGE_BYTES + C::QSLOTS * C::Q_BYTES + C::ML_BYTES + C::CTRL_BYTES, warp,
                              lane);
     return;

@@ -32,6 +32,8 @@ constexpr int kAutoInKernelTiles = 8;      // mode -1: in-kernel merge from this
 constexpr int kInKernelMergeSpans = kMaxMergeRun;   // a cut unit followed by at most this many spans is merged inside the decode kernel
 int g_host_zero_copy = -1;                // pdattn_set_host_zero_copy: -1 default (when possible), 0 never, 1 as -1
 int g_prefix_engine = -1;                 // pdattn_set_prefix_engine: -1 default (tcgen05), 0 warp MMAs, 1 tcgen05
+int g_short_path = -1;                    // pdattn_set_short_piece_path: -1 by batch shape, 0 never, 1 whenever it applies
+constexpr int kAutoShortTilesX2 = 3;      // mode -1: the short-piece kernel below 1.5 tiles per unit on average
 thread_local std::vector<int32_t> g_start_tiles_host;   // scratch of the grouped path (no call parameter lives here)
 
 // What one decode call is, beyond the plain arguments: every entry point fills one of these and hands it to
@@ -54,6 +56,7 @@ struct DevInfo;
 struct LaunchCtx {
   int block_size;
   bool chain, probe, fp8;
+  bool win;                 // the short-piece instantiation of the chained-merge kernel (8-row tiles, bf16 cache)
   DevInfo* di;
   cudaStream_t stream;
 };
@@ -108,6 +111,7 @@ struct DevInfo {
   bool attr_set[2][2][3] = {};      // [D==128][NT==2][page size / 32]
   bool probe_attr_set[2][2][3] = {};
   bool chain_attr_set[2][2][3] = {};
+  bool win_attr_set[2][3] = {};     // [D==128][page size / 32]
   bool fp8_attr_set[2][2][3] = {};  // [D==128][NT==2][page size / 32]
   bool prefix_fp8_attr_set[2][3] = {};
   bool prefix_attr_set[2][3] = {};  // [D==128][page size / 32]
@@ -315,6 +319,17 @@ pdattn_status launch_bs(const CUtensorMap& mk, const CUtensorMap& mv, const Deco
       fdone = true;
     }
     launch_dependent(k8, grid, C8::NTHREADS, C8::CHAIN_DYN_BYTES, stream, dependent, mk, mv, P);
+  } else if (lc.chain && lc.win && NT == 1) {
+    if constexpr (NT == 1) {
+      auto win = decode_kernel<D, NT, BS, false, true, 2, true>;
+      bool& wdone = di->win_attr_set[D == 128][BS / 32];
+      if (!wdone) {
+        cudaError_t we = cudaFuncSetAttribute(win, cudaFuncAttributeMaxDynamicSharedMemorySize, C::CHAIN_DYN_BYTES);
+        if (we != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", we);
+        wdone = true;
+      }
+      launch_dependent(win, grid, C::NTHREADS, C::CHAIN_DYN_BYTES, stream, dependent, mk, mv, P);
+    }
   } else if (lc.chain) {
     auto chain = decode_kernel<D, NT, BS, false, true>;
     bool& cdone = di->chain_attr_set[D == 128][NT == 2][BS / 32];
@@ -489,6 +504,12 @@ pdattn_status pdattn_append_kv_fp8(const void* k_new, const void* v_new, void* k
       static_cast<uint8_t*>(k_cache), static_cast<uint8_t*>(v_cache), k_scale, v_scale, block_table, context_lens,
       num_kv_heads, head_dim, block_size, max_blocks_per_seq, num_blocks, static_cast<int32_t*>(workspace));
   if (e != cudaSuccess) return cuda_fail("append_fp8_kernel launch", e);
+  return PDATTN_OK;
+}
+
+pdattn_status pdattn_set_short_piece_path(int mode) {
+  if (mode < -1 || mode > 1) return PDATTN_INVALID_ARG;
+  g_short_path = mode;
   return PDATTN_OK;
 }
 
@@ -981,6 +1002,7 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
                  ? kAutoDynPerCta
                  : 0);
   int grid = n_ctas, combine_grid = 0, n_spans_host = -1;
+  bool win = false;
   if (a->context_lens_host) {
     const int max_param_spans = cd.static_scratch ? n_ctas : MAX_PARAM_SPANS;
     if (!plan_spans(a->context_lens_host, start_tiles_host, a->num_seqs, a->num_kv_heads, n_ctas, dyn_per_cta,
@@ -994,9 +1016,18 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
     // 1 - 2 % on the long-context configurations.
     if (g_merge_mode == -1 && P.plan.total < static_cast<int64_t>(kAutoInKernelTiles) * a->num_seqs * a->num_kv_heads)
       P.inkernel_max = 0;
-    if (P.inkernel_max > 0) {
-      // if every cut unit is short enough for the decode kernel's own merge, combine_kernel has nothing to do
-      // and is not launched
+    // Batches of mostly one-tile pieces (below 1.5 tiles per unit on average) take the short-piece instantiation:
+    // every warp walks the spans 32 units at a time and the tenth warp stages the query rows instead of merging.
+    if (chain && !fp8 && !cd.probe && G * T <= 8 &&
+        (g_short_path == 1 ||
+         (g_short_path == -1 && 2 * static_cast<int64_t>(P.plan.total) <
+                                    static_cast<int64_t>(kAutoShortTilesX2) * a->num_seqs * a->num_kv_heads))) {
+      win = true;
+      P.inkernel_max = 0;
+    }
+    {
+      // if every cut unit is short enough for the decode kernel's own merge (or no unit is cut at all, as in a
+      // batch of one-tile sequences), combine_kernel has nothing to do and is not launched
       bool all_short = true;
       for (int k = 0; k < n_spans_host && all_short; ++k) all_short = merge_run(P.spans[k].merge) <= P.inkernel_max;
       if (all_short) combine_grid = 0;
@@ -1033,7 +1064,7 @@ pdattn_status decode_common(const pdattn_args* a, const CallDesc& cd, pdattn_str
                a->kv_head_stride, a->kv_token_stride, fp8 ? kMapV8 : rank, &mv);
   if (s != PDATTN_OK) return s;
   P.box5d = rank == 5;
-  const LaunchCtx lc{a->block_size, chain, cd.probe, fp8, di, stream};
+  const LaunchCtx lc{a->block_size, chain, cd.probe, fp8, win, di, stream};
 
   if (grouped) {
     // shared prompt tiles first: one pass per (group, kv head) for the query rows of all samples

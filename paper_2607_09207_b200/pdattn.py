@@ -32,7 +32,7 @@ EXPORTS = [
     "pdattn_host_staging_size", "pdattn_decode_host", "pdattn_plan_host", "pdattn_check",
     "pdattn_last_launch_count", "pdattn_status_string", "pdattn_last_cuda_error", "pdattn_profile_events",
     "pdattn_gather_probe", "pdattn_stream_read_probe", "pdattn_wait_limit_probe", "pdattn_set_dynamic_spans",
-    "pdattn_set_merge_mode", "pdattn_set_prefix_engine", "pdattn_set_host_zero_copy",
+    "pdattn_set_merge_mode", "pdattn_set_prefix_engine", "pdattn_set_host_zero_copy", "pdattn_set_short_piece_path",
     "pdattn_decode_static_scratch", "pdattn_append_kv",
     "pdattn_grouped_workspace_size", "pdattn_decode_grouped",
     "pdattn_multi_workspace_size", "pdattn_decode_multi", "pdattn_decode_fp8", "pdattn_append_kv_fp8", "pdattn_decode_fp8_multi",
@@ -92,6 +92,7 @@ def lib():
         L.pdattn_set_dynamic_spans.argtypes = [i32]
         L.pdattn_set_merge_mode.argtypes = [i32]
         L.pdattn_set_prefix_engine.argtypes = [i32]
+        L.pdattn_set_short_piece_path.argtypes = [i32]
         L.pdattn_set_host_zero_copy.argtypes = [i32]
         L.pdattn_decode_static_scratch.argtypes = [ctypes.POINTER(Args), vp, vp]
         L.pdattn_grouped_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
@@ -475,6 +476,14 @@ def set_merge_mode(mode: int):
     st = lib().pdattn_set_merge_mode(mode)
     if st != OK:
         raise PdattnError(st, "pdattn_set_merge_mode")
+
+
+def set_short_piece_path(mode: int):
+    """-1: the short-piece kernel instantiation for batches below 1.5 tiles per unit on average (default); 0: never; 1: whenever
+    it applies (chained merge, bf16 cache, at most 8 query rows per KV head, host lengths)."""
+    st = lib().pdattn_set_short_piece_path(mode)
+    if st != OK:
+        raise PdattnError(st, "pdattn_set_short_piece_path")
 
 
 def set_prefix_engine(engine: int):

@@ -27,10 +27,11 @@ def pytest_collection_modifyitems(config, items):
 
 
 # The GPU parity modules run once per merge mode: the barrier merge with the combine kernel, the chained merge
-# with the final merge of cut units inside the decode kernel (the default), and the chained merge with the
-# combine kernel must each pass every case, whatever the library would pick by itself.
+# with the final merge of cut units inside the decode kernel (the default), the chained merge with the
+# combine kernel, and the short-piece instantiation of the latter (forced on for every batch it can run) must
+# each pass every case, whatever the library would pick by itself.  Values: (merge mode, short-piece path).
 MERGE_MODE_MODULES = ("test_gpu_parity", "test_gpu_grouped", "test_gpu_decode_loop", "test_gpu_multi_token")
-MERGE_MODES = {"barrier": 0, "chain": 1, "chain_combine": 2}
+MERGE_MODES = {"barrier": (0, -1), "chain": (1, -1), "chain_combine": (2, -1), "chain_short": (2, 1)}
 
 
 # ... and the grouped-decode module once per kernel for the shared prompt tiles.
@@ -67,11 +68,13 @@ def merge_mode(request):
         yield None
         return
     from paper_2607_09207_b200 import pdattn
-    pdattn.set_merge_mode(MERGE_MODES[name])
+    pdattn.set_merge_mode(MERGE_MODES[name][0])
+    pdattn.set_short_piece_path(MERGE_MODES[name][1])
     try:
         yield name
     finally:
         pdattn.set_merge_mode(-1)
+        pdattn.set_short_piece_path(-1)
 
 
 # The fp64 oracle's output for a benchmark configuration at full size, every (sequence, head) row.  The

@@ -79,6 +79,11 @@ def test_tuning_setters_check_their_ranges():
         assert L.pdattn_set_host_zero_copy(mode) == pdattn.OK
     assert L.pdattn_set_host_zero_copy(2) == pdattn.INVALID_ARG
     assert L.pdattn_set_host_zero_copy(-1) == pdattn.OK
+    for mode in (-1, 0, 1):
+        assert L.pdattn_set_short_piece_path(mode) == pdattn.OK
+    for mode in (-2, 2):
+        assert L.pdattn_set_short_piece_path(mode) == pdattn.INVALID_ARG
+    assert L.pdattn_set_short_piece_path(-1) == pdattn.OK
 
 
 def test_workspace_size_and_shape_checks():

@@ -96,6 +96,43 @@ def test_batches_of_two_to_eleven_tile_pieces(Hq, Hkv, d, bs):
     assert st == pdattn.OK and torch.equal(out, again)      # the order of every sum is fixed
 
 
+@pytest.mark.parametrize("Hq,Hkv,d,bs", [(28, 4, 128, 16), (8, 2, 64, 32), (5, 5, 128, 64), (16, 2, 64, 16)])
+@pytest.mark.parametrize("kind", ["one_tile", "ragged", "few_tiles"])
+def test_short_piece_kernel_same_bits_as_the_default_kernel(Hq, Hkv, d, bs, kind):
+    """The short-piece instantiation (every warp walks 32 units at a time, a warp of its own stages the query
+    rows) against the oracle, and bit for bit against the all-purpose instantiation: same tile dealing, same
+    order of every sum.  A batch in which no sequence is cut needs no combine launch."""
+    rng = np.random.default_rng(31)
+    S = 1500
+    lens = {"one_tile": rng.integers(1, 65, size=S), "ragged": rng.integers(0, 260, size=S),
+            "few_tiles": rng.integers(40, 700, size=S)}[kind]
+    if kind == "ragged":
+        lens[rng.integers(S, size=40)] = 0                    # empty sequences inside the 32-unit windows
+        lens[rng.integers(S, size=3)] = rng.integers(3000, 9000, size=3)   # and a few long ones cut over many spans
+    w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, bs=bs, seed=37, device=DEV)
+    try:
+        pdattn.set_merge_mode(2)
+        pdattn.set_short_piece_path(0)
+        base, st = run(w)
+        assert st == pdattn.OK
+        pdattn.set_short_piece_path(1)
+        out = check_against_oracle(w, f"short-piece kernel, {kind}", pairs=sample_pairs(w, 800, seed=41))
+        assert torch.equal(out, base)
+        for _ in range(3):
+            again, st = run(w)
+            assert st == pdattn.OK and torch.equal(out, again)
+        # by itself the library takes this kernel for batches of mostly one-tile sequences
+        pdattn.set_merge_mode(-1)
+        pdattn.set_short_piece_path(-1)
+        auto, st = run(w)
+        assert st == pdattn.OK and torch.equal(out, auto)
+        if kind == "one_tile":
+            assert pdattn.last_launch_count() == 1            # nothing is cut: no combine launch
+    finally:
+        pdattn.set_merge_mode(-1)
+        pdattn.set_short_piece_path(-1)
+
+
 def test_single_long_sequence_is_split_over_all_sms():
     w = W.make_custom([40000], Hq=7, Hkv=1, d=128, seed=6, device=DEV)
     check_against_oracle(w, "one long sequence")

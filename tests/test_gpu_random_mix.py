@@ -42,10 +42,11 @@ def test_random_mix_of_everything(seed):
             lens = rng.integers(0, hi, size=S)
             if kind == "mixed": lens[rng.integers(S)] = int(rng.integers(20000, 60000))
             mode = int(rng.choice([-1, 0, 1, 2])); dyn = int(rng.choice([-1, 0, 3, 8])); host = bool(rng.integers(2))
-            pdattn.set_merge_mode(mode); pdattn.set_dynamic_spans(dyn)
+            short = int(rng.choice([-1, 0, 1]))
+            pdattn.set_merge_mode(mode); pdattn.set_dynamic_spans(dyn); pdattn.set_short_piece_path(short)
             variant = rng.choice(["plain", "multi", "fp8", "grouped", "fp8multi"])
             G = Hq // Hkv
-            desc = f"{variant} Hq={Hq} Hkv={Hkv} d={d} bs={bs} S={S} {kind} mode={mode} dyn={dyn} host={host}"
+            desc = f"{variant} Hq={Hq} Hkv={Hkv} d={d} bs={bs} S={S} {kind} mode={mode} dyn={dyn} short={short} host={host}"
             try:
                 w = W.make_custom(lens, Hq=Hq, Hkv=Hkv, d=d, bs=bs, seed=int(rng.integers(1 << 30)), device=DEV)
                 wc = w.to("cpu")
@@ -108,6 +109,7 @@ def test_random_mix_of_everything(seed):
     finally:
         pdattn.set_merge_mode(-1)
         pdattn.set_dynamic_spans(-1)
+        pdattn.set_short_piece_path(-1)
         pdattn.set_prefix_engine(-1)
     assert not failures, "\n".join(failures)
     assert n == 60
