@@ -56,9 +56,11 @@ def parse():
     ap.add_argument("--fp8", action="store_true",
                     help="time pdattn_decode_fp8 over an e4m3 copy of the same pools (half the KV bytes per step) "
                          "instead of the bf16 step; head_dim 128 configurations only")
-    ap.add_argument("--short-batches", action="store_true",
-                    help="also time batches of 4096 short contexts under both merge modes, and a large GRPO batch "
-                         "early in its rollout under both prefix kernels (secondary results, N = 1)")
+    ap.add_argument("--short-batches", nargs="?", const="all", default=None, metavar="NAME",
+                    help="also time batches of 4096 short contexts under every merge mode and with the short-piece "
+                         "kernel off, and a large GRPO batch early in its rollout under both prefix kernels "
+                         "(secondary results, N = 1); with NAME (4096x64, 4096x128, 4096xU[50,400], 4096x512, grpo) "
+                         "only that batch, e.g. for a profiler capture of one small case")
     ap.add_argument("--grouped", action="store_true",
                     help="config 3 only: time pdattn_decode_grouped (shared prompt pages read once per group)")
     ap.add_argument("--no-all-configs", action="store_true",
@@ -549,7 +551,7 @@ def main():
                                                "unique_kv_gbs": uniq / (t_grouped * 1e-3) / 1e9}
 
         if args.short_batches:
-            extras["short_context_batches"] = short_batches(pdattn, W, dev, timed)
+            extras["short_context_batches"] = short_batches(pdattn, W, dev, timed, args.short_batches)
         if args.cfg == 2 and args.num_seqs is None and not args.no_all_configs:
             extras["configs"] = other_configs(pdattn, W, dev, stream, local, peak, with_oracle=not args.no_cpu_baseline)
 
@@ -620,14 +622,18 @@ def main():
         dist.destroy_process_group()
 
 
-def short_batches(pdattn, W, dev, timed):
+def short_batches(pdattn, W, dev, timed, only="all"):
     """Batches whose pieces are one to a few tiles long: 4096 sequences of the 7B shape under the barrier
-    and the chained merge of the decode kernel, and 512 GRPO groups of 8 (40 q / 8 KV heads) that share a
-    1024-token prompt and have generated 1..64 tokens, under both kernels for the shared tiles."""
+    and the chained merge of the decode kernel (and, in the default mode, with the short-piece instantiation
+    switched off), and 512 GRPO groups of 8 (40 q / 8 KV heads) that share a 1024-token prompt and have
+    generated 1..64 tokens, under both kernels for the shared tiles."""
     res = {}
     rng = np.random.default_rng(0)
+    ragged = rng.integers(50, 400, size=4096)
     for name, lens in [("4096x64", np.full(4096, 64)), ("4096x128", np.full(4096, 128)),
-                       ("4096xU[50,400]", rng.integers(50, 400, size=4096)), ("4096x512", np.full(4096, 512))]:
+                       ("4096xU[50,400]", ragged), ("4096x512", np.full(4096, 512))]:
+        if only not in ("all", name):
+            continue
         w = W.make_custom(lens, Hq=28, Hkv=4, d=128, bs=16, seed=3, device=dev, poison=False)
         ws = pdattn.alloc_workspace(w.num_seqs, 28, 4, 128, 16, device=dev)
         out = torch.empty_like(w.q)
@@ -637,11 +643,20 @@ def short_batches(pdattn, W, dev, timed):
             pdattn.set_merge_mode(mode)
             row[key] = timed(lambda: pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale,
                                                       out, ws, context_lens_host=w.context_lens_host))
+        row["launches_per_step_default"] = pdattn.last_launch_count()
+        pdattn.set_short_piece_path(0)
+        row["default_short_piece_kernel_off_ms"] = timed(
+            lambda: pdattn.decode_ex(w.q, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.scale, out, ws,
+                                     context_lens_host=w.context_lens_host))
+        pdattn.set_short_piece_path(-1)
         pdattn.set_merge_mode(-1)
+        row["default_kv_gbs"] = row["kv_bytes"] / (row["default_ms"] * 1e-3) / 1e9
         assert pdattn.check(ws) == pdattn.OK
         res[name] = row
         del w, ws, out
         torch.cuda.empty_cache()
+    if only not in ("all", "grpo"):
+        return res
     lens = 1024 + rng.integers(1, 65, size=4096)
     w = W.make_custom(lens, Hq=40, Hkv=8, d=128, bs=16, seed=3, device=dev, poison=False, shared_prefix_pages=64, group=8)
     gws = pdattn.alloc_grouped_workspace(w.num_seqs, 40, 8, 128, device=dev)
