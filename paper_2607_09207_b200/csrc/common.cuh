@@ -27,6 +27,9 @@ namespace pdattn {
 
 constexpr int TILE = kTileTokens;                // tokens per pipeline stage
 constexpr int MAX_SPANS = 2048;                  // spans per call (static + run-time); sizes the workspace
+#ifndef PDATTN_DRAW_AHEAD
+#define PDATTN_DRAW_AHEAD 12   // tiles left in a span when the producer draws the CTA's next run-time span
+#endif
 constexpr int MAX_PARAM_SPANS = 768;             // spans that can travel in kernel parameters
 constexpr int SPAN_QUEUE = 32;                   // in-CTA queue of run-time span ids
 constexpr int MAX_STAGES = 14;

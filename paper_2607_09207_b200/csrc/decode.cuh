@@ -755,17 +755,28 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const int pw = warp - NCW;
     constexpr int IDS_PER_BATCH = 32;
     constexpr int TILES_PER_BATCH = IDS_PER_BATCH / C::PAGES;
+    constexpr int DRAW_AHEAD = PDATTN_DRAW_AHEAD;
     bool any_bad = false;
     int span = cta;
     for (int k = 0; span >= 0; ++k) {
-      // draw the next run-time span now; its id is only consumed after this span's tiles are issued
-      int nxt = -1;
-      if (pw == 0 && lane == 0 && pp.n_dyn > 0) {
-        const int j = atomicAdd(&P.hdr->counter, 1);
-        nxt = j < pp.n_dyn ? pp.n_static + j : -1;
-      }
       const SpanStart sp = P.use_ws_plan ? P.spans_ws[span] : P.spans[span];
       const int sp_end = P.use_ws_plan ? P.spans_ws[span + 1].flat : P.spans[span + 1].flat;
+      // The next run-time span is drawn when this span has DRAW_AHEAD tiles left to issue: early enough to hide the
+      // atomic's round trip (its result is only consumed after this span's tiles are issued), late enough that a
+      // CTA does not sit on a reserved span for the length of a whole span while other CTAs run dry.
+      int nxt = -1;
+      bool drawn = !(pw == 0 && pp.n_dyn > 0);
+      const int draw_at = it + (sp_end - sp.flat) - DRAW_AHEAD;
+      auto maybe_draw = [&](int it_now) {
+        if (!drawn && it_now >= draw_at) {
+          drawn = true;
+          if (lane == 0) {
+            const int j = atomicAdd(&P.hdr->counter, 1);
+            nxt = j < pp.n_dyn ? pp.n_static + j : -1;
+          }
+        }
+      };
+      maybe_draw(it);
       // ---- the tiles of one piece that this warp issues (`it`: the CTA's tile counter at the piece's first tile)
       auto issue_piece = [&](const Piece& pc) -> bool {
         const int32_t* row = P.block_table + static_cast<int64_t>(pc.s) * P.MB;
@@ -788,6 +799,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             ids_cur = ids_nxt;
             ids_nxt = page_id(pbase + rel * C::PAGES + IDS_PER_BATCH + lane);
           }
+          maybe_draw(it);
           if (C::NPW > 1 && it % C::NPW != pw) continue;
           const int slot = it % NST;
           const uint32_t phase = (it / NST) & 1;
@@ -879,6 +891,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         PieceWindow W;
         while (!aborted && walk.next(W, it)) {
           const int it_end = it + W.total;
+          maybe_draw(it_end);
           int first = pw - W.it0 % C::NPW;          // the first tile of the lane's piece that is this warp's
           if (first < 0) first += C::NPW;
           uint32_t m_mine = __ballot_sync(0xffffffffu, W.take > 0 && first < W.take);
@@ -927,6 +940,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
       }
       if (aborted) break;
+      maybe_draw(draw_at);
       if (pw == 0) {
         if (lane == 0) {
           const int slot = k % SPAN_QUEUE;

@@ -33,6 +33,14 @@ namespace pdattn {
 constexpr int kTileTokens = PDATTN_TILE_TOKENS;
 constexpr int kPieceCostTiles = PDATTN_PIECE_COST;
 constexpr int kMaxDynPerCta = 8;      // at most this many run-time spans per CTA
+#ifndef PDATTN_DYN_EIGHTHS
+#define PDATTN_DYN_EIGHTHS 2
+#endif
+constexpr int kDynEighths = PDATTN_DYN_EIGHTHS;   // share of the cost stream that is cut into run-time spans, in eighths
+#ifndef PDATTN_TAPER
+#define PDATTN_TAPER 3
+#endif
+constexpr int kTaper = PDATTN_TAPER;   // taper of the run-time spans, in quarters (0: equal spans)
 constexpr int kMinDynCost = 8;        // a run-time span is never cheaper than this
 constexpr int kStaticOnlyBelow = 16;  // less cost per CTA than this: no run-time spans
 
@@ -100,9 +108,10 @@ PDATTN_HD inline PlanParams make_plan_params(int64_t total_cost, int64_t total_t
   p.cost_static = total_cost;
   p.total = static_cast<int>(total_tiles);
   if (n_dyn_max > 0 && total_cost >= static_cast<int64_t>(n_static) * kStaticOnlyBelow) {
-    const int64_t cd = total_cost / 4;
+    const int64_t cd = total_cost * kDynEighths / 8;
     int64_t d = (cd + n_dyn_max - 1) / n_dyn_max;
-    if (d < kMinDynCost) d = kMinDynCost;
+    // (the smallest span of the taper, (4 - kTaper) / 4 of the mean, is held to the minimum)
+    if (d * (4 - kTaper) < kMinDynCost * 4) d = (kMinDynCost * 4 + 3 - kTaper) / (4 - kTaper);
     p.n_dyn = static_cast<int>((cd + d - 1) / d);
     p.cost_static = total_cost - cd;
   }
@@ -111,8 +120,10 @@ PDATTN_HD inline PlanParams make_plan_params(int64_t total_cost, int64_t total_t
 // cost coordinate at which span i begins (i == n_static + n_dyn gives the end of the stream)
 PDATTN_HD inline int64_t span_cost_start(const PlanParams& p, int i) {
   if (i <= p.n_static) return p.cost_static * i / p.n_static;
-  const int j = i - p.n_static;
-  return p.cost_static + (p.cost_total - p.cost_static) * j / p.n_dyn;
+  // run-time spans shrink linearly from (4 + kTaper) / 4 of their mean cost to (4 - kTaper) / 4 of it: the CTAs draw
+  // them in this order, so the ones that decide when the last CTA finishes are the small ones
+  const int64_t j = i - p.n_static, n = p.n_dyn;
+  return p.cost_static + (p.cost_total - p.cost_static) * (j * ((4 + kTaper) * n - kTaper * j)) / (4 * n * n);
 }
 // cost of one sequence: Hkv units of nt tiles each
 PDATTN_HD inline int64_t seq_cost(int64_t nt, int hkv) { return nt > 0 ? (nt + kPieceCostTiles) * hkv : 0; }
