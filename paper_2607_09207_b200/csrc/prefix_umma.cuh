@@ -588,8 +588,8 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           stage_q(nu.u, n + 1);
         }
         const bool mine = pt >= 2 || owner;     // a one-tile unit leaves the other team without a state
-        wait_all(&ctrl->unit_done, n & 1);
-        tc_fence_after();
+        // The teams' (m, l) are final as soon as their own last tile's softmax is done, so they are exchanged and
+        // the common reference and the two factors computed while the unit's last products still run.
         if (!is_lo) xs[tm * 64 + rho] = mine ? m : NEG_INF;
         xs[128 + (is_lo ? 128 : 0) + tm * 64 + rho] = mine ? l : 0.f;
         all_barrier();
@@ -597,6 +597,10 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         const float mt = fmaxf(m0, m1);
         const float mtu = (mt == NEG_INF) ? 0.f : mt;
         const float f0 = fast_exp2(m0 - mtu), f1 = fast_exp2(m1 - mtu);   // 0 for a team without a state
+        // (read here, before the second barrier: after it nobody touches this area until the next unit writes it)
+        const float lsum = (xs[128 + rho] + xs[256 + rho]) * f0 + (xs[192 + rho] + xs[320 + rho]) * f1;
+        wait_all(&ctrl->unit_done, n & 1);
+        tc_fence_after();
         const int c0 = tm * (D / 2);
         uint4* xrow = reinterpret_cast<uint4*>(xo) + rho * (D / 8);       // a row of bf16: D / 8 chunks of 16 bytes
         auto combined = [&](int q, float (&v)[32]) {   // columns c0 + 32 q .. + 31 of this lane, both teams, common reference
@@ -637,11 +641,11 @@ prefix_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           }
           if (tm == 0) {
             slotp[rh] = mt;
-            slotp[C::HP + rh] = (xs[128 + rho] + xs[256 + rho]) * f0 + (xs[192 + rho] + xs[320 + rho]) * f1;
+            slotp[C::HP + rh] = lsum;
           }
         }
-        // (no barrier here: the next unit's writes to these areas come after its first barrier, which every
-        // thread reaches only after the reads above)
+        // (no barrier here: the next unit's writes to the (m, l) area come after this unit's second barrier, which
+        // every read of it precedes, and those to the bf16 rows after the next unit's first barrier)
       }
       uc = nu;
     }
