@@ -251,6 +251,27 @@ def test_partitioner_balances_cost_not_tiles():
     assert np.corrcoef(units, tiles)[0, 1] < -0.8       # more units to start -> fewer tiles
 
 
+def test_runtime_spans_are_a_quarter_of_the_cost_and_shrink_along_the_stream():
+    """Config 2 with up to 4 run-time spans per CTA: the static spans share 3/4 of the cost evenly, the run-time spans
+    the rest, falling linearly from 1.75 to 0.25 of their mean cost (to within the cut unit's start-up); there are
+    as many of them as keeps the smallest at 8 cost units (the partitioner's minimum), and none is empty."""
+    lens = W.config_lengths(2)
+    cover, plan = walk_spans(lens, 4, 148, dyn=4)
+    assert plan.n_static == 148 and 148 < plan.n_dynamic <= 4 * 148
+    costs = np.array([span_cost(m) for m in cover], dtype=np.float64)
+    stat, dyn = costs[:148], costs[148:]
+    assert all(len(m) > 0 for m in cover)
+    assert stat.max() - stat.min() <= 2 * PIECE_COST + 1
+    total = stat.sum() + dyn.sum()
+    assert abs(dyn.sum() / total - 0.25) < 0.01
+    mean = dyn.mean()
+    n = len(dyn)
+    want = mean * (1.75 - 1.5 * (np.arange(n) + 0.5) / n)
+    assert np.abs(dyn - want).max() <= 2 * PIECE_COST + 2
+    assert dyn[:8].mean() > 5 * dyn[-8:].mean()
+    assert 8 - 1 <= 0.25 * mean <= 8 + 1                 # the smallest span's nominal cost
+
+
 def test_partitioner_spreads_the_straggler_phase_over_all_sms():
     """8 sequences x 4 KV heads = 32 units must still occupy all 148 CTAs."""
     lens = W.config_lengths(5)
