@@ -280,7 +280,9 @@ pdattn_status pdattn_decode_host_fp8(const void* q_host, const int32_t* block_ta
  * costs its tiles plus 2 for starting it, so a CTA that walks many short sequences gets fewer
  * tiles than one inside a long sequence.  n_static spans, one per CTA, cover the stream; with
  * dynamic_per_cta > 0 they cover only its first three quarters (by cost) and up to n_ctas *
- * dynamic_per_cta short spans cover the rest, taken at run time by whichever CTA is free.
+ * dynamic_per_cta short spans cover the rest, taken at run time, in stream order, by whichever CTA is free;
+ * their cost falls linearly along the stream from 1.75 to 0.25 of their mean, and there are no more of them
+ * than keeps the smallest at 8 cost units.
  * spans: HOST int32 [4 * (max_spans + 1)], one (unit, tile, flat, merge) entry per span plus an end
  * marker: span i starts at tile `tile` of unit `unit`, which is tile number `flat` of the stream,
  * and holds flat[i + 1] - flat[i] tiles (possibly none).  n_static + n_dynamic <= max_spans.

@@ -254,7 +254,7 @@ struct Cfg {
   static constexpr int CTRL_BYTES = 1280;
   static constexpr int NCW = PDATTN_NCW;                               // consumer warps
   static constexpr int ML_BYTES = NCW * HP * 2 * 4;
-  static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged by producer 0
+  static constexpr int QSLOTS = 4;                     // query rows of upcoming pieces, staged ahead of the consumers
   static constexpr int Q_BYTES = HP * D * 2;           // one slot: the packed query heads of one KV head
   static constexpr int NSTAGES_FIT = (SMEM_MAX - 1024 - QSLOTS * Q_BYTES - ML_BYTES - CTRL_BYTES) / STAGE_BYTES;
   static constexpr int NSTAGES = (NSTAGES_FIT > MAX_STAGES ? MAX_STAGES : NSTAGES_FIT) / NCW * NCW;
@@ -418,8 +418,8 @@ struct WindowWalker {
 // ------------------------------------------------------------------------------------------
 // Span sequencing inside a CTA.  Every warp walks the same sequence of spans: first the CTA's
 // static span, then run-time spans.  Lane 0 of producer warp 0 draws run-time spans from the
-// global counter (one atomic per span, issued a whole span ahead of its use) and publishes the
-// ids through a small shared-memory queue; every other warp reads them from there.
+// global counter (one atomic per span, issued a dozen tiles before the current span's last) and
+// publishes the ids through a small shared-memory queue; every other warp reads them from there.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ int ld_acquire_shared(const int32_t* p) {
   int v;

@@ -1187,7 +1187,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
               }
             }
           }
-          bar_consumers<NCT>();   // everyone has read this round's accumulators
+          bar_consumers<NCT>();   // everyone has read this pass's accumulators
         }
         if (warp == w_last && !aborted) {
           fence_proxy_async();    // our stores into the slot are ordered before the TMA write that refills it

@@ -3,8 +3,9 @@
 // The batch is flattened into a stream of fixed-size token tiles, unit-major (unit = sequence *
 // Hkv + kv_head; unit u has ceil(L_s / tile) tiles), and the stream is cut into contiguous spans:
 //   - n_static spans, one per CTA;
-//   - optionally n_dyn short spans over the last quarter of the stream, handed out at run time to
-//     whichever CTA finishes first.
+//   - optionally n_dyn short spans over the last quarter of the stream, handed out at run time, in
+//     stream order, to whichever CTA is free; they shrink along the stream (kTaper), so that the
+//     ones handed out last are the cheapest.
 // Spans are balanced by COST, not by tile count: a unit costs its tiles plus kPieceCostTiles for
 // starting it (query rows, page-table row, merge of the warp states, output); a sweep of that
 // constant on the 7B-shaped batch put the best value at 2.  In cost coordinates unit u covers
